@@ -395,6 +395,15 @@ def test_find_split_validity_rules():
     no = oracle.find_split(hg, hh, 0, 20, 20, 1.0, 1.0, True,
                            oracle.make_params(min_data_in_leaf=1, min_gain=1e9))
     assert not no.valid                           # gain must exceed the floor
+    # a side whose hessian mass is zero is never a candidate (Eq. 7 would divide by zero)
+    z = oracle.find_split(np.array([[5, -5, 0, 0]], np.int64), np.array([[0, 20, 0, 0]], np.int64), 0, 20, 20,
+                          1.0, 1.0, False, oracle.make_params(min_data_in_leaf=0))
+    assert not z.valid
+    # estimated rows per side are rounded to nearest: 7/20 of 30 rows = 10.5 -> 11
+    hg2 = np.array([[9, -9, 0, 0]], np.int64)
+    hh2 = np.array([[7, 13, 0, 0]], np.int64)
+    e = oracle.find_split(hg2, hh2, 0, 20, 30, 1.0, 1.0, False, oracle.make_params(min_data_in_leaf=11))
+    assert e.valid and (e.nl_est, e.nr_est) == (11, 19)
     flat = oracle.find_split(np.zeros((1, nb), np.int64), hh, 0, 20, 20, 1.0, 1.0, True,
                              oracle.make_params(min_data_in_leaf=1))
     assert not flat.valid                         # zero gain is not a split
@@ -568,6 +577,35 @@ def test_first_split_is_the_root_argmax():
                           False, prm)
     assert (t.feature[0], t.bin[0]) == (s.feature, s.bin) and t.gain[0] == s.gain
     assert t.leaf_count[0] == int((data[:, s.feature] <= s.bin).sum())
+
+
+def test_every_split_is_the_best_first_choice():
+    # replay the growth from the recorded nodes: at each step the split taken must be the largest-gain
+    # candidate among the current leaves, each found from that leaf's own rows and integer totals
+    data, y, _ = toy_classification(n=3000, seed=6)
+    prm = oracle.make_params(bits=3, num_leaves=6, seed=4)
+    scores = np.zeros(len(y), np.float32)
+    t = oracle.train_tree(data, 32, y, scores, prm, 0)
+    g, h = oracle.gradients(0, np.zeros(len(y), np.float32), y)
+    q = oracle.quantize(g, h, bits=3, seed=4, tree=0)
+    gq, hq = q.gq.astype(np.int64), q.hq.astype(np.int64)
+
+    def best_of(rows):
+        hg, hh = oracle.histogram(data, 32, q.gq, q.hq, rows.astype(np.uint32))
+        return oracle.find_split(hg, hh, gq[rows].sum(), hq[rows].sum(), len(rows), q.gmax, q.hmax, False, prm)
+
+    leaves = {0: np.arange(len(y))}
+    for node in range(t.num_leaves - 1):
+        cands = {l: best_of(r) for l, r in leaves.items()}
+        pick = max((l for l in cands if cands[l].valid), key=lambda l: (cands[l].gain, -l))
+        s = cands[pick]
+        assert (t.feature[node], t.bin[node]) == (s.feature, s.bin) and t.gain[node] == s.gain
+        rows = leaves[pick]
+        go_left = data[rows, s.feature] <= s.bin
+        assert gq[rows[go_left]].sum() == s.gl and hq[rows[go_left]].sum() == s.hl
+        leaves[pick], leaves[node + 1] = rows[go_left], rows[~go_left]
+    for l, rows in leaves.items():
+        assert t.leaf_count[l] == len(rows)
 
 
 def test_training_loss_decreases_and_tracks_high_precision():

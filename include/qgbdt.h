@@ -1,0 +1,184 @@
+/*
+ * qgbdt.h -- C ABI of the quantized-GBDT hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library trains gradient-boosted trees from gradients quantized to 2..8 bits
+ * by stochastic rounding, with integer histograms ("Quantized Training of Gradient
+ * Boosting Decision Trees", arXiv 2207.09682).  Every step below runs in hand-written
+ * CUDA kernels; there is no CPU fallback.
+ *
+ * Conventions
+ *  - Every call returns 0 (QGBDT_OK) or a negative error code; qgbdt_last_error()
+ *    gives the message of the last failure on that context.  Nothing throws or aborts.
+ *  - Pointers named d_* are DEVICE pointers owned by the caller; they must stay valid
+ *    until the stream work of the call has finished.  Pointers named h_* (and all
+ *    scalar out-parameters) are HOST pointers owned by the caller.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *    that only take device pointers are asynchronous on that stream; calls that return
+ *    host scalars synchronise the stream before returning (stated per call).
+ *  - A context belongs to the CUDA device that was current when it was created, owns
+ *    its work buffers (relaid bin matrix, row-index lists, packed gradient codes,
+ *    histogram pool, scratch) and frees them in qgbdt_destroy().  A context is not
+ *    thread-safe.
+ *  - Histogram layout: hist[feature][bin], one 64-bit word per bin holding the hessian
+ *    sum in the low 32 bits (unsigned) and the gradient sum in the high 32 bits
+ *    (signed): word = (int64)G * 2^32 + H  (Sec. 6.2, packed gradient and hessian).
+ *  - Leaf numbering: before any split there is one leaf, 0, holding all rows in
+ *    ascending order.  Splitting leaf l keeps l as the left child (bin <= threshold)
+ *    and gives the right child the next unused leaf number.
+ */
+#ifndef QGBDT_H
+#define QGBDT_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QGBDT_OK 0
+#define QGBDT_ERR_ARG (-1)      /* null pointer, size or parameter out of range           */
+#define QGBDT_ERR_STATE (-2)    /* call out of order (e.g. histogram before quantize)     */
+#define QGBDT_ERR_OVERFLOW (-3) /* integer sums could exceed the 32+32-bit histogram word */
+#define QGBDT_ERR_CUDA (-4)     /* a CUDA runtime call or kernel failed                   */
+#define QGBDT_ERR_ALLOC (-5)    /* device or host allocation failed                       */
+#define QGBDT_ERR_VALUE (-6)    /* non-finite gradient, negative hessian, |g| or h >= 256,
+                                   or a bin code >= n_bins                                */
+
+typedef struct qgbdt_ctx qgbdt_ctx;
+
+/* Training parameters.  Defaults of the paper's runs: learning_rate 0.1, 255 leaves. */
+typedef struct {
+    int32_t bits;             /* B, gradient bits, 2..8 (Sec. 4.1)                              */
+    int32_t objective;        /* 0: logistic loss, labels in {0,1}; 1: squared loss (hessian 1) */
+    int32_t num_leaves;       /* leaves per tree, 1..4096 (leaf-wise growth, Sec. 3)            */
+    int32_t num_trees;        /* informational; qgbdt_train takes its own count                */
+    int32_t min_data_in_leaf; /* a split needs this many (estimated) rows on both sides         */
+    double learning_rate;     /* leaf outputs are learning_rate * w* (Eq. 3)                    */
+    double lambda_l2;         /* added to every hessian sum in Eq. 3 / Eq. 7 (paper: 0)         */
+    double min_sum_hessian;   /* a split needs this much dequantized hessian on both sides      */
+    double min_gain;          /* a split needs gain > min_gain                                  */
+    uint64_t seed;            /* seed of the stochastic-rounding hash                           */
+    int32_t hess_levels_mode; /* 0: delta_h = max h / (2^B - 2) (Eq. 5); 1: max h / (2^B - 1)   */
+    int32_t rounding;         /* 0: stochastic rounding; 1: round to nearest (Eq. 8)            */
+} qgbdt_params;
+
+/* One histogram bin: little-endian view of the packed 64-bit word. */
+typedef struct {
+    uint32_t h; /* sum of quantized hessians */
+    int32_t g;  /* sum of quantized gradients */
+} qgbdt_bin;
+
+/* Best split of one leaf (Eq. 7).  Rows with bin <= `bin` of `feature` go left. */
+typedef struct {
+    int32_t feature, bin;
+    double gain;
+    int64_t gl, hl, gr, hr; /* integer gradient / hessian sums of the two sides */
+    int64_t nl_est, nr_est; /* rows per side estimated from hessian sums (exact for constant hessian) */
+    int32_t valid;          /* 0: the leaf has no admissible split */
+} qgbdt_split;
+
+/* Trees written by qgbdt_train: HOST arrays allocated by the caller.  L = params.num_leaves.
+ * Tree k uses node slots [k*(L-1), (k+1)*(L-1)) and leaf slots [k*L, (k+1)*L).
+ * Node i of a tree is the i-th split made; a child c >= 0 is a node, c < 0 is leaf ~c. */
+typedef struct {
+    int32_t *num_leaves; /* [num_trees]                                   */
+    int32_t *feature;    /* [num_trees * (L-1)]                           */
+    int32_t *bin;        /* [num_trees * (L-1)] threshold bin             */
+    int32_t *left;       /* [num_trees * (L-1)]                           */
+    int32_t *right;      /* [num_trees * (L-1)]                           */
+    double *gain;        /* [num_trees * (L-1)]                           */
+    float *leaf_value;   /* [num_trees * L], already times learning_rate  */
+    int64_t *leaf_count; /* [num_trees * L] rows per leaf                 */
+} qgbdt_model;
+
+/* Creates a context on the current CUDA device.  Fails with QGBDT_ERR_ARG on parameters
+ * out of range and QGBDT_ERR_CUDA when no usable device is present. */
+int qgbdt_create(qgbdt_ctx **ctx, const qgbdt_params *params);
+int qgbdt_destroy(qgbdt_ctx *ctx);
+/* Message of the last error on this context (owned by the context; "" if none). */
+const char *qgbdt_last_error(const qgbdt_ctx *ctx);
+
+/* Loads the bin matrix data[N][J] of Algorithm 1: one uint8 bin code per (row, feature),
+ * every code < n_bins (2..256).  layout 0: row-major, element (i, j) at d_bins[i*ld + j];
+ * layout 1: column-major, element (i, j) at d_bins[j*ld + i].  The matrix is copied into
+ * an internal feature-tiled layout, so d_bins may be freed once the stream work is done.
+ * Resets the leaf state to the single root leaf.  Synchronises (it checks the codes and
+ * returns QGBDT_ERR_VALUE for a code >= n_bins).  n_rows < 2^31. */
+int qgbdt_load_binned(qgbdt_ctx *ctx, const uint8_t *d_bins, int64_t n_rows, int32_t n_features,
+                      int32_t n_bins, int32_t layout, int64_t ld, void *stream);
+/* Same with the matrix in HOST memory (pinned or pageable); the copy to the device is part
+ * of the call. */
+int qgbdt_load_binned_host(qgbdt_ctx *ctx, const uint8_t *h_bins, int64_t n_rows, int32_t n_features,
+                           int32_t n_bins, int32_t layout, int64_t ld, void *stream);
+
+/* Eq. 1: gradients of the context's objective at the current scores.  d_h may be NULL for
+ * the squared loss (constant hessian).  Asynchronous. */
+int qgbdt_compute_gradients(qgbdt_ctx *ctx, const float *d_scores, const float *d_labels,
+                            float *d_g, float *d_h, void *stream);
+
+/* Eq. 5, 6, 8: quantizes the gradients of all rows for boosting iteration `tree`:
+ * delta_g = max|g| / (2^(B-1) - 1), delta_h = max h / (2^B - 2), then stochastic rounding
+ * with a counter hash of (seed, tree, row).  d_h == NULL: constant hessian, not quantized
+ * (every row counts 1, delta_h = 1).  The packed per-row codes stay inside the context for
+ * the histogram calls.  Optional outputs: d_gq [n_rows] int8, d_hq [n_rows] uint8 (device),
+ * and the host scalars g_scale = delta_g, h_scale = delta_h, G_total, H_total (integer sums
+ * over all rows).  Synchronises.  QGBDT_ERR_VALUE on bad gradient values. */
+int qgbdt_quantize_gradients(qgbdt_ctx *ctx, const float *d_g, const float *d_h, uint32_t tree,
+                             int8_t *d_gq, uint8_t *d_hq, double *g_scale, double *h_scale,
+                             int64_t *G_total, int64_t *H_total, void *stream);
+
+/* Algorithm 1 with integer gradients for the rows of `leaf`; d_hist [n_features][n_bins] is
+ * overwritten.  Asynchronous. */
+int qgbdt_build_histograms(qgbdt_ctx *ctx, int32_t leaf, qgbdt_bin *d_hist, void *stream);
+/* The same for an explicit row list d_rows[n] (any order, duplicates counted twice). */
+int qgbdt_build_histograms_rows(qgbdt_ctx *ctx, const uint32_t *d_rows, int64_t n, qgbdt_bin *d_hist,
+                                void *stream);
+/* Histogram subtraction: d_large = d_parent - d_small, bin by bin (the larger sibling's
+ * histogram from its parent's and its smaller sibling's).  d_large may alias d_parent.
+ * Asynchronous. */
+int qgbdt_subtract_histograms(qgbdt_ctx *ctx, const qgbdt_bin *d_parent, const qgbdt_bin *d_small,
+                              qgbdt_bin *d_large, void *stream);
+
+/* Eq. 7: scans all (feature, threshold bin) candidates of a leaf whose integer totals are
+ * G, H over n_rows rows, gain in double precision from the integer sums and the scales of
+ * the last quantize call; ties go to the lowest (feature, bin).  Synchronises. */
+int qgbdt_find_best_split(qgbdt_ctx *ctx, const qgbdt_bin *d_hist, int64_t G, int64_t H, int64_t n_rows,
+                          qgbdt_split *h_out, void *stream);
+
+/* Stable partition of the rows of `leaf` by (feature, bin): rows with bin code <= bin stay
+ * in `leaf`, the others form leaf *right_leaf; relative order is kept.  Synchronises. */
+int qgbdt_split_leaf(qgbdt_ctx *ctx, int32_t leaf, int32_t feature, int32_t bin, int32_t *right_leaf,
+                     int64_t *n_left, int64_t *n_right, void *stream);
+/* Borrowed view of a leaf's row list (device memory inside the context; valid until the
+ * next split or reset). */
+int qgbdt_get_leaf_rows(qgbdt_ctx *ctx, int32_t leaf, const uint32_t **d_rows, int64_t *n);
+/* Back to the single root leaf (all rows, ascending).  Asynchronous. */
+int qgbdt_reset_leaves(qgbdt_ctx *ctx, void *stream);
+
+/* Eq. 3 with the ORIGINAL gradients (leaf-value refitting, Sec. 4.2): for every current
+ * leaf, w = -sum g / (sum h + lambda_l2) over its rows, sums taken in 2^-30 fixed point
+ * (order-independent).  h_w [current leaves] receives w, h_value the leaf outputs
+ * (float)(learning_rate * w); either may be NULL.  d_h == NULL: hessian 1.  Synchronises. */
+int qgbdt_refit_leaves(qgbdt_ctx *ctx, const float *d_g, const float *d_h, double *h_w, float *h_value,
+                       void *stream);
+
+/* Fig. 1 workflow: trains boosting iterations first_tree .. first_tree + num_trees - 1
+ * (gradients, quantization, leaf-wise growth with integer histograms and histogram
+ * subtraction, refit, score update).  d_labels [n_rows]; d_scores [n_rows] holds the
+ * current predictions on entry and the updated ones on return.  `model` (host) receives
+ * the trees, tree k of this call in slot k.  Synchronises. */
+int qgbdt_train(qgbdt_ctx *ctx, const float *d_labels, float *d_scores, uint32_t first_tree,
+                int32_t num_trees, qgbdt_model *model, void *stream);
+/* Same with labels and scores in HOST memory; both copies are part of the call. */
+int qgbdt_train_host(qgbdt_ctx *ctx, const float *h_labels, float *h_scores, uint32_t first_tree,
+                     int32_t num_trees, qgbdt_model *model, void *stream);
+
+/* Counters of the work done by qgbdt_train since the context was created:
+ * kernel launches, histogram builds, and rows x features accumulated by them. */
+int qgbdt_get_counters(const qgbdt_ctx *ctx, int64_t *kernel_launches, int64_t *hist_builds,
+                       int64_t *hist_row_features);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QGBDT_H */

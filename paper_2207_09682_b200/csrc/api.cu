@@ -1,0 +1,423 @@
+// C ABI of libqgbdt: context management, argument checks, and the host-side sequencing of
+// the kernels.  No arithmetic of the method happens on the host except picking the leaf
+// with the largest stored gain and bookkeeping of leaf ranges.
+#include <cstdarg>
+#include <cstring>
+#include <new>
+
+#include "qgbdt_internal.cuh"
+
+int qg_fail(qgbdt_ctx *c, int code, const char *fmt, ...) {
+    if (c) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(c->err, sizeof(c->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+static_assert(sizeof(qgbdt_params) == 72 && sizeof(qgbdt_split) == 72 && sizeof(qgbdt_bin) == 8,
+              "ABI struct sizes are part of the interface");
+
+namespace {
+
+constexpr size_t PINNED_BYTES = 128 * 1024;
+constexpr size_t PINNED_SCALARS = 64 * 1024;  // offset of the small-scalar area
+constexpr int MAX_LEAVES = 4096;
+
+template <typename T>
+int dev_alloc(qgbdt_ctx *c, T **p, size_t count) {
+    void *q = nullptr;
+    cudaError_t e = cudaMalloc(&q, count * sizeof(T) > 0 ? count * sizeof(T) : 16);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return qg_fail(c, QGBDT_ERR_ALLOC, "cudaMalloc of %zu bytes failed: %s", count * sizeof(T), cudaGetErrorString(e));
+    }
+    *p = reinterpret_cast<T *>(q);
+    return QGBDT_OK;
+}
+
+template <typename T>
+void dev_free(T *&p) {
+    if (p) cudaFree(p);
+    p = nullptr;
+}
+
+void free_data(qgbdt_ctx *c) {
+    for (void *p : c->tile_allocs) cudaFree(p);
+    c->tile_allocs.clear();
+    c->tiles.clear();
+    dev_free(c->d_tiles);
+    dev_free(c->d_codes);
+    dev_free(c->d_idx);
+    dev_free(c->d_idx_tmp);
+    dev_free(c->d_part_counts);
+    dev_free(c->d_part_bits);
+    dev_free(c->d_feat_best);
+    dev_free(c->d_g);
+    dev_free(c->d_h);
+    dev_free(c->d_hist_pool);
+    c->loaded = false;
+    c->quantized = false;
+}
+
+int next_pow2(int v) {
+    int p = 1;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+// Feature tiles: full tiles of 128 features, then the remainder either padded to a power-of-two
+// number of words (cheap padding, or a matrix narrower than one tile: one row = one aligned
+// segment, which keeps row gathers sector-exact) or split into power-of-two pieces.
+void plan_tiles(int F, std::vector<TileDesc> &out) {
+    int f = 0;
+    auto add = [&](int nf, int words) {
+        TileDesc t;
+        t.data = nullptr;
+        t.f0 = f;
+        t.nf = nf;
+        int lw = 0;
+        while ((1 << lw) < words) ++lw;
+        t.logW = lw;
+        t.words_used = (nf + 3) / 4;
+        out.push_back(t);
+        f += nf;
+    };
+    while (F - f >= 128) add(128, 32);
+    while (F - f > 0) {
+        const int rem = F - f;
+        const int w = (rem + 3) / 4;
+        const int P = next_pow2(w);
+        if (F < 128 || (P - w) * 4 * 20 <= F) {
+            add(rem, P);
+        } else {
+            int q = P / 2;  // largest power of two below w
+            add(q * 4, q);
+        }
+    }
+}
+
+int check_loaded(qgbdt_ctx *c) {
+    if (!c) return QGBDT_ERR_ARG;
+    if (!c->loaded) return qg_fail(c, QGBDT_ERR_STATE, "no bin matrix loaded");
+    return QGBDT_OK;
+}
+
+void reset_leaf_state(qgbdt_ctx *c) {
+    c->n_leaves = 1;
+    c->leaf_off.assign(c->prm.num_leaves, 0);
+    c->leaf_n.assign(c->prm.num_leaves, 0);
+    c->leaf_n[0] = c->N;
+}
+
+void rec_to_split(const SplitRec &r, int64_t G, int64_t H, int64_t n_rows, bool const_h, qgbdt_split *out) {
+    memset(out, 0, sizeof(*out));
+    out->feature = -1;
+    out->bin = -1;
+    if (!r.valid) return;
+    out->valid = 1;
+    out->feature = r.feature;
+    out->bin = r.bin;
+    out->gain = r.gain;
+    out->gl = r.gl;
+    out->hl = r.hl;
+    out->gr = G - r.gl;
+    out->hr = H - r.hl;
+    // row estimate of the candidate (same integer formula as the scan kernel)
+    out->nl_est = const_h ? r.hl
+                          : (int64_t)(((unsigned long long)r.hl * (unsigned long long)n_rows + (unsigned long long)(H / 2)) /
+                                      (unsigned long long)H);
+    out->nr_est = n_rows - out->nl_est;
+}
+
+int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_features, int32_t n_bins,
+                int32_t layout, int64_t ld, cudaStream_t st) {
+    free_data(c);
+    c->N = n_rows;
+    c->F = n_features;
+    c->nb = n_bins;
+    c->code_bytes = c->prm.bits <= 4 ? 1 : 2;
+    plan_tiles(n_features, c->tiles);
+    int rc;
+    for (TileDesc &t : c->tiles) {
+        uint32_t *p = nullptr;
+        if ((rc = dev_alloc(c, &p, (size_t)n_rows << t.logW)) != QGBDT_OK) return rc;
+        c->tile_allocs.push_back(p);
+        t.data = p;
+    }
+    if ((rc = dev_alloc(c, &c->d_tiles, c->tiles.size())) != QGBDT_OK) return rc;
+    QG_CUDA(c, cudaMemcpyAsync(c->d_tiles, c->tiles.data(), sizeof(TileDesc) * c->tiles.size(),
+                               cudaMemcpyHostToDevice, st));
+    if ((rc = dev_alloc(c, &c->d_codes, (size_t)n_rows * 2 + 16)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_idx, (size_t)n_rows)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_idx_tmp, (size_t)n_rows)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_part_bits, ((size_t)n_rows + 2048) / 32 + 64)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_feat_best, (size_t)n_features)) != QGBDT_OK) return rc;
+    QG_CUDA(c, cudaMemsetAsync(c->d_state, 0, sizeof(DevState), st));
+    if ((rc = qg_relayout(c, d_bins, layout, ld, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_iota(c, st)) != QGBDT_OK) return rc;
+    DevState *hs = reinterpret_cast<DevState *>(reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS);
+    QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaStreamSynchronize(st));
+    if (hs->bad_value) {
+        free_data(c);
+        return qg_fail(c, QGBDT_ERR_VALUE, "a bin code is >= n_bins (%d)", n_bins);
+    }
+    c->loaded = true;
+    reset_leaf_state(c);
+    return QGBDT_OK;
+}
+
+int check_load_args(qgbdt_ctx *c, const uint8_t *bins, int64_t n_rows, int32_t n_features, int32_t n_bins,
+                    int32_t layout, int64_t ld) {
+    if (!c) return QGBDT_ERR_ARG;
+    if (!bins) return qg_fail(c, QGBDT_ERR_ARG, "bins is NULL");
+    if (n_rows < 1 || n_rows >= (1ll << 31)) return qg_fail(c, QGBDT_ERR_ARG, "n_rows must be in [1, 2^31)");
+    if (n_features < 1 || n_features > (1 << 20)) return qg_fail(c, QGBDT_ERR_ARG, "n_features out of range");
+    if (n_bins < 2 || n_bins > 256) return qg_fail(c, QGBDT_ERR_ARG, "n_bins must be in [2, 256]");
+    if (layout != 0 && layout != 1) return qg_fail(c, QGBDT_ERR_ARG, "layout must be 0 or 1");
+    if (ld < (layout == 0 ? (int64_t)n_features : n_rows)) return qg_fail(c, QGBDT_ERR_ARG, "ld too small");
+    const int64_t kg = qg_levels_g(c->prm.bits), kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
+    if (n_rows * kg > 2147483647ll || n_rows * kh > 4294967295ll)
+        return qg_fail(c, QGBDT_ERR_OVERFLOW, "n_rows * levels exceeds the 32+32-bit histogram word");
+    return QGBDT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int qgbdt_create(qgbdt_ctx **out, const qgbdt_params *p) {
+    if (!out || !p) return QGBDT_ERR_ARG;
+    *out = nullptr;
+    if (p->bits < 2 || p->bits > 8 || (p->objective != 0 && p->objective != 1) || p->num_leaves < 1 ||
+        p->num_leaves > MAX_LEAVES || p->min_data_in_leaf < 0 || !(p->learning_rate == p->learning_rate) ||
+        p->lambda_l2 < 0 || (p->hess_levels_mode != 0 && p->hess_levels_mode != 1) ||
+        (p->rounding != 0 && p->rounding != 1))
+        return QGBDT_ERR_ARG;
+    qgbdt_ctx *c = new (std::nothrow) qgbdt_ctx();
+    if (!c) return QGBDT_ERR_ALLOC;
+    c->prm = *p;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return QGBDT_ERR_CUDA;
+    }
+    c->sm_count = prop.multiProcessorCount;
+    c->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    const int L = p->num_leaves;
+    bool ok = cudaMalloc(reinterpret_cast<void **>(&c->d_state), sizeof(DevState)) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void **>(&c->d_split_out), sizeof(SplitRec) * 4) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_sums), sizeof(long long) * 2 * L) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_table), sizeof(uint32_t) * 2 * L) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_value), sizeof(float) * L) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_w), sizeof(double) * L) == cudaSuccess &&
+              cudaMallocHost(&c->h_pinned, PINNED_BYTES) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        qgbdt_destroy(c);
+        return QGBDT_ERR_ALLOC;
+    }
+    *out = c;
+    return QGBDT_OK;
+}
+
+int qgbdt_destroy(qgbdt_ctx *c) {
+    if (!c) return QGBDT_ERR_ARG;
+    free_data(c);
+    dev_free(c->d_state);
+    dev_free(c->d_split_out);
+    dev_free(c->d_leaf_sums);
+    dev_free(c->d_leaf_table);
+    dev_free(c->d_leaf_value);
+    dev_free(c->d_leaf_w);
+    if (c->h_pinned) cudaFreeHost(c->h_pinned);
+    delete c;
+    return QGBDT_OK;
+}
+
+const char *qgbdt_last_error(const qgbdt_ctx *c) { return c ? c->err : "null context"; }
+
+int qgbdt_load_binned(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_features, int32_t n_bins,
+                      int32_t layout, int64_t ld, void *stream) {
+    int rc = check_load_args(c, d_bins, n_rows, n_features, n_bins, layout, ld);
+    if (rc != QGBDT_OK) return rc;
+    return load_common(c, d_bins, n_rows, n_features, n_bins, layout, ld, (cudaStream_t)stream);
+}
+
+int qgbdt_load_binned_host(qgbdt_ctx *c, const uint8_t *h_bins, int64_t n_rows, int32_t n_features, int32_t n_bins,
+                           int32_t layout, int64_t ld, void *stream) {
+    int rc = check_load_args(c, h_bins, n_rows, n_features, n_bins, layout, ld);
+    if (rc != QGBDT_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bytes = (size_t)ld * (size_t)(layout == 0 ? n_rows : n_features);
+    uint8_t *tmp = nullptr;
+    if ((rc = dev_alloc(c, &tmp, bytes)) != QGBDT_OK) return rc;
+    cudaError_t e = cudaMemcpyAsync(tmp, h_bins, bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) {
+        cudaFree(tmp);
+        return qg_fail(c, QGBDT_ERR_CUDA, "copy of the bin matrix failed: %s", cudaGetErrorString(e));
+    }
+    rc = load_common(c, tmp, n_rows, n_features, n_bins, layout, ld, st);
+    cudaStreamSynchronize(st);
+    cudaFree(tmp);
+    return rc;
+}
+
+int qgbdt_compute_gradients(qgbdt_ctx *c, const float *d_scores, const float *d_labels, float *d_g, float *d_h,
+                            void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!d_scores || !d_labels || !d_g || (c->prm.objective == 0 && !d_h))
+        return qg_fail(c, QGBDT_ERR_ARG, "null pointer");
+    return qg_gradients(c, d_scores, d_labels, d_g, d_h, false, (cudaStream_t)stream);
+}
+
+int qgbdt_quantize_gradients(qgbdt_ctx *c, const float *d_g, const float *d_h, uint32_t tree, int8_t *d_gq,
+                             uint8_t *d_hq, double *g_scale, double *h_scale, int64_t *G_total, int64_t *H_total,
+                             void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!d_g) return qg_fail(c, QGBDT_ERR_ARG, "d_g is NULL");
+    cudaStream_t st = (cudaStream_t)stream;
+    c->quantized = false;
+    c->const_hess = d_h == nullptr;
+    if ((rc = qg_absmax(c, d_g, d_h, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_quantize(c, d_g, d_h, tree, d_gq, d_hq, st)) != QGBDT_OK) return rc;
+    DevState *hs = reinterpret_cast<DevState *>(reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS);
+    QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaStreamSynchronize(st));
+    if (hs->bad_value)
+        return qg_fail(c, QGBDT_ERR_VALUE, "gradient or hessian out of domain (non-finite, h < 0, or magnitude >= 256)");
+    memcpy(&c->gmax, &hs->gmax_bits, 4);
+    memcpy(&c->hmax, &hs->hmax_bits, 4);
+    if (c->const_hess) c->hmax = 1.0f;
+    c->quantized = true;
+    const int kg = qg_levels_g(c->prm.bits), kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
+    if (g_scale) *g_scale = (double)c->gmax / (double)kg;
+    if (h_scale) *h_scale = c->const_hess ? 1.0 : (double)c->hmax / (double)kh;
+    if (G_total) *G_total = hs->tot_g;
+    if (H_total) *H_total = hs->tot_h;
+    return QGBDT_OK;
+}
+
+int qgbdt_build_histograms(qgbdt_ctx *c, int32_t leaf, qgbdt_bin *d_hist, void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!c->quantized) return qg_fail(c, QGBDT_ERR_STATE, "quantize gradients before building histograms");
+    if (!d_hist) return qg_fail(c, QGBDT_ERR_ARG, "d_hist is NULL");
+    if (leaf < 0 || leaf >= c->n_leaves) return qg_fail(c, QGBDT_ERR_ARG, "leaf %d does not exist", leaf);
+    const bool root = c->n_leaves == 1 && c->idx_is_identity;
+    return qg_hist(c, root ? nullptr : c->d_idx, c->leaf_off[leaf], c->leaf_n[leaf],
+                   reinterpret_cast<unsigned long long *>(d_hist), (cudaStream_t)stream);
+}
+
+int qgbdt_build_histograms_rows(qgbdt_ctx *c, const uint32_t *d_rows, int64_t n, qgbdt_bin *d_hist, void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!c->quantized) return qg_fail(c, QGBDT_ERR_STATE, "quantize gradients before building histograms");
+    if (!d_hist || (n > 0 && !d_rows) || n < 0 || n >= (1ll << 32)) return qg_fail(c, QGBDT_ERR_ARG, "bad argument");
+    return qg_hist(c, d_rows, 0, n, reinterpret_cast<unsigned long long *>(d_hist), (cudaStream_t)stream);
+}
+
+int qgbdt_subtract_histograms(qgbdt_ctx *c, const qgbdt_bin *d_parent, const qgbdt_bin *d_small, qgbdt_bin *d_large,
+                              void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!d_parent || !d_small || !d_large) return qg_fail(c, QGBDT_ERR_ARG, "null pointer");
+    return qg_subtract(c, reinterpret_cast<const unsigned long long *>(d_parent),
+                       reinterpret_cast<const unsigned long long *>(d_small),
+                       reinterpret_cast<unsigned long long *>(d_large), (cudaStream_t)stream);
+}
+
+int qgbdt_find_best_split(qgbdt_ctx *c, const qgbdt_bin *d_hist, int64_t G, int64_t H, int64_t n_rows,
+                          qgbdt_split *h_out, void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!c->quantized) return qg_fail(c, QGBDT_ERR_STATE, "quantize gradients before searching splits");
+    if (!d_hist || !h_out || n_rows < 0 || H < 0) return qg_fail(c, QGBDT_ERR_ARG, "bad argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((rc = qg_find_split(c, reinterpret_cast<const unsigned long long *>(d_hist), G, H, n_rows, c->d_split_out,
+                            st)) != QGBDT_OK)
+        return rc;
+    SplitRec *hr = reinterpret_cast<SplitRec *>(reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS + 256);
+    QG_CUDA(c, cudaMemcpyAsync(hr, c->d_split_out, sizeof(SplitRec), cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaStreamSynchronize(st));
+    rec_to_split(*hr, G, H, n_rows, c->const_hess, h_out);
+    return QGBDT_OK;
+}
+
+int qgbdt_split_leaf(qgbdt_ctx *c, int32_t leaf, int32_t feature, int32_t bin, int32_t *right_leaf, int64_t *n_left,
+                     int64_t *n_right, void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (leaf < 0 || leaf >= c->n_leaves) return qg_fail(c, QGBDT_ERR_ARG, "leaf %d does not exist", leaf);
+    if (c->n_leaves >= c->prm.num_leaves) return qg_fail(c, QGBDT_ERR_STATE, "the tree already has num_leaves leaves");
+    if (feature < 0 || feature >= c->F || bin < 0 || bin >= c->nb) return qg_fail(c, QGBDT_ERR_ARG, "bad (feature, bin)");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t off = c->leaf_off[leaf], n = c->leaf_n[leaf];
+    int64_t nl = 0;
+    if (n > 0) {
+        if ((rc = qg_partition(c, off, n, feature, bin, st)) != QGBDT_OK) return rc;
+        DevState *hs = reinterpret_cast<DevState *>(reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS);
+        QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
+        QG_CUDA(c, cudaStreamSynchronize(st));
+        nl = hs->part_nl;
+    }
+    const int r = c->n_leaves++;
+    c->leaf_n[leaf] = nl;
+    c->leaf_off[r] = off + nl;
+    c->leaf_n[r] = n - nl;
+    if (right_leaf) *right_leaf = r;
+    if (n_left) *n_left = nl;
+    if (n_right) *n_right = n - nl;
+    return QGBDT_OK;
+}
+
+int qgbdt_get_leaf_rows(qgbdt_ctx *c, int32_t leaf, const uint32_t **d_rows, int64_t *n) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (leaf < 0 || leaf >= c->n_leaves || !d_rows || !n) return qg_fail(c, QGBDT_ERR_ARG, "bad argument");
+    *d_rows = c->d_idx + c->leaf_off[leaf];
+    *n = c->leaf_n[leaf];
+    return QGBDT_OK;
+}
+
+int qgbdt_reset_leaves(qgbdt_ctx *c, void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    reset_leaf_state(c);
+    return qg_iota(c, (cudaStream_t)stream);
+}
+
+int qgbdt_refit_leaves(qgbdt_ctx *c, const float *d_g, const float *d_h, double *h_w, float *h_value, void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!d_g) return qg_fail(c, QGBDT_ERR_ARG, "d_g is NULL");
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((rc = qg_refit(c, d_g, d_h, st)) != QGBDT_OK) return rc;
+    const int L = c->n_leaves;
+    char *base = reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS + 1024;
+    double *hw = reinterpret_cast<double *>(base);
+    float *hv = reinterpret_cast<float *>(base + sizeof(double) * MAX_LEAVES);
+    QG_CUDA(c, cudaMemcpyAsync(hw, c->d_leaf_w, sizeof(double) * L, cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaMemcpyAsync(hv, c->d_leaf_value, sizeof(float) * L, cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaStreamSynchronize(st));
+    if (h_w) memcpy(h_w, hw, sizeof(double) * L);
+    if (h_value) memcpy(h_value, hv, sizeof(float) * L);
+    return QGBDT_OK;
+}
+
+int qgbdt_get_counters(const qgbdt_ctx *c, int64_t *kernel_launches, int64_t *hist_builds, int64_t *hist_row_features) {
+    if (!c) return QGBDT_ERR_ARG;
+    if (kernel_launches) *kernel_launches = c->n_launches;
+    if (hist_builds) *hist_builds = c->n_hist_builds;
+    if (hist_row_features) *hist_row_features = c->n_hist_row_features;
+    return QGBDT_OK;
+}
+
+}  // extern "C"

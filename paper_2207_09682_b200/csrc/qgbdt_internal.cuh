@@ -1,0 +1,145 @@
+// Internal declarations shared by the CUDA sources of libqgbdt (never installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <cstdio>
+#include <vector>
+
+#include "qgbdt.h"
+
+// ---------------------------------------------------------------------------
+// Data layout in device memory
+//
+// Bin matrix: split by features into tiles of at most 128 features.  A tile stores
+// its features row-major, W = 2^logW 32-bit words per row (W in 1..32), four
+// consecutive features per word (feature 4a+k of the tile in byte k of word a).
+// Features beyond the tile's real width are stored as code 0 and never reported.
+// A warp that reads 32 consecutive words therefore reads R = 32/W whole rows; lane
+// l holds word a = l % W of row slot b = l / W.
+//
+// Packed gradient codes (Sec. 6.2 packs g and h of a sample the same way as the
+// bins): B <= 4: one byte per row, signed gradient in the high nibble, hessian in
+// the low nibble; B >= 5: two bytes, signed gradient in the high byte.
+//
+// Row lists: one uint32 array of N entries; leaf l owns [leaf_off[l], +leaf_n[l]).
+// ---------------------------------------------------------------------------
+
+struct TileDesc {
+    const uint32_t *data;  // [N][W] words
+    int32_t f0;            // first feature of the tile
+    int32_t nf;            // real features in the tile (<= 4 * W)
+    int32_t logW;          // log2 of words per row
+    int32_t words_used;    // ceil(nf / 4)
+};
+
+// Scalars produced and consumed on the device within one boosting iteration.
+struct DevState {
+    unsigned int gmax_bits;  // max |g| as float bits (non-negative floats order like uints)
+    unsigned int hmax_bits;  // max h as float bits
+    int bad_value;           // set when a gradient / hessian / bin code is out of domain
+    unsigned int part_nl;    // rows that went left in the last partition
+    long long tot_g, tot_h;  // integer sums over all rows of the last quantization
+};
+
+// Per-feature best candidate, then the leaf's best split (same fields as qgbdt_split).
+struct SplitRec {
+    double gain;
+    long long gl, hl;
+    int feature, bin;
+    int valid, pad;
+};
+
+struct qgbdt_ctx {
+    qgbdt_params prm;
+    int device = 0;
+    int sm_count = 0;
+    int max_smem_optin = 0;
+    // data
+    int64_t N = 0;
+    int F = 0, nb = 0;
+    bool loaded = false;
+    std::vector<TileDesc> tiles;
+    TileDesc *d_tiles = nullptr;
+    std::vector<void *> tile_allocs;
+    // quantized gradients
+    uint8_t *d_codes = nullptr;  // [N * code_bytes]
+    int code_bytes = 1;
+    bool quantized = false;
+    bool const_hess = false;
+    float gmax = 0.f, hmax = 0.f;
+    // leaves
+    int n_leaves = 1;
+    std::vector<int64_t> leaf_off, leaf_n;
+    uint32_t *d_idx = nullptr, *d_idx_tmp = nullptr;
+    bool idx_is_identity = false;
+    // scratch
+    DevState *d_state = nullptr;
+    uint32_t *d_part_counts = nullptr;  // per partition block: rows going left, then its exclusive scan
+    uint32_t *d_part_bits = nullptr;    // one predicate bit per row of the leaf being split
+    SplitRec *d_feat_best = nullptr;    // [F]
+    SplitRec *d_split_out = nullptr;    // [2]
+    long long *d_leaf_sums = nullptr;   // [L][2] fixed-point refit sums
+    uint32_t *d_leaf_table = nullptr;   // [L][2] (offset, leaf) sorted by offset, then [L] counts
+    float *d_leaf_value = nullptr;      // [L]
+    double *d_leaf_w = nullptr;         // [L]
+    void *h_pinned = nullptr;           // small pinned staging area
+    // training buffers (allocated on first qgbdt_train)
+    float *d_g = nullptr, *d_h = nullptr;
+    unsigned long long *d_hist_pool = nullptr;  // [L][F][nb]
+    // counters
+    int64_t n_launches = 0, n_hist_builds = 0, n_hist_row_features = 0;
+    char err[512] = {0};
+};
+
+int qg_fail(qgbdt_ctx *c, int code, const char *fmt, ...);
+
+#define QG_CUDA(c, expr)                                                                       \
+    do {                                                                                       \
+        cudaError_t e_ = (expr);                                                               \
+        if (e_ != cudaSuccess)                                                                 \
+            return qg_fail((c), QGBDT_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+#define QG_LAUNCH_CHECK(c)                                                                    \
+    do {                                                                                      \
+        (c)->n_launches++;                                                                    \
+        cudaError_t e_ = cudaGetLastError();                                                  \
+        if (e_ != cudaSuccess)                                                                \
+            return qg_fail((c), QGBDT_ERR_CUDA, "kernel launch failed at %s:%d: %s", __FILE__, \
+                           __LINE__, cudaGetErrorString(e_));                                  \
+    } while (0)
+
+static inline int qg_levels_g(int bits) { return (1 << (bits - 1)) - 1; }
+static inline int qg_levels_h(int bits, int mode) { return mode == 0 ? (1 << bits) - 2 : (1 << bits) - 1; }
+
+// ---- launchers implemented in the kernel files (all asynchronous on `st`) ----
+
+// load.cu
+int qg_relayout(qgbdt_ctx *c, const uint8_t *d_bins, int layout, int64_t ld, cudaStream_t st);
+int qg_iota(qgbdt_ctx *c, cudaStream_t st);
+
+// quantize.cu
+int qg_gradients(qgbdt_ctx *c, const float *d_scores, const float *d_labels, float *d_g, float *d_h,
+                 bool reduce_max, cudaStream_t st);
+int qg_absmax(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st);
+int qg_quantize(qgbdt_ctx *c, const float *d_g, const float *d_h, uint32_t tree, int8_t *d_gq,
+                uint8_t *d_hq, cudaStream_t st);
+
+// hist.cu
+int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsigned long long *d_hist,
+            cudaStream_t st);
+int qg_subtract(qgbdt_ctx *c, const unsigned long long *d_parent, const unsigned long long *d_small,
+                unsigned long long *d_large, cudaStream_t st);
+
+// split.cu
+int qg_find_split(qgbdt_ctx *c, const unsigned long long *d_hist, long long G, long long H, long long n_rows,
+                  SplitRec *d_out, cudaStream_t st);
+
+// partition.cu
+int qg_partition(qgbdt_ctx *c, int64_t off, int64_t n, int feature, int bin, cudaStream_t st);
+
+// refit.cu
+int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st);
+int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st);

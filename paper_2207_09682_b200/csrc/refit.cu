@@ -1,0 +1,158 @@
+// Eq. 3 with the original gradients (leaf-value refitting, Sec. 4.2) and the score update.
+// Sums are taken in 2^-30 fixed point: each term is rounded once, the 64-bit integer sum is
+// exact, so the result does not depend on the order in which rows are added.
+#include "qgbdt_internal.cuh"
+
+namespace {
+
+constexpr int REFIT_THREADS = 256;
+constexpr int REFIT_ITEMS = 16;
+constexpr int REFIT_BLOCK = REFIT_THREADS * REFIT_ITEMS;
+constexpr int REFIT_LOCAL = 64;  // leaf slots a block can accumulate in shared memory
+
+// Slot (index into the offset-sorted leaf table) of position p: last slot with offs[s] <= p.
+__device__ inline int slot_of(const uint32_t *offs, int n_leaves, uint32_t p) {
+    int lo = 0, hi = n_leaves - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (offs[mid] <= p) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__device__ inline long long to_fixed(float v) { return __double2ll_rn(__dmul_rn((double)v, 1073741824.0)); }
+
+// table: [n_leaves] offsets ascending, then [n_leaves] leaf ids.  sums: [n_leaves][2] by slot.
+__global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__restrict__ idx, uint32_t n,
+                                                              const uint32_t *__restrict__ table, int n_leaves,
+                                                              const float *__restrict__ g, const float *__restrict__ h,
+                                                              long long *__restrict__ sums) {
+    extern __shared__ uint32_t offs[];  // n_leaves offsets
+    __shared__ unsigned long long acc[REFIT_LOCAL][2];
+    for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) offs[i] = table[i];
+    for (int i = threadIdx.x; i < REFIT_LOCAL * 2; i += REFIT_THREADS) (&acc[0][0])[i] = 0ull;
+    __syncthreads();
+    const uint32_t p0 = blockIdx.x * REFIT_BLOCK;
+    const uint32_t p1 = min(n, p0 + REFIT_BLOCK);
+    const int s_lo = slot_of(offs, n_leaves, p0);
+    const int lane = threadIdx.x & 31;
+#pragma unroll 4
+    for (int j = 0; j < REFIT_ITEMS; ++j) {
+        const uint32_t p = p0 + j * REFIT_THREADS + threadIdx.x;
+        const bool ok = p < p1;
+        int s = -1;
+        long long gf = 0, hf = 0;
+        if (ok) {
+            s = slot_of(offs, n_leaves, p);
+            const uint32_t row = idx[p];
+            gf = to_fixed(g[row]);
+            hf = h ? to_fixed(h[row]) : 1073741824LL;
+        }
+        const int s0 = __shfl_sync(0xffffffffu, s, 0);
+        if (__all_sync(0xffffffffu, s == s0)) {
+            if (s0 < 0) continue;  // whole warp past the end
+            for (int o = 16; o > 0; o >>= 1) {
+                gf += __shfl_xor_sync(0xffffffffu, gf, o);
+                hf += __shfl_xor_sync(0xffffffffu, hf, o);
+            }
+            if (lane == 0) {
+                if (s0 - s_lo < REFIT_LOCAL) {
+                    atomicAdd(&acc[s0 - s_lo][0], (unsigned long long)gf);
+                    atomicAdd(&acc[s0 - s_lo][1], (unsigned long long)hf);
+                } else {
+                    atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * s0]), (unsigned long long)gf);
+                    atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * s0 + 1]), (unsigned long long)hf);
+                }
+            }
+        } else if (ok) {
+            if (s - s_lo < REFIT_LOCAL) {
+                atomicAdd(&acc[s - s_lo][0], (unsigned long long)gf);
+                atomicAdd(&acc[s - s_lo][1], (unsigned long long)hf);
+            } else {
+                atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * s]), (unsigned long long)gf);
+                atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * s + 1]), (unsigned long long)hf);
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < REFIT_LOCAL; i += REFIT_THREADS) {
+        if (s_lo + i < n_leaves && (acc[i][0] | acc[i][1]) != 0ull) {
+            atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * (s_lo + i)]), acc[i][0]);
+            atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * (s_lo + i) + 1]), acc[i][1]);
+        }
+    }
+}
+
+// w = -sum g / (sum h + lambda); output (float)(learning_rate * w); written by leaf id.
+__global__ void k_leaf_values(const long long *__restrict__ sums, const uint32_t *__restrict__ table, int n_leaves,
+                              double lambda, double lr, double *__restrict__ w_out, float *__restrict__ v_out) {
+    for (int s = blockIdx.x * blockDim.x + threadIdx.x; s < n_leaves; s += gridDim.x * blockDim.x) {
+        const int leaf = (int)table[n_leaves + s];
+        const double den = __dadd_rn((double)sums[2 * s + 1], __dmul_rn(lambda, 1073741824.0));
+        const double w = den > 0.0 ? __ddiv_rn(-(double)sums[2 * s], den) : 0.0;
+        w_out[leaf] = w;
+        v_out[leaf] = __double2float_rn(__dmul_rn(lr, w));
+    }
+}
+
+__global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *__restrict__ idx, uint32_t n,
+                                                                const uint32_t *__restrict__ table, int n_leaves,
+                                                                const float *__restrict__ values,
+                                                                float *__restrict__ scores) {
+    extern __shared__ uint32_t offs[];
+    for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) offs[i] = table[i];
+    __syncthreads();
+    for (uint32_t p = blockIdx.x * REFIT_THREADS + threadIdx.x; p < n; p += gridDim.x * REFIT_THREADS) {
+        const int s = slot_of(offs, n_leaves, p);
+        const uint32_t row = idx[p];
+        scores[row] = __fadd_rn(scores[row], values[table[n_leaves + s]]);
+    }
+}
+
+// Writes the offset-sorted leaf table into pinned memory and queues its copy to the device.
+int upload_table(qgbdt_ctx *c, cudaStream_t st) {
+    const int L = c->n_leaves;
+    uint32_t *tab = reinterpret_cast<uint32_t *>(c->h_pinned);
+    std::vector<int> order(L);
+    for (int i = 0; i < L; ++i) order[i] = i;
+    for (int i = 1; i < L; ++i) {  // insertion sort by offset (lists are short and nearly sorted)
+        const int v = order[i];
+        int j = i - 1;
+        while (j >= 0 && c->leaf_off[order[j]] > c->leaf_off[v]) { order[j + 1] = order[j]; --j; }
+        order[j + 1] = v;
+    }
+    for (int s = 0; s < L; ++s) {
+        tab[s] = (uint32_t)c->leaf_off[order[s]];
+        tab[L + s] = (uint32_t)order[s];
+    }
+    QG_CUDA(c, cudaMemcpyAsync(c->d_leaf_table, tab, sizeof(uint32_t) * 2 * L, cudaMemcpyHostToDevice, st));
+    return QGBDT_OK;
+}
+
+}  // namespace
+
+int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st) {
+    const int L = c->n_leaves;
+    int rc = upload_table(c, st);
+    if (rc != QGBDT_OK) return rc;
+    QG_CUDA(c, cudaMemsetAsync(c->d_leaf_sums, 0, sizeof(long long) * 2 * L, st));
+    const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
+    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, (uint32_t)c->N, c->d_leaf_table, L,
+                                                                     d_g, d_h, c->d_leaf_sums);
+    QG_LAUNCH_CHECK(c);
+    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, c->d_leaf_table, L, c->prm.lambda_l2,
+                                                   c->prm.learning_rate, c->d_leaf_w, c->d_leaf_value);
+    QG_LAUNCH_CHECK(c);
+    return QGBDT_OK;
+}
+
+// Requires the leaf table uploaded by the preceding qg_refit on the same stream.
+int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st) {
+    const int L = c->n_leaves;
+    unsigned blocks = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
+    if (blocks > (unsigned)c->sm_count * 16) blocks = (unsigned)c->sm_count * 16;
+    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, (uint32_t)c->N, c->d_leaf_table, L,
+                                                                       c->d_leaf_value, d_scores);
+    QG_LAUNCH_CHECK(c);
+    return QGBDT_OK;
+}

@@ -92,7 +92,7 @@ class _DeviceView:
     """CUDA array interface over borrowed device memory holding n 32-bit words."""
 
     def __init__(self, ptr: int, n: int):
-        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (ptr, True), "version": 2}
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (ptr, False), "version": 2}
 
 
 class HostModel:

@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized-GBDT hot path on B200.
+
+A step is one boosting iteration (one tree) of the whole path -- gradients, quantization,
+leaf-wise growth with integer histograms, subtraction, split search, partition, refit, score
+update -- on a synthetic workload shaped like the paper's largest dense dataset
+(10.5 M rows x 28 features, 255 bins, squared loss, 4-bit gradients, 255 leaves).
+
+Metric: histogram row-features per second = rows x features that Algorithm 1 has to visit
+(the root plus the smaller child of every split) divided by the time of the WHOLE step.
+ms_per_step is ms per tree.  `roofline` is the histogram kernel alone: algorithmic bytes of
+all its launches inside the timed region over their summed CUDA-event durations, against the
+measured HBM copy bandwidth.  `cpu_baseline` is the CPU oracle on a bounded row sample.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOAD_ROWS = {"large": 10_500_000, "tall": 1_000_000, "tiny": 50_000, "wide": 400_000}
+CPU_SAMPLE_ROWS = {"large": 3_000_000, "tall": 1_000_000, "tiny": 50_000, "wide": 20_000}
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self) -> dict:
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for name, v in zip(names, r[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                pass
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def needed_hist_rows(tree: dict, n_rows: int) -> int:
+    """Rows Algorithm 1 must visit for one tree: the root plus the smaller child of every split."""
+    nl = tree["num_leaves"]
+    if nl <= 1:
+        return n_rows
+    count = {}
+
+    def size(c):
+        if c < 0:
+            return int(tree["leaf_count"][~c])
+        if c not in count:
+            count[c] = size(int(tree["left"][c])) + size(int(tree["right"][c]))
+        return count[c]
+
+    total = n_rows
+    for i in range(nl - 1):
+        total += min(size(int(tree["left"][i])), size(int(tree["right"][i])))
+    return total
+
+
+def oracle_leg(wl_name: str, rows: int, steps: int, warmup: int, data=None, y=None, n_bins=None, params=None) -> dict:
+    """Times the CPU oracle (as it stands, one thread) on a bounded row sample of the workload."""
+    import numpy as np
+    import oracle
+    from paper_2207_09682_b200 import synth
+    if data is None:
+        wl = synth.CONFIGS[wl_name](device="cpu", rows=rows)
+        data, y, n_bins, params = wl.bins.numpy(), wl.labels.numpy(), wl.n_bins, wl.params
+    prm = oracle.make_params(**dict(params, num_trees=1, seed=1))
+    scores = np.zeros(rows, np.float32)
+    rf, secs = 0, 0.0
+    for k in range(warmup + steps):
+        t0 = time.perf_counter()
+        t = oracle.train_tree(data, n_bins, y, scores, prm, k)
+        dt = time.perf_counter() - t0
+        if k >= warmup:
+            tree = dict(num_leaves=t.num_leaves, left=t.left, right=t.right, leaf_count=t.leaf_count)
+            rf += needed_hist_rows(tree, rows) * data.shape[1]
+            secs += dt
+    return {"value": rf / secs, "unit": "row-features/s", "cores": 1, "kind": "oracle",
+            "sample": "%d trees of %d leaves on the first-generated %d rows x %d features of workload '%s'"
+                      % (steps, prm.num_leaves, rows, data.shape[1], wl_name),
+            "ms_per_tree": 1e3 * secs / steps}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows = min(args.rows or WORKLOAD_ROWS[args.workload], CPU_SAMPLE_ROWS[args.workload])
+    steps, warmup = args.steps, args.warmup
+    leg = oracle_leg(args.workload, rows, steps, warmup)
+    line = {"impl": "reference", "metric": "hist_row_features_per_s", "value": leg["value"], "unit": "row-features/s",
+            "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "ms_per_step": leg["ms_per_tree"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": args.workload, "rows": rows, "note": "CPU oracle on a bounded row sample"},
+            "cpu_baseline": {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": leg["value"], "unit": "row-features/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes, reps=20):
+    """Stand-alone root and 50%-subset histogram builds, L2 flushed between repetitions."""
+    import numpy as np
+    hist = ctx.new_hist()
+    rows = synth.subset_rows(n, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    out = {}
+    for name, r in (("root", None), ("subset50", rows)):
+        ts = []
+        for i in range(reps + 3):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            if r is None:
+                ctx.build_histograms(0, hist)
+            else:
+                ctx.build_histograms_rows(r, hist)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1))
+        nr = n if r is None else int(r.numel())
+        ms = float(np.median(ts))
+        nbytes = nr * (features + code_bytes + (0 if r is None else 4)) + features * n_bins * 8
+        out[name] = {"rows": nr, "us": 1e3 * ms, "row_features_per_s": nr * features / (ms * 1e-3),
+                     "gbs": nbytes / (ms * 1e6), "note": "includes the memset of the output histogram"}
+    return out
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2207_09682_b200 import binding, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    rows = args.rows or WORKLOAD_ROWS[args.workload]
+    wl = synth.CONFIGS[args.workload](device="cuda", rows=rows, seed=synth.MASTER_SEED + 100 + rank)
+    n, features = wl.bins.shape
+    n_bins = wl.n_bins
+    kw = dict(wl.params, num_trees=1, seed=1 + rank)
+    ctx = binding.Context(binding.make_params(**kw))
+    ctx.load_binned(wl.bins, wl.n_bins)
+    scores = torch.zeros(n, device="cuda")
+    K, W = args.steps, args.warmup
+
+    ctx.train(wl.labels, scores, 0, W)                       # warm-up trees 0 .. W-1
+    torch.cuda.synchronize()
+    c0 = ctx.get_counters()
+    ctx.profile_histograms(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clocks:
+        e0.record()
+        model = ctx.train(wl.labels, scores, W, K)           # the timed K steps
+        e1.record()
+        torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    prof = ctx.get_histogram_profile()
+    ctx.profile_histograms(False)
+    c1 = ctx.get_counters()
+    rf = c1["hist_row_features"] - c0["hist_row_features"]
+    launches = c1["kernel_launches"] - c0["kernel_launches"]
+    leaves = [int(x) for x in model.num_leaves]
+
+    t = torch.tensor([ms, float(rf), float(launches)], dtype=torch.float64, device="cuda")
+    if dist:
+        tmax = t.clone()
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        ms, rf, launches = float(tmax[0]), float(t[1]), float(t[2])
+    if rank != 0:
+        dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    achieved = prof["total_bytes"] / (prof["total_ms"] * 1e6) if prof["total_ms"] > 0 else 0.0
+    code_bytes = 1 if kw["bits"] <= 4 else 2
+    line = {
+        "metric": "hist_row_features_per_s", "value": rf / (ms * 1e-3), "unit": "row-features/s",
+        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": args.workload, "rows": n, "features": features, "bins": wl.n_bins,
+                   "bits": kw["bits"], "num_leaves": kw["num_leaves"], "objective": kw["objective"],
+                   "l2_policy": "inputs larger than L2 (bin matrix %d MB)" % (n * ((features + 3) // 4 * 4) >> 20),
+                   "multi_gpu": "replicas only: one independent shard per GPU, no collective",
+                   "leaves_per_tree": [min(leaves), max(leaves)]},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_kind": peak_kind, "kernel": "k_hist",
+                     "launches": prof["builds"], "total_ms": prof["total_ms"],
+                     "share_of_step": prof["total_ms"] / ms if ms else None},
+        "clocks": clocks.summary(),
+    }
+
+    # stand-alone histogram builds on the same data (root leaf and a 50 % subset)
+    g = torch.empty(n, device="cuda")
+    h = torch.empty(n, device="cuda") if kw["objective"] == 0 else None
+    ctx.reset_leaves()
+    ctx.compute_gradients(scores, wl.labels, g, h)
+    ctx.quantize_gradients(g, h, tree=W + K)
+    builds = time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes)
+    for b in builds.values():
+        b["frac"] = b["gbs"] / peak
+    line["hist_builds"] = builds
+
+    # end to end through the C ABI with host buffers: every step copies the bin matrix, labels and
+    # scores from pinned host memory and reads the scores back
+    host_data = None
+    if not args.no_e2e:
+        hb = wl.bins.cpu().pin_memory()
+        hl = wl.labels.cpu().pin_memory()
+        host_data = (hb.numpy(), hl.numpy())
+        hs = torch.zeros(n).pin_memory()
+        ctx.close()
+        del wl, scores
+        torch.cuda.empty_cache()
+        ctx2 = binding.Context(binding.make_params(**kw))
+        e_steps = max(1, min(K, 5))
+        rf2, t_e2e = 0, 0.0
+        for k in range(1 + e_steps):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            ctx2.load_binned(hb, n_bins)
+            m2 = ctx2.train(hl, hs, k, 1)
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            if k >= 1:
+                t_e2e += dt
+                rf2 += needed_hist_rows(m2.tree(0), n) * features
+        line["e2e"] = {"value": rf2 / t_e2e, "unit": "row-features/s", "h2d_bytes_per_step": int(hb.numel() + 8 * n),
+                       "d2h_bytes_per_step": int(4 * n), "steps": e_steps, "ms_per_step": 1e3 * t_e2e / e_steps}
+        ctx2.close()
+
+    if not args.no_cpu_baseline:
+        if host_data is None:
+            leg = oracle_leg(args.workload, min(n, CPU_SAMPLE_ROWS[args.workload]), 1, 0)
+        else:   # the very arrays the GPU path was timed on, all rows, one tree
+            leg = oracle_leg(args.workload, n, 1, 0, host_data[0], host_data[1], n_bins, kw)
+        line["cpu_baseline"] = {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=sorted(WORKLOAD_ROWS))
+    ap.add_argument("--rows", type=int, default=0, help="override the workload's row count (profiling captures)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

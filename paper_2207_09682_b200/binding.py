@@ -21,7 +21,7 @@ EXPORTS = [
     "qgbdt_compute_gradients", "qgbdt_quantize_gradients", "qgbdt_build_histograms",
     "qgbdt_build_histograms_rows", "qgbdt_subtract_histograms", "qgbdt_find_best_split", "qgbdt_split_leaf",
     "qgbdt_get_leaf_rows", "qgbdt_reset_leaves", "qgbdt_refit_leaves", "qgbdt_train", "qgbdt_train_host",
-    "qgbdt_get_counters",
+    "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile",
 ]
 
 
@@ -247,6 +247,20 @@ class Context:
         a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
         self._check(self.lib.qgbdt_get_counters(self.h, C.byref(a), C.byref(b), C.byref(c)))
         return dict(kernel_launches=a.value, hist_builds=b.value, hist_row_features=c.value)
+
+
+def _profile_histograms(self, enable: bool):
+    self._check(self.lib.qgbdt_profile_histograms(self.h, C.c_int32(1 if enable else 0)))
+
+
+def _get_histogram_profile(self) -> dict:
+    ms, nbytes, builds = C.c_double(), C.c_int64(), C.c_int64()
+    self._check(self.lib.qgbdt_get_histogram_profile(self.h, C.byref(ms), C.byref(nbytes), C.byref(builds)))
+    return dict(total_ms=ms.value, total_bytes=nbytes.value, builds=builds.value)
+
+
+Context.profile_histograms = _profile_histograms
+Context.get_histogram_profile = _get_histogram_profile
 
 
 def unpack_hist(hist: torch.Tensor) -> tuple[np.ndarray, np.ndarray]:

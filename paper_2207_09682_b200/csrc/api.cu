@@ -236,6 +236,7 @@ int qgbdt_destroy(qgbdt_ctx *c) {
     dev_free(c->d_leaf_value);
     dev_free(c->d_leaf_w);
     if (c->h_pinned) cudaFreeHost(c->h_pinned);
+    for (cudaEvent_t e : c->hist_events) cudaEventDestroy(e);
     delete c;
     return QGBDT_OK;
 }
@@ -417,6 +418,33 @@ int qgbdt_get_counters(const qgbdt_ctx *c, int64_t *kernel_launches, int64_t *hi
     if (kernel_launches) *kernel_launches = c->n_launches;
     if (hist_builds) *hist_builds = c->n_hist_builds;
     if (hist_row_features) *hist_row_features = c->n_hist_row_features;
+    return QGBDT_OK;
+}
+
+int qgbdt_profile_histograms(qgbdt_ctx *c, int32_t enable) {
+    if (!c) return QGBDT_ERR_ARG;
+    c->profile_hist = enable != 0;
+    c->hist_events_used = 0;
+    c->hist_prof_bytes = 0;
+    c->hist_prof_launches = 0;
+    return QGBDT_OK;
+}
+
+int qgbdt_get_histogram_profile(qgbdt_ctx *c, double *total_ms, int64_t *total_bytes, int64_t *builds) {
+    if (!c) return QGBDT_ERR_ARG;
+    double ms = 0.0;
+    for (size_t i = 0; i + 1 < c->hist_events_used; i += 2) {
+        QG_CUDA(c, cudaEventSynchronize(c->hist_events[i + 1]));
+        float t = 0.f;
+        QG_CUDA(c, cudaEventElapsedTime(&t, c->hist_events[i], c->hist_events[i + 1]));
+        ms += t;
+    }
+    if (total_ms) *total_ms = ms;
+    if (total_bytes) *total_bytes = c->hist_prof_bytes;
+    if (builds) *builds = c->hist_prof_launches;
+    c->hist_events_used = 0;
+    c->hist_prof_bytes = 0;
+    c->hist_prof_launches = 0;
     return QGBDT_OK;
 }
 

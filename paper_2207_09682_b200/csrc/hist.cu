@@ -246,16 +246,40 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
     const unsigned long long units = (unsigned long long)((n + ROW_BLOCK - 1) / ROW_BLOCK) * a.n_tiles;
     unsigned grid = (unsigned)(units < (unsigned long long)c->sm_count ? units : (unsigned long long)c->sm_count);
 
-    if (!wide) {
-        return launch_hist<1, false, 4>(c, a, grid, st);
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (c->profile_hist) {
+        if (c->hist_events_used + 2 > c->hist_events.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                QG_CUDA(c, cudaEventCreate(&e));
+                c->hist_events.push_back(e);
+            }
+        }
+        ev0 = c->hist_events[c->hist_events_used++];
+        ev1 = c->hist_events[c->hist_events_used++];
+        // algorithmic bytes of this build: bin codes + packed gradient code (+ row index) per row, histogram out
+        c->hist_prof_bytes += n * (c->F + c->code_bytes + (d_rows ? 4 : 0)) + (int64_t)hist_bytes;
+        c->hist_prof_launches++;
+        QG_CUDA(c, cudaEventRecord(ev0, st));
     }
-    // 32+32 local bins: two words per bin; all four bytes fit only for small bin counts
-    const size_t full = (size_t)4 * c->nb * 32 * 4 * 2;
-    if (full <= (size_t)c->max_smem_optin) return launch_hist<2, true, 4>(c, a, grid, st);
-    int rc = launch_hist<2, true, 2>(c, a, grid, st);
-    if (rc != QGBDT_OK) return rc;
-    a.k0 = 2;
-    return launch_hist<2, true, 2>(c, a, grid, st);
+    int rc;
+    if (!wide) {
+        rc = launch_hist<1, false, 4>(c, a, grid, st);
+    } else {
+        // 32+32 local bins: two words per bin; all four bytes fit only for small bin counts
+        const size_t full = (size_t)4 * c->nb * 32 * 4 * 2;
+        if (full <= (size_t)c->max_smem_optin) {
+            rc = launch_hist<2, true, 4>(c, a, grid, st);
+        } else {
+            rc = launch_hist<2, true, 2>(c, a, grid, st);
+            if (rc == QGBDT_OK) {
+                a.k0 = 2;
+                rc = launch_hist<2, true, 2>(c, a, grid, st);
+            }
+        }
+    }
+    if (rc == QGBDT_OK && ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
+    return rc;
 }
 
 int qg_subtract(qgbdt_ctx *c, const unsigned long long *d_parent, const unsigned long long *d_small,

@@ -90,6 +90,11 @@ struct qgbdt_ctx {
     unsigned long long *d_hist_pool = nullptr;  // [L][F][nb]
     // counters
     int64_t n_launches = 0, n_hist_builds = 0, n_hist_row_features = 0;
+    // optional per-launch timing of the histogram kernel (event pairs on the launching stream)
+    bool profile_hist = false;
+    std::vector<cudaEvent_t> hist_events;  // start/stop pairs, reused
+    size_t hist_events_used = 0;
+    int64_t hist_prof_bytes = 0, hist_prof_launches = 0;
     char err[512] = {0};
 };
 

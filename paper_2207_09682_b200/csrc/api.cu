@@ -49,6 +49,8 @@ void free_data(qgbdt_ctx *c) {
     c->tile_allocs.clear();
     c->tiles.clear();
     dev_free(c->d_tiles);
+    dev_free(c->d_cta_map);
+    dev_free(c->d_partial);
     dev_free(c->d_codes);
     dev_free(c->d_idx);
     dev_free(c->d_idx_tmp);
@@ -99,6 +101,37 @@ void plan_tiles(int F, std::vector<TileDesc> &out) {
     }
 }
 
+// Histogram plan: CTAs are shared out among the tiles in proportion to their width in words
+// (the cost of a row is one warp instruction slot per 32 words); with more tiles than SMs every
+// tile gets one CTA.  Fills parts / cta0 of the tiles and returns the CTA -> (tile, part) map.
+void plan_hist_ctas(int sm_count, std::vector<TileDesc> &tiles, std::vector<int2> &map, int &max_parts) {
+    const int T = (int)tiles.size();
+    long long total_w = 0;
+    for (const TileDesc &t : tiles) total_w += 1 << t.logW;
+    int used = 0;
+    for (TileDesc &t : tiles) {
+        long long p = T >= sm_count ? 1 : (long long)sm_count * (1 << t.logW) / total_w;
+        t.parts = (int)(p < 1 ? 1 : p);
+        used += t.parts;
+    }
+    // hand the CTAs left over by the rounding to the tiles with the most words per part
+    while (T < sm_count && used < sm_count) {
+        int best = 0;
+        for (int i = 1; i < T; ++i)
+            if ((long long)(1 << tiles[i].logW) * tiles[best].parts > (long long)(1 << tiles[best].logW) * tiles[i].parts)
+                best = i;
+        tiles[best].parts++;
+        used++;
+    }
+    map.clear();
+    max_parts = 1;
+    for (int i = 0; i < T; ++i) {
+        tiles[i].cta0 = (int)map.size();
+        for (int p = 0; p < tiles[i].parts; ++p) map.push_back(make_int2(i, p));
+        if (tiles[i].parts > max_parts) max_parts = tiles[i].parts;
+    }
+}
+
 int check_loaded(qgbdt_ctx *c) {
     if (!c) return QGBDT_ERR_ARG;
     if (!c->loaded) return qg_fail(c, QGBDT_ERR_STATE, "no bin matrix loaded");
@@ -138,8 +171,11 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     c->N = n_rows;
     c->F = n_features;
     c->nb = n_bins;
-    c->code_bytes = c->prm.bits <= 4 ? 1 : 2;
+    c->code_bytes = 2;
     plan_tiles(n_features, c->tiles);
+    std::vector<int2> cta_map;
+    plan_hist_ctas(c->sm_count, c->tiles, cta_map, c->max_parts);
+    c->hist_grid = (int)cta_map.size();
     int rc;
     for (TileDesc &t : c->tiles) {
         uint32_t *p = nullptr;
@@ -150,7 +186,13 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     if ((rc = dev_alloc(c, &c->d_tiles, c->tiles.size())) != QGBDT_OK) return rc;
     QG_CUDA(c, cudaMemcpyAsync(c->d_tiles, c->tiles.data(), sizeof(TileDesc) * c->tiles.size(),
                                cudaMemcpyHostToDevice, st));
-    if ((rc = dev_alloc(c, &c->d_codes, (size_t)n_rows * 2 + 16)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_cta_map, cta_map.size())) != QGBDT_OK) return rc;
+    // pageable source: the copy has left the host buffer when the call returns
+    QG_CUDA(c, cudaMemcpyAsync(c->d_cta_map, cta_map.data(), sizeof(int2) * cta_map.size(), cudaMemcpyHostToDevice, st));
+    if (c->max_parts > 1 &&
+        (rc = dev_alloc(c, &c->d_partial, (size_t)c->hist_grid * 4 * n_bins * 32)) != QGBDT_OK)
+        return rc;
+    if ((rc = dev_alloc(c, &c->d_codes, ((size_t)n_rows + 15) / 16 * 16 * 2 + 16)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx, (size_t)n_rows)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx_tmp, (size_t)n_rows)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8)) != QGBDT_OK) return rc;
@@ -367,6 +409,7 @@ int qgbdt_split_leaf(qgbdt_ctx *c, int32_t leaf, int32_t feature, int32_t bin, i
         DevState *hs = reinterpret_cast<DevState *>(reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS);
         QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
         QG_CUDA(c, cudaStreamSynchronize(st));
+        if (hs->kernel_error) return qg_fail(c, QGBDT_ERR_CUDA, "a histogram kernel refused its launch configuration");
         nl = hs->part_nl;
     }
     const int r = c->n_leaves++;

@@ -1,195 +1,383 @@
 // Algorithm 1 with integer gradients: per-CTA shared-memory histograms with packed
 // gradient+hessian bins (Sec. 6.1 hierarchical buffers, Sec. 6.2 packing), merged into the
-// leaf's 32+32-bit histogram with 64-bit global atomics; and histogram subtraction.
+// leaf's 32+32-bit histogram in two stages; and histogram subtraction.
 //
-// Shared-memory layout (the part that differs from the paper's V100 design): the local
-// histogram is indexed [byte k of the word][bin][lane].  Lane l of a warp always adds into
-// column l, i.e. bank l, so the 32 shared atomics of one warp instruction never collide,
-// whatever the bin codes are (uniform or 90 % in one bin).  A lane owns word a = l % W of
-// row slot b = l / W; column l of slab k therefore holds feature 4a+k of the tile, and the
-// R = 32/W row slots are R private replicas that the flush adds up.
+// What differs from the paper's V100 design (one 16+16 local histogram per CUDA block, merged
+// with atomics):
 //
-// Local bin width: B <= 4 uses one 32-bit word per bin, gradient sum in the high 16 bits
-// (signed), hessian sum in the low 16 bits; the CTA flushes before any lane slot has added
-// more rows than fit (flush_rows).  B >= 5 uses two 32-bit words per bin (32+32 local).
+//  * Bank-private columns.  The local histogram is indexed [bin][byte k of the word][lane].
+//    Lane l of a warp always adds into column l, i.e. shared-memory bank l, so the 32 atomics
+//    of one warp instruction never collide, whatever the bin codes are (uniform, or 90 % in
+//    one bin).  A lane owns word a = l % W of row slot l / W; the R = 32/W row slots are R
+//    private replicas that the flush adds up.  Measured: one conflict-free warp atomic per
+//    clock per SM.
+//  * One-instruction addressing.  The local histogram starts on a 64 KB boundary of the shared
+//    window and a bin is 256 bytes apart from the next, so the address of (bin, lane) is the
+//    lane's base address with its second byte replaced by the bin code: a single byte permute
+//    of the loaded word yields the atomic's address, and the per-row increment (gradient << 16
+//    + hessian) is one more permute of the row's 16-bit code.
+//  * Rolling prefetch.  Every lane keeps U units of four rows in flight in registers and
+//    refills a slot as soon as it has been consumed.
+//  * Two-stage merge.  A CTA stores its partial histogram with plain coalesced stores; a small
+//    kernel sums the partials of each feature tile.  (64-bit global atomics from 148 CTAs on
+//    the same 7 k bins cost about as much as half of the whole build.)
+//
+// Local bin width: B <= 5 uses one 32-bit word per bin, gradient sum in the high 16 bits
+// (signed), hessian sum in the low 16 bits; the CTA flushes before any column can have added
+// more rows than fit.  B >= 6 uses one 64-bit word per bin (32+32) and two passes over the
+// rows, each pass taking two of the four bytes of a word.
 #include "qgbdt_internal.cuh"
 
 namespace {
 
 constexpr int HIST_THREADS = 1024;
 constexpr int HIST_WARPS = HIST_THREADS / 32;
-constexpr int ROW_BLOCK = 2048;  // rows per work unit
-constexpr int UNROLL = 8;
+constexpr int HIST_SMEM = 192 * 1024;     // 128 KB histogram on a 64 KB boundary + the room below it
+constexpr uint32_t MIN_ROWS_PER_CTA = 4096;
+constexpr int U_ROOT = 3;                 // units in flight per lane, contiguous rows
+constexpr int U_LIST = 2;                 // units in flight per lane, row list (plus as many index units)
 
 struct HistArgs {
     const TileDesc *tiles;
-    int n_tiles;
-    const uint8_t *codes;
-    const uint32_t *rows;  // row list, or nullptr: rows off .. off+n-1
-    uint32_t off, n;
+    const int2 *cta_map;           // CTA -> (tile, part)
+    const uint16_t *codes;         // per-row code (g8 << 8 | h8), transposed inside blocks of 16 rows
+    const uint32_t *rows;          // row list, or nullptr: rows 0 .. n-1
+    uint32_t off, n;               // list: entries rows[off .. off+n)
     int nb;
-    unsigned long long *hist;  // [F][nb]
-    uint32_t flush_rows;       // rows one lane slot may add between flushes (16+16 local only)
-    int k0;                    // first byte of the word handled by this launch
+    unsigned long long *hist;      // [F][nb]
+    unsigned long long *partial;   // [CTA][4][nb][32]
+    uint32_t flush_rows;           // rows one column may add between flushes (16+16 local only)
+    int pass;                      // 32+32 local only: bytes 2*pass, 2*pass+1 of every word
+    DevState *state;
 };
 
-template <int CODE_BYTES>
-__device__ inline uint32_t load_code(const uint8_t *codes, uint32_t row) {
-    if (CODE_BYTES == 1) return codes[row];
-    return reinterpret_cast<const uint16_t *>(codes)[row];
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(s));
+    return d;
 }
 
-// Adds the CTA's local histogram of the current tile into the leaf histogram and clears it.
-template <bool WIDE, int KC>
-__device__ inline void flush_local(int *sh, const TileDesc &td, int nb, int k0, unsigned long long *hist) {
+template <int IMM>
+__device__ __forceinline__ void red32(uint32_t addr, int v) {
+    asm volatile("red.shared.add.u32 [%0+%1], %2;" ::"r"(addr), "n"(IMM), "r"(v) : "memory");
+}
+
+template <int IMM>
+__device__ __forceinline__ void red64(uint32_t addr, uint32_t lo, uint32_t hi) {
+    asm volatile("{ .reg .b64 t; mov.b64 t, {%2, %3}; red.shared.add.u64 [%0+%1], t; }" ::"r"(addr), "n"(IMM),
+                 "r"(lo), "r"(hi)
+                 : "memory");
+}
+
+__device__ __forceinline__ uint32_t ldg32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint2 ldg64(const uint2 *p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint32_t ldg16(const uint16_t *p) {
+    uint32_t v;
+    asm volatile("{ .reg .u16 t; ld.global.nc.L1::no_allocate.u16 t, [%1]; cvt.u32.u16 %0, t; }" : "=r"(v) : "l"(p));
+    return v;
+}
+
+// Position of a row's code: inside every block of 16 rows the 4 x 4 arrangement is transposed,
+// so that the codes of rows 4j + s (j = 0..3) of a block are adjacent.
+__device__ __forceinline__ uint32_t code_pos(uint32_t row) {
+    return (row & ~15u) | ((row & 3u) << 2) | ((row >> 2) & 3u);
+}
+
+// One row's word: its bin codes -> shared atomics.  `half` selects the 16-bit code in the low
+// or high half of c.
+template <bool WIDE>
+__device__ __forceinline__ void add_word(uint32_t base, uint32_t w, uint32_t c, int half, int pass) {
+    if (!WIDE) {
+        // inc = g * 65536 + h: byte 0 = h, byte 1 = 0, byte 2 = g, byte 3 = sign of g
+        const int inc = (int)prmt(c, 0u, half ? 0xB342u : 0x9140u);
+        red32<0>(prmt(w, base, 0x7604u), inc);
+        red32<128>(prmt(w, base, 0x7614u), inc);
+        red32<65536>(prmt(w, base, 0x7624u), inc);
+        red32<65536 + 128>(prmt(w, base, 0x7634u), inc);
+    } else {
+        const uint32_t lo = prmt(c, 0u, half ? 0x4442u : 0x4440u);   // h
+        const uint32_t hi = prmt(c, 0u, half ? 0xBBB3u : 0x9991u);   // g, sign-extended
+        const uint32_t s0 = 0x7604u | ((uint32_t)(2 * pass) << 4), s1 = s0 + 0x10u;
+        red64<0>(prmt(w, base, s0), lo, hi);
+        red64<65536>(prmt(w, base, s1), lo, hi);
+    }
+}
+
+struct Out {
+    unsigned long long *ptr;   // partial slot of this CTA, or the final histogram
+    bool direct;               // final layout hist[f][bin] instead of partial [k][bin][a]
+    bool first;                // nothing stored yet: store instead of accumulate
+};
+
+// Adds the CTA's local histogram into its output and clears it.
+template <bool WIDE>
+__device__ inline void flush_local(int *hp, const TileDesc &td, int nb, int pass, Out &out) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int W = 1 << td.logW;
-    for (int r = warp; r < KC * nb; r += HIST_WARPS) {
+    const int nk = WIDE ? 2 : 4;
+    for (int r = warp; r < nk * nb; r += HIST_WARPS) {
         const int kk = r / nb, bin = r - kk * nb;
-        int G;
-        unsigned int H;
+        long long G;
+        unsigned long long H;
+        int k;
         if (!WIDE) {
-            const int v = sh[r * 32 + lane];
-            sh[r * 32 + lane] = 0;
+            k = kk;
+            int *p = hp + (kk >> 1) * 16384 + bin * 64 + (kk & 1) * 32 + lane;
+            const int v = *p;
+            *p = 0;
             G = v >> 16;
             H = (unsigned int)(v & 0xFFFF);
         } else {
-            G = sh[(2 * r) * 32 + lane];
-            H = (unsigned int)sh[(2 * r + 1) * 32 + lane];
-            sh[(2 * r) * 32 + lane] = 0;
-            sh[(2 * r + 1) * 32 + lane] = 0;
+            k = 2 * pass + kk;
+            unsigned long long *p = reinterpret_cast<unsigned long long *>(hp) + kk * 8192 + bin * 32 + lane;
+            const unsigned long long v = *p;
+            *p = 0ull;
+            G = (long long)(int)(v >> 32);
+            H = v & 0xFFFFFFFFull;
         }
         for (int o = W; o < 32; o <<= 1) {
             G += __shfl_xor_sync(0xffffffffu, G, o);
             H += __shfl_xor_sync(0xffffffffu, H, o);
         }
-        const int fl = 4 * lane + k0 + kk;
-        if (lane < W && fl < td.nf && (G != 0 || H != 0u)) {
-            const long long packed = (long long)G * 4294967296LL + (long long)H;
-            atomicAdd(&hist[(size_t)(td.f0 + fl) * nb + bin], (unsigned long long)packed);
+        const int fl = 4 * lane + k;
+        if (lane < W && fl < td.nf) {
+            unsigned long long *q = out.direct ? out.ptr + (size_t)(td.f0 + fl) * nb + bin
+                                               : out.ptr + (size_t)(k * nb + bin) * W + lane;
+            unsigned long long v = (unsigned long long)(G * 4294967296LL + (long long)H);
+            if (!out.first) v += *q;
+            *q = v;
         }
     }
+    out.first = false;
 }
 
-// Persistent CTAs over work units (tile, block of ROW_BLOCK rows), tile-major, split evenly
-// and contiguously, so a CTA changes tile (and flushes for that) at most a few times.
-template <int CODE_BYTES, bool WIDE, int KC>
+// CTAs of the static plan that take part in a build of n rows of a tile.
+__device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
+    uint32_t want = (n + MIN_ROWS_PER_CTA - 1) / MIN_ROWS_PER_CTA;
+    if (want < 1) want = 1;
+    return want < parts ? want : parts;
+}
+
+// The work of a lane is cut into units of four rows.  Contiguous rows: unit v covers rows
+// 16 (v / 4) + 4 j + v % 4, j = 0..3, whose codes are the four adjacent 16-bit values codes[4v ..].
+// Row list: warp-unit q covers list entries 4 R q .. 4 R (q + 1) - 1, entry 4 R q + R j + slot for
+// the lane's j-th row.  A warp instruction spans R units (one per row slot): a "warp-unit".
+template <bool WIDE, bool LIST>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
-    extern __shared__ int sh[];
+    extern __shared__ __align__(1024) int sh[];
+    const int2 me = a.cta_map[blockIdx.x];
+    const TileDesc td = a.tiles[me.x];
+    const uint32_t n = a.n;
+    const uint32_t P = effective_parts((uint32_t)td.parts, n);
+    const uint32_t part = (uint32_t)me.y;
+    if (part >= P) return;
+
+    const uint32_t sbase = smem_u32(sh);
+    const uint32_t h0 = (sbase + 65535u) & ~65535u;
+    uint32_t dyn_size;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_size));
+    if (h0 + 131072u > sbase + dyn_size) {   // the launch below leaves room; never write out of bounds
+        if (threadIdx.x == 0) atomicExch(&a.state->kernel_error, 1);
+        return;
+    }
+    int *hp = sh + (h0 - sbase) / 4;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int n_words = KC * a.nb * 32 * (WIDE ? 2 : 1);
-    for (int i = threadIdx.x; i < n_words; i += HIST_THREADS) sh[i] = 0;
+    for (int i = threadIdx.x; i < a.nb * 64; i += HIST_THREADS) {
+        hp[i] = 0;
+        hp[16384 + i] = 0;
+    }
     __syncthreads();
 
-    const uint32_t n = a.n;
-    const uint32_t nblk = (n + ROW_BLOCK - 1) / ROW_BLOCK;
-    const unsigned long long units = (unsigned long long)nblk * a.n_tiles;
-    const uint32_t u0 = (uint32_t)(units * blockIdx.x / gridDim.x);
-    const uint32_t u1 = (uint32_t)(units * (blockIdx.x + 1) / gridDim.x);
+    const int logW = td.logW, logR = 5 - logW;
+    const uint32_t R = 1u << logR;
+    const uint32_t wa = lane & ((1u << logW) - 1);
+    const uint32_t slot = lane >> logW;
+    const uint32_t base = h0 + lane * (WIDE ? 8 : 4);
+    const uint32_t *tile = td.data;
+    const int pass = a.pass;
 
-    int cur_tile = -1;
-    TileDesc td = {};
-    uint32_t slot_rows = 0;
-    bool dirty = false;
-    int *const my_col = sh + lane;
+    Out out;
+    out.direct = P == 1;
+    out.first = true;   // the two passes of the 32+32 mode write different features
+    out.ptr = out.direct ? a.hist : a.partial + (size_t)blockIdx.x * 4 * a.nb * 32;
 
-    for (uint32_t u = u0; u < u1; ++u) {
-        const int t = (int)(u / nblk);
-        const uint32_t blk = u - (uint32_t)t * nblk;
-        if (t != cur_tile) {
-            if (dirty) {
-                __syncthreads();
-                flush_local<WIDE, KC>(sh, td, a.nb, a.k0, a.hist);
-                __syncthreads();
-                dirty = false;
-            }
-            td = a.tiles[t];
-            cur_tile = t;
-            slot_rows = 0;
+    // ---- range of this part in warp-units [0, q1) from its first unit, and the leftover rows /
+    //      entries [s0, s1) that are done one by one
+    uint32_t q1, s0, s1, first_unit = 0, first_q = 0;
+    if (!LIST) {
+        const uint32_t B = n >> 4;                                   // full blocks of 16 rows
+        const uint32_t b0 = (uint32_t)((unsigned long long)B * part / P);
+        const uint32_t b1 = (uint32_t)((unsigned long long)B * (part + 1) / P);
+        first_unit = b0 << 2;
+        if (logR >= 2) {                                             // a warp-unit is R / 4 whole blocks
+            const uint32_t bpw = R >> 2;
+            q1 = (b1 - b0) / bpw;
+            s0 = (b0 + q1 * bpw) << 4;
+        } else {                                                     // 4 / R warp-units per block
+            q1 = (b1 - b0) << (2 - logR);
+            s0 = b1 << 4;
         }
-        const int logW = td.logW;
-        const int logR = 5 - logW;
-        const uint32_t row0 = blk * ROW_BLOCK;
-        const uint32_t rows_here = min((uint32_t)ROW_BLOCK, n - row0);
-        const uint32_t groups = (rows_here + (1u << logR) - 1) >> logR;
-        if (!WIDE) {
-            if (slot_rows + groups > a.flush_rows) {
-                __syncthreads();
-                flush_local<WIDE, KC>(sh, td, a.nb, a.k0, a.hist);
-                __syncthreads();
-                slot_rows = 0;
-            }
-            slot_rows += groups;
-        }
-        dirty = true;
-        const uint32_t wa = lane & ((1u << logW) - 1);  // word of the row held by this lane
-        const uint32_t slot = lane >> logW;             // row slot of this lane
-        const bool lane_used = wa < (uint32_t)td.words_used;
-        const uint32_t *tile = td.data;
-
-        for (uint32_t g0 = warp; g0 < groups; g0 += HIST_WARPS * UNROLL) {
-            uint32_t row[UNROLL];
-            bool ok[UNROLL];
-#pragma unroll
-            for (int j = 0; j < UNROLL; ++j) {
-                const uint32_t gi = g0 + j * HIST_WARPS;
-                const uint32_t p = row0 + (gi << logR) + slot;
-                ok[j] = lane_used && gi < groups && p < n;
-                row[j] = 0;
-                if (ok[j]) row[j] = a.rows ? a.rows[a.off + p] : a.off + p;
-            }
-            uint32_t word[UNROLL], code[UNROLL];
-#pragma unroll
-            for (int j = 0; j < UNROLL; ++j) {
-                word[j] = 0;
-                code[j] = 0;
-                if (ok[j]) {
-                    word[j] = tile[((size_t)row[j] << logW) + wa];
-                    code[j] = load_code<CODE_BYTES>(a.codes, row[j]);
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < UNROLL; ++j) {
-                if (!ok[j]) continue;
-                const uint32_t w = word[j] >> (8 * a.k0);
-                if (!WIDE) {
-                    // 4-bit codes: gradient in the high nibble (signed), hessian in the low nibble
-                    int gq, hq;
-                    if (CODE_BYTES == 1) {
-                        gq = ((int)(int8_t)code[j]) >> 4;
-                        hq = (int)(code[j] & 0xF);
-                    } else {
-                        gq = (int)(int8_t)(code[j] >> 8);
-                        hq = (int)(code[j] & 0xFF);
-                    }
-                    const int inc = gq * 65536 + hq;
-#pragma unroll
-                    for (int k = 0; k < KC; ++k) {
-                        const uint32_t bin = (w >> (8 * k)) & 0xFF;
-                        atomicAdd(my_col + (k * a.nb + bin) * 32, inc);
-                    }
-                } else {
-                    int gq, hq;
-                    if (CODE_BYTES == 1) {
-                        gq = ((int)(int8_t)code[j]) >> 4;
-                        hq = (int)(code[j] & 0xF);
-                    } else {
-                        gq = (int)(int8_t)(code[j] >> 8);
-                        hq = (int)(code[j] & 0xFF);
-                    }
-#pragma unroll
-                    for (int k = 0; k < KC; ++k) {
-                        const uint32_t bin = (w >> (8 * k)) & 0xFF;
-                        atomicAdd(my_col + (2 * (k * a.nb + bin)) * 32, gq);
-                        atomicAdd(my_col + (2 * (k * a.nb + bin) + 1) * 32, hq);
-                    }
-                }
-            }
-        }
+        s1 = part + 1 == P ? n : b1 << 4;
+    } else {
+        const uint32_t per = 4u << logR;                             // entries per warp-unit
+        const uint32_t Q = n / per;                                  // full warp-units
+        first_q = (uint32_t)((unsigned long long)Q * part / P);
+        q1 = (uint32_t)((unsigned long long)Q * (part + 1) / P) - first_q;
+        s0 = part + 1 == P ? Q * per : 0;
+        s1 = part + 1 == P ? n : 0;
     }
-    if (dirty) {
-        __syncthreads();
-        flush_local<WIDE, KC>(sh, td, a.nb, a.k0, a.hist);
+
+    // ---- leftover rows first (the column counters are still zero): R rows per warp instruction
+    uint32_t col_rows = 0;   // rows any one column may hold since the last flush
+    if (s1 > s0) {
+        for (uint32_t i = s0 + warp * R + slot; i < s1; i += HIST_WARPS * R) {
+            const uint32_t row = LIST ? a.rows[a.off + i] : i;
+            const uint32_t w = tile[((size_t)row << logW) + wa];
+            const uint32_t c = a.codes[code_pos(row)];
+            add_word<WIDE>(base, w, c, 0, pass);
+        }
+        col_rows = (s1 - s0 + R - 1) >> logR;
+    }
+
+    // ---- fast warp-units, in epochs that keep every 16+16 column below its limit
+    uint32_t q = 0;
+    while (q < q1) {
+        uint32_t epoch = q1 - q;   // warp-units of this epoch, all warps together
+        if (!WIDE) {
+            const uint32_t room = a.flush_rows > col_rows ? a.flush_rows - col_rows : 0;
+            const uint32_t fit = room >> 2;                          // every warp-unit adds 4 rows to each column
+            if (fit == 0) {
+                __syncthreads();
+                flush_local<WIDE>(hp, td, a.nb, pass, out);
+                __syncthreads();
+                col_rows = 0;
+                continue;
+            }
+            if (fit < epoch) epoch = fit;
+        }
+        // this warp's warp-units: q + warp, q + warp + 32, ... < q + epoch
+        const uint32_t nq = epoch > (uint32_t)warp ? (epoch - warp + HIST_WARPS - 1) / HIST_WARPS : 0;
+        if (!LIST) {
+            const uint32_t v = first_unit + ((q + warp) << logR) + slot;         // first unit of this lane
+            const uint32_t row0 = ((v >> 2) << 4) + (v & 3u);
+            const uint32_t *pw = tile + ((size_t)row0 << logW) + wa;
+            const uint2 *pc = reinterpret_cast<const uint2 *>(a.codes) + v;
+            const uint32_t jstride = 4u << logW;                                  // words between rows 4 apart
+            constexpr uint32_t QW = 32 * 128;                                     // words per 32 warp-units
+            const uint32_t qc = 32u << logR;                                      // units per 32 warp-units
+            uint32_t w[U_ROOT][4];
+            uint2 c[U_ROOT];
+#pragma unroll
+            for (int u = 0; u < U_ROOT; ++u) {
+                if ((uint32_t)u < nq) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) w[u][j] = ldg32(pw + (size_t)u * QW + j * jstride);
+                    c[u] = ldg64(pc + (size_t)u * qc);
+                }
+            }
+            for (uint32_t i = 0; i < nq; i += U_ROOT) {
+#pragma unroll
+                for (int u = 0; u < U_ROOT; ++u) {
+                    if (i + u < nq) {
+                        add_word<WIDE>(base, w[u][0], c[u].x, 0, pass);
+                        add_word<WIDE>(base, w[u][1], c[u].x, 1, pass);
+                        add_word<WIDE>(base, w[u][2], c[u].y, 0, pass);
+                        add_word<WIDE>(base, w[u][3], c[u].y, 1, pass);
+                        const uint32_t nx = i + u + U_ROOT;
+                        if (nx < nq) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) w[u][j] = ldg32(pw + (size_t)nx * QW + j * jstride);
+                            c[u] = ldg64(pc + (size_t)nx * qc);
+                        }
+                    }
+                }
+            }
+        } else {
+            // entry of (warp-unit wu, j): off + (4 wu << logR) + (j << logR) + slot
+            const uint32_t *pr = a.rows + a.off + ((size_t)(first_q + q + warp) << (logR + 2)) + slot;
+            const uint32_t qs = 128u << logR;                                     // entries per 32 warp-units
+            uint32_t idx[U_LIST][4], w[U_LIST][4], c[U_LIST][4];
+#pragma unroll
+            for (int u = 0; u < U_LIST; ++u)
+                if ((uint32_t)u < nq) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) idx[u][j] = pr[(size_t)u * qs + ((uint32_t)j << logR)];
+                }
+#pragma unroll
+            for (int u = 0; u < U_LIST; ++u)
+                if ((uint32_t)u < nq) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        w[u][j] = ldg32(tile + ((size_t)idx[u][j] << logW) + wa);
+                        c[u][j] = ldg16(a.codes + code_pos(idx[u][j]));
+                    }
+                    if ((uint32_t)u + U_LIST < nq) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) idx[u][j] = pr[(size_t)(u + U_LIST) * qs + ((uint32_t)j << logR)];
+                    }
+                }
+            for (uint32_t i = 0; i < nq; i += U_LIST) {
+#pragma unroll
+                for (int u = 0; u < U_LIST; ++u) {
+                    if (i + u < nq) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) add_word<WIDE>(base, w[u][j], c[u][j], 0, pass);
+                        const uint32_t nx = i + u + U_LIST;
+                        if (nx < nq) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                w[u][j] = ldg32(tile + ((size_t)idx[u][j] << logW) + wa);
+                                c[u][j] = ldg16(a.codes + code_pos(idx[u][j]));
+                            }
+                            if (nx + U_LIST < nq) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    idx[u][j] = pr[(size_t)(nx + U_LIST) * qs + ((uint32_t)j << logR)];
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        q += epoch;
+        col_rows += 4 * epoch;
+    }
+    __syncthreads();
+    flush_local<WIDE>(hp, td, a.nb, pass, out);
+}
+
+// Sums the partial histograms of every tile that was built by more than one CTA.
+__global__ void __launch_bounds__(256) k_hist_reduce(const TileDesc *__restrict__ tiles, uint32_t n, int nb,
+                                                     const unsigned long long *__restrict__ partial,
+                                                     unsigned long long *__restrict__ hist) {
+    const TileDesc td = tiles[blockIdx.y];
+    const uint32_t P = effective_parts((uint32_t)td.parts, n);
+    if (P <= 1) return;
+    const int W = 1 << td.logW;
+    const uint32_t total = 4u * nb * W;
+    const size_t stride = (size_t)4 * nb * 32;
+    for (uint32_t e = blockIdx.x * 256 + threadIdx.x; e < total; e += gridDim.x * 256) {
+        const uint32_t a = e & (W - 1);
+        const uint32_t kb = e >> td.logW;          // k * nb + bin
+        const uint32_t k = kb / nb, bin = kb - k * nb;
+        const uint32_t fl = 4 * a + k;
+        if (fl >= (uint32_t)td.nf) continue;
+        const unsigned long long *p = partial + (size_t)td.cta0 * stride + e;
+        unsigned long long s = 0;
+        for (uint32_t i = 0; i < P; ++i) s += p[i * stride];
+        hist[(size_t)(td.f0 + fl) * nb + bin] = s;
     }
 }
 
@@ -201,16 +389,15 @@ __global__ void k_subtract(const unsigned long long *__restrict__ parent, const 
         large[i] = parent[i] - small[i];
 }
 
-template <int CODE_BYTES, bool WIDE, int KC>
-int launch_hist(qgbdt_ctx *c, const HistArgs &args, unsigned grid, cudaStream_t st) {
-    const size_t smem = (size_t)KC * c->nb * 32 * 4 * (WIDE ? 2 : 1);
-    auto kern = k_hist<CODE_BYTES, WIDE, KC>;
-    static size_t configured = 48 * 1024;  // per instantiation: largest opt-in size set so far
-    if (smem > configured) {
-        QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = smem;
+template <bool WIDE, bool LIST>
+int launch_hist(qgbdt_ctx *c, const HistArgs &args, cudaStream_t st) {
+    auto kern = k_hist<WIDE, LIST>;
+    static bool configured = false;   // per instantiation
+    if (!configured) {
+        QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
+        configured = true;
     }
-    kern<<<grid, HIST_THREADS, smem, st>>>(args);
+    kern<<<(unsigned)c->hist_grid, HIST_THREADS, HIST_SMEM, st>>>(args);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
 }
@@ -220,31 +407,33 @@ int launch_hist(qgbdt_ctx *c, const HistArgs &args, unsigned grid, cudaStream_t 
 int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsigned long long *d_hist,
             cudaStream_t st) {
     const size_t hist_bytes = (size_t)c->F * c->nb * sizeof(unsigned long long);
-    QG_CUDA(c, cudaMemsetAsync(d_hist, 0, hist_bytes, st));
     c->n_hist_builds++;
     c->n_hist_row_features += n * c->F;
-    if (n <= 0) return QGBDT_OK;
+    if (n <= 0) {
+        QG_CUDA(c, cudaMemsetAsync(d_hist, 0, hist_bytes, st));
+        return QGBDT_OK;
+    }
+    if (!d_rows && off != 0) return qg_fail(c, QGBDT_ERR_ARG, "a contiguous build starts at row 0");
 
     const int bits = c->prm.bits;
     const int kg = qg_levels_g(bits);
     const int kh = c->const_hess ? 1 : qg_levels_h(bits, c->prm.hess_levels_mode);
-    const bool wide = c->code_bytes == 2;
+    const bool wide = bits >= 6;
 
     HistArgs a;
     a.tiles = c->d_tiles;
-    a.n_tiles = (int)c->tiles.size();
-    a.codes = c->d_codes;
+    a.cta_map = c->d_cta_map;
+    a.codes = reinterpret_cast<const uint16_t *>(c->d_codes);
     a.rows = d_rows;
     a.off = (uint32_t)off;
     a.n = (uint32_t)n;
     a.nb = c->nb;
     a.hist = d_hist;
-    a.k0 = 0;
+    a.partial = c->d_partial;
     const uint32_t by_h = 65535u / (uint32_t)kh, by_g = 32767u / (uint32_t)kg;
     a.flush_rows = by_h < by_g ? by_h : by_g;
-
-    const unsigned long long units = (unsigned long long)((n + ROW_BLOCK - 1) / ROW_BLOCK) * a.n_tiles;
-    unsigned grid = (unsigned)(units < (unsigned long long)c->sm_count ? units : (unsigned long long)c->sm_count);
+    a.pass = 0;
+    a.state = c->d_state;
 
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     if (c->profile_hist) {
@@ -257,29 +446,29 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
         }
         ev0 = c->hist_events[c->hist_events_used++];
         ev1 = c->hist_events[c->hist_events_used++];
-        // algorithmic bytes of this build: bin codes + packed gradient code (+ row index) per row, histogram out
+        // algorithmic bytes of this build: bin codes + gradient code (+ row index) per row, histogram out
         c->hist_prof_bytes += n * (c->F + c->code_bytes + (d_rows ? 4 : 0)) + (int64_t)hist_bytes;
         c->hist_prof_launches++;
         QG_CUDA(c, cudaEventRecord(ev0, st));
     }
     int rc;
     if (!wide) {
-        rc = launch_hist<1, false, 4>(c, a, grid, st);
+        rc = d_rows ? launch_hist<false, true>(c, a, st) : launch_hist<false, false>(c, a, st);
     } else {
-        // 32+32 local bins: two words per bin; all four bytes fit only for small bin counts
-        const size_t full = (size_t)4 * c->nb * 32 * 4 * 2;
-        if (full <= (size_t)c->max_smem_optin) {
-            rc = launch_hist<2, true, 4>(c, a, grid, st);
-        } else {
-            rc = launch_hist<2, true, 2>(c, a, grid, st);
-            if (rc == QGBDT_OK) {
-                a.k0 = 2;
-                rc = launch_hist<2, true, 2>(c, a, grid, st);
-            }
+        rc = d_rows ? launch_hist<true, true>(c, a, st) : launch_hist<true, false>(c, a, st);
+        if (rc == QGBDT_OK) {
+            a.pass = 1;
+            rc = d_rows ? launch_hist<true, true>(c, a, st) : launch_hist<true, false>(c, a, st);
         }
     }
-    if (rc == QGBDT_OK && ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
-    return rc;
+    if (rc != QGBDT_OK) return rc;
+    if (c->max_parts > 1 && effective_parts((uint32_t)c->max_parts, (uint32_t)n) > 1) {
+        const dim3 grid((unsigned)((4 * c->nb * 32 + 255) / 256), (unsigned)c->tiles.size());
+        k_hist_reduce<<<grid, 256, 0, st>>>(c->d_tiles, (uint32_t)n, c->nb, c->d_partial, d_hist);
+        QG_LAUNCH_CHECK(c);
+    }
+    if (ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
+    return QGBDT_OK;
 }
 
 int qg_subtract(qgbdt_ctx *c, const unsigned long long *d_parent, const unsigned long long *d_small,

@@ -20,8 +20,14 @@
 // l holds word a = l % W of row slot b = l / W.
 //
 // Packed gradient codes (Sec. 6.2 packs g and h of a sample the same way as the
-// bins): B <= 4: one byte per row, signed gradient in the high nibble, hessian in
-// the low nibble; B >= 5: two bytes, signed gradient in the high byte.
+// bins): two bytes per row, signed gradient in the high byte, hessian in the low
+// byte.  Inside every block of 16 rows the codes are stored 4 x 4 transposed (the
+// code of row 16 b + 4 j + s sits at position 16 b + 4 s + j), so that a lane of the
+// histogram kernel reads the codes of its four rows with one 8-byte load.
+//
+// Histogram plan: every tile owns `parts` consecutive CTAs starting at `cta0` (in
+// proportion to its width); cta_map[cta] = (tile, part).  A build of n rows uses the
+// first min(parts, ceil(n / 4096)) of them.
 //
 // Row lists: one uint32 array of N entries; leaf l owns [leaf_off[l], +leaf_n[l]).
 // ---------------------------------------------------------------------------
@@ -32,6 +38,8 @@ struct TileDesc {
     int32_t nf;            // real features in the tile (<= 4 * W)
     int32_t logW;          // log2 of words per row
     int32_t words_used;    // ceil(nf / 4)
+    int32_t parts;         // CTAs of the histogram plan that work on this tile
+    int32_t cta0;          // first of them
 };
 
 // Scalars produced and consumed on the device within one boosting iteration.
@@ -39,6 +47,7 @@ struct DevState {
     unsigned int gmax_bits;  // max |g| as float bits (non-negative floats order like uints)
     unsigned int hmax_bits;  // max h as float bits
     int bad_value;           // set when a gradient / hessian / bin code is out of domain
+    int kernel_error;        // set by a kernel that refused to run (checked at the next synchronising call)
     unsigned int part_nl;    // rows that went left in the last partition
     long long tot_g, tot_h;  // integer sums over all rows of the last quantization
 };
@@ -62,10 +71,13 @@ struct qgbdt_ctx {
     bool loaded = false;
     std::vector<TileDesc> tiles;
     TileDesc *d_tiles = nullptr;
+    int2 *d_cta_map = nullptr;               // [hist_grid]
+    int hist_grid = 0, max_parts = 1;
+    unsigned long long *d_partial = nullptr;  // [hist_grid][4][nb][32] partial histograms (only if max_parts > 1)
     std::vector<void *> tile_allocs;
     // quantized gradients
-    uint8_t *d_codes = nullptr;  // [N * code_bytes]
-    int code_bytes = 1;
+    uint8_t *d_codes = nullptr;  // [round_up(N, 16)] 16-bit codes
+    int code_bytes = 2;
     bool quantized = false;
     bool const_hess = false;
     float gmax = 0.f, hmax = 0.f;

@@ -124,9 +124,8 @@ __device__ inline int round_level(float x, int rounding, uint32_t u) {
     return (int)f + (u < t ? 1 : 0);
 }
 
-// Eq. 6 + Eq. 8 for every row; writes the packed per-row code, optional unpacked copies,
+// Eq. 6 + Eq. 8 for every row; writes the packed 16-bit per-row code, optional unpacked copies,
 // and adds the integer totals (one atomic pair per block).
-template <int CODE_BYTES>
 __global__ void k_quantize(const float *__restrict__ g, const float *__restrict__ h, long long n, int kg, int kh,
                            int rounding, uint32_t key, DevState *state, uint8_t *__restrict__ codes,
                            int8_t *__restrict__ gq_out, uint8_t *__restrict__ hq_out) {
@@ -149,11 +148,9 @@ __global__ void k_quantize(const float *__restrict__ g, const float *__restrict_
             y = y < 0.f ? 0.f : y;
             hq = round_level(y, rounding, mix32(r + 0x6A09E667u) >> 8);
         }
-        if (CODE_BYTES == 1) {
-            codes[i] = (uint8_t)(((gq & 0xF) << 4) | hq);
-        } else {
-            reinterpret_cast<uint16_t *>(codes)[i] = (uint16_t)(((gq & 0xFF) << 8) | hq);
-        }
+        // 4 x 4 transposed inside blocks of 16 rows (see the layout notes of the internal header)
+        const long long pos = (i & ~15LL) | ((i & 3) << 2) | ((i >> 2) & 3);
+        reinterpret_cast<uint16_t *>(codes)[pos] = (uint16_t)(((gq & 0xFF) << 8) | hq);
         if (gq_out) gq_out[i] = (int8_t)gq;
         if (hq_out) hq_out[i] = (uint8_t)hq;
         sg += gq;
@@ -219,12 +216,8 @@ int qg_quantize(qgbdt_ctx *c, const float *d_g, const float *d_h, uint32_t tree,
     const uint32_t key = mix32(mix32(mix32(seed_lo ^ 0x6A09E667u) + seed_hi) ^ tree);
     const int kg = qg_levels_g(c->prm.bits), kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
     const unsigned grid = grid_for(c, c->N, 256, 8);
-    if (c->code_bytes == 1)
-        k_quantize<1><<<grid, 256, 0, st>>>(d_g, d_h, c->N, kg, kh, c->prm.rounding, key, c->d_state, c->d_codes,
-                                            d_gq, d_hq);
-    else
-        k_quantize<2><<<grid, 256, 0, st>>>(d_g, d_h, c->N, kg, kh, c->prm.rounding, key, c->d_state, c->d_codes,
-                                            d_gq, d_hq);
+    k_quantize<<<grid, 256, 0, st>>>(d_g, d_h, c->N, kg, kh, c->prm.rounding, key, c->d_state, c->d_codes, d_gq,
+                                     d_hq);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
 }

@@ -70,6 +70,7 @@ int train_one_tree(qgbdt_ctx *c, const float *d_labels, float *d_scores, uint32_
         if ((rc = qg_partition(c, off, n, s.feature, s.bin, st)) != QGBDT_OK) return rc;
         QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
         QG_CUDA(c, cudaStreamSynchronize(st));
+        if (hs->kernel_error) return qg_fail(c, QGBDT_ERR_CUDA, "a histogram kernel refused its launch configuration");
         const int64_t nl = hs->part_nl, nr = n - nl;
         const int node = c->n_leaves - 1, right = c->n_leaves;
         nf[node] = s.feature;

@@ -49,9 +49,9 @@ void free_data(qgbdt_ctx *c) {
     c->tile_allocs.clear();
     c->tiles.clear();
     dev_free(c->d_tiles);
-    dev_free(c->d_cta_map);
     dev_free(c->d_partial);
     dev_free(c->d_codes);
+    dev_free(c->d_codes_nat);
     dev_free(c->d_idx);
     dev_free(c->d_idx_tmp);
     dev_free(c->d_part_counts);
@@ -103,8 +103,8 @@ void plan_tiles(int F, std::vector<TileDesc> &out) {
 
 // Histogram plan: CTAs are shared out among the tiles in proportion to their width in words
 // (the cost of a row is one warp instruction slot per 32 words); with more tiles than SMs every
-// tile gets one CTA.  Fills parts / cta0 of the tiles and returns the CTA -> (tile, part) map.
-void plan_hist_ctas(int sm_count, std::vector<TileDesc> &tiles, std::vector<int2> &map, int &max_parts) {
+// tile gets one CTA.  Fills parts / cta0 of the tiles; part p of a tile owns partial-histogram slot cta0 + p.
+void plan_hist_ctas(int sm_count, std::vector<TileDesc> &tiles, int &n_ctas, int &max_parts) {
     const int T = (int)tiles.size();
     long long total_w = 0;
     for (const TileDesc &t : tiles) total_w += 1 << t.logW;
@@ -123,11 +123,11 @@ void plan_hist_ctas(int sm_count, std::vector<TileDesc> &tiles, std::vector<int2
         tiles[best].parts++;
         used++;
     }
-    map.clear();
+    n_ctas = 0;
     max_parts = 1;
     for (int i = 0; i < T; ++i) {
-        tiles[i].cta0 = (int)map.size();
-        for (int p = 0; p < tiles[i].parts; ++p) map.push_back(make_int2(i, p));
+        tiles[i].cta0 = n_ctas;
+        n_ctas += tiles[i].parts;
         if (tiles[i].parts > max_parts) max_parts = tiles[i].parts;
     }
 }
@@ -173,9 +173,7 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     c->nb = n_bins;
     c->code_bytes = 2;
     plan_tiles(n_features, c->tiles);
-    std::vector<int2> cta_map;
-    plan_hist_ctas(c->sm_count, c->tiles, cta_map, c->max_parts);
-    c->hist_grid = (int)cta_map.size();
+    plan_hist_ctas(c->sm_count, c->tiles, c->hist_grid, c->max_parts);
     int rc;
     for (TileDesc &t : c->tiles) {
         uint32_t *p = nullptr;
@@ -186,13 +184,11 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     if ((rc = dev_alloc(c, &c->d_tiles, c->tiles.size())) != QGBDT_OK) return rc;
     QG_CUDA(c, cudaMemcpyAsync(c->d_tiles, c->tiles.data(), sizeof(TileDesc) * c->tiles.size(),
                                cudaMemcpyHostToDevice, st));
-    if ((rc = dev_alloc(c, &c->d_cta_map, cta_map.size())) != QGBDT_OK) return rc;
-    // pageable source: the copy has left the host buffer when the call returns
-    QG_CUDA(c, cudaMemcpyAsync(c->d_cta_map, cta_map.data(), sizeof(int2) * cta_map.size(), cudaMemcpyHostToDevice, st));
     if (c->max_parts > 1 &&
         (rc = dev_alloc(c, &c->d_partial, (size_t)c->hist_grid * 4 * n_bins * 32)) != QGBDT_OK)
         return rc;
     if ((rc = dev_alloc(c, &c->d_codes, ((size_t)n_rows + 15) / 16 * 16 * 2 + 16)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_codes_nat, (size_t)n_rows * 2 + 16)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx, (size_t)n_rows)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx_tmp, (size_t)n_rows)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8)) != QGBDT_OK) return rc;

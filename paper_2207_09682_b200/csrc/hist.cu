@@ -8,8 +8,8 @@
 //  * Bank-private columns.  The local histogram is indexed [bin][byte k of the word][lane].
 //    Lane l of a warp always adds into column l, i.e. shared-memory bank l, so the 32 atomics
 //    of one warp instruction never collide, whatever the bin codes are (uniform, or 90 % in
-//    one bin).  A lane owns word a = l % W of row slot l / W; the R = 32/W row slots are R
-//    private replicas that the flush adds up.  Measured: one conflict-free warp atomic per
+//    one bin).  A lane owns word a = l / R of row slot l % R; the R = 32/W row slots are R
+//    private replicas in adjacent words that the flush adds up.  Measured: one conflict-free warp atomic per
 //    clock per SM.
 //  * One-instruction addressing.  The local histogram starts on a 64 KB boundary of the shared
 //    window and a bin is 256 bytes apart from the next, so the address of (bin, lane) is the
@@ -34,13 +34,14 @@ constexpr int HIST_THREADS = 1024;
 constexpr int HIST_WARPS = HIST_THREADS / 32;
 constexpr int HIST_SMEM = 192 * 1024;     // 128 KB histogram on a 64 KB boundary + the room below it
 constexpr uint32_t MIN_ROWS_PER_CTA = 4096;
-constexpr int U_ROOT = 3;                 // units in flight per lane, contiguous rows
+constexpr int U_ROOT = 4;                 // units in flight per lane, contiguous rows
 constexpr int U_LIST = 2;                 // units in flight per lane, row list (plus as many index units)
 
 struct HistArgs {
     const TileDesc *tiles;
-    const int2 *cta_map;           // CTA -> (tile, part)
     const uint16_t *codes;         // per-row code (g8 << 8 | h8), transposed inside blocks of 16 rows
+    const uint16_t *codes_nat;     // the same codes in row order (row lists and leftover rows)
+    int tile0;                     // first tile of this launch
     const uint32_t *rows;          // row list, or nullptr: rows 0 .. n-1
     uint32_t off, n;               // list: entries rows[off .. off+n)
     int nb;
@@ -89,12 +90,6 @@ __device__ __forceinline__ uint32_t ldg16(const uint16_t *p) {
     return v;
 }
 
-// Position of a row's code: inside every block of 16 rows the 4 x 4 arrangement is transposed,
-// so that the codes of rows 4j + s (j = 0..3) of a block are adjacent.
-__device__ __forceinline__ uint32_t code_pos(uint32_t row) {
-    return (row & ~15u) | ((row & 3u) << 2) | ((row >> 2) & 3u);
-}
-
 // One row's word: its bin codes -> shared atomics.  `half` selects the 16-bit code in the low
 // or high half of c.
 template <bool WIDE>
@@ -121,43 +116,53 @@ struct Out {
     bool first;                // nothing stored yet: store instead of accumulate
 };
 
-// Adds the CTA's local histogram into its output and clears it.
+// Adds the CTA's local histogram into its output and clears it.  The R replicas of a column
+// (the row slots of word a) are R adjacent shared words, so one thread sums them from vector
+// loads and writes one packed 64-bit bin.
 template <bool WIDE>
-__device__ inline void flush_local(int *hp, const TileDesc &td, int nb, int pass, Out &out) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int W = 1 << td.logW;
-    const int nk = WIDE ? 2 : 4;
-    for (int r = warp; r < nk * nb; r += HIST_WARPS) {
-        const int kk = r / nb, bin = r - kk * nb;
-        long long G;
-        unsigned long long H;
-        int k;
-        if (!WIDE) {
-            k = kk;
-            int *p = hp + (kk >> 1) * 16384 + bin * 64 + (kk & 1) * 32 + lane;
-            const int v = *p;
-            *p = 0;
-            G = v >> 16;
-            H = (unsigned int)(v & 0xFFFF);
-        } else {
-            k = 2 * pass + kk;
-            unsigned long long *p = reinterpret_cast<unsigned long long *>(hp) + kk * 8192 + bin * 32 + lane;
-            const unsigned long long v = *p;
-            *p = 0ull;
-            G = (long long)(int)(v >> 32);
-            H = v & 0xFFFFFFFFull;
-        }
-        for (int o = W; o < 32; o <<= 1) {
-            G += __shfl_xor_sync(0xffffffffu, G, o);
-            H += __shfl_xor_sync(0xffffffffu, H, o);
-        }
-        const int fl = 4 * lane + k;
-        if (lane < W && fl < td.nf) {
-            unsigned long long *q = out.direct ? out.ptr + (size_t)(td.f0 + fl) * nb + bin
-                                               : out.ptr + (size_t)(k * nb + bin) * W + lane;
-            unsigned long long v = (unsigned long long)(G * 4294967296LL + (long long)H);
-            if (!out.first) v += *q;
-            *q = v;
+__device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, int nb, int pass, Out &out) {
+    const int W = 1 << logW, R = 32 >> logW;
+    const int per_k = nb << logW;                                   // outputs per byte position k
+    for (int kk = 0; kk < (WIDE ? 2 : 4); ++kk) {
+        const int k = WIDE ? 2 * pass + kk : kk;
+        for (int e = threadIdx.x; e < per_k; e += HIST_THREADS) {
+            const int a = e & (W - 1), bin = e >> logW;
+            unsigned long long v;
+            if (!WIDE) {
+                int *p = hp + (kk >> 1) * 16384 + bin * 64 + (kk & 1) * 32 + a * R;
+                int G = 0, H = 0;
+                if (R >= 4) {
+                    for (int r = 0; r < R; r += 4) {
+                        const int4 x = *reinterpret_cast<const int4 *>(p + r);
+                        *reinterpret_cast<int4 *>(p + r) = make_int4(0, 0, 0, 0);
+                        G += (x.x >> 16) + (x.y >> 16) + (x.z >> 16) + (x.w >> 16);
+                        H += (x.x & 0xFFFF) + (x.y & 0xFFFF) + (x.z & 0xFFFF) + (x.w & 0xFFFF);
+                    }
+                } else {
+                    for (int r = 0; r < R; ++r) {
+                        const int x = p[r];
+                        p[r] = 0;
+                        G += x >> 16;
+                        H += x & 0xFFFF;
+                    }
+                }
+                v = (unsigned long long)((long long)G * 4294967296LL + (long long)H);
+            } else {
+                // packed 32+32 words add up as they are: no field can overflow (checked at load time)
+                unsigned long long *p = reinterpret_cast<unsigned long long *>(hp) + kk * 8192 + bin * 32 + a * R;
+                v = 0;
+                for (int r = 0; r < R; ++r) {
+                    v += p[r];
+                    p[r] = 0ull;
+                }
+            }
+            const int fl = 4 * a + k;
+            if (fl < td.nf) {
+                unsigned long long *q = out.direct ? out.ptr + (size_t)(td.f0 + fl) * nb + bin
+                                                   : out.ptr + (size_t)k * nb * W + e;
+                if (!out.first) v += *q;
+                *q = v;
+            }
         }
     }
     out.first = false;
@@ -174,14 +179,16 @@ __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) 
 // 16 (v / 4) + 4 j + v % 4, j = 0..3, whose codes are the four adjacent 16-bit values codes[4v ..].
 // Row list: warp-unit q covers list entries 4 R q .. 4 R (q + 1) - 1, entry 4 R q + R j + slot for
 // the lane's j-th row.  A warp instruction spans R units (one per row slot): a "warp-unit".
-template <bool WIDE, bool LIST>
+//
+// LOGW_T >= 0 fixes the tile width at compile time (all strides become immediates); -1 reads it
+// from the tile.  The grid is (part, tile - tile0).
+template <int LOGW_T, bool WIDE, bool LIST>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     extern __shared__ __align__(1024) int sh[];
-    const int2 me = a.cta_map[blockIdx.x];
-    const TileDesc td = a.tiles[me.x];
+    const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
     const uint32_t n = a.n;
     const uint32_t P = effective_parts((uint32_t)td.parts, n);
-    const uint32_t part = (uint32_t)me.y;
+    const uint32_t part = blockIdx.x;
     if (part >= P) return;
 
     const uint32_t sbase = smem_u32(sh);
@@ -193,17 +200,19 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
         return;
     }
     int *hp = sh + (h0 - sbase) / 4;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
     for (int i = threadIdx.x; i < a.nb * 64; i += HIST_THREADS) {
         hp[i] = 0;
         hp[16384 + i] = 0;
     }
     __syncthreads();
 
-    const int logW = td.logW, logR = 5 - logW;
+    const int logW = LOGW_T >= 0 ? LOGW_T : td.logW;
+    const int logR = 5 - logW;
     const uint32_t R = 1u << logR;
-    const uint32_t wa = lane & ((1u << logW) - 1);
-    const uint32_t slot = lane >> logW;
+    const uint32_t wa = lane >> logR;           // word of the row held by this lane
+    const uint32_t slot = lane & (R - 1);       // row slot of this lane (adjacent lanes: replicas of a column)
     const uint32_t base = h0 + lane * (WIDE ? 8 : 4);
     const uint32_t *tile = td.data;
     const int pass = a.pass;
@@ -211,7 +220,7 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     Out out;
     out.direct = P == 1;
     out.first = true;   // the two passes of the 32+32 mode write different features
-    out.ptr = out.direct ? a.hist : a.partial + (size_t)blockIdx.x * 4 * a.nb * 32;
+    out.ptr = out.direct ? a.hist : a.partial + (size_t)(td.cta0 + part) * 4 * a.nb * 32;
 
     // ---- range of this part in warp-units [0, q1) from its first unit, and the leftover rows /
     //      entries [s0, s1) that are done one by one
@@ -245,13 +254,14 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
         for (uint32_t i = s0 + warp * R + slot; i < s1; i += HIST_WARPS * R) {
             const uint32_t row = LIST ? a.rows[a.off + i] : i;
             const uint32_t w = tile[((size_t)row << logW) + wa];
-            const uint32_t c = a.codes[code_pos(row)];
+            const uint32_t c = a.codes_nat[row];
             add_word<WIDE>(base, w, c, 0, pass);
         }
         col_rows = (s1 - s0 + R - 1) >> logR;
     }
 
     // ---- fast warp-units, in epochs that keep every 16+16 column below its limit
+    constexpr int U = LIST ? U_LIST : U_ROOT;
     uint32_t q = 0;
     while (q < q1) {
         uint32_t epoch = q1 - q;   // warp-units of this epoch, all warps together
@@ -260,7 +270,7 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
             const uint32_t fit = room >> 2;                          // every warp-unit adds 4 rows to each column
             if (fit == 0) {
                 __syncthreads();
-                flush_local<WIDE>(hp, td, a.nb, pass, out);
+                flush_local<WIDE>(hp, td, logW, a.nb, pass, out);
                 __syncthreads();
                 col_rows = 0;
                 continue;
@@ -277,88 +287,116 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
             const uint32_t jstride = 4u << logW;                                  // words between rows 4 apart
             constexpr uint32_t QW = 32 * 128;                                     // words per 32 warp-units
             const uint32_t qc = 32u << logR;                                      // units per 32 warp-units
-            uint32_t w[U_ROOT][4];
-            uint2 c[U_ROOT];
+            uint32_t w[U][4];
+            uint2 c[U];
+#define QG_LOAD_UNIT(u)                                                                  \
+    {                                                                                    \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) w[u][j] = ldg32(pw + (u) * QW + j * jstride); \
+        c[u] = ldg64(pc + (u) * qc);                                                     \
+    }
+#define QG_USE_UNIT(u)                                       \
+    {                                                        \
+        add_word<WIDE>(base, w[u][0], c[u].x, 0, pass);      \
+        add_word<WIDE>(base, w[u][1], c[u].x, 1, pass);      \
+        add_word<WIDE>(base, w[u][2], c[u].y, 0, pass);      \
+        add_word<WIDE>(base, w[u][3], c[u].y, 1, pass);      \
+    }
 #pragma unroll
-            for (int u = 0; u < U_ROOT; ++u) {
-                if ((uint32_t)u < nq) {
+            for (int u = 0; u < U; ++u)
+                if ((uint32_t)u < nq) QG_LOAD_UNIT(u)
+            pw += U * QW;
+            pc += U * qc;
+            uint32_t i = 0;
+            for (; i + 2 * U <= nq; i += U) {   // units i .. i+U-1 are in registers, the next U exist
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) w[u][j] = ldg32(pw + (size_t)u * QW + j * jstride);
-                    c[u] = ldg64(pc + (size_t)u * qc);
+                for (int u = 0; u < U; ++u) {
+                    QG_USE_UNIT(u)
+                    QG_LOAD_UNIT(u)
                 }
+                pw += U * QW;
+                pc += U * qc;
             }
-            for (uint32_t i = 0; i < nq; i += U_ROOT) {
+            for (; i < nq; i += U) {
 #pragma unroll
-                for (int u = 0; u < U_ROOT; ++u) {
+                for (int u = 0; u < U; ++u) {
                     if (i + u < nq) {
-                        add_word<WIDE>(base, w[u][0], c[u].x, 0, pass);
-                        add_word<WIDE>(base, w[u][1], c[u].x, 1, pass);
-                        add_word<WIDE>(base, w[u][2], c[u].y, 0, pass);
-                        add_word<WIDE>(base, w[u][3], c[u].y, 1, pass);
-                        const uint32_t nx = i + u + U_ROOT;
-                        if (nx < nq) {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) w[u][j] = ldg32(pw + (size_t)nx * QW + j * jstride);
-                            c[u] = ldg64(pc + (size_t)nx * qc);
-                        }
+                        QG_USE_UNIT(u)
+                        if (i + u + U < nq) QG_LOAD_UNIT(u)
                     }
                 }
+                pw += U * QW;
+                pc += U * qc;
             }
+#undef QG_LOAD_UNIT
+#undef QG_USE_UNIT
         } else {
             // entry of (warp-unit wu, j): off + (4 wu << logR) + (j << logR) + slot
             const uint32_t *pr = a.rows + a.off + ((size_t)(first_q + q + warp) << (logR + 2)) + slot;
             const uint32_t qs = 128u << logR;                                     // entries per 32 warp-units
-            uint32_t idx[U_LIST][4], w[U_LIST][4], c[U_LIST][4];
+            const uint32_t *tw = tile + wa;
+            uint32_t idx[U][4], w[U][4], c[U][4];
+#define QG_LOAD_IDX(u)                                                                              \
+    {                                                                                               \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) idx[u][j] = pr[(u) * qs + ((uint32_t)j << logR)]; \
+    }
+#define QG_LOAD_DATA(u)                                                \
+    {                                                                  \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) {                \
+            w[u][j] = ldg32(tw + ((size_t)idx[u][j] << logW));         \
+            c[u][j] = ldg16(a.codes_nat + idx[u][j]);                  \
+        }                                                              \
+    }
+#define QG_USE_DATA(u)                                                                           \
+    {                                                                                            \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) add_word<WIDE>(base, w[u][j], c[u][j], 0, pass); \
+    }
 #pragma unroll
-            for (int u = 0; u < U_LIST; ++u)
+            for (int u = 0; u < U; ++u)
+                if ((uint32_t)u < nq) QG_LOAD_IDX(u)
+            pr += U * qs;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
                 if ((uint32_t)u < nq) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) idx[u][j] = pr[(size_t)u * qs + ((uint32_t)j << logR)];
+                    QG_LOAD_DATA(u)
+                    if ((uint32_t)u + U < nq) QG_LOAD_IDX(u)
                 }
+            pr += U * qs;
+            uint32_t i = 0;
+            for (; i + 3 * U <= nq; i += U) {   // data of units i .. i+U-1 and indices of the next U are in registers
 #pragma unroll
-            for (int u = 0; u < U_LIST; ++u)
-                if ((uint32_t)u < nq) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        w[u][j] = ldg32(tile + ((size_t)idx[u][j] << logW) + wa);
-                        c[u][j] = ldg16(a.codes + code_pos(idx[u][j]));
-                    }
-                    if ((uint32_t)u + U_LIST < nq) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) idx[u][j] = pr[(size_t)(u + U_LIST) * qs + ((uint32_t)j << logR)];
-                    }
+                for (int u = 0; u < U; ++u) {
+                    QG_USE_DATA(u)
+                    QG_LOAD_DATA(u)
+                    QG_LOAD_IDX(u)
                 }
-            for (uint32_t i = 0; i < nq; i += U_LIST) {
+                pr += U * qs;
+            }
+            for (; i < nq; i += U) {
 #pragma unroll
-                for (int u = 0; u < U_LIST; ++u) {
+                for (int u = 0; u < U; ++u) {
                     if (i + u < nq) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) add_word<WIDE>(base, w[u][j], c[u][j], 0, pass);
-                        const uint32_t nx = i + u + U_LIST;
-                        if (nx < nq) {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                w[u][j] = ldg32(tile + ((size_t)idx[u][j] << logW) + wa);
-                                c[u][j] = ldg16(a.codes + code_pos(idx[u][j]));
-                            }
-                            if (nx + U_LIST < nq) {
-#pragma unroll
-                                for (int j = 0; j < 4; ++j)
-                                    idx[u][j] = pr[(size_t)(nx + U_LIST) * qs + ((uint32_t)j << logR)];
-                            }
+                        QG_USE_DATA(u)
+                        if (i + u + U < nq) {
+                            QG_LOAD_DATA(u)
+                            if (i + u + 2 * U < nq) QG_LOAD_IDX(u)
                         }
                     }
                 }
+                pr += U * qs;
             }
+#undef QG_LOAD_IDX
+#undef QG_LOAD_DATA
+#undef QG_USE_DATA
         }
         q += epoch;
         col_rows += 4 * epoch;
     }
     __syncthreads();
-    flush_local<WIDE>(hp, td, a.nb, pass, out);
+    flush_local<WIDE>(hp, td, logW, a.nb, pass, out);
 }
 
-// Sums the partial histograms of every tile that was built by more than one CTA.
+// Sums the partial histograms of every tile that was built by more than one CTA.  A block takes
+// 32 consecutive partial entries; its eight thread groups each add every eighth partial.
 __global__ void __launch_bounds__(256) k_hist_reduce(const TileDesc *__restrict__ tiles, uint32_t n, int nb,
                                                      const unsigned long long *__restrict__ partial,
                                                      unsigned long long *__restrict__ hist) {
@@ -368,16 +406,32 @@ __global__ void __launch_bounds__(256) k_hist_reduce(const TileDesc *__restrict_
     const int W = 1 << td.logW;
     const uint32_t total = 4u * nb * W;
     const size_t stride = (size_t)4 * nb * 32;
-    for (uint32_t e = blockIdx.x * 256 + threadIdx.x; e < total; e += gridDim.x * 256) {
-        const uint32_t a = e & (W - 1);
-        const uint32_t kb = e >> td.logW;          // k * nb + bin
-        const uint32_t k = kb / nb, bin = kb - k * nb;
-        const uint32_t fl = 4 * a + k;
-        if (fl >= (uint32_t)td.nf) continue;
-        const unsigned long long *p = partial + (size_t)td.cta0 * stride + e;
+    __shared__ unsigned long long acc[8][32];
+    const uint32_t ex = threadIdx.x & 31, pg = threadIdx.x >> 5;
+    for (uint32_t e0 = blockIdx.x * 32; e0 < total; e0 += gridDim.x * 32) {
+        const uint32_t e = e0 + ex;
         unsigned long long s = 0;
-        for (uint32_t i = 0; i < P; ++i) s += p[i * stride];
-        hist[(size_t)(td.f0 + fl) * nb + bin] = s;
+        if (e < total) {
+            const unsigned long long *p = partial + (size_t)td.cta0 * stride + e;
+            uint32_t i = pg;
+            for (; i + 24 < P; i += 32) {
+                const unsigned long long x0 = p[(size_t)i * stride], x1 = p[(size_t)(i + 8) * stride];
+                const unsigned long long x2 = p[(size_t)(i + 16) * stride], x3 = p[(size_t)(i + 24) * stride];
+                s += (x0 + x1) + (x2 + x3);
+            }
+            for (; i < P; i += 8) s += p[(size_t)i * stride];
+        }
+        acc[pg][ex] = s;
+        __syncthreads();
+        if (pg == 0 && e < total) {
+            for (int g = 1; g < 8; ++g) s += acc[g][ex];
+            const uint32_t a = e & (W - 1);
+            const uint32_t kb = e >> td.logW;          // k * nb + bin
+            const uint32_t k = kb / nb, bin = kb - k * nb;
+            const uint32_t fl = 4 * a + k;
+            if (fl < (uint32_t)td.nf) hist[(size_t)(td.f0 + fl) * nb + bin] = s;
+        }
+        __syncthreads();
     }
 }
 
@@ -389,16 +443,37 @@ __global__ void k_subtract(const unsigned long long *__restrict__ parent, const 
         large[i] = parent[i] - small[i];
 }
 
-template <bool WIDE, bool LIST>
-int launch_hist(qgbdt_ctx *c, const HistArgs &args, cudaStream_t st) {
-    auto kern = k_hist<WIDE, LIST>;
+template <int LOGW_T, bool WIDE, bool LIST>
+int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st) {
+    auto kern = k_hist<LOGW_T, WIDE, LIST>;
     static bool configured = false;   // per instantiation
     if (!configured) {
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
         configured = true;
     }
-    kern<<<(unsigned)c->hist_grid, HIST_THREADS, HIST_SMEM, st>>>(args);
+    const dim3 grid(effective_parts((uint32_t)c->max_parts, args.n), (unsigned)n_tiles);
+    kern<<<grid, HIST_THREADS, HIST_SMEM, st>>>(args);
     QG_LAUNCH_CHECK(c);
+    return QGBDT_OK;
+}
+
+// One launch per run of tiles of equal width (the full 128-feature tiles, then the remainder).
+template <bool WIDE, bool LIST>
+int launch_hist(qgbdt_ctx *c, HistArgs args, cudaStream_t st) {
+    const int T = (int)c->tiles.size();
+    for (int t0 = 0; t0 < T;) {
+        int t1 = t0 + 1;
+        while (t1 < T && c->tiles[t1].logW == c->tiles[t0].logW) ++t1;
+        args.tile0 = t0;
+        int rc;
+        switch (c->tiles[t0].logW) {
+            case 5: rc = launch_one<5, WIDE, LIST>(c, args, t1 - t0, st); break;
+            case 3: rc = launch_one<3, WIDE, LIST>(c, args, t1 - t0, st); break;
+            default: rc = launch_one<-1, WIDE, LIST>(c, args, t1 - t0, st); break;
+        }
+        if (rc != QGBDT_OK) return rc;
+        t0 = t1;
+    }
     return QGBDT_OK;
 }
 
@@ -422,8 +497,9 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
 
     HistArgs a;
     a.tiles = c->d_tiles;
-    a.cta_map = c->d_cta_map;
     a.codes = reinterpret_cast<const uint16_t *>(c->d_codes);
+    a.codes_nat = reinterpret_cast<const uint16_t *>(c->d_codes_nat);
+    a.tile0 = 0;
     a.rows = d_rows;
     a.off = (uint32_t)off;
     a.n = (uint32_t)n;
@@ -463,7 +539,7 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
     }
     if (rc != QGBDT_OK) return rc;
     if (c->max_parts > 1 && effective_parts((uint32_t)c->max_parts, (uint32_t)n) > 1) {
-        const dim3 grid((unsigned)((4 * c->nb * 32 + 255) / 256), (unsigned)c->tiles.size());
+        const dim3 grid((unsigned)((4 * c->nb * 32 + 31) / 32), (unsigned)c->tiles.size());
         k_hist_reduce<<<grid, 256, 0, st>>>(c->d_tiles, (uint32_t)n, c->nb, c->d_partial, d_hist);
         QG_LAUNCH_CHECK(c);
     }

@@ -26,8 +26,8 @@
 // histogram kernel reads the codes of its four rows with one 8-byte load.
 //
 // Histogram plan: every tile owns `parts` consecutive CTAs starting at `cta0` (in
-// proportion to its width); cta_map[cta] = (tile, part).  A build of n rows uses the
-// first min(parts, ceil(n / 4096)) of them.
+// proportion to its width); the grid is (part, tile).  A build of n rows uses the first
+// min(parts, ceil(n / 4096)) parts of every tile.
 //
 // Row lists: one uint32 array of N entries; leaf l owns [leaf_off[l], +leaf_n[l]).
 // ---------------------------------------------------------------------------
@@ -71,12 +71,12 @@ struct qgbdt_ctx {
     bool loaded = false;
     std::vector<TileDesc> tiles;
     TileDesc *d_tiles = nullptr;
-    int2 *d_cta_map = nullptr;               // [hist_grid]
     int hist_grid = 0, max_parts = 1;
     unsigned long long *d_partial = nullptr;  // [hist_grid][4][nb][32] partial histograms (only if max_parts > 1)
     std::vector<void *> tile_allocs;
     // quantized gradients
-    uint8_t *d_codes = nullptr;  // [round_up(N, 16)] 16-bit codes
+    uint8_t *d_codes = nullptr;  // [round_up(N, 16)] 16-bit codes, transposed inside blocks of 16 rows
+    uint8_t *d_codes_nat = nullptr;  // [N] the same codes in row order (read through row lists)
     int code_bytes = 2;
     bool quantized = false;
     bool const_hess = false;

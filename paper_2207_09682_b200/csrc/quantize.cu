@@ -128,7 +128,7 @@ __device__ inline int round_level(float x, int rounding, uint32_t u) {
 // and adds the integer totals (one atomic pair per block).
 __global__ void k_quantize(const float *__restrict__ g, const float *__restrict__ h, long long n, int kg, int kh,
                            int rounding, uint32_t key, DevState *state, uint8_t *__restrict__ codes,
-                           int8_t *__restrict__ gq_out, uint8_t *__restrict__ hq_out) {
+                           uint16_t *__restrict__ codes_nat, int8_t *__restrict__ gq_out, uint8_t *__restrict__ hq_out) {
     const float gmax = __uint_as_float(state->gmax_bits);
     const float hmax = h ? __uint_as_float(state->hmax_bits) : 1.0f;
     const float inv_g = gmax > 0.f ? __fdiv_rn((float)kg, gmax) : 0.f;
@@ -150,7 +150,9 @@ __global__ void k_quantize(const float *__restrict__ g, const float *__restrict_
         }
         // 4 x 4 transposed inside blocks of 16 rows (see the layout notes of the internal header)
         const long long pos = (i & ~15LL) | ((i & 3) << 2) | ((i >> 2) & 3);
-        reinterpret_cast<uint16_t *>(codes)[pos] = (uint16_t)(((gq & 0xFF) << 8) | hq);
+        const uint16_t code = (uint16_t)(((gq & 0xFF) << 8) | hq);
+        reinterpret_cast<uint16_t *>(codes)[pos] = code;
+        codes_nat[i] = code;
         if (gq_out) gq_out[i] = (int8_t)gq;
         if (hq_out) hq_out[i] = (uint8_t)hq;
         sg += gq;
@@ -216,8 +218,8 @@ int qg_quantize(qgbdt_ctx *c, const float *d_g, const float *d_h, uint32_t tree,
     const uint32_t key = mix32(mix32(mix32(seed_lo ^ 0x6A09E667u) + seed_hi) ^ tree);
     const int kg = qg_levels_g(c->prm.bits), kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
     const unsigned grid = grid_for(c, c->N, 256, 8);
-    k_quantize<<<grid, 256, 0, st>>>(d_g, d_h, c->N, kg, kh, c->prm.rounding, key, c->d_state, c->d_codes, d_gq,
-                                     d_hq);
+    k_quantize<<<grid, 256, 0, st>>>(d_g, d_h, c->N, kg, kh, c->prm.rounding, key, c->d_state, c->d_codes,
+                                     reinterpret_cast<uint16_t *>(c->d_codes_nat), d_gq, d_hq);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
 }

@@ -101,34 +101,27 @@ void plan_tiles(int F, std::vector<TileDesc> &out) {
     }
 }
 
-// Histogram plan: CTAs are shared out among the tiles in proportion to their width in words
-// (the cost of a row is one warp instruction slot per 32 words); with more tiles than SMs every
-// tile gets one CTA.  Fills parts / cta0 of the tiles; part p of a tile owns partial-histogram slot cta0 + p.
+// Histogram plan.  Tiles of equal width form a group that is built by one launch (the full
+// 128-feature tiles, then the remainder tiles); a group's tiles share the SMs equally, and with
+// more tiles than SMs every tile gets one CTA.  Fills parts / cta0 of the tiles; part p of a tile
+// owns partial-histogram slot cta0 + p.
 void plan_hist_ctas(int sm_count, std::vector<TileDesc> &tiles, int &n_ctas, int &max_parts) {
     const int T = (int)tiles.size();
-    long long total_w = 0;
-    for (const TileDesc &t : tiles) total_w += 1 << t.logW;
-    int used = 0;
-    for (TileDesc &t : tiles) {
-        long long p = T >= sm_count ? 1 : (long long)sm_count * (1 << t.logW) / total_w;
-        t.parts = (int)(p < 1 ? 1 : p);
-        used += t.parts;
-    }
-    // hand the CTAs left over by the rounding to the tiles with the most words per part
-    while (T < sm_count && used < sm_count) {
-        int best = 0;
-        for (int i = 1; i < T; ++i)
-            if ((long long)(1 << tiles[i].logW) * tiles[best].parts > (long long)(1 << tiles[best].logW) * tiles[i].parts)
-                best = i;
-        tiles[best].parts++;
-        used++;
-    }
     n_ctas = 0;
     max_parts = 1;
-    for (int i = 0; i < T; ++i) {
-        tiles[i].cta0 = n_ctas;
-        n_ctas += tiles[i].parts;
-        if (tiles[i].parts > max_parts) max_parts = tiles[i].parts;
+    for (int t0 = 0; t0 < T;) {
+        int t1 = t0 + 1;
+        while (t1 < T && tiles[t1].logW == tiles[t0].logW) ++t1;
+        const int g = t1 - t0;
+        for (int i = t0; i < t1; ++i) {
+            int p = sm_count / g + (i - t0 < sm_count % g ? 1 : 0);
+            if (p < 1) p = 1;
+            tiles[i].parts = p;
+            tiles[i].cta0 = n_ctas;
+            n_ctas += p;
+            if (p > max_parts) max_parts = p;
+        }
+        t0 = t1;
     }
 }
 

@@ -24,8 +24,8 @@
 //
 // Local bin width: B <= 5 uses one 32-bit word per bin, gradient sum in the high 16 bits
 // (signed), hessian sum in the low 16 bits; the CTA flushes before any column can have added
-// more rows than fit.  B >= 6 uses one 64-bit word per bin (32+32) and two passes over the
-// rows, each pass taking two of the four bytes of a word.
+// more rows than fit.  B >= 6 uses two 32-bit words per bin (32+32, a hessian plane and a gradient
+// plane) and two passes over the rows, each pass taking two of the four bytes of a word.
 #include "qgbdt_internal.cuh"
 
 namespace {
@@ -65,13 +65,6 @@ __device__ __forceinline__ void red32(uint32_t addr, int v) {
     asm volatile("red.shared.add.u32 [%0+%1], %2;" ::"r"(addr), "n"(IMM), "r"(v) : "memory");
 }
 
-template <int IMM>
-__device__ __forceinline__ void red64(uint32_t addr, uint32_t lo, uint32_t hi) {
-    asm volatile("{ .reg .b64 t; mov.b64 t, {%2, %3}; red.shared.add.u64 [%0+%1], t; }" ::"r"(addr), "n"(IMM),
-                 "r"(lo), "r"(hi)
-                 : "memory");
-}
-
 __device__ __forceinline__ uint32_t ldg32(const uint32_t *p) {
     uint32_t v;
     asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
@@ -102,11 +95,15 @@ __device__ __forceinline__ void add_word(uint32_t base, uint32_t w, uint32_t c, 
         red32<65536>(prmt(w, base, 0x7624u), inc);
         red32<65536 + 128>(prmt(w, base, 0x7634u), inc);
     } else {
-        const uint32_t lo = prmt(c, 0u, half ? 0x4442u : 0x4440u);   // h
-        const uint32_t hi = prmt(c, 0u, half ? 0xBBB3u : 0x9991u);   // g, sign-extended
+        // 32+32 local bins: the hessian plane at +0 and the gradient plane at +128 of a bin's 256 bytes
+        const int h = (int)prmt(c, 0u, half ? 0x4442u : 0x4440u);
+        const int g = (int)prmt(c, 0u, half ? 0xBBB3u : 0x9991u);   // sign-extended
         const uint32_t s0 = 0x7604u | ((uint32_t)(2 * pass) << 4), s1 = s0 + 0x10u;
-        red64<0>(prmt(w, base, s0), lo, hi);
-        red64<65536>(prmt(w, base, s1), lo, hi);
+        const uint32_t a0 = prmt(w, base, s0), a1 = prmt(w, base, s1);
+        red32<0>(a0, h);
+        red32<128>(a0, g);
+        red32<65536>(a1, h);
+        red32<65536 + 128>(a1, g);
     }
 }
 
@@ -148,13 +145,17 @@ __device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, 
                 }
                 v = (unsigned long long)((long long)G * 4294967296LL + (long long)H);
             } else {
-                // packed 32+32 words add up as they are: no field can overflow (checked at load time)
-                unsigned long long *p = reinterpret_cast<unsigned long long *>(hp) + kk * 8192 + bin * 32 + a * R;
-                v = 0;
+                // two 32-bit planes per bin; no field can overflow (checked at load time)
+                int *p = hp + kk * 16384 + bin * 64 + a * R;
+                long long G = 0;
+                unsigned long long H = 0;
                 for (int r = 0; r < R; ++r) {
-                    v += p[r];
-                    p[r] = 0ull;
+                    H += (unsigned int)p[r];
+                    G += p[32 + r];
+                    p[r] = 0;
+                    p[32 + r] = 0;
                 }
+                v = (unsigned long long)(G * 4294967296LL + (long long)H);
             }
             const int fl = 4 * a + k;
             if (fl < td.nf) {
@@ -213,7 +214,7 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     const uint32_t R = 1u << logR;
     const uint32_t wa = lane >> logR;           // word of the row held by this lane
     const uint32_t slot = lane & (R - 1);       // row slot of this lane (adjacent lanes: replicas of a column)
-    const uint32_t base = h0 + lane * (WIDE ? 8 : 4);
+    const uint32_t base = h0 + lane * 4;
     const uint32_t *tile = td.data;
     const int pass = a.pass;
 
@@ -451,7 +452,10 @@ int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st)
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
         configured = true;
     }
-    const dim3 grid(effective_parts((uint32_t)c->max_parts, args.n), (unsigned)n_tiles);
+    int group_parts = 1;
+    for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
+        if (c->tiles[t].parts > group_parts) group_parts = c->tiles[t].parts;
+    const dim3 grid(effective_parts((uint32_t)group_parts, args.n), (unsigned)n_tiles);
     kern<<<grid, HIST_THREADS, HIST_SMEM, st>>>(args);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;

@@ -25,8 +25,8 @@
 // code of row 16 b + 4 j + s sits at position 16 b + 4 s + j), so that a lane of the
 // histogram kernel reads the codes of its four rows with one 8-byte load.
 //
-// Histogram plan: every tile owns `parts` consecutive CTAs starting at `cta0` (in
-// proportion to its width); the grid is (part, tile).  A build of n rows uses the first
+// Histogram plan: tiles of equal width are built by one launch and share the SMs equally;
+// a tile owns `parts` partial-histogram slots starting at `cta0`; the grid is (part, tile).  A build of n rows uses the first
 // min(parts, ceil(n / 4096)) parts of every tile.
 //
 // Row lists: one uint32 array of N entries; leaf l owns [leaf_off[l], +leaf_n[l]).

@@ -60,6 +60,18 @@ void free_data(qgbdt_ctx *c) {
     dev_free(c->d_g);
     dev_free(c->d_h);
     dev_free(c->d_hist_pool);
+    dev_free(c->d_leaves);
+    dev_free(c->d_cand);
+    dev_free(c->d_feat_tile);
+    dev_free(c->d_m_num_leaves);
+    dev_free(c->d_m_feature);
+    dev_free(c->d_m_bin);
+    dev_free(c->d_m_left);
+    dev_free(c->d_m_right);
+    dev_free(c->d_m_gain);
+    dev_free(c->d_m_leaf_value);
+    dev_free(c->d_m_leaf_count);
+    c->model_cap = 0;
     c->loaded = false;
     c->quantized = false;
 }
@@ -184,7 +196,14 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     if ((rc = dev_alloc(c, &c->d_codes_nat, (size_t)n_rows * 2 + 16)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx, (size_t)n_rows)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx_tmp, (size_t)n_rows)) != QGBDT_OK) return rc;
-    if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8 + (size_t)c->sm_count * 32)) != QGBDT_OK) return rc;
+    {
+        std::vector<int32_t> ft((size_t)n_features);
+        for (size_t t = 0; t < c->tiles.size(); ++t)
+            for (int f = c->tiles[t].f0; f < c->tiles[t].f0 + c->tiles[t].nf; ++f) ft[f] = (int32_t)t;
+        if ((rc = dev_alloc(c, &c->d_feat_tile, (size_t)n_features)) != QGBDT_OK) return rc;
+        QG_CUDA(c, cudaMemcpy(c->d_feat_tile, ft.data(), sizeof(int32_t) * ft.size(), cudaMemcpyHostToDevice));
+    }
     if ((rc = dev_alloc(c, &c->d_part_bits, ((size_t)n_rows + 2048) / 32 + 64)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_feat_best, (size_t)n_features)) != QGBDT_OK) return rc;
     QG_CUDA(c, cudaMemsetAsync(c->d_state, 0, sizeof(DevState), st));
@@ -244,7 +263,7 @@ int qgbdt_create(qgbdt_ctx **out, const qgbdt_params *p) {
     bool ok = cudaMalloc(reinterpret_cast<void **>(&c->d_state), sizeof(DevState)) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_split_out), sizeof(SplitRec) * 4) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_sums), sizeof(long long) * 2 * L) == cudaSuccess &&
-              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_table), sizeof(uint32_t) * 2 * L) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_table), sizeof(uint32_t) * 3 * L) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_value), sizeof(float) * L) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_w), sizeof(double) * L) == cudaSuccess &&
               cudaMallocHost(&c->h_pinned, PINNED_BYTES) == cudaSuccess;
@@ -261,6 +280,7 @@ int qgbdt_destroy(qgbdt_ctx *c) {
     if (!c) return QGBDT_ERR_ARG;
     free_data(c);
     dev_free(c->d_state);
+    dev_free(c->d_gs);
     dev_free(c->d_split_out);
     dev_free(c->d_leaf_sums);
     dev_free(c->d_leaf_table);
@@ -306,7 +326,7 @@ int qgbdt_compute_gradients(qgbdt_ctx *c, const float *d_scores, const float *d_
     if (rc != QGBDT_OK) return rc;
     if (!d_scores || !d_labels || !d_g || (c->prm.objective == 0 && !d_h))
         return qg_fail(c, QGBDT_ERR_ARG, "null pointer");
-    return qg_gradients(c, d_scores, d_labels, d_g, d_h, false, (cudaStream_t)stream);
+    return qg_gradients(c, d_scores, d_labels, d_g, d_h, false, false, (cudaStream_t)stream);
 }
 
 int qgbdt_quantize_gradients(qgbdt_ctx *c, const float *d_g, const float *d_h, uint32_t tree, int8_t *d_gq,

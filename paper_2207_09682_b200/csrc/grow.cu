@@ -1,0 +1,390 @@
+// Leaf-wise (best-first) growth of one tree (Sec. 3) with every decision taken on the device:
+// the host enqueues a fixed sequence of kernels per split and never waits for a result.
+//
+// Per split: (1) k_grow_flags: one predicate bit per row of the leaf being split and the number
+// of left rows per warp range; (2) k_grow_scatter: stable scatter of the row indices into the
+// other index buffer (left rows first); (3) the histogram kernel on the smaller child's rows
+// (Algorithm 1); (4) k_grow_finish: per feature, the smaller child's histogram from the partial
+// histograms, the larger child's as parent minus smaller, both children's best splits (Eq. 7);
+// the last block to finish records the split in the tree, creates the leaf records and picks
+// the leaf with the largest gain for the next split.
+#include "split_scan.cuh"
+
+namespace {
+
+constexpr int PART_THREADS = 256;
+constexpr int PART_WARPS = PART_THREADS / 32;
+constexpr int FIN_WARPS = 8;
+constexpr uint32_t MIN_ROWS_PER_CTA = 4096;   // same rule as the histogram kernel
+
+__device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
+    uint32_t want = (n + MIN_ROWS_PER_CTA - 1) / MIN_ROWS_PER_CTA;
+    if (want < 1) want = 1;
+    return want < parts ? want : parts;
+}
+
+struct GrowArgs {
+    GrowState *gs;
+    LeafRec *leaves;
+    const DevState *state;
+    const TileDesc *tiles;
+    const int32_t *feat_tile;
+    uint32_t *idx0, *idx1;           // the two row-index buffers
+    uint32_t *bits, *counts;         // predicate bits of the leaf being split, left rows per warp range
+    int n_count;                     // warp ranges (= warps of the flag / scatter grids)
+    unsigned long long *pool;        // [L][F][nb]
+    const unsigned long long *partial;
+    SplitRec *cand;                  // [finish blocks][2]
+    int F, nb, L;
+    SplitParams sp;                  // G, H, n_s are filled per leaf on the device
+    // tree output (device arrays of the current tree)
+    int32_t *m_feature, *m_bin, *m_left, *m_right;
+    double *m_gain;
+};
+
+__global__ void k_grow_begin(GrowState *gs, LeafRec *leaves, const DevState *state, uint32_t N) {
+    LeafRec r;
+    r.off = 0; r.n = N; r.buf = -1; r.slot = 0;
+    r.G = state->tot_g; r.H = state->tot_h;
+    r.best = qg_invalid_rec();
+    r.parent_node = -1; r.parent_side = 0;
+    leaves[0] = r;
+    gs->n_leaves = 1;
+    gs->done = 0;
+    gs->finish_count = 0;
+}
+
+// Words of 32 rows [w0, w1) of warp gw when nw words are shared out among n_count warps.
+__device__ inline void warp_range(uint32_t nw, uint32_t gw, uint32_t n_count, uint32_t &w0, uint32_t &w1) {
+    w0 = (uint32_t)((unsigned long long)nw * gw / n_count);
+    w1 = (uint32_t)((unsigned long long)nw * (gw + 1) / n_count);
+}
+
+__global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
+    const GrowState *gs = a.gs;
+    if (gs->done) return;
+    const int lane = threadIdx.x & 31;
+    const uint32_t gw = blockIdx.x * PART_WARPS + (threadIdx.x >> 5);
+    const uint32_t n = gs->n, off = gs->off;
+    const uint32_t nw = (n + 31) >> 5;
+    uint32_t w0, w1;
+    warp_range(nw, gw, (uint32_t)a.n_count, w0, w1);
+    const uint32_t *src = gs->buf < 0 ? nullptr : (gs->buf ? a.idx1 : a.idx0);
+    const TileDesc td = a.tiles[gs->tile];
+    const uint32_t *col = td.data + gs->word;
+    const int logW = td.logW, shift = 8 * gs->byte;
+    const uint32_t thr = (uint32_t)gs->bin;
+    uint32_t lefts = 0;
+    for (uint32_t w = w0; w < w1; ++w) {
+        const uint32_t e = (w << 5) + lane;
+        bool left = false;
+        if (e < n) {
+            const uint32_t row = src ? src[off + e] : off + e;
+            left = ((col[(size_t)row << logW] >> shift) & 0xFFu) <= thr;
+        }
+        const uint32_t b = __ballot_sync(0xffffffffu, left);
+        if (lane == 0) a.bits[w] = b;
+        lefts += __popc(b);
+    }
+    if (lane == 0) a.counts[gw] = lefts;
+}
+
+__global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
+    GrowState *gs = a.gs;
+    if (gs->done) return;
+    const int lane = threadIdx.x & 31;
+    const uint32_t gw = blockIdx.x * PART_WARPS + (threadIdx.x >> 5);
+    const uint32_t n = gs->n, off = gs->off;
+    const uint32_t nw = (n + 31) >> 5;
+    uint32_t w0, w1;
+    warp_range(nw, gw, (uint32_t)a.n_count, w0, w1);
+    if (w1 <= w0 && gw != 0) return;
+    // left rows before this warp's range, and in the whole leaf
+    uint32_t before = 0, total = 0;
+    for (uint32_t j = lane; j < (uint32_t)a.n_count; j += 32) {
+        const uint32_t v = a.counts[j];
+        total += v;
+        if (j < gw) before += v;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, o);
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+    }
+    if (gw == 0 && lane == 0) gs->nl = total;
+    const uint32_t *src = gs->buf < 0 ? nullptr : (gs->buf ? a.idx1 : a.idx0);
+    uint32_t *dst = gs->buf == 0 ? a.idx1 : a.idx0;
+    for (uint32_t w = w0; w < w1; ++w) {
+        const uint32_t bw = a.bits[w];
+        const uint32_t e = (w << 5) + lane;
+        if (e < n) {
+            const uint32_t row = src ? src[off + e] : off + e;
+            const uint32_t rank_l = __popc(bw & ((1u << lane) - 1u));
+            const bool left = (bw >> lane) & 1u;
+            const uint32_t dest = left ? before + rank_l : total + ((w << 5) - before) + (lane - rank_l);
+            dst[off + dest] = row;
+        }
+        before += __popc(bw);
+    }
+}
+
+__device__ inline SplitRec load_rec_cg(const SplitRec *p) {   // bypasses L1: written by another block of this kernel
+    const long long *q = reinterpret_cast<const long long *>(p);
+    long long v[5];
+#pragma unroll
+    for (int i = 0; i < 5; ++i) v[i] = __ldcg(q + i);
+    SplitRec r;
+    memcpy(&r, v, sizeof(r));
+    return r;
+}
+static_assert(sizeof(SplitRec) == 40, "SplitRec is copied as five 64-bit words");
+
+// ROOT: scans the root histogram (pool slot 0).  Otherwise: completes the split recorded in the
+// grow state.  One warp per feature.
+template <bool ROOT>
+__global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
+    GrowState *gs = a.gs;
+    if (gs->done) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int f = blockIdx.x * FIN_WARPS + warp;
+    const int n_leaves = gs->n_leaves;
+    const size_t hw = (size_t)a.F * a.nb;
+
+    // the two children: "small" was built by Algorithm 1, "large" is parent - small
+    const uint32_t n = ROOT ? a.leaves[0].n : gs->n, nl = ROOT ? n : gs->nl, nr = n - nl;
+    const bool small_is_left = nl <= nr;
+    SplitParams pS = a.sp, pL = a.sp;
+    if (ROOT) {
+        pS.G = a.leaves[0].G; pS.H = a.leaves[0].H; pS.n_s = n;
+    } else {
+        const long long gl = gs->gl, hl = gs->hl, gr = gs->PG - gl, hr = gs->PH - hl;
+        pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl : nr;
+        pL.G = small_is_left ? gr : gl; pL.H = small_is_left ? hr : hl; pL.n_s = small_is_left ? nr : nl;
+    }
+    SplitRec rS = qg_invalid_rec(), rL = qg_invalid_rec();
+    if (f < a.F) {
+        double dg, dh;
+        qg_scales(a.state, pS, dg, dh);
+        const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
+        const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
+        const TileDesc td = a.tiles[a.feat_tile[f]];
+        const int fl = f - td.f0, W = 1 << td.logW;
+        const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)td.parts, (uint32_t)pS.n_s);
+        const size_t pstride = (size_t)4 * a.nb * 32;
+        const unsigned long long *part = a.partial + (size_t)td.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
+        unsigned long long *S = a.pool + (ROOT ? 0 : (size_t)n_leaves * hw) + (size_t)f * a.nb;
+        unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)gs->parent_slot * hw + (size_t)f * a.nb;
+        ScanState scS, scL;
+        qg_scan_init(scS);
+        qg_scan_init(scL);
+        for (int base = 0; base < a.nb; base += 32) {
+            const int b = base + lane;
+            unsigned long long s = 0, l = 0;
+            if (b < a.nb) {
+                if (ROOT) {
+                    s = S[b];
+                } else {
+                    if (P > 1) {
+                        const unsigned long long *q = part + (size_t)b * W;
+                        for (uint32_t i = 0; i < P; ++i) s += q[i * pstride];
+                        S[b] = s;
+                    } else {
+                        s = S[b];
+                    }
+                    l = Pp[b] - s;   // no field borrows: every child sum is at most the parent's
+                    Pp[b] = l;
+                }
+            }
+            qg_scan_step(scS, s, b, a.nb, pS, dg, dh, tpS);
+            if (!ROOT) qg_scan_step(scL, l, b, a.nb, pL, dg, dh, tpL);
+        }
+        rS = qg_scan_finish(scS, f);
+        if (!ROOT) rL = qg_scan_finish(scL, f);
+    }
+
+    // best of the block, then of the grid (last block through)
+    __shared__ SplitRec sm[2][FIN_WARPS * 32];
+    __shared__ bool is_last;
+    if (lane == 0) { sm[0][warp] = rS; sm[1][warp] = rL; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        SplitRec bS = sm[0][0], bL = sm[1][0];
+        for (int w = 1; w < FIN_WARPS; ++w) {
+            if (qg_rec_better(sm[0][w], bS)) bS = sm[0][w];
+            if (qg_rec_better(sm[1][w], bL)) bL = sm[1][w];
+        }
+        a.cand[2 * blockIdx.x] = bS;
+        a.cand[2 * blockIdx.x + 1] = bL;
+        __threadfence();
+        is_last = atomicAdd(&gs->finish_count, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    SplitRec bS = qg_invalid_rec(), bL = qg_invalid_rec();
+    for (int i = threadIdx.x; i < (int)gridDim.x; i += FIN_WARPS * 32) {
+        const SplitRec x = load_rec_cg(a.cand + 2 * i), y = load_rec_cg(a.cand + 2 * i + 1);
+        if (qg_rec_better(x, bS)) bS = x;
+        if (qg_rec_better(y, bL)) bL = y;
+    }
+    sm[0][threadIdx.x] = bS;
+    sm[1][threadIdx.x] = bL;
+    __syncthreads();
+    for (int st = FIN_WARPS * 16; st > 0; st >>= 1) {
+        if ((int)threadIdx.x < st) {
+            if (qg_rec_better(sm[0][threadIdx.x + st], sm[0][threadIdx.x])) sm[0][threadIdx.x] = sm[0][threadIdx.x + st];
+            if (qg_rec_better(sm[1][threadIdx.x + st], sm[1][threadIdx.x])) sm[1][threadIdx.x] = sm[1][threadIdx.x + st];
+        }
+        __syncthreads();
+    }
+    int leaves_now = n_leaves;
+    if (threadIdx.x == 0) {
+        bS = sm[0][0];
+        bL = sm[1][0];
+        if (ROOT) {
+            a.leaves[0].best = bS;
+        } else {
+            const int pick = gs->pick, right = n_leaves, node = n_leaves - 1;
+            const LeafRec par = a.leaves[pick];
+            a.m_feature[node] = gs->feature;
+            a.m_bin[node] = gs->bin;
+            a.m_left[node] = ~pick;
+            a.m_right[node] = ~right;
+            a.m_gain[node] = gs->gain;
+            if (par.parent_node >= 0) {
+                if (par.parent_side == 0) a.m_left[par.parent_node] = node;
+                else a.m_right[par.parent_node] = node;
+            }
+            const int dstbuf = gs->buf == 0 ? 1 : 0;
+            LeafRec lf, rt;
+            lf.off = par.off; lf.n = nl; lf.buf = dstbuf;
+            lf.G = gs->gl; lf.H = gs->hl;
+            lf.parent_node = node; lf.parent_side = 0;
+            rt.off = par.off + nl; rt.n = nr; rt.buf = dstbuf;
+            rt.G = gs->PG - gs->gl; rt.H = gs->PH - gs->hl;
+            rt.parent_node = node; rt.parent_side = 1;
+            lf.slot = small_is_left ? n_leaves : par.slot;
+            rt.slot = small_is_left ? par.slot : n_leaves;
+            lf.best = small_is_left ? bS : bL;
+            rt.best = small_is_left ? bL : bS;
+            a.leaves[pick] = lf;
+            a.leaves[right] = rt;
+            gs->n_leaves = n_leaves + 1;
+            gs->hist_rows += small_is_left ? nl : nr;
+            gs->hist_builds += 1;
+        }
+        gs->finish_count = 0;
+    }
+    if (!ROOT) leaves_now = n_leaves + 1;
+    __syncthreads();
+
+    // the next leaf to split: largest gain, lowest leaf number on equal gain
+    __shared__ double pg[FIN_WARPS * 32];
+    __shared__ int pi[FIN_WARPS * 32];
+    double bg = 0.0;
+    int bi = -1;
+    if (leaves_now < a.L) {
+        for (int i = threadIdx.x; i < leaves_now; i += FIN_WARPS * 32) {
+            const SplitRec &r = a.leaves[i].best;
+            if (r.valid && (bi < 0 || r.gain > bg)) { bg = r.gain; bi = i; }
+        }
+    }
+    pg[threadIdx.x] = bg;
+    pi[threadIdx.x] = bi;
+    __syncthreads();
+    for (int st = FIN_WARPS * 16; st > 0; st >>= 1) {
+        if ((int)threadIdx.x < st) {
+            const double og = pg[threadIdx.x + st];
+            const int oi = pi[threadIdx.x + st];
+            const int mi = pi[threadIdx.x];
+            if (oi >= 0 && (mi < 0 || og > pg[threadIdx.x] || (og == pg[threadIdx.x] && oi < mi))) {
+                pg[threadIdx.x] = og;
+                pi[threadIdx.x] = oi;
+            }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const int pick = pi[0];
+        if (pick < 0) {
+            gs->done = 1;
+        } else {
+            const LeafRec lr = a.leaves[pick];
+            const TileDesc td = a.tiles[a.feat_tile[lr.best.feature]];
+            const int fl = lr.best.feature - td.f0;
+            gs->pick = pick;
+            gs->feature = lr.best.feature;
+            gs->bin = lr.best.bin;
+            gs->tile = a.feat_tile[lr.best.feature];
+            gs->word = fl >> 2;
+            gs->byte = fl & 3;
+            gs->off = lr.off;
+            gs->n = lr.n;
+            gs->buf = lr.buf;
+            gs->gl = lr.best.gl;
+            gs->hl = lr.best.hl;
+            gs->PG = lr.G;
+            gs->PH = lr.H;
+            gs->gain = lr.best.gain;
+            gs->parent_slot = lr.slot;
+        }
+    }
+}
+
+}  // namespace
+
+// Grows the tree of boosting iteration slot `tree_slot` of the current train call.  Gradients must
+// have been quantized on the same stream (the state holds the totals and maxima).  Asynchronous.
+int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
+    const int L = c->prm.num_leaves;
+    GrowArgs a;
+    a.gs = c->d_gs;
+    a.leaves = c->d_leaves;
+    a.state = c->d_state;
+    a.tiles = c->d_tiles;
+    a.feat_tile = c->d_feat_tile;
+    a.idx0 = c->d_idx;
+    a.idx1 = c->d_idx_tmp;
+    a.bits = c->d_part_bits;
+    a.counts = c->d_part_counts;
+    const int part_blocks = c->sm_count * 4;
+    a.n_count = part_blocks * PART_WARPS;
+    a.pool = c->d_hist_pool;
+    a.partial = c->d_partial;
+    a.cand = c->d_cand;
+    a.F = c->F;
+    a.nb = c->nb;
+    a.L = L;
+    a.sp.G = a.sp.H = a.sp.n_s = 0;
+    a.sp.kg = qg_levels_g(c->prm.bits);
+    a.sp.kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
+    a.sp.const_h = c->const_hess ? 1 : 0;
+    a.sp.min_data = c->prm.min_data_in_leaf;
+    a.sp.min_sum_h = c->prm.min_sum_hessian;
+    a.sp.min_gain = c->prm.min_gain;
+    a.sp.lambda = c->prm.lambda_l2;
+    const size_t no = (size_t)tree_slot * (L > 1 ? L - 1 : 1);
+    a.m_feature = c->d_m_feature + no;
+    a.m_bin = c->d_m_bin + no;
+    a.m_left = c->d_m_left + no;
+    a.m_right = c->d_m_right + no;
+    a.m_gain = c->d_m_gain + no;
+
+    k_grow_begin<<<1, 1, 0, st>>>(c->d_gs, c->d_leaves, c->d_state, (uint32_t)c->N);
+    QG_LAUNCH_CHECK(c);
+    int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
+    if (rc != QGBDT_OK) return rc;
+    const unsigned fin_blocks = (unsigned)((c->F + FIN_WARPS - 1) / FIN_WARPS);
+    k_grow_finish<true><<<fin_blocks, FIN_WARPS * 32, 0, st>>>(a);
+    QG_LAUNCH_CHECK(c);
+    for (int split = 1; split < L; ++split) {
+        k_grow_flags<<<part_blocks, PART_THREADS, 0, st>>>(a);
+        QG_LAUNCH_CHECK(c);
+        k_grow_scatter<<<part_blocks, PART_THREADS, 0, st>>>(a);
+        QG_LAUNCH_CHECK(c);
+        if ((rc = qg_hist_grow(c, st)) != QGBDT_OK) return rc;
+        k_grow_finish<false><<<fin_blocks, FIN_WARPS * 32, 0, st>>>(a);
+        QG_LAUNCH_CHECK(c);
+    }
+    return QGBDT_OK;
+}

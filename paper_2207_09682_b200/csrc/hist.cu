@@ -42,6 +42,11 @@ struct HistArgs {
     const uint16_t *codes;         // per-row code (g8 << 8 | h8), transposed inside blocks of 16 rows
     const uint16_t *codes_nat;     // the same codes in row order (row lists and leftover rows)
     int tile0;                     // first tile of this launch
+    // tree growth: the rows are the smaller child of the split recorded in *gs (nullptr otherwise)
+    const GrowState *gs;
+    const uint32_t *idx0, *idx1;   // the two row-index buffers
+    unsigned long long *pool;      // histogram pool, slot stride F * nb words
+    size_t hist_words;
     const uint32_t *rows;          // row list, or nullptr: rows 0 .. n-1
     uint32_t off, n;               // list: entries rows[off .. off+n)
     int nb;
@@ -187,6 +192,17 @@ template <int LOGW_T, bool WIDE, bool LIST>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     extern __shared__ __align__(1024) int sh[];
     const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
+    if (LIST && a.gs) {
+        // the smaller child (ties: the left one) in the buffer the scatter kernel wrote; its
+        // histogram goes to the pool slot numbered like the leaf about to be created
+        const GrowState *gs = a.gs;
+        if (gs->done) return;
+        const uint32_t nl = gs->nl, nr = gs->n - nl;
+        a.rows = gs->buf == 0 ? a.idx1 : a.idx0;
+        a.off = nl <= nr ? gs->off : gs->off + nl;
+        a.n = nl <= nr ? nl : nr;
+        a.hist = a.pool + (size_t)gs->n_leaves * a.hist_words;
+    }
     const uint32_t n = a.n;
     const uint32_t P = effective_parts((uint32_t)td.parts, n);
     const uint32_t part = blockIdx.x;
@@ -232,9 +248,9 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
         const uint32_t b1 = (uint32_t)((unsigned long long)B * (part + 1) / P);
         first_unit = b0 << 2;
         if (logR >= 2) {                                             // a warp-unit is R / 4 whole blocks
-            const uint32_t bpw = R >> 2;
-            q1 = (b1 - b0) / bpw;
-            s0 = (b0 + q1 * bpw) << 4;
+            const int lb = logR >= 2 ? logR - 2 : 0;                 // log2 of blocks per warp-unit
+            q1 = (b1 - b0) >> lb;
+            s0 = (b0 + (q1 << lb)) << 4;
         } else {                                                     // 4 / R warp-units per block
             q1 = (b1 - b0) << (2 - logR);
             s0 = b1 << 4;
@@ -455,7 +471,7 @@ int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st)
     int group_parts = 1;
     for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
         if (c->tiles[t].parts > group_parts) group_parts = c->tiles[t].parts;
-    const dim3 grid(effective_parts((uint32_t)group_parts, args.n), (unsigned)n_tiles);
+    const dim3 grid(args.gs ? (unsigned)group_parts : effective_parts((uint32_t)group_parts, args.n), (unsigned)n_tiles);
     kern<<<grid, HIST_THREADS, HIST_SMEM, st>>>(args);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
@@ -504,6 +520,10 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
     a.codes = reinterpret_cast<const uint16_t *>(c->d_codes);
     a.codes_nat = reinterpret_cast<const uint16_t *>(c->d_codes_nat);
     a.tile0 = 0;
+    a.gs = nullptr;
+    a.idx0 = a.idx1 = nullptr;
+    a.pool = nullptr;
+    a.hist_words = 0;
     a.rows = d_rows;
     a.off = (uint32_t)off;
     a.n = (uint32_t)n;
@@ -549,6 +569,59 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
     }
     if (ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
     return QGBDT_OK;
+}
+
+// Histogram of the smaller child of the split recorded in the grow state (sizes known only on
+// the device): partial histograms or, for a small child, the finished histogram in its pool slot.
+int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
+    const int bits = c->prm.bits;
+    const int kg = qg_levels_g(bits);
+    const int kh = c->const_hess ? 1 : qg_levels_h(bits, c->prm.hess_levels_mode);
+    HistArgs a;
+    a.tiles = c->d_tiles;
+    a.codes = reinterpret_cast<const uint16_t *>(c->d_codes);
+    a.codes_nat = reinterpret_cast<const uint16_t *>(c->d_codes_nat);
+    a.tile0 = 0;
+    a.gs = c->d_gs;
+    a.idx0 = c->d_idx;
+    a.idx1 = c->d_idx_tmp;
+    a.pool = c->d_hist_pool;
+    a.hist_words = (size_t)c->F * c->nb;
+    a.rows = nullptr;
+    a.off = 0;
+    a.n = 0;
+    a.nb = c->nb;
+    a.hist = nullptr;
+    a.partial = c->d_partial;
+    const uint32_t by_h = 65535u / (uint32_t)kh, by_g = 32767u / (uint32_t)kg;
+    a.flush_rows = by_h < by_g ? by_h : by_g;
+    a.pass = 0;
+    a.state = c->d_state;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (c->profile_hist) {
+        if (c->hist_events_used + 2 > c->hist_events.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                QG_CUDA(c, cudaEventCreate(&e));
+                c->hist_events.push_back(e);
+            }
+        }
+        ev0 = c->hist_events[c->hist_events_used++];
+        ev1 = c->hist_events[c->hist_events_used++];
+        QG_CUDA(c, cudaEventRecord(ev0, st));
+    }
+    int rc;
+    if (bits < 6) {
+        rc = launch_hist<false, true>(c, a, st);
+    } else {
+        rc = launch_hist<true, true>(c, a, st);
+        if (rc == QGBDT_OK) {
+            a.pass = 1;
+            rc = launch_hist<true, true>(c, a, st);
+        }
+    }
+    if (rc == QGBDT_OK && ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
+    return rc;
 }
 
 int qg_subtract(qgbdt_ctx *c, const unsigned long long *d_parent, const unsigned long long *d_small,

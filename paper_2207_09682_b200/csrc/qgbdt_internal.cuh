@@ -60,6 +60,34 @@ struct SplitRec {
     int valid, pad;
 };
 
+// One leaf of the tree being grown (device memory).  Its rows are entries [off, off + n) of the
+// row-index buffer `buf` (0 or 1; -1: the identity list of the root).
+struct LeafRec {
+    uint32_t off, n;
+    int32_t buf;
+    int32_t slot;            // histogram slot in the pool
+    long long G, H;          // integer gradient / hessian totals
+    SplitRec best;           // best split of the leaf
+    int32_t parent_node, parent_side;
+};
+
+// State of leaf-wise growth kept on the device, so that a tree grows without the host looking:
+// the split being executed and counters.
+struct GrowState {
+    int32_t n_leaves, done;
+    int32_t pick, feature, bin;      // leaf being split and its winning candidate
+    int32_t tile, word, byte;        // where the split feature sits in the tiled matrix
+    uint32_t off, n;                 // rows of the leaf being split
+    int32_t buf;                     // their index buffer
+    uint32_t nl;                     // rows that go left (written by the scatter kernel)
+    long long gl, hl, PG, PH;        // left totals of the candidate, totals of the leaf
+    double gain;
+    int32_t parent_slot;
+    unsigned int finish_count;       // blocks of the finishing kernel that are through
+    unsigned long long hist_rows;    // rows visited by histogram builds of row lists
+    unsigned long long hist_builds;
+};
+
 struct qgbdt_ctx {
     qgbdt_params prm;
     int device = 0;
@@ -100,6 +128,17 @@ struct qgbdt_ctx {
     // training buffers (allocated on first qgbdt_train)
     float *d_g = nullptr, *d_h = nullptr;
     unsigned long long *d_hist_pool = nullptr;  // [L][F][nb]
+    LeafRec *d_leaves = nullptr;                // [L]
+    GrowState *d_gs = nullptr;
+    SplitRec *d_cand = nullptr;                 // [finish blocks][2] per-block best candidates of the two children
+    int32_t *d_feat_tile = nullptr;             // [F] tile of every feature
+    // trees of the current qgbdt_train call, on the device until the call ends
+    int model_cap = 0;                          // trees the arrays below can hold
+    int32_t *d_m_num_leaves = nullptr, *d_m_feature = nullptr, *d_m_bin = nullptr, *d_m_left = nullptr,
+            *d_m_right = nullptr;
+    double *d_m_gain = nullptr;
+    float *d_m_leaf_value = nullptr;
+    long long *d_m_leaf_count = nullptr;
     // counters
     int64_t n_launches = 0, n_hist_builds = 0, n_hist_row_features = 0;
     // optional per-launch timing of the histogram kernel (event pairs on the launching stream)
@@ -139,7 +178,7 @@ int qg_iota(qgbdt_ctx *c, cudaStream_t st);
 
 // quantize.cu
 int qg_gradients(qgbdt_ctx *c, const float *d_scores, const float *d_labels, float *d_g, float *d_h,
-                 bool reduce_max, cudaStream_t st);
+                 bool reduce_max, bool clear_bad, cudaStream_t st);
 int qg_absmax(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st);
 int qg_quantize(qgbdt_ctx *c, const float *d_g, const float *d_h, uint32_t tree, int8_t *d_gq,
                 uint8_t *d_hq, cudaStream_t st);
@@ -160,3 +199,10 @@ int qg_partition(qgbdt_ctx *c, int64_t off, int64_t n, int feature, int bin, cud
 // refit.cu
 int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st);
 int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st);
+// the same two for a tree grown on the device (leaf table from the device leaf records)
+int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_scores, int tree_slot, cudaStream_t st);
+
+// grow.cu: one tree by leaf-wise growth, every decision taken on the device
+int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st);
+// hist.cu: histogram of the smaller child of the split recorded in the grow state
+int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st);

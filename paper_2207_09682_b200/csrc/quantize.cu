@@ -175,10 +175,12 @@ __global__ void k_quantize(const float *__restrict__ g, const float *__restrict_
     }
 }
 
-__global__ void k_reset_state(DevState *state) {
+// The out-of-domain flag is sticky over the trees of one train call: only the caller-facing
+// quantize call and the start of a train call clear it.
+__global__ void k_reset_state(DevState *state, int clear_bad) {
     state->gmax_bits = 0;
     state->hmax_bits = 0;
-    state->bad_value = 0;
+    if (clear_bad) state->bad_value = 0;
     state->tot_g = 0;
     state->tot_h = 0;
 }
@@ -193,9 +195,9 @@ inline unsigned grid_for(const qgbdt_ctx *c, long long n, int threads, int per_s
 }  // namespace
 
 int qg_gradients(qgbdt_ctx *c, const float *d_scores, const float *d_labels, float *d_g, float *d_h,
-                 bool reduce_max, cudaStream_t st) {
+                 bool reduce_max, bool clear_bad, cudaStream_t st) {
     if (reduce_max) {
-        k_reset_state<<<1, 1, 0, st>>>(c->d_state);
+        k_reset_state<<<1, 1, 0, st>>>(c->d_state, clear_bad ? 1 : 0);
         QG_LAUNCH_CHECK(c);
     }
     k_gradients<<<grid_for(c, c->N, 256, 8), 256, 0, st>>>(c->prm.objective, d_scores, d_labels, c->N, d_g, d_h,
@@ -205,7 +207,7 @@ int qg_gradients(qgbdt_ctx *c, const float *d_scores, const float *d_labels, flo
 }
 
 int qg_absmax(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st) {
-    k_reset_state<<<1, 1, 0, st>>>(c->d_state);
+    k_reset_state<<<1, 1, 0, st>>>(c->d_state, 1);
     QG_LAUNCH_CHECK(c);
     k_absmax<<<grid_for(c, c->N, 256, 8), 256, 0, st>>>(d_g, d_h, c->N, c->d_state);
     QG_LAUNCH_CHECK(c);

@@ -23,11 +23,24 @@ __device__ inline int slot_of(const uint32_t *offs, int n_leaves, uint32_t p) {
 __device__ inline long long to_fixed(float v) { return __double2ll_rn(__dmul_rn((double)v, 1073741824.0)); }
 
 // table: [n_leaves] offsets ascending, then [n_leaves] leaf ids.  sums: [n_leaves][2] by slot.
-__global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__restrict__ idx, uint32_t n,
+// gs != nullptr: a tree grown on the device: the leaf count comes from *gs and the table's third
+// part [n_leaves] says which index buffer holds a leaf's rows (-1: the identity list).
+__device__ inline uint32_t leaf_row(const uint32_t *idx0, const uint32_t *idx1, const uint32_t *table, int n_leaves,
+                                    bool grown, int s, uint32_t p) {
+    if (!grown) return idx0[p];
+    const int buf = (int)table[2 * n_leaves + s];
+    return buf < 0 ? p : (buf ? idx1[p] : idx0[p]);
+}
+
+__global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__restrict__ idx,
+                                                              const uint32_t *__restrict__ idx1, uint32_t n,
                                                               const uint32_t *__restrict__ table, int n_leaves,
-                                                              const float *__restrict__ g, const float *__restrict__ h,
+                                                              const GrowState *gs, const float *__restrict__ g,
+                                                              const float *__restrict__ h,
                                                               long long *__restrict__ sums) {
     extern __shared__ uint32_t offs[];  // n_leaves offsets
+    const bool grown = gs != nullptr;
+    if (grown) n_leaves = gs->n_leaves;
     __shared__ unsigned long long acc[REFIT_LOCAL][2];
     for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) offs[i] = table[i];
     for (int i = threadIdx.x; i < REFIT_LOCAL * 2; i += REFIT_THREADS) (&acc[0][0])[i] = 0ull;
@@ -44,7 +57,7 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__
         long long gf = 0, hf = 0;
         if (ok) {
             s = slot_of(offs, n_leaves, p);
-            const uint32_t row = idx[p];
+            const uint32_t row = leaf_row(idx, idx1, table, n_leaves, grown, s, p);
             gf = to_fixed(g[row]);
             hf = h ? to_fixed(h[row]) : 1073741824LL;
         }
@@ -85,7 +98,9 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__
 
 // w = -sum g / (sum h + lambda); output (float)(learning_rate * w); written by leaf id.
 __global__ void k_leaf_values(const long long *__restrict__ sums, const uint32_t *__restrict__ table, int n_leaves,
-                              double lambda, double lr, double *__restrict__ w_out, float *__restrict__ v_out) {
+                              const GrowState *gs, double lambda, double lr, double *__restrict__ w_out,
+                              float *__restrict__ v_out) {
+    if (gs) n_leaves = gs->n_leaves;
     for (int s = blockIdx.x * blockDim.x + threadIdx.x; s < n_leaves; s += gridDim.x * blockDim.x) {
         const int leaf = (int)table[n_leaves + s];
         const double den = __dadd_rn((double)sums[2 * s + 1], __dmul_rn(lambda, 1073741824.0));
@@ -95,18 +110,48 @@ __global__ void k_leaf_values(const long long *__restrict__ sums, const uint32_t
     }
 }
 
-__global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *__restrict__ idx, uint32_t n,
+__global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *__restrict__ idx,
+                                                                const uint32_t *__restrict__ idx1, uint32_t n,
                                                                 const uint32_t *__restrict__ table, int n_leaves,
+                                                                const GrowState *gs,
                                                                 const float *__restrict__ values,
                                                                 float *__restrict__ scores) {
     extern __shared__ uint32_t offs[];
+    const bool grown = gs != nullptr;
+    if (grown) n_leaves = gs->n_leaves;
     for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) offs[i] = table[i];
     __syncthreads();
     for (uint32_t p = blockIdx.x * REFIT_THREADS + threadIdx.x; p < n; p += gridDim.x * REFIT_THREADS) {
         const int s = slot_of(offs, n_leaves, p);
-        const uint32_t row = idx[p];
+        const uint32_t row = leaf_row(idx, idx1, table, n_leaves, grown, s, p);
         scores[row] = __fadd_rn(scores[row], values[table[n_leaves + s]]);
     }
+}
+
+// Leaf table of a tree grown on the device: leaves ranked by (offset, empty first, leaf number);
+// [L] offsets, [L] leaf numbers, [L] index buffers.  Also zeroes the sums and stores the tree's
+// leaf count and rows per leaf.  One block.
+__global__ void __launch_bounds__(256) k_leaf_table(const LeafRec *__restrict__ leaves, const GrowState *gs,
+                                                    uint32_t *__restrict__ table, long long *__restrict__ sums,
+                                                    int32_t *__restrict__ m_num_leaves,
+                                                    long long *__restrict__ m_leaf_count) {
+    const int L = gs->n_leaves;
+    for (int i = threadIdx.x; i < L; i += 256) {
+        const uint32_t off = leaves[i].off, n = leaves[i].n;
+        int rank = 0;
+        for (int j = 0; j < L; ++j) {
+            const uint32_t oj = leaves[j].off, nj = leaves[j].n;
+            const bool before = oj < off || (oj == off && ((nj == 0) > (n == 0) || ((nj == 0) == (n == 0) && j < i)));
+            rank += before ? 1 : 0;
+        }
+        table[rank] = off;
+        table[L + rank] = (uint32_t)i;
+        table[2 * L + rank] = (uint32_t)leaves[i].buf;
+        sums[2 * i] = 0;
+        sums[2 * i + 1] = 0;
+        m_leaf_count[i] = n;
+    }
+    if (threadIdx.x == 0) *m_num_leaves = L;
 }
 
 // Writes the offset-sorted leaf table into pinned memory and queues its copy to the device.
@@ -137,10 +182,10 @@ int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st) 
     if (rc != QGBDT_OK) return rc;
     QG_CUDA(c, cudaMemsetAsync(c->d_leaf_sums, 0, sizeof(long long) * 2 * L, st));
     const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
-    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, (uint32_t)c->N, c->d_leaf_table, L,
-                                                                     d_g, d_h, c->d_leaf_sums);
+    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, nullptr, (uint32_t)c->N, c->d_leaf_table,
+                                                                     L, nullptr, d_g, d_h, c->d_leaf_sums);
     QG_LAUNCH_CHECK(c);
-    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, c->d_leaf_table, L, c->prm.lambda_l2,
+    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, c->d_leaf_table, L, nullptr, c->prm.lambda_l2,
                                                    c->prm.learning_rate, c->d_leaf_w, c->d_leaf_value);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
@@ -151,8 +196,34 @@ int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st) {
     const int L = c->n_leaves;
     unsigned blocks = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
     if (blocks > (unsigned)c->sm_count * 16) blocks = (unsigned)c->sm_count * 16;
-    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, (uint32_t)c->N, c->d_leaf_table, L,
-                                                                       c->d_leaf_value, d_scores);
+    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, nullptr, (uint32_t)c->N,
+                                                                       c->d_leaf_table, L, nullptr, c->d_leaf_value,
+                                                                       d_scores);
+    QG_LAUNCH_CHECK(c);
+    return QGBDT_OK;
+}
+
+// Refit (Eq. 3 with the original gradients) and score update for the tree just grown on the
+// device; leaf values and counts go to slot `tree_slot` of the device-side model arrays.
+int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_scores, int tree_slot, cudaStream_t st) {
+    const int L = c->prm.num_leaves;   // upper bound; the kernels read the real count from the grow state
+    k_leaf_table<<<1, 256, 0, st>>>(c->d_leaves, c->d_gs, c->d_leaf_table, c->d_leaf_sums,
+                                    c->d_m_num_leaves + tree_slot, c->d_m_leaf_count + (size_t)tree_slot * L);
+    QG_LAUNCH_CHECK(c);
+    const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
+    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, c->d_idx_tmp, (uint32_t)c->N,
+                                                                     c->d_leaf_table, L, c->d_gs, d_g, d_h,
+                                                                     c->d_leaf_sums);
+    QG_LAUNCH_CHECK(c);
+    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, c->d_leaf_table, L, c->d_gs, c->prm.lambda_l2,
+                                                   c->prm.learning_rate, c->d_leaf_w,
+                                                   c->d_m_leaf_value + (size_t)tree_slot * L);
+    QG_LAUNCH_CHECK(c);
+    unsigned ab = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
+    if (ab > (unsigned)c->sm_count * 16) ab = (unsigned)c->sm_count * 16;
+    k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, c->d_idx_tmp, (uint32_t)c->N,
+                                                                   c->d_leaf_table, L, c->d_gs,
+                                                                   c->d_m_leaf_value + (size_t)tree_slot * L, d_scores);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
 }

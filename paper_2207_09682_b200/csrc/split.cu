@@ -2,30 +2,9 @@
 // (prefix sums over bins by warp shuffles), gains in double precision with every operation
 // individually rounded; a second kernel takes the best feature.  Ties: lowest feature,
 // then lowest bin.
-#include "qgbdt_internal.cuh"
+#include "split_scan.cuh"
 
 namespace {
-
-struct SplitParams {
-    long long G, H, n_s;
-    int kg, kh, const_h, min_data;
-    double min_sum_h, min_gain, lambda;
-};
-
-__device__ inline double gain_term(long long G, long long H, double dg, double dh, double lambda) {
-    const double gd = __dmul_rn((double)G, dg);
-    const double hd = __dadd_rn(__dmul_rn((double)H, dh), lambda);
-    return __ddiv_rn(__dmul_rn(gd, gd), hd);
-}
-
-// a strictly better than b?  (gain first; equal gains: the lower position wins)
-__device__ inline bool better(bool av, double ag, int apos, bool bv, double bg, int bpos) {
-    if (!av) return false;
-    if (!bv) return true;
-    if (ag > bg) return true;
-    if (ag < bg) return false;
-    return apos < bpos;
-}
 
 constexpr int SCAN_WARPS = 8;
 
@@ -35,74 +14,27 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) k_split_scan(const unsigned l
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int f = blockIdx.x * SCAN_WARPS + warp;
     if (f >= F) return;
-    const double dg = __ddiv_rn((double)__uint_as_float(state->gmax_bits), (double)p.kg);
-    const double dh = p.const_h ? 1.0 : __ddiv_rn((double)__uint_as_float(state->hmax_bits), (double)p.kh);
-    const double tp = gain_term(p.G, p.H, dg, dh, p.lambda);
-
-    long long carry_g = 0, carry_h = 0;
-    bool bv = false;
-    double bgain = 0.0;
-    int bbin = -1;
-    long long bgl = 0, bhl = 0;
+    double dg, dh;
+    qg_scales(state, p, dg, dh);
+    const double tp = qg_gain_term(p.G, p.H, dg, dh, p.lambda);
+    ScanState s;
+    qg_scan_init(s);
     for (int base = 0; base < nb - 1; base += 32) {
         const int t = base + lane;
-        long long g = 0, h = 0;
-        if (t < nb - 1) {
-            const unsigned long long v = hist[(size_t)f * nb + t];
-            g = (long long)(int)(v >> 32);
-            h = (long long)(unsigned int)(v & 0xFFFFFFFFull);
-        }
-        for (int o = 1; o < 32; o <<= 1) {
-            const long long ug = __shfl_up_sync(0xffffffffu, g, o);
-            const long long uh = __shfl_up_sync(0xffffffffu, h, o);
-            if (lane >= o) { g += ug; h += uh; }
-        }
-        const long long gl = carry_g + g, hl = carry_h + h;
-        carry_g += __shfl_sync(0xffffffffu, g, 31);
-        carry_h += __shfl_sync(0xffffffffu, h, 31);
-        if (t < nb - 1) {
-            const long long gr = p.G - gl, hr = p.H - hl;
-            if (hl > 0 && hr > 0) {
-                long long nl;
-                if (p.const_h) nl = hl;
-                else nl = (long long)(((unsigned long long)hl * (unsigned long long)p.n_s +
-                                       (unsigned long long)(p.H / 2)) / (unsigned long long)p.H);
-                const long long nr = p.n_s - nl;
-                if (nl >= p.min_data && nr >= p.min_data &&
-                    !(__dmul_rn((double)hl, dh) < p.min_sum_h) && !(__dmul_rn((double)hr, dh) < p.min_sum_h)) {
-                    const double tl = gain_term(gl, hl, dg, dh, p.lambda);
-                    const double tr = gain_term(gr, hr, dg, dh, p.lambda);
-                    const double gain = __dmul_rn(0.5, __dsub_rn(__dadd_rn(tl, tr), tp));
-                    if (gain > p.min_gain && (!bv || gain > bgain)) {
-                        bv = true; bgain = gain; bbin = t; bgl = gl; bhl = hl;
-                    }
-                }
-            }
-        }
+        const unsigned long long v = t < nb - 1 ? hist[(size_t)f * nb + t] : 0ull;
+        qg_scan_step(s, v, t, nb, p, dg, dh, tp);
     }
-    for (int o = 16; o > 0; o >>= 1) {
-        const bool ov = __shfl_xor_sync(0xffffffffu, (int)bv, o) != 0;
-        const double og = __shfl_xor_sync(0xffffffffu, bgain, o);
-        const int ob = __shfl_xor_sync(0xffffffffu, bbin, o);
-        const long long ogl = __shfl_xor_sync(0xffffffffu, bgl, o);
-        const long long ohl = __shfl_xor_sync(0xffffffffu, bhl, o);
-        if (better(ov, og, ob, bv, bgain, bbin)) { bv = ov; bgain = og; bbin = ob; bgl = ogl; bhl = ohl; }
-    }
-    if (lane == 0) {
-        SplitRec r;
-        r.gain = bgain; r.gl = bgl; r.hl = bhl; r.feature = f; r.bin = bbin; r.valid = bv ? 1 : 0; r.pad = 0;
-        feat_best[f] = r;
-    }
+    const SplitRec r = qg_scan_finish(s, f);
+    if (lane == 0) feat_best[f] = r;
 }
 
 __global__ void __launch_bounds__(256) k_split_reduce(const SplitRec *__restrict__ feat_best, int F,
                                                       SplitRec *__restrict__ out) {
     __shared__ SplitRec sm[256];
-    SplitRec b;
-    b.valid = 0; b.gain = 0.0; b.feature = -1; b.bin = -1; b.gl = 0; b.hl = 0; b.pad = 0;
+    SplitRec b = qg_invalid_rec();
     for (int f = threadIdx.x; f < F; f += 256) {
         const SplitRec r = feat_best[f];
-        if (better(r.valid != 0, r.gain, r.feature, b.valid != 0, b.gain, b.feature)) b = r;
+        if (qg_rec_better(r, b)) b = r;
     }
     sm[threadIdx.x] = b;
     __syncthreads();
@@ -110,7 +42,7 @@ __global__ void __launch_bounds__(256) k_split_reduce(const SplitRec *__restrict
         if (threadIdx.x < s) {
             const SplitRec o = sm[threadIdx.x + s];
             SplitRec &m = sm[threadIdx.x];
-            if (better(o.valid != 0, o.gain, o.feature, m.valid != 0, m.gain, m.feature)) m = o;
+            if (qg_rec_better(o, m)) m = o;
         }
         __syncthreads();
     }

@@ -10,144 +10,69 @@
 
 namespace {
 
-struct HostSplit {
-    SplitRec rec;
-    long long G, H;  // totals of the leaf the record belongs to
-};
-
-int train_one_tree(qgbdt_ctx *c, const float *d_labels, float *d_scores, uint32_t tree, int slot,
-                   qgbdt_model *model, cudaStream_t st) {
-    const int L = c->prm.num_leaves;
-    const size_t hist_words = (size_t)c->F * c->nb;
+// One boosting iteration, enqueued without waiting for any result.
+int train_one_tree(qgbdt_ctx *c, const float *d_labels, float *d_scores, uint32_t tree, int slot, bool first,
+                   cudaStream_t st) {
     const bool const_h = c->prm.objective == 1;
     int rc;
-    char *scal = reinterpret_cast<char *>(c->h_pinned) + 64 * 1024;
-    DevState *hs = reinterpret_cast<DevState *>(scal);
-    SplitRec *hrec = reinterpret_cast<SplitRec *>(scal + 256);
-
     c->const_hess = const_h;
     c->quantized = false;
-    if ((rc = qg_gradients(c, d_scores, d_labels, c->d_g, const_h ? nullptr : c->d_h, true, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_gradients(c, d_scores, d_labels, c->d_g, const_h ? nullptr : c->d_h, true, first, st)) != QGBDT_OK)
+        return rc;
     if ((rc = qg_quantize(c, c->d_g, const_h ? nullptr : c->d_h, tree, nullptr, nullptr, st)) != QGBDT_OK) return rc;
-    c->n_leaves = 1;
-    c->leaf_off.assign(L, 0);
-    c->leaf_n.assign(L, 0);
-    c->leaf_n[0] = c->N;
-    if (!c->idx_is_identity && (rc = qg_iota(c, st)) != QGBDT_OK) return rc;
-    QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
-    QG_CUDA(c, cudaStreamSynchronize(st));
-    if (hs->bad_value) return qg_fail(c, QGBDT_ERR_VALUE, "gradient or hessian out of domain in tree %u", tree);
-    memcpy(&c->gmax, &hs->gmax_bits, 4);
-    memcpy(&c->hmax, &hs->hmax_bits, 4);
-    if (const_h) c->hmax = 1.0f;
     c->quantized = true;
+    if ((rc = qg_grow_tree(c, slot, st)) != QGBDT_OK) return rc;
+    return qg_refit_grown(c, c->d_g, const_h ? nullptr : c->d_h, d_scores, slot, st);
+}
 
-    std::vector<HostSplit> best(L);
-    std::vector<int> hist_slot(L, 0), parent_node(L, -1), parent_side(L, 0);
-    int next_slot = 1;
-    auto hist_of = [&](int s) { return c->d_hist_pool + (size_t)s * hist_words; };
-
-    best[0].G = hs->tot_g;
-    best[0].H = hs->tot_h;
-    if ((rc = qg_hist(c, nullptr, 0, c->N, hist_of(0), st)) != QGBDT_OK) return rc;
-    if ((rc = qg_find_split(c, hist_of(0), best[0].G, best[0].H, c->N, c->d_split_out, st)) != QGBDT_OK) return rc;
-    QG_CUDA(c, cudaMemcpyAsync(hrec, c->d_split_out, sizeof(SplitRec), cudaMemcpyDeviceToHost, st));
-    QG_CUDA(c, cudaStreamSynchronize(st));
-    best[0].rec = hrec[0];
-
-    int32_t *nf = model->feature + (size_t)slot * (L - 1), *nbn = model->bin + (size_t)slot * (L - 1);
-    int32_t *nl_ = model->left + (size_t)slot * (L - 1), *nr_ = model->right + (size_t)slot * (L - 1);
-    double *ng = model->gain + (size_t)slot * (L - 1);
-
-    while (c->n_leaves < L) {
-        int pick = -1;
-        for (int l = 0; l < c->n_leaves; ++l)
-            if (best[l].rec.valid && (pick < 0 || best[l].rec.gain > best[pick].rec.gain)) pick = l;
-        if (pick < 0) break;
-        const SplitRec s = best[pick].rec;
-        const long long PG = best[pick].G, PH = best[pick].H;
-        const int64_t off = c->leaf_off[pick], n = c->leaf_n[pick];
-        if ((rc = qg_partition(c, off, n, s.feature, s.bin, st)) != QGBDT_OK) return rc;
-        QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
-        QG_CUDA(c, cudaStreamSynchronize(st));
-        if (hs->kernel_error) return qg_fail(c, QGBDT_ERR_CUDA, "a histogram kernel refused its launch configuration");
-        const int64_t nl = hs->part_nl, nr = n - nl;
-        const int node = c->n_leaves - 1, right = c->n_leaves;
-        nf[node] = s.feature;
-        nbn[node] = s.bin;
-        nl_[node] = ~pick;
-        nr_[node] = ~right;
-        ng[node] = s.gain;
-        if (parent_node[pick] >= 0) {
-            if (parent_side[pick] == 0) nl_[parent_node[pick]] = node;
-            else nr_[parent_node[pick]] = node;
-        }
-        parent_node[pick] = node; parent_side[pick] = 0;
-        parent_node[right] = node; parent_side[right] = 1;
-        c->leaf_n[pick] = nl;
-        c->leaf_off[right] = off + nl;
-        c->leaf_n[right] = nr;
-        c->n_leaves++;
-        best[pick].G = s.gl; best[pick].H = s.hl;
-        best[right].G = PG - s.gl; best[right].H = PH - s.hl;
-
-        // smaller child by Algorithm 1, larger child = parent - smaller (ties: left is "smaller")
-        const int small = nl <= nr ? pick : right, large = nl <= nr ? right : pick;
-        const int pslot = hist_slot[pick];
-        hist_slot[small] = next_slot++;
-        hist_slot[large] = pslot;
-        if ((rc = qg_hist(c, c->d_idx, c->leaf_off[small], c->leaf_n[small], hist_of(hist_slot[small]), st)) != QGBDT_OK)
-            return rc;
-        if ((rc = qg_subtract(c, hist_of(pslot), hist_of(hist_slot[small]), hist_of(pslot), st)) != QGBDT_OK) return rc;
-        if ((rc = qg_find_split(c, hist_of(hist_slot[pick]), best[pick].G, best[pick].H, nl, c->d_split_out, st)) != QGBDT_OK)
-            return rc;
-        if ((rc = qg_find_split(c, hist_of(hist_slot[right]), best[right].G, best[right].H, nr, c->d_split_out + 1, st)) !=
-            QGBDT_OK)
-            return rc;
-        QG_CUDA(c, cudaMemcpyAsync(hrec, c->d_split_out, 2 * sizeof(SplitRec), cudaMemcpyDeviceToHost, st));
-        QG_CUDA(c, cudaStreamSynchronize(st));
-        best[pick].rec = hrec[0];
-        best[right].rec = hrec[1];
+template <typename T>
+int alloc_dev(qgbdt_ctx *c, T **p, size_t count, const char *what) {
+    void *q = nullptr;
+    if (cudaMalloc(&q, (count ? count : 1) * sizeof(T)) != cudaSuccess) {
+        cudaGetLastError();
+        return qg_fail(c, QGBDT_ERR_ALLOC, "%s allocation of %zu bytes failed", what, count * sizeof(T));
     }
-
-    if ((rc = qg_refit(c, c->d_g, const_h ? nullptr : c->d_h, st)) != QGBDT_OK) return rc;
-    if ((rc = qg_apply_leaf_values(c, d_scores, st)) != QGBDT_OK) return rc;
-    float *hv = reinterpret_cast<float *>(scal + 1024);
-    QG_CUDA(c, cudaMemcpyAsync(hv, c->d_leaf_value, sizeof(float) * c->n_leaves, cudaMemcpyDeviceToHost, st));
-    QG_CUDA(c, cudaStreamSynchronize(st));
-    model->num_leaves[slot] = c->n_leaves;
-    for (int l = 0; l < c->n_leaves; ++l) {
-        model->leaf_value[(size_t)slot * L + l] = hv[l];
-        model->leaf_count[(size_t)slot * L + l] = c->leaf_n[l];
-    }
+    *p = reinterpret_cast<T *>(q);
     return QGBDT_OK;
 }
 
-int ensure_train_buffers(qgbdt_ctx *c) {
-    if (!c->d_g) {
-        void *p = nullptr;
-        if (cudaMalloc(&p, sizeof(float) * (size_t)c->N) != cudaSuccess) {
-            cudaGetLastError();
-            return qg_fail(c, QGBDT_ERR_ALLOC, "gradient buffer allocation failed");
-        }
-        c->d_g = reinterpret_cast<float *>(p);
+template <typename T>
+void free_dev(T *&p) {
+    if (p) cudaFree(p);
+    p = nullptr;
+}
+
+int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
+    const int L = c->prm.num_leaves;
+    int rc;
+    if (!c->d_g && (rc = alloc_dev(c, &c->d_g, (size_t)c->N, "gradient buffer")) != QGBDT_OK) return rc;
+    if (!c->d_h && c->prm.objective == 0 && (rc = alloc_dev(c, &c->d_h, (size_t)c->N, "hessian buffer")) != QGBDT_OK)
+        return rc;
+    if (!c->d_hist_pool &&
+        (rc = alloc_dev(c, &c->d_hist_pool, (size_t)L * c->F * c->nb, "histogram pool")) != QGBDT_OK)
+        return rc;
+    if (!c->d_leaves && (rc = alloc_dev(c, &c->d_leaves, (size_t)L, "leaf records")) != QGBDT_OK) return rc;
+    if (!c->d_cand && (rc = alloc_dev(c, &c->d_cand, (size_t)2 * ((c->F + 7) / 8), "candidate records")) != QGBDT_OK)
+        return rc;
+    if (!c->d_gs) {
+        if ((rc = alloc_dev(c, &c->d_gs, 1, "grow state")) != QGBDT_OK) return rc;
+        QG_CUDA(c, cudaMemsetAsync(c->d_gs, 0, sizeof(GrowState), st));
     }
-    if (!c->d_h && c->prm.objective == 0) {
-        void *p = nullptr;
-        if (cudaMalloc(&p, sizeof(float) * (size_t)c->N) != cudaSuccess) {
-            cudaGetLastError();
-            return qg_fail(c, QGBDT_ERR_ALLOC, "hessian buffer allocation failed");
-        }
-        c->d_h = reinterpret_cast<float *>(p);
-    }
-    if (!c->d_hist_pool) {
-        void *p = nullptr;
-        const size_t bytes = (size_t)c->prm.num_leaves * c->F * c->nb * sizeof(unsigned long long);
-        if (cudaMalloc(&p, bytes) != cudaSuccess) {
-            cudaGetLastError();
-            return qg_fail(c, QGBDT_ERR_ALLOC, "histogram pool allocation of %zu bytes failed", bytes);
-        }
-        c->d_hist_pool = reinterpret_cast<unsigned long long *>(p);
+    if (num_trees > c->model_cap) {
+        free_dev(c->d_m_num_leaves); free_dev(c->d_m_feature); free_dev(c->d_m_bin); free_dev(c->d_m_left);
+        free_dev(c->d_m_right); free_dev(c->d_m_gain); free_dev(c->d_m_leaf_value); free_dev(c->d_m_leaf_count);
+        c->model_cap = 0;
+        const size_t nn = (size_t)num_trees * (L > 1 ? L - 1 : 1), nl = (size_t)num_trees * L;
+        if ((rc = alloc_dev(c, &c->d_m_num_leaves, (size_t)num_trees, "model")) != QGBDT_OK ||
+            (rc = alloc_dev(c, &c->d_m_feature, nn, "model")) != QGBDT_OK ||
+            (rc = alloc_dev(c, &c->d_m_bin, nn, "model")) != QGBDT_OK ||
+            (rc = alloc_dev(c, &c->d_m_left, nn, "model")) != QGBDT_OK ||
+            (rc = alloc_dev(c, &c->d_m_right, nn, "model")) != QGBDT_OK ||
+            (rc = alloc_dev(c, &c->d_m_gain, nn, "model")) != QGBDT_OK ||
+            (rc = alloc_dev(c, &c->d_m_leaf_value, nl, "model")) != QGBDT_OK ||
+            (rc = alloc_dev(c, &c->d_m_leaf_count, nl, "model")) != QGBDT_OK)
+            return rc;
+        c->model_cap = num_trees;
     }
     return QGBDT_OK;
 }
@@ -166,11 +91,54 @@ int qgbdt_train(qgbdt_ctx *c, const float *d_labels, float *d_scores, uint32_t f
     if (!c) return QGBDT_ERR_ARG;
     if (!c->loaded) return qg_fail(c, QGBDT_ERR_STATE, "no bin matrix loaded");
     if (!d_labels || !d_scores || num_trees < 0 || !model_ok(model)) return qg_fail(c, QGBDT_ERR_ARG, "bad argument");
-    int rc = ensure_train_buffers(c);
-    if (rc != QGBDT_OK) return rc;
+    if (num_trees == 0) return QGBDT_OK;
     cudaStream_t st = (cudaStream_t)stream;
-    for (int k = 0; k < num_trees; ++k)
-        if ((rc = train_one_tree(c, d_labels, d_scores, first_tree + (uint32_t)k, k, model, st)) != QGBDT_OK) return rc;
+    int rc = ensure_train_buffers(c, num_trees, st);
+    if (rc != QGBDT_OK) return rc;
+    const int L = c->prm.num_leaves;
+    char *scal = reinterpret_cast<char *>(c->h_pinned) + 64 * 1024;
+    DevState *hs = reinterpret_cast<DevState *>(scal);
+    GrowState *hg = reinterpret_cast<GrowState *>(scal + 256);
+    GrowState before;
+    QG_CUDA(c, cudaMemcpyAsync(hg, c->d_gs, sizeof(GrowState), cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaStreamSynchronize(st));
+    before = *hg;
+    for (int k = 0; k < num_trees; ++k) {
+        if ((rc = train_one_tree(c, d_labels, d_scores, first_tree + (uint32_t)k, k, k == 0, st)) != QGBDT_OK) return rc;
+    }
+    // the trees, the flags and the counters come back once, after the last tree
+    const size_t nn = (size_t)num_trees * (L > 1 ? L - 1 : 1), nl = (size_t)num_trees * L;
+    QG_CUDA(c, cudaMemcpyAsync(model->num_leaves, c->d_m_num_leaves, sizeof(int32_t) * num_trees, cudaMemcpyDeviceToHost, st));
+    if (L > 1) {
+        QG_CUDA(c, cudaMemcpyAsync(model->feature, c->d_m_feature, sizeof(int32_t) * nn, cudaMemcpyDeviceToHost, st));
+        QG_CUDA(c, cudaMemcpyAsync(model->bin, c->d_m_bin, sizeof(int32_t) * nn, cudaMemcpyDeviceToHost, st));
+        QG_CUDA(c, cudaMemcpyAsync(model->left, c->d_m_left, sizeof(int32_t) * nn, cudaMemcpyDeviceToHost, st));
+        QG_CUDA(c, cudaMemcpyAsync(model->right, c->d_m_right, sizeof(int32_t) * nn, cudaMemcpyDeviceToHost, st));
+        QG_CUDA(c, cudaMemcpyAsync(model->gain, c->d_m_gain, sizeof(double) * nn, cudaMemcpyDeviceToHost, st));
+    }
+    QG_CUDA(c, cudaMemcpyAsync(model->leaf_value, c->d_m_leaf_value, sizeof(float) * nl, cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaMemcpyAsync(model->leaf_count, c->d_m_leaf_count, sizeof(long long) * nl, cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
+    QG_CUDA(c, cudaMemcpyAsync(hg, c->d_gs, sizeof(GrowState), cudaMemcpyDeviceToHost, st));
+    // leave the step-wise interface in a defined state: one root leaf, rows ascending
+    c->n_leaves = 1;
+    c->leaf_off.assign(L, 0);
+    c->leaf_n.assign(L, 0);
+    c->leaf_n[0] = c->N;
+    if ((rc = qg_iota(c, st)) != QGBDT_OK) return rc;
+    QG_CUDA(c, cudaStreamSynchronize(st));
+    c->n_hist_builds += (int64_t)(hg->hist_builds - before.hist_builds);
+    c->n_hist_row_features += (int64_t)(hg->hist_rows - before.hist_rows) * c->F;
+    c->hist_prof_bytes += (int64_t)(hg->hist_rows - before.hist_rows) * (c->F + c->code_bytes + 4) +
+                          (int64_t)(hg->hist_builds - before.hist_builds) * c->F * c->nb * 8;
+    c->hist_prof_launches += (int64_t)(hg->hist_builds - before.hist_builds);
+    memcpy(&c->gmax, &hs->gmax_bits, 4);
+    memcpy(&c->hmax, &hs->hmax_bits, 4);
+    if (c->prm.objective == 1) c->hmax = 1.0f;
+    if (hs->kernel_error) return qg_fail(c, QGBDT_ERR_CUDA, "a histogram kernel refused its launch configuration");
+    if (hs->bad_value)
+        return qg_fail(c, QGBDT_ERR_VALUE, "gradient or hessian out of domain during trees %u .. %u", first_tree,
+                       first_tree + (uint32_t)num_trees - 1);
     return QGBDT_OK;
 }
 

@@ -34,7 +34,7 @@ struct GrowArgs {
     int n_count;                     // warp ranges (= warps of the flag / scatter grids)
     unsigned long long *pool;        // [L][F][nb]
     const unsigned long long *partial;
-    SplitRec *cand;                  // [finish blocks][2]
+    SplitRec *cand;                  // [F][2] best candidates of every feature for the two children
     int F, nb, L;
     SplitParams sp;                  // G, H, n_s are filled per leaf on the device
     // tree output (device arrays of the current tree)
@@ -54,10 +54,15 @@ __global__ void k_grow_begin(GrowState *gs, LeafRec *leaves, const DevState *sta
     gs->finish_count = 0;
 }
 
-// Words of 32 rows [w0, w1) of warp gw when nw words are shared out among n_count warps.
-__device__ inline void warp_range(uint32_t nw, uint32_t gw, uint32_t n_count, uint32_t &w0, uint32_t &w1) {
-    w0 = (uint32_t)((unsigned long long)nw * gw / n_count);
-    w1 = (uint32_t)((unsigned long long)nw * (gw + 1) / n_count);
+// Words of 32 rows [w0, w1) of warp gw: every warp takes the same number of consecutive words
+// (at least 4), so the warps with work are a prefix [0, active) of the grid.
+__device__ inline void warp_range(uint32_t nw, uint32_t gw, uint32_t n_count, uint32_t &w0, uint32_t &w1,
+                                  uint32_t &active) {
+    uint32_t per = (nw + n_count - 1) / n_count;
+    if (per < 4) per = 4;
+    active = (nw + per - 1) / per;
+    w0 = gw * per < nw ? gw * per : nw;
+    w1 = w0 + per < nw ? w0 + per : nw;
 }
 
 __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
@@ -67,8 +72,9 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
     const uint32_t gw = blockIdx.x * PART_WARPS + (threadIdx.x >> 5);
     const uint32_t n = gs->n, off = gs->off;
     const uint32_t nw = (n + 31) >> 5;
-    uint32_t w0, w1;
-    warp_range(nw, gw, (uint32_t)a.n_count, w0, w1);
+    uint32_t w0, w1, active;
+    warp_range(nw, gw, (uint32_t)a.n_count, w0, w1, active);
+    if (gw >= active) return;
     const uint32_t *src = gs->buf < 0 ? nullptr : (gs->buf ? a.idx1 : a.idx0);
     const TileDesc td = a.tiles[gs->tile];
     const uint32_t *col = td.data + gs->word;
@@ -96,12 +102,12 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
     const uint32_t gw = blockIdx.x * PART_WARPS + (threadIdx.x >> 5);
     const uint32_t n = gs->n, off = gs->off;
     const uint32_t nw = (n + 31) >> 5;
-    uint32_t w0, w1;
-    warp_range(nw, gw, (uint32_t)a.n_count, w0, w1);
-    if (w1 <= w0 && gw != 0) return;
+    uint32_t w0, w1, active;
+    warp_range(nw, gw, (uint32_t)a.n_count, w0, w1, active);
+    if (gw >= active && gw != 0) return;
     // left rows before this warp's range, and in the whole leaf
     uint32_t before = 0, total = 0;
-    for (uint32_t j = lane; j < (uint32_t)a.n_count; j += 32) {
+    for (uint32_t j = lane; j < active; j += 32) {
         const uint32_t v = a.counts[j];
         total += v;
         if (j < gw) before += v;
@@ -139,13 +145,13 @@ __device__ inline SplitRec load_rec_cg(const SplitRec *p) {   // bypasses L1: wr
 static_assert(sizeof(SplitRec) == 40, "SplitRec is copied as five 64-bit words");
 
 // ROOT: scans the root histogram (pool slot 0).  Otherwise: completes the split recorded in the
-// grow state.  One warp per feature.
+// grow state.  One block per feature.
 template <bool ROOT>
 __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     GrowState *gs = a.gs;
     if (gs->done) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int f = blockIdx.x * FIN_WARPS + warp;
+    const int f = blockIdx.x;   // one block per feature
     const int n_leaves = gs->n_leaves;
     const size_t hw = (size_t)a.F * a.nb;
 
@@ -160,63 +166,74 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
         pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl : nr;
         pL.G = small_is_left ? gr : gl; pL.H = small_is_left ? hr : hl; pL.n_s = small_is_left ? nr : nl;
     }
-    SplitRec rS = qg_invalid_rec(), rL = qg_invalid_rec();
-    if (f < a.F) {
-        double dg, dh;
-        qg_scales(a.state, pS, dg, dh);
-        const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
-        const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
-        const TileDesc td = a.tiles[a.feat_tile[f]];
-        const int fl = f - td.f0, W = 1 << td.logW;
-        const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)td.parts, (uint32_t)pS.n_s);
-        const size_t pstride = (size_t)4 * a.nb * 32;
-        const unsigned long long *part = a.partial + (size_t)td.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
-        unsigned long long *S = a.pool + (ROOT ? 0 : (size_t)n_leaves * hw) + (size_t)f * a.nb;
-        unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)gs->parent_slot * hw + (size_t)f * a.nb;
-        ScanState scS, scL;
-        qg_scan_init(scS);
-        qg_scan_init(scL);
-        for (int base = 0; base < a.nb; base += 32) {
-            const int b = base + lane;
-            unsigned long long s = 0, l = 0;
-            if (b < a.nb) {
-                if (ROOT) {
-                    s = S[b];
-                } else {
-                    if (P > 1) {
-                        const unsigned long long *q = part + (size_t)b * W;
-                        for (uint32_t i = 0; i < P; ++i) s += q[i * pstride];
-                        S[b] = s;
-                    } else {
-                        s = S[b];
-                    }
-                    l = Pp[b] - s;   // no field borrows: every child sum is at most the parent's
-                    Pp[b] = l;
-                }
-            }
-            qg_scan_step(scS, s, b, a.nb, pS, dg, dh, tpS);
-            if (!ROOT) qg_scan_step(scL, l, b, a.nb, pL, dg, dh, tpL);
-        }
-        rS = qg_scan_finish(scS, f);
-        if (!ROOT) rL = qg_scan_finish(scL, f);
-    }
-
-    // best of the block, then of the grid (last block through)
+    // ---- phase A: one thread per bin (groups of 256 bins): the smaller child's sum over the
+    //      partial histograms, the larger child's bin by subtraction; both kept for the scans
+    __shared__ unsigned long long binS[256], binL[256];
     __shared__ SplitRec sm[2][FIN_WARPS * 32];
     __shared__ bool is_last;
-    if (lane == 0) { sm[0][warp] = rS; sm[1][warp] = rL; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        SplitRec bS = sm[0][0], bL = sm[1][0];
-        for (int w = 1; w < FIN_WARPS; ++w) {
-            if (qg_rec_better(sm[0][w], bS)) bS = sm[0][w];
-            if (qg_rec_better(sm[1][w], bL)) bL = sm[1][w];
+    double dg, dh;
+    qg_scales(a.state, pS, dg, dh);
+    const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
+    const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
+    const TileDesc td = a.tiles[a.feat_tile[f]];
+    const int fl = f - td.f0, W = 1 << td.logW;
+    const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)td.parts, (uint32_t)pS.n_s);
+    const size_t pstride = (size_t)4 * a.nb * 32;
+    const unsigned long long *part = a.partial + (size_t)td.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
+    unsigned long long *S = a.pool + (ROOT ? 0 : (size_t)n_leaves * hw) + (size_t)f * a.nb;
+    unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)gs->parent_slot * hw + (size_t)f * a.nb;
+    ScanState sc;
+    qg_scan_init(sc);
+    for (int base = 0; base < a.nb; base += 256) {
+        const int b = base + (int)threadIdx.x;
+        unsigned long long s = 0, l = 0;
+        if (b < a.nb) {
+            if (ROOT) {
+                s = S[b];
+            } else {
+                if (P > 1) {
+                    const unsigned long long *q = part + (size_t)b * W;
+                    unsigned long long s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+                    uint32_t i = 0;
+                    for (; i + 8 <= P; i += 8) {
+                        const unsigned long long x0 = q[(size_t)i * pstride], x1 = q[(size_t)(i + 1) * pstride];
+                        const unsigned long long x2 = q[(size_t)(i + 2) * pstride], x3 = q[(size_t)(i + 3) * pstride];
+                        const unsigned long long x4 = q[(size_t)(i + 4) * pstride], x5 = q[(size_t)(i + 5) * pstride];
+                        const unsigned long long x6 = q[(size_t)(i + 6) * pstride], x7 = q[(size_t)(i + 7) * pstride];
+                        s0 += x0 + x4; s1 += x1 + x5; s2 += x2 + x6; s3 += x3 + x7;
+                    }
+                    for (; i < P; ++i) s0 += q[(size_t)i * pstride];
+                    s = (s0 + s1) + (s2 + s3);
+                    S[b] = s;
+                } else {
+                    s = S[b];
+                }
+                l = Pp[b] - s;   // no field borrows: every child sum is at most the parent's
+                Pp[b] = l;
+            }
         }
-        a.cand[2 * blockIdx.x] = bS;
-        a.cand[2 * blockIdx.x + 1] = bL;
-        __threadfence();
-        is_last = atomicAdd(&gs->finish_count, 1u) == gridDim.x - 1;
+        binS[threadIdx.x] = s;
+        binL[threadIdx.x] = l;
+        __syncthreads();
+        // ---- phase B: warp 0 scans the smaller child's bins, warp 1 the larger child's
+        if (warp < (ROOT ? 1 : 2)) {
+            const unsigned long long *bins = warp == 0 ? binS : binL;
+            const SplitParams &pp = warp == 0 ? pS : pL;
+            const double tp = warp == 0 ? tpS : tpL;
+            for (int g = 0; g < 256 && base + g < a.nb; g += 32)
+                qg_scan_step(sc, bins[g + lane], base + g + lane, a.nb, pp, dg, dh, tp);
+        }
+        __syncthreads();
     }
+    if (warp < 2) {
+        const SplitRec r = (ROOT && warp == 1) ? qg_invalid_rec() : qg_scan_finish(sc, f);
+        if (lane == 0) {
+            a.cand[2 * f + warp] = r;
+            __threadfence();
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(&gs->finish_count, 1u) == gridDim.x - 1;
     __syncthreads();
     if (!is_last) return;
     __threadfence();
@@ -374,7 +391,7 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     QG_LAUNCH_CHECK(c);
     int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
     if (rc != QGBDT_OK) return rc;
-    const unsigned fin_blocks = (unsigned)((c->F + FIN_WARPS - 1) / FIN_WARPS);
+    const unsigned fin_blocks = (unsigned)c->F;
     k_grow_finish<true><<<fin_blocks, FIN_WARPS * 32, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     for (int split = 1; split < L; ++split) {

@@ -130,7 +130,7 @@ struct qgbdt_ctx {
     unsigned long long *d_hist_pool = nullptr;  // [L][F][nb]
     LeafRec *d_leaves = nullptr;                // [L]
     GrowState *d_gs = nullptr;
-    SplitRec *d_cand = nullptr;                 // [finish blocks][2] per-block best candidates of the two children
+    SplitRec *d_cand = nullptr;                 // [F][2] per-feature best candidates of the two children
     int32_t *d_feat_tile = nullptr;             // [F] tile of every feature
     // trees of the current qgbdt_train call, on the device until the call ends
     int model_cap = 0;                          // trees the arrays below can hold

@@ -52,7 +52,7 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
         (rc = alloc_dev(c, &c->d_hist_pool, (size_t)L * c->F * c->nb, "histogram pool")) != QGBDT_OK)
         return rc;
     if (!c->d_leaves && (rc = alloc_dev(c, &c->d_leaves, (size_t)L, "leaf records")) != QGBDT_OK) return rc;
-    if (!c->d_cand && (rc = alloc_dev(c, &c->d_cand, (size_t)2 * ((c->F + 7) / 8), "candidate records")) != QGBDT_OK)
+    if (!c->d_cand && (rc = alloc_dev(c, &c->d_cand, (size_t)2 * c->F, "candidate records")) != QGBDT_OK)
         return rc;
     if (!c->d_gs) {
         if ((rc = alloc_dev(c, &c->d_gs, 1, "grow state")) != QGBDT_OK) return rc;

@@ -186,6 +186,33 @@ int qgbdt_get_counters(const qgbdt_ctx *ctx, int64_t *kernel_launches, int64_t *
 int qgbdt_profile_histograms(qgbdt_ctx *ctx, int32_t enable);
 int qgbdt_get_histogram_profile(qgbdt_ctx *ctx, double *total_ms, int64_t *total_bytes, int64_t *builds);
 
+/* Histogram build that allocates nothing (the paper has no counterpart; it exists for callers
+ * that are not allowed to call cudaMalloc: code running inside a memory pool that owns the
+ * device, inside a loop where an allocation would stall the GPU, or in a plug-in whose host
+ * bans allocator calls).  It needs no context.  It computes the same histogram as
+ * qgbdt_build_histograms / qgbdt_build_histograms_rows from the caller's own arrays:
+ *   d_bins  row-major bin matrix, element (i, j) at d_bins[i*ld + j], codes < n_bins
+ *   d_gq    [n_rows] int8 quantized gradients, d_hq [n_rows] uint8 quantized hessians
+ *           (the optional outputs of qgbdt_quantize_gradients)
+ *   d_rows  [n] row list, or NULL for all rows (then n must equal n_rows)
+ *   d_hist  [n_features][n_bins], overwritten
+ *   d_status  optional device word the caller clears: set to 1 when a row index or a bin code
+ *           was out of range (such entries are skipped)
+ * All pointers are device pointers owned by the caller.  The per-CTA partial histograms live in
+ * a fixed 4 MiB array inside the library image (every GPU that loads the library holds it until
+ * the process ends), so n_features * n_bins may be at most 16384; larger problems are refused
+ * with QGBDT_ERR_ARG and need a context.  The call makes no cudaMalloc / cudaFree and calls no
+ * allocating routine.  The first call on a device looks up the array's device address; make
+ * that first call outside any stream capture.  All calls share the one array, which keeps the
+ * previous call's sums (each call clears what it uses): two calls whose kernels overlap on the
+ * GPU -- different streams, or different host threads on different streams -- race; keep them on
+ * one stream or order them with events.  Asynchronous on `stream`.  On failure
+ * qgbdt_noalloc_last_error() gives the reason (per host thread). */
+int qgbdt_build_histograms_noalloc(const uint8_t *d_bins, int64_t n_rows, int32_t n_features, int32_t n_bins,
+                                   int64_t ld, const int8_t *d_gq, const uint8_t *d_hq, const uint32_t *d_rows,
+                                   int64_t n, qgbdt_bin *d_hist, int32_t *d_status, void *stream);
+const char *qgbdt_noalloc_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,6 +22,7 @@ EXPORTS = [
     "qgbdt_build_histograms_rows", "qgbdt_subtract_histograms", "qgbdt_find_best_split", "qgbdt_split_leaf",
     "qgbdt_get_leaf_rows", "qgbdt_reset_leaves", "qgbdt_refit_leaves", "qgbdt_train", "qgbdt_train_host",
     "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile",
+    "qgbdt_build_histograms_noalloc", "qgbdt_noalloc_last_error",
 ]
 
 
@@ -261,6 +262,21 @@ def _get_histogram_profile(self) -> dict:
 
 Context.profile_histograms = _profile_histograms
 Context.get_histogram_profile = _get_histogram_profile
+
+
+def build_histograms_noalloc(bins: torch.Tensor, n_bins: int, gq: torch.Tensor, hq: torch.Tensor,
+                             hist: torch.Tensor, rows: torch.Tensor = None, status: torch.Tensor = None, stream=None):
+    """The context-free, allocation-free histogram call: bins uint8 [N, F] row-major, gq int8 [N],
+    hq uint8 [N], hist int64 [F, n_bins] (overwritten), rows optional int32 list.  Marshalling only."""
+    lib = load_library()
+    lib.qgbdt_noalloc_last_error.restype = C.c_char_p
+    n_rows, f = bins.shape
+    n = n_rows if rows is None else rows.numel()
+    rc = lib.qgbdt_build_histograms_noalloc(_dptr(bins), C.c_int64(n_rows), C.c_int32(f), C.c_int32(n_bins),
+                                            C.c_int64(bins.stride(0)), _dptr(gq), _dptr(hq), _dptr(rows), C.c_int64(n),
+                                            _dptr(hist), _dptr(status), _stream(stream))
+    if rc != OK:
+        raise QgbdtError(rc, lib.qgbdt_noalloc_last_error().decode())
 
 
 def unpack_hist(hist: torch.Tensor) -> tuple[np.ndarray, np.ndarray]:

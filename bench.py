@@ -148,11 +148,13 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes, reps=20):
-    """Stand-alone root and 50%-subset histogram builds, back to back on inputs larger than L2.
+def time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes, reps=10, batch=10):
+    """Stand-alone root and 50%-subset histogram builds on inputs larger than L2.
 
-    (Writing a buffer to flush L2 would leave it full of dirty lines whose write-back is then
-    charged to the next build; the bin matrix itself is larger than L2, so nothing is reused.)"""
+    `batch` builds are enqueued back to back between two CUDA events so that the GPU never waits
+    for the host; the time per build is the median over `reps` such batches.  (Writing a buffer
+    to flush L2 would leave it full of dirty lines whose write-back is then charged to the next
+    build; the bin matrix itself is larger than L2, so nothing is reused between builds.)"""
     import numpy as np
     hist = ctx.new_hist()
     rows = synth.subset_rows(n, device="cuda")
@@ -162,20 +164,46 @@ def time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes, reps=20
         for i in range(reps + 3):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            if r is None:
-                ctx.build_histograms(0, hist)
-            else:
-                ctx.build_histograms_rows(r, hist)
+            for _ in range(batch):
+                if r is None:
+                    ctx.build_histograms(0, hist)
+                else:
+                    ctx.build_histograms_rows(r, hist)
             e1.record()
             torch.cuda.synchronize()
             if i >= 3:
-                ts.append(e0.elapsed_time(e1))
+                ts.append(e0.elapsed_time(e1) / batch)
         nr = n if r is None else int(r.numel())
         ms = float(np.median(ts))
         nbytes = nr * (features + code_bytes + (0 if r is None else 4)) + features * n_bins * 8
         out[name] = {"rows": nr, "us": 1e3 * ms, "row_features_per_s": nr * features / (ms * 1e-3),
-                     "gbs": nbytes / (ms * 1e6), "note": "partial-histogram kernel + merge kernel"}
+                     "gbs": nbytes / (ms * 1e6), "note": "partial-histogram kernel + merge kernel, %d builds per timing" % batch}
     return out
+
+
+def run_sweep(args):
+    """Histogram-kernel sweep (rows x features x bins x gradient bits, root and 50 % subset builds);
+    prints one text line per point.  Not a benchmark line: a table for the design notes."""
+    import torch
+    from paper_2207_09682_b200 import binding, synth
+    torch.cuda.set_device(0)
+    peak, kind = measured_peak()
+    print("# rows features bins bits | root us  GB/s  frac | subset50 us  GB/s  frac   (frac of %s %.0f GB/s)" % (kind, peak))
+    for n in (1_000_000, 4_000_000, 16_000_000):
+        for f in (28, 136, 1000):
+            for nb in (16, 64, 255):
+                bins = synth.sweep_bins(n, f, nb, device="cuda")
+                g, h = synth.sweep_gradients(n, device="cuda")
+                for bits in (2, 3, 4, 8):
+                    ctx = binding.Context(binding.make_params(bits=bits))
+                    ctx.load_binned(bins, nb)
+                    ctx.quantize_gradients(g, h)
+                    b = time_hist_builds(ctx, torch, synth, n, f, nb, 2, reps=3, batch=5)
+                    print("%9d %5d %4d %2d | %9.1f %7.0f %5.3f | %9.1f %7.0f %5.3f" % (
+                        n, f, nb, bits, b["root"]["us"], b["root"]["gbs"], b["root"]["gbs"] / peak,
+                        b["subset50"]["us"], b["subset50"]["gbs"], b["subset50"]["gbs"] / peak), flush=True)
+                    ctx.close()
+                del bins
 
 
 def run_ours(args):
@@ -315,8 +343,11 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override the workload's row count (profiling captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="print the histogram-kernel sweep table instead")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

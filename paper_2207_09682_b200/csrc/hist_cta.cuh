@@ -1,0 +1,393 @@
+// Device code of the histogram build (Algorithm 1 with integer gradients), shared by the
+// stand-alone kernel and by the tree-growing kernel.  See hist.cu for the design notes.
+#pragma once
+
+#include "qgbdt_internal.cuh"
+
+namespace {
+
+constexpr int HIST_THREADS = 1024;
+constexpr int HIST_WARPS = HIST_THREADS / 32;
+constexpr int HIST_SMEM = 192 * 1024;     // 128 KB histogram on a 64 KB boundary + the room below it
+constexpr uint32_t MIN_ROWS_PER_CTA = 4096;
+constexpr int U_ROOT = 4;                 // units in flight per lane, contiguous rows
+constexpr int U_LIST = 2;                 // units in flight per lane, row list (plus as many index units)
+
+struct HistArgs {
+    const TileDesc *tiles;
+    const uint16_t *codes;         // per-row code (g8 << 8 | h8), transposed inside blocks of 16 rows
+    const uint16_t *codes_nat;     // the same codes in row order (row lists and leftover rows)
+    int tile0;                     // first tile of this launch
+    const uint32_t *rows;          // row list (LIST 1), or nullptr: rows 0 .. n-1 (LIST 0)
+    const uint2 *ents;             // (row, code) pairs written by the tree-growing scatter (LIST 2)
+    uint32_t off, n;               // list: entries rows[off .. off+n)
+    int nb;
+    unsigned long long *hist;      // [F][nb]
+    unsigned long long *partial;   // [CTA][4][nb][32]
+    uint32_t flush_rows;           // rows one column may add between flushes (16+16 local only)
+    int pass;                      // 32+32 local only: bytes 2*pass, 2*pass+1 of every word
+    DevState *state;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t s) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(s));
+    return d;
+}
+
+template <int IMM>
+__device__ __forceinline__ void red32(uint32_t addr, int v) {
+    asm volatile("red.shared.add.u32 [%0+%1], %2;" ::"r"(addr), "n"(IMM), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ uint32_t ldg32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint2 ldg64(const uint2 *p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint32_t ldg16(const uint16_t *p) {
+    uint32_t v;
+    asm volatile("{ .reg .u16 t; ld.global.nc.L1::no_allocate.u16 t, [%1]; cvt.u32.u16 %0, t; }" : "=r"(v) : "l"(p));
+    return v;
+}
+
+// One row's word: its bin codes -> shared atomics.  `half` selects the 16-bit code in the low
+// or high half of c.
+template <bool WIDE>
+__device__ __forceinline__ void add_word(uint32_t base, uint32_t w, uint32_t c, int half, int pass) {
+    if (!WIDE) {
+        // inc = g * 65536 + h: byte 0 = h, byte 1 = 0, byte 2 = g, byte 3 = sign of g
+        const int inc = (int)prmt(c, 0u, half ? 0xB342u : 0x9140u);
+        red32<0>(prmt(w, base, 0x7604u), inc);
+        red32<128>(prmt(w, base, 0x7614u), inc);
+        red32<65536>(prmt(w, base, 0x7624u), inc);
+        red32<65536 + 128>(prmt(w, base, 0x7634u), inc);
+    } else {
+        // 32+32 local bins: the hessian plane at +0 and the gradient plane at +128 of a bin's 256 bytes
+        const int h = (int)prmt(c, 0u, half ? 0x4442u : 0x4440u);
+        const int g = (int)prmt(c, 0u, half ? 0xBBB3u : 0x9991u);   // sign-extended
+        const uint32_t s0 = 0x7604u | ((uint32_t)(2 * pass) << 4), s1 = s0 + 0x10u;
+        const uint32_t a0 = prmt(w, base, s0), a1 = prmt(w, base, s1);
+        red32<0>(a0, h);
+        red32<128>(a0, g);
+        red32<65536>(a1, h);
+        red32<65536 + 128>(a1, g);
+    }
+}
+
+struct Out {
+    unsigned long long *ptr;   // partial slot of this CTA, or the final histogram
+    bool direct;               // final layout hist[f][bin] instead of partial [k][bin][a]
+    bool first;                // nothing stored yet: store instead of accumulate
+};
+
+// Adds the CTA's local histogram into its output and clears it.  The R replicas of a column
+// (the row slots of word a) are R adjacent shared words, so one thread sums them from vector
+// loads and writes one packed 64-bit bin.
+template <bool WIDE>
+__device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, int nb, int pass, Out &out) {
+    const int W = 1 << logW, R = 32 >> logW;
+    const int per_k = nb << logW;                                   // outputs per byte position k
+    for (int kk = 0; kk < (WIDE ? 2 : 4); ++kk) {
+        const int k = WIDE ? 2 * pass + kk : kk;
+        for (int e = threadIdx.x; e < per_k; e += HIST_THREADS) {
+            const int a = e & (W - 1), bin = e >> logW;
+            unsigned long long v;
+            if (!WIDE) {
+                int *p = hp + (kk >> 1) * 16384 + bin * 64 + (kk & 1) * 32 + a * R;
+                int G = 0, H = 0;
+                if (R >= 4) {
+                    for (int r = 0; r < R; r += 4) {
+                        const int4 x = *reinterpret_cast<const int4 *>(p + r);
+                        *reinterpret_cast<int4 *>(p + r) = make_int4(0, 0, 0, 0);
+                        G += (x.x >> 16) + (x.y >> 16) + (x.z >> 16) + (x.w >> 16);
+                        H += (x.x & 0xFFFF) + (x.y & 0xFFFF) + (x.z & 0xFFFF) + (x.w & 0xFFFF);
+                    }
+                } else {
+                    for (int r = 0; r < R; ++r) {
+                        const int x = p[r];
+                        p[r] = 0;
+                        G += x >> 16;
+                        H += x & 0xFFFF;
+                    }
+                }
+                v = (unsigned long long)((long long)G * 4294967296LL + (long long)H);
+            } else {
+                // two 32-bit planes per bin; no field can overflow (checked at load time)
+                int *p = hp + kk * 16384 + bin * 64 + a * R;
+                long long G = 0;
+                unsigned long long H = 0;
+                for (int r = 0; r < R; ++r) {
+                    H += (unsigned int)p[r];
+                    G += p[32 + r];
+                    p[r] = 0;
+                    p[32 + r] = 0;
+                }
+                v = (unsigned long long)(G * 4294967296LL + (long long)H);
+            }
+            const int fl = 4 * a + k;
+            if (fl < td.nf) {
+                unsigned long long *q = out.direct ? out.ptr + (size_t)(td.f0 + fl) * nb + bin
+                                                   : out.ptr + (size_t)k * nb * W + e;
+                if (!out.first) v += *q;
+                *q = v;
+            }
+        }
+    }
+    out.first = false;
+}
+
+// CTAs of the static plan that take part in a build of n rows of a tile.
+__device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
+    uint32_t want = (n + MIN_ROWS_PER_CTA - 1) / MIN_ROWS_PER_CTA;
+    if (want < 1) want = 1;
+    return want < parts ? want : parts;
+}
+
+// The work of a lane is cut into units of four rows.  Contiguous rows: unit v covers rows
+// 16 (v / 4) + 4 j + v % 4, j = 0..3, whose codes are the four adjacent 16-bit values codes[4v ..].
+// Row list: warp-unit q covers list entries 4 R q .. 4 R (q + 1) - 1, entry 4 R q + R j + slot for
+// the lane's j-th row.  A warp instruction spans R units (one per row slot): a "warp-unit".
+//
+// LOGW_T >= 0 fixes the tile width at compile time (all strides become immediates); -1 reads it
+// from the tile.  The grid is (part, tile - tile0).
+// One CTA's share (part `part` of P) of the histogram of a.n rows for tile td.  `sh` is the
+// CTA's dynamic shared memory (HIST_SMEM bytes).  Ends with the CTA's local histogram flushed.
+template <int LOGW_T, bool WIDE, int LIST>
+__device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, const uint32_t part, const uint32_t P,
+                                         int *sh) {
+    const uint32_t n = a.n;
+
+    const uint32_t sbase = smem_u32(sh);
+    const uint32_t h0 = (sbase + 65535u) & ~65535u;
+    uint32_t dyn_size;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_size));
+    if (h0 + 131072u > sbase + dyn_size) {   // the launches leave room; never write out of bounds
+        if (threadIdx.x == 0) atomicExch(&a.state->kernel_error, 1);
+        return;
+    }
+    int *hp = sh + (h0 - sbase) / 4;
+    const int lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
+    for (int i = threadIdx.x; i < a.nb * 64; i += HIST_THREADS) {
+        hp[i] = 0;
+        hp[16384 + i] = 0;
+    }
+    __syncthreads();
+
+    const int logW = LOGW_T >= 0 ? LOGW_T : td.logW;
+    const int logR = 5 - logW;
+    const uint32_t R = 1u << logR;
+    const uint32_t wa = lane >> logR;           // word of the row held by this lane
+    const uint32_t slot = lane & (R - 1);       // row slot of this lane (adjacent lanes: replicas of a column)
+    const uint32_t base = h0 + lane * 4;
+    const uint32_t *tile = td.data;
+    const int pass = a.pass;
+
+    Out out;
+    out.direct = P == 1;
+    out.first = true;   // the two passes of the 32+32 mode write different features
+    out.ptr = out.direct ? a.hist : a.partial + (size_t)(td.cta0 + part) * 4 * a.nb * 32;
+
+    // ---- range of this part in warp-units [0, q1) from its first unit, and the leftover rows /
+    //      entries [s0, s1) that are done one by one
+    uint32_t q1, s0, s1, first_unit = 0, first_q = 0;
+    if (!LIST) {
+        const uint32_t B = n >> 4;                                   // full blocks of 16 rows
+        const uint32_t b0 = (uint32_t)((unsigned long long)B * part / P);
+        const uint32_t b1 = (uint32_t)((unsigned long long)B * (part + 1) / P);
+        first_unit = b0 << 2;
+        if (logR >= 2) {                                             // a warp-unit is R / 4 whole blocks
+            const int lb = logR >= 2 ? logR - 2 : 0;                 // log2 of blocks per warp-unit
+            q1 = (b1 - b0) >> lb;
+            s0 = (b0 + (q1 << lb)) << 4;
+        } else {                                                     // 4 / R warp-units per block
+            q1 = (b1 - b0) << (2 - logR);
+            s0 = b1 << 4;
+        }
+        s1 = part + 1 == P ? n : b1 << 4;
+    } else {
+        const uint32_t per = 4u << logR;                             // entries per warp-unit
+        const uint32_t Q = n / per;                                  // full warp-units
+        first_q = (uint32_t)((unsigned long long)Q * part / P);
+        q1 = (uint32_t)((unsigned long long)Q * (part + 1) / P) - first_q;
+        s0 = part + 1 == P ? Q * per : 0;
+        s1 = part + 1 == P ? n : 0;
+    }
+
+    // ---- leftover rows first (the column counters are still zero): R rows per warp instruction
+    uint32_t col_rows = 0;   // rows any one column may hold since the last flush
+    if (s1 > s0) {
+        for (uint32_t i = s0 + warp * R + slot; i < s1; i += HIST_WARPS * R) {
+            uint32_t row, c;
+            if (LIST == 2) {
+                const uint2 e = __ldcg(a.ents + a.off + i);
+                row = e.x;
+                c = e.y;
+            } else {
+                row = LIST ? a.rows[a.off + i] : i;
+                c = a.codes_nat[row];
+            }
+            const uint32_t w = tile[((size_t)row << logW) + wa];
+            add_word<WIDE>(base, w, c, 0, pass);
+        }
+        col_rows = (s1 - s0 + R - 1) >> logR;
+    }
+
+    // ---- fast warp-units, in epochs that keep every 16+16 column below its limit
+    constexpr int U = LIST ? U_LIST : U_ROOT;
+    uint32_t q = 0;
+    while (q < q1) {
+        uint32_t epoch = q1 - q;   // warp-units of this epoch, all warps together
+        if (!WIDE) {
+            const uint32_t room = a.flush_rows > col_rows ? a.flush_rows - col_rows : 0;
+            const uint32_t fit = room >> 2;                          // every warp-unit adds 4 rows to each column
+            if (fit == 0) {
+                __syncthreads();
+                flush_local<WIDE>(hp, td, logW, a.nb, pass, out);
+                __syncthreads();
+                col_rows = 0;
+                continue;
+            }
+            if (fit < epoch) epoch = fit;
+        }
+        // this warp's warp-units: q + warp, q + warp + 32, ... < q + epoch
+        const uint32_t nq = epoch > (uint32_t)warp ? (epoch - warp + HIST_WARPS - 1) / HIST_WARPS : 0;
+        if (!LIST) {
+            const uint32_t v = first_unit + ((q + warp) << logR) + slot;         // first unit of this lane
+            const uint32_t row0 = ((v >> 2) << 4) + (v & 3u);
+            const uint32_t *pw = tile + ((size_t)row0 << logW) + wa;
+            const uint2 *pc = reinterpret_cast<const uint2 *>(a.codes) + v;
+            const uint32_t jstride = 4u << logW;                                  // words between rows 4 apart
+            constexpr uint32_t QW = 32 * 128;                                     // words per 32 warp-units
+            const uint32_t qc = 32u << logR;                                      // units per 32 warp-units
+            uint32_t w[U][4];
+            uint2 c[U];
+#define QG_LOAD_UNIT(u)                                                                  \
+    {                                                                                    \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) w[u][j] = ldg32(pw + (u) * QW + j * jstride); \
+        c[u] = ldg64(pc + (u) * qc);                                                     \
+    }
+#define QG_USE_UNIT(u)                                       \
+    {                                                        \
+        add_word<WIDE>(base, w[u][0], c[u].x, 0, pass);      \
+        add_word<WIDE>(base, w[u][1], c[u].x, 1, pass);      \
+        add_word<WIDE>(base, w[u][2], c[u].y, 0, pass);      \
+        add_word<WIDE>(base, w[u][3], c[u].y, 1, pass);      \
+    }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if ((uint32_t)u < nq) QG_LOAD_UNIT(u)
+            pw += U * QW;
+            pc += U * qc;
+            uint32_t i = 0;
+            for (; i + 2 * U <= nq; i += U) {   // units i .. i+U-1 are in registers, the next U exist
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    QG_USE_UNIT(u)
+                    QG_LOAD_UNIT(u)
+                }
+                pw += U * QW;
+                pc += U * qc;
+            }
+            for (; i < nq; i += U) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (i + u < nq) {
+                        QG_USE_UNIT(u)
+                        if (i + u + U < nq) QG_LOAD_UNIT(u)
+                    }
+                }
+                pw += U * QW;
+                pc += U * qc;
+            }
+#undef QG_LOAD_UNIT
+#undef QG_USE_UNIT
+        } else {
+            // entry of (warp-unit wu, j): off + (4 wu << logR) + (j << logR) + slot
+            const size_t e0 = a.off + ((size_t)(first_q + q + warp) << (logR + 2)) + slot;
+            const uint32_t *pr = LIST == 2 ? nullptr : a.rows + e0;
+            const uint2 *pe = LIST == 2 ? a.ents + e0 : nullptr;
+            const uint32_t qs = 128u << logR;                                     // entries per 32 warp-units
+            const uint32_t *tw = tile + wa;
+            uint32_t idx[U][4], w[U][4], c[U][4];
+            uint32_t cn[LIST == 2 ? U : 1][4];   // codes that came with the indices (pair entries)
+#define QG_LOAD_IDX(u)                                                                \
+    {                                                                                 \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) {                               \
+            if (LIST == 2) {                                                          \
+                const uint2 e = __ldcg(pe + (u) * qs + ((uint32_t)j << logR));        \
+                idx[u][j] = e.x;                                                      \
+                cn[LIST == 2 ? (u) : 0][j] = e.y;                                     \
+            } else {                                                                  \
+                idx[u][j] = pr[(u) * qs + ((uint32_t)j << logR)];                     \
+            }                                                                         \
+        }                                                                             \
+    }
+#define QG_LOAD_DATA(u)                                                \
+    {                                                                  \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) {                \
+            w[u][j] = ldg32(tw + ((size_t)idx[u][j] << logW));         \
+            if (LIST == 2) c[u][j] = cn[LIST == 2 ? (u) : 0][j];       \
+            else c[u][j] = ldg16(a.codes_nat + idx[u][j]);             \
+        }                                                              \
+    }
+#define QG_USE_DATA(u)                                                                           \
+    {                                                                                            \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) add_word<WIDE>(base, w[u][j], c[u][j], 0, pass); \
+    }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if ((uint32_t)u < nq) QG_LOAD_IDX(u)
+            if (LIST == 2) pe += U * qs; else pr += U * qs;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if ((uint32_t)u < nq) {
+                    QG_LOAD_DATA(u)
+                    if ((uint32_t)u + U < nq) QG_LOAD_IDX(u)
+                }
+            if (LIST == 2) pe += U * qs; else pr += U * qs;
+            uint32_t i = 0;
+            for (; i + 3 * U <= nq; i += U) {   // data of units i .. i+U-1 and indices of the next U are in registers
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    QG_USE_DATA(u)
+                    QG_LOAD_DATA(u)
+                    QG_LOAD_IDX(u)
+                }
+                if (LIST == 2) pe += U * qs; else pr += U * qs;
+            }
+            for (; i < nq; i += U) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (i + u < nq) {
+                        QG_USE_DATA(u)
+                        if (i + u + U < nq) {
+                            QG_LOAD_DATA(u)
+                            if (i + u + 2 * U < nq) QG_LOAD_IDX(u)
+                        }
+                    }
+                }
+                if (LIST == 2) pe += U * qs; else pr += U * qs;
+            }
+#undef QG_LOAD_IDX
+#undef QG_LOAD_DATA
+#undef QG_USE_DATA
+        }
+        q += epoch;
+        col_rows += 4 * epoch;
+    }
+    __syncthreads();
+    flush_local<WIDE>(hp, td, logW, a.nb, pass, out);
+}
+
+}  // namespace

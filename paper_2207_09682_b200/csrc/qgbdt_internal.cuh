@@ -204,5 +204,4 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
 
 // grow.cu: one tree by leaf-wise growth, every decision taken on the device
 int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st);
-// hist.cu: histogram of the smaller child of the split recorded in the grow state
-int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st);
+

@@ -61,6 +61,8 @@ void free_data(qgbdt_ctx *c) {
     dev_free(c->d_h);
     dev_free(c->d_hist_pool);
     dev_free(c->d_leaves);
+    dev_free(c->d_ent0);
+    dev_free(c->d_ent1);
     dev_free(c->d_cand);
     dev_free(c->d_feat_tile);
     dev_free(c->d_m_num_leaves);

@@ -61,7 +61,7 @@ struct SplitRec {
 };
 
 // One leaf of the tree being grown (device memory).  Its rows are entries [off, off + n) of the
-// row-index buffer `buf` (0 or 1; -1: the identity list of the root).
+// (row, code) pair buffer `buf` (0 or 1; -1: the identity list of the root).
 struct LeafRec {
     uint32_t off, n;
     int32_t buf;
@@ -71,20 +71,10 @@ struct LeafRec {
     int32_t parent_node, parent_side;
 };
 
-// State of leaf-wise growth kept on the device, so that a tree grows without the host looking:
-// the split being executed and counters.
+// What the tree-growing kernel leaves behind for the refit kernels and the counters.
 struct GrowState {
-    int32_t n_leaves, done;
-    int32_t pick, feature, bin;      // leaf being split and its winning candidate
-    int32_t tile, word, byte;        // where the split feature sits in the tiled matrix
-    uint32_t off, n;                 // rows of the leaf being split
-    int32_t buf;                     // their index buffer
-    uint32_t nl;                     // rows that go left (written by the scatter kernel)
-    long long gl, hl, PG, PH;        // left totals of the candidate, totals of the leaf
-    double gain;
-    int32_t parent_slot;
-    unsigned int finish_count;       // blocks of the finishing kernel that are through
-    unsigned long long hist_rows;    // rows visited by histogram builds of row lists
+    int32_t n_leaves, pad;
+    unsigned long long hist_rows;    // rows visited by histogram builds of row lists (all trees so far)
     unsigned long long hist_builds;
 };
 
@@ -129,6 +119,7 @@ struct qgbdt_ctx {
     float *d_g = nullptr, *d_h = nullptr;
     unsigned long long *d_hist_pool = nullptr;  // [L][F][nb]
     LeafRec *d_leaves = nullptr;                // [L]
+    uint2 *d_ent0 = nullptr, *d_ent1 = nullptr; // [N] (row, gradient code) pairs of the leaves, two buffers
     GrowState *d_gs = nullptr;
     SplitRec *d_cand = nullptr;                 // [F][2] per-feature best candidates of the two children
     int32_t *d_feat_tile = nullptr;             // [F] tile of every feature

@@ -24,16 +24,17 @@ __device__ inline long long to_fixed(float v) { return __double2ll_rn(__dmul_rn(
 
 // table: [n_leaves] offsets ascending, then [n_leaves] leaf ids.  sums: [n_leaves][2] by slot.
 // gs != nullptr: a tree grown on the device: the leaf count comes from *gs and the table's third
-// part [n_leaves] says which index buffer holds a leaf's rows (-1: the identity list).
-__device__ inline uint32_t leaf_row(const uint32_t *idx0, const uint32_t *idx1, const uint32_t *table, int n_leaves,
-                                    bool grown, int s, uint32_t p) {
-    if (!grown) return idx0[p];
+// part [n_leaves] says which (row, code) pair buffer holds a leaf's rows (-1: the identity list).
+__device__ inline uint32_t leaf_row(const uint32_t *idx, const uint2 *ent0, const uint2 *ent1, const uint32_t *table,
+                                    int n_leaves, bool grown, int s, uint32_t p) {
+    if (!grown) return idx[p];
     const int buf = (int)table[2 * n_leaves + s];
-    return buf < 0 ? p : (buf ? idx1[p] : idx0[p]);
+    return buf < 0 ? p : (buf ? ent1[p].x : ent0[p].x);
 }
 
 __global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__restrict__ idx,
-                                                              const uint32_t *__restrict__ idx1, uint32_t n,
+                                                              const uint2 *__restrict__ ent0,
+                                                              const uint2 *__restrict__ ent1, uint32_t n,
                                                               const uint32_t *__restrict__ table, int n_leaves,
                                                               const GrowState *gs, const float *__restrict__ g,
                                                               const float *__restrict__ h,
@@ -57,7 +58,7 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__
         long long gf = 0, hf = 0;
         if (ok) {
             s = slot_of(offs, n_leaves, p);
-            const uint32_t row = leaf_row(idx, idx1, table, n_leaves, grown, s, p);
+            const uint32_t row = leaf_row(idx, ent0, ent1, table, n_leaves, grown, s, p);
             gf = to_fixed(g[row]);
             hf = h ? to_fixed(h[row]) : 1073741824LL;
         }
@@ -111,7 +112,8 @@ __global__ void k_leaf_values(const long long *__restrict__ sums, const uint32_t
 }
 
 __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *__restrict__ idx,
-                                                                const uint32_t *__restrict__ idx1, uint32_t n,
+                                                                const uint2 *__restrict__ ent0,
+                                                                const uint2 *__restrict__ ent1, uint32_t n,
                                                                 const uint32_t *__restrict__ table, int n_leaves,
                                                                 const GrowState *gs,
                                                                 const float *__restrict__ values,
@@ -123,7 +125,7 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *
     __syncthreads();
     for (uint32_t p = blockIdx.x * REFIT_THREADS + threadIdx.x; p < n; p += gridDim.x * REFIT_THREADS) {
         const int s = slot_of(offs, n_leaves, p);
-        const uint32_t row = leaf_row(idx, idx1, table, n_leaves, grown, s, p);
+        const uint32_t row = leaf_row(idx, ent0, ent1, table, n_leaves, grown, s, p);
         scores[row] = __fadd_rn(scores[row], values[table[n_leaves + s]]);
     }
 }
@@ -182,8 +184,9 @@ int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st) 
     if (rc != QGBDT_OK) return rc;
     QG_CUDA(c, cudaMemsetAsync(c->d_leaf_sums, 0, sizeof(long long) * 2 * L, st));
     const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
-    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, nullptr, (uint32_t)c->N, c->d_leaf_table,
-                                                                     L, nullptr, d_g, d_h, c->d_leaf_sums);
+    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, nullptr, nullptr, (uint32_t)c->N,
+                                                                     c->d_leaf_table, L, nullptr, d_g, d_h,
+                                                                     c->d_leaf_sums);
     QG_LAUNCH_CHECK(c);
     k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, c->d_leaf_table, L, nullptr, c->prm.lambda_l2,
                                                    c->prm.learning_rate, c->d_leaf_w, c->d_leaf_value);
@@ -196,7 +199,7 @@ int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st) {
     const int L = c->n_leaves;
     unsigned blocks = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
     if (blocks > (unsigned)c->sm_count * 16) blocks = (unsigned)c->sm_count * 16;
-    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, nullptr, (uint32_t)c->N,
+    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, nullptr, nullptr, (uint32_t)c->N,
                                                                        c->d_leaf_table, L, nullptr, c->d_leaf_value,
                                                                        d_scores);
     QG_LAUNCH_CHECK(c);
@@ -211,7 +214,7 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
                                     c->d_m_num_leaves + tree_slot, c->d_m_leaf_count + (size_t)tree_slot * L);
     QG_LAUNCH_CHECK(c);
     const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
-    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, c->d_idx_tmp, (uint32_t)c->N,
+    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
                                                                      c->d_leaf_table, L, c->d_gs, d_g, d_h,
                                                                      c->d_leaf_sums);
     QG_LAUNCH_CHECK(c);
@@ -221,7 +224,7 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
     QG_LAUNCH_CHECK(c);
     unsigned ab = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
     if (ab > (unsigned)c->sm_count * 16) ab = (unsigned)c->sm_count * 16;
-    k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, c->d_idx_tmp, (uint32_t)c->N,
+    k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
                                                                    c->d_leaf_table, L, c->d_gs,
                                                                    c->d_m_leaf_value + (size_t)tree_slot * L, d_scores);
     QG_LAUNCH_CHECK(c);

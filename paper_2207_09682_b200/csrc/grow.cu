@@ -22,6 +22,9 @@ namespace cg = cooperative_groups;
 
 namespace {
 
+constexpr int GROW_THREADS = 512;   // 128 registers per thread: the phases keep their state out of local memory
+constexpr int GROW_WARPS = GROW_THREADS / 32;
+
 struct GrowArgs {
     GrowState *gs;
     LeafRec *leaves;
@@ -76,41 +79,49 @@ __device__ inline void warp_range(uint32_t nw, uint32_t gw, uint32_t n_count, ui
 // The split being executed, identical in every CTA.
 struct Cur {
     int pick, feature, bin, buf, slot, parent_node, parent_side;
+    const uint32_t *col;   // word of the split feature in row 0 of its tile
+    int logW, shift;       // words per row (log2) of that tile, bit position of the feature's byte
     uint32_t off, n;
     long long gl, hl, PG, PH;
     double gain;
 };
 
-// (B) predicate bits and left counts.
-__device__ __noinline__ void phase_flags(const GrowArgs &a, const Cur &cur, uint32_t gw, uint32_t n_count, int lane) {
+// (B) predicate bits and left counts.  Four words of 32 rows at a time, so that the dependent
+// loads (pair -> bin word) of the four are in flight together.
+__device__ __forceinline__ void phase_flags(const GrowArgs &a, const Cur &cur, uint32_t gw, uint32_t n_count, int lane) {
     const uint32_t nw = (cur.n + 31) >> 5;
     uint32_t w0, w1, active;
     warp_range(nw, gw, n_count, w0, w1, active);
     if (gw >= active) return;
     const uint2 *src = cur.buf < 0 ? nullptr : (cur.buf ? a.ent1 : a.ent0);
-    const int t = a.feat_tile[cur.feature];
-    const TileDesc td = a.h.tiles[t];
-    const int fl = cur.feature - td.f0;
-    const uint32_t *col = td.data + (fl >> 2);
-    const int logW = td.logW, shift = 8 * (fl & 3);
-    const uint32_t thr = (uint32_t)cur.bin;
+    const uint32_t *col = cur.col;
+    const int logW = cur.logW, shift = cur.shift;
+    const uint32_t thr = (uint32_t)cur.bin, n = cur.n, off = cur.off;
     uint32_t lefts = 0;
-    for (uint32_t w = w0; w < w1; ++w) {
-        const uint32_t e = (w << 5) + lane;
-        bool left = false;
-        if (e < cur.n) {
-            const uint32_t row = src ? __ldcg(&src[cur.off + e].x) : cur.off + e;
-            left = ((col[(size_t)row << logW] >> shift) & 0xFFu) <= thr;
+    for (uint32_t w = w0; w < w1; w += 4) {
+        uint32_t row[4], word[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t e = ((w + k) << 5) + lane;
+            row[k] = (w + k < w1 && e < n) ? (src ? __ldcg(&src[off + e].x) : off + e) : 0xFFFFFFFFu;
         }
-        const uint32_t b = __ballot_sync(0xffffffffu, left);
-        if (lane == 0) a.bits[w] = b;
-        lefts += __popc(b);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) word[k] = row[k] != 0xFFFFFFFFu ? col[(size_t)row[k] << logW] : 0xFFFFFFFFu;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool left = row[k] != 0xFFFFFFFFu && ((word[k] >> shift) & 0xFFu) <= thr;
+            const uint32_t b = __ballot_sync(0xffffffffu, left);
+            if (w + k < w1) {
+                if (lane == 0) a.bits[w + k] = b;
+                lefts += __popc(b);
+            }
+        }
     }
     if (lane == 0) a.counts[gw] = lefts;
 }
 
 // Left rows before warp gw's range and in the whole leaf (sums of the warp counts).
-__device__ __noinline__ void count_lefts(const GrowArgs &a, const Cur &cur, uint32_t gw, uint32_t n_count, int lane,
+__device__ __forceinline__ void count_lefts(const GrowArgs &a, const Cur &cur, uint32_t gw, uint32_t n_count, int lane,
                                    uint32_t &before, uint32_t &total) {
     const uint32_t nw = (cur.n + 31) >> 5;
     uint32_t w0, w1, active;
@@ -129,7 +140,7 @@ __device__ __noinline__ void count_lefts(const GrowArgs &a, const Cur &cur, uint
 }
 
 // (C) stable scatter of (row, code) pairs: left rows first, relative order kept.
-__device__ __noinline__ void phase_scatter(const GrowArgs &a, const Cur &cur, uint32_t gw, uint32_t n_count, int lane,
+__device__ __forceinline__ void phase_scatter(const GrowArgs &a, const Cur &cur, uint32_t gw, uint32_t n_count, int lane,
                                      uint32_t before, uint32_t total) {
     const uint32_t nw = (cur.n + 31) >> 5;
     uint32_t w0, w1, active;
@@ -137,23 +148,35 @@ __device__ __noinline__ void phase_scatter(const GrowArgs &a, const Cur &cur, ui
     if (gw >= active) return;
     const uint2 *src = cur.buf < 0 ? nullptr : (cur.buf ? a.ent1 : a.ent0);
     uint2 *dst = cur.buf == 0 ? a.ent1 : a.ent0;
-    for (uint32_t w = w0; w < w1; ++w) {
-        const uint32_t bw = __ldcg(a.bits + w);
-        const uint32_t e = (w << 5) + lane;
-        if (e < cur.n) {
-            uint2 ent;
-            if (src) {
-                ent = __ldcg(src + cur.off + e);
-            } else {
-                ent.x = cur.off + e;
-                ent.y = a.h.codes_nat[ent.x];
+    const uint32_t n = cur.n, off = cur.off;
+    for (uint32_t w = w0; w < w1; w += 4) {
+        uint32_t bw[4];
+        uint2 ent[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t e = ((w + k) << 5) + lane;
+            const bool ok = w + k < w1 && e < n;
+            bw[k] = w + k < w1 ? __ldcg(a.bits + w + k) : 0u;
+            if (ok) {
+                if (src) {
+                    ent[k] = __ldcg(src + off + e);
+                } else {
+                    ent[k].x = off + e;
+                    ent[k].y = a.h.codes_nat[off + e];
+                }
             }
-            const uint32_t rank_l = __popc(bw & ((1u << lane) - 1u));
-            const bool left = (bw >> lane) & 1u;
-            const uint32_t dest = left ? before + rank_l : total + ((w << 5) - before) + (lane - rank_l);
-            dst[cur.off + dest] = ent;
         }
-        before += __popc(bw);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t e = ((w + k) << 5) + lane;
+            if (w + k < w1 && e < n) {
+                const uint32_t rank_l = __popc(bw[k] & ((1u << lane) - 1u));
+                const bool left = (bw[k] >> lane) & 1u;
+                const uint32_t dest = left ? before + rank_l : total + (((w + k) << 5) - before) + (lane - rank_l);
+                dst[off + dest] = ent[k];
+            }
+            before += __popc(bw[k]);
+        }
     }
 }
 
@@ -172,7 +195,7 @@ struct FinishCtx {
 // of the smaller child and takes the larger child's bin by subtraction; warps 0 and 1 of the
 // group then scan the two children's bins.
 template <bool ROOT>
-__device__ __noinline__ void finish_feature(const GrowArgs &a, const FinishCtx &fc, int f, int grp,
+__device__ __forceinline__ void finish_feature(const GrowArgs &a, const FinishCtx &fc, int f, int grp,
                                       unsigned long long *binS, unsigned long long *binL) {
     const int gt = threadIdx.x & 255, gwarp = gt >> 5, lane = gt & 31;
     const int nb = a.h.nb;
@@ -195,17 +218,13 @@ __device__ __noinline__ void finish_feature(const GrowArgs &a, const FinishCtx &
             } else {
                 if (P > 1) {
                     const unsigned long long *q = part + (size_t)b * W;
-                    unsigned long long s0 = 0, s1 = 0, s2 = 0, s3 = 0;
-                    uint32_t i = 0;
-                    for (; i + 8 <= P; i += 8) {
-                        const unsigned long long x0 = __ldcg(q + (size_t)i * pstride), x1 = __ldcg(q + (size_t)(i + 1) * pstride);
-                        const unsigned long long x2 = __ldcg(q + (size_t)(i + 2) * pstride), x3 = __ldcg(q + (size_t)(i + 3) * pstride);
-                        const unsigned long long x4 = __ldcg(q + (size_t)(i + 4) * pstride), x5 = __ldcg(q + (size_t)(i + 5) * pstride);
-                        const unsigned long long x6 = __ldcg(q + (size_t)(i + 6) * pstride), x7 = __ldcg(q + (size_t)(i + 7) * pstride);
-                        s0 += x0 + x4; s1 += x1 + x5; s2 += x2 + x6; s3 += x3 + x7;
+                    for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
+                        unsigned long long x[16];
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? __ldcg(q + (size_t)(i0 + k) * pstride) : 0ull;
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) s += x[k];
                     }
-                    for (; i < P; ++i) s0 += __ldcg(q + (size_t)i * pstride);
-                    s = (s0 + s1) + (s2 + s3);
                     S[b] = s;
                 } else {
                     s = __ldcg(S + b);
@@ -247,29 +266,31 @@ __device__ inline SplitRec warp_best(SplitRec r) {
     return r;
 }
 
-// (F) best candidate over all features for child `side` (0 small, 1 large); the result is valid
-// in every thread.  s_red: [32] scratch.
-__device__ __noinline__ SplitRec reduce_cand(const GrowArgs &a, int side, SplitRec *s_red) {
-    SplitRec b = qg_invalid_rec();
-    for (int f = threadIdx.x; f < a.F; f += HIST_THREADS) {
-        const SplitRec x = load_rec_cg(a.cand + 2 * f + side);
-        if (qg_rec_better(x, b)) b = x;
+// (F) best candidates over all features for the two children (0 small, 1 large); the results are
+// valid in every thread.  s_red: [2][32] scratch.
+__device__ __forceinline__ void reduce_cand(const GrowArgs &a, SplitRec *s_red, SplitRec &outS, SplitRec &outL) {
+    SplitRec bS = qg_invalid_rec(), bL = qg_invalid_rec();
+    for (int f = threadIdx.x; f < a.F; f += GROW_THREADS) {
+        const SplitRec x = load_rec_cg(a.cand + 2 * f), y = load_rec_cg(a.cand + 2 * f + 1);
+        if (qg_rec_better(x, bS)) bS = x;
+        if (qg_rec_better(y, bL)) bL = y;
     }
-    b = warp_best(b);
+    bS = warp_best(bS);
+    bL = warp_best(bL);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __syncthreads();
-    if (lane == 0) s_red[warp] = b;
+    if (lane == 0) { s_red[warp] = bS; s_red[32 + warp] = bL; }
     __syncthreads();
-    b = s_red[lane];
-    return warp_best(b);
+    outS = warp_best(lane < GROW_WARPS ? s_red[lane] : qg_invalid_rec());
+    outL = warp_best(lane < GROW_WARPS ? s_red[32 + lane] : qg_invalid_rec());
 }
 
 // Leaf with the largest gain (lowest number on equal gain) among sh_gain[0 .. n), or -1.
-__device__ __noinline__ int pick_leaf(const double *sh_gain, int n, double *s_pg, int *s_pi) {
+__device__ __forceinline__ int pick_leaf(const double *sh_gain, int n, double *s_pg, int *s_pi) {
     const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
     double bg = NEG;
     int bi = -1;
-    for (int i = threadIdx.x; i < n; i += HIST_THREADS) {
+    for (int i = threadIdx.x; i < n; i += GROW_THREADS) {
         const double g = sh_gain[i];
         if (g > bg) { bg = g; bi = i; }   // ascending i: the first maximum stays
     }
@@ -282,8 +303,8 @@ __device__ __noinline__ int pick_leaf(const double *sh_gain, int n, double *s_pg
     __syncthreads();
     if (lane == 0) { s_pg[warp] = bg; s_pi[warp] = bi; }
     __syncthreads();
-    bg = s_pg[lane];
-    bi = s_pi[lane];
+    bg = lane < GROW_WARPS ? s_pg[lane] : NEG;
+    bi = lane < GROW_WARPS ? s_pi[lane] : -1;
     for (int o = 16; o > 0; o >>= 1) {
         const double og = __shfl_xor_sync(0xffffffffu, bg, o);
         const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
@@ -295,24 +316,35 @@ __device__ __noinline__ int pick_leaf(const double *sh_gain, int n, double *s_pg
 template <bool WIDE>
 __device__ __forceinline__ void run_hist_unit(HistArgs &ha, const TileDesc &td, uint32_t part, uint32_t P, int *sh) {
     for (int pass = 0; pass < (WIDE ? 2 : 1); ++pass) {
-        ha.pass = pass;
+        if (WIDE) {
+            if (threadIdx.x == 0) ha.pass = pass;
+            __syncthreads();
+        }
         switch (td.logW) {
-            case 5: hist_cta<5, WIDE, 2>(ha, td, part, P, sh); break;
-            case 3: hist_cta<3, WIDE, 2>(ha, td, part, P, sh); break;
-            default: hist_cta<-1, WIDE, 2>(ha, td, part, P, sh); break;
+            case 5: hist_cta<GROW_THREADS, 5, WIDE, 2>(ha, td, part, P, sh); break;
+            case 3: hist_cta<GROW_THREADS, 3, WIDE, 2>(ha, td, part, P, sh); break;
+            default: hist_cta<GROW_THREADS, -1, WIDE, 2>(ha, td, part, P, sh); break;
         }
         __syncthreads();   // the local histogram is reused by the next pass / unit
     }
 }
 
 template <bool WIDE>
-__global__ void __launch_bounds__(HIST_THREADS, 1) k_grow(GrowArgs a) {
+__global__ void __launch_bounds__(GROW_THREADS, 1) k_grow(const GrowArgs args) {
     extern __shared__ __align__(1024) int sh[];
+    // arguments and per-split context live in shared memory: with 210 KB of it carved out there is
+    // hardly any L1 left for per-thread local copies
+    __shared__ GrowArgs s_args;
+    __shared__ FinishCtx s_fc;
+    __shared__ HistArgs s_ha;
+    if (threadIdx.x == 0) s_args = args;
+    __syncthreads();
+    const GrowArgs &a = s_args;
     cg::grid_group grid = cg::this_grid();
     const uint32_t G = gridDim.x, cta = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
-    const uint32_t n_count = G * HIST_WARPS, gw = cta * HIST_WARPS + warp;
+    const uint32_t n_count = G * GROW_WARPS, gw = (uint32_t)warp * G + cta;   // neighbouring ranges on different SMs
     const int grp = tid >> 8;
     const int nb = a.h.nb;
     const size_t hw = (size_t)a.F * nb;
@@ -327,30 +359,35 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_grow(GrowArgs a) {
         return;   // every CTA takes this branch: no barrier is left waiting
     }
     double *sh_gain = reinterpret_cast<double *>(sh);
-    __shared__ unsigned long long s_bins[4][2][256];
-    __shared__ SplitRec s_red[32];
+    __shared__ unsigned long long s_bins[GROW_THREADS / 256][2][256];
+    __shared__ SplitRec s_red[64];
     __shared__ double s_pg[32];
     __shared__ int s_pi[32];
     __shared__ Cur s_cur;
     __shared__ LeafRec s_child[2];
     __shared__ int s_child_id[2];
     const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
-    for (int i = tid; i < a.L; i += HIST_THREADS) sh_gain[i] = NEG;
+    for (int i = tid; i < a.L; i += GROW_THREADS) sh_gain[i] = NEG;
 
     // ---- root: scan its histogram (pool slot 0, built before this kernel)
     const long long G0 = a.state->tot_g, H0 = a.state->tot_h;
-    FinishCtx fc;
-    fc.pS = a.sp; fc.pL = a.sp;
-    fc.pS.G = G0; fc.pS.H = H0; fc.pS.n_s = a.N;
-    qg_scales(a.state, fc.pS, fc.dg, fc.dh);
-    fc.tpS = qg_gain_term(G0, H0, fc.dg, fc.dh, fc.pS.lambda);
-    fc.tpL = 0.0;
-    fc.n_small = a.N; fc.new_slot = 0; fc.parent_slot = 0;
-    for (int f = (int)cta * 4 + grp; f < a.F; f += (int)G * 4) finish_feature<true>(a, fc, f, grp, s_bins[grp][0], s_bins[grp][1]);
+    FinishCtx &fc = s_fc;
+    if (tid == 0) {
+        fc.pS = a.sp; fc.pL = a.sp;
+        fc.pS.G = G0; fc.pS.H = H0; fc.pS.n_s = a.N;
+        qg_scales(a.state, fc.pS, fc.dg, fc.dh);
+        fc.tpS = qg_gain_term(G0, H0, fc.dg, fc.dh, fc.pS.lambda);
+        fc.tpL = 0.0;
+        fc.n_small = a.N; fc.new_slot = 0; fc.parent_slot = 0;
+        s_ha = a.h;
+    }
+    __syncthreads();
+    for (int f = (int)cta * (GROW_THREADS / 256) + grp; f < a.F; f += (int)G * (GROW_THREADS / 256)) finish_feature<true>(a, fc, f, grp, s_bins[grp][0], s_bins[grp][1]);
     __syncthreads();
     grid.sync();
     {
-        const SplitRec b = reduce_cand(a, 0, s_red);
+        SplitRec b, unused;
+        reduce_cand(a, s_red, b, unused);
         if (tid == 0) {
             LeafRec r;
             r.off = 0; r.n = a.N; r.buf = -1; r.slot = 0; r.G = G0; r.H = H0; r.best = b;
@@ -375,11 +412,18 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_grow(GrowArgs a) {
             Cur c;
             c.pick = pick; c.feature = r.best.feature; c.bin = r.best.bin; c.buf = r.buf; c.slot = r.slot;
             c.parent_node = r.parent_node; c.parent_side = r.parent_side;
+            {
+                const TileDesc td = a.h.tiles[a.feat_tile[r.best.feature]];
+                const int fl = r.best.feature - td.f0;
+                c.col = td.data + (fl >> 2);
+                c.logW = td.logW;
+                c.shift = 8 * (fl & 3);
+            }
             c.off = r.off; c.n = r.n; c.gl = r.best.gl; c.hl = r.best.hl; c.PG = r.G; c.PH = r.H; c.gain = r.best.gain;
             s_cur = c;
         }
         __syncthreads();
-        const Cur cur = s_cur;
+        const Cur &cur = s_cur;
 
         // ---- (B) flags
         phase_flags(a, cur, gw, n_count, lane);
@@ -394,12 +438,15 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_grow(GrowArgs a) {
         grid.sync();
         // ---- (D) histogram of the smaller child (ties: the left one) into pool slot n_leaves
         {
-            HistArgs ha = a.h;
-            ha.ents = cur.buf == 0 ? a.ent1 : a.ent0;
-            ha.rows = nullptr;
-            ha.off = small_is_left ? cur.off : cur.off + nl;
-            ha.n = n_small;
-            ha.hist = a.pool + (size_t)n_leaves * hw;
+            HistArgs &ha = s_ha;
+            if (tid == 0) {
+                ha.ents = cur.buf == 0 ? a.ent1 : a.ent0;
+                ha.rows = nullptr;
+                ha.off = small_is_left ? cur.off : cur.off + nl;
+                ha.n = n_small;
+                ha.hist = a.pool + (size_t)n_leaves * hw;
+            }
+            __syncthreads();
             uint32_t ubase = 0;
             for (int t = 0; t < a.n_tiles; ++t) {
                 const TileDesc td = a.h.tiles[t];
@@ -410,21 +457,22 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_grow(GrowArgs a) {
         }
         grid.sync();
         // ---- (E) per feature: merge, subtract, scan
-        {
+        if (tid == 0) {
             const long long gl = cur.gl, hl = cur.hl, gr = cur.PG - gl, hr = cur.PH - hl;
             fc.pS.G = small_is_left ? gl : gr; fc.pS.H = small_is_left ? hl : hr; fc.pS.n_s = small_is_left ? nl : nr;
             fc.pL.G = small_is_left ? gr : gl; fc.pL.H = small_is_left ? hr : hl; fc.pL.n_s = small_is_left ? nr : nl;
             fc.tpS = qg_gain_term(fc.pS.G, fc.pS.H, fc.dg, fc.dh, fc.pS.lambda);
             fc.tpL = qg_gain_term(fc.pL.G, fc.pL.H, fc.dg, fc.dh, fc.pL.lambda);
             fc.n_small = n_small; fc.new_slot = n_leaves; fc.parent_slot = cur.slot;
-            for (int f = (int)cta * 4 + grp; f < a.F; f += (int)G * 4)
-                finish_feature<false>(a, fc, f, grp, s_bins[grp][0], s_bins[grp][1]);
         }
+        __syncthreads();
+        for (int f = (int)cta * (GROW_THREADS / 256) + grp; f < a.F; f += (int)G * (GROW_THREADS / 256))
+            finish_feature<false>(a, fc, f, grp, s_bins[grp][0], s_bins[grp][1]);
         __syncthreads();
         grid.sync();
         // ---- (F) every CTA: the children's best splits, the new leaves, the gains
-        const SplitRec bS = reduce_cand(a, 0, s_red);
-        const SplitRec bL = reduce_cand(a, 1, s_red);
+        SplitRec bS, bL;
+        reduce_cand(a, s_red, bS, bL);
         if (tid == 0) {
             const int right = n_leaves, node = n_leaves - 1;
             const int dstbuf = cur.buf == 0 ? 1 : 0;
@@ -528,13 +576,13 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
         int coop = 0, per_sm = 0;
         QG_CUDA(c, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
-        QG_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, HIST_THREADS, HIST_SMEM));
+        QG_CUDA(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, GROW_THREADS, HIST_SMEM));
         if (!coop || per_sm < 1)
             return qg_fail(c, QGBDT_ERR_CUDA, "the device cannot co-schedule one tree-growing CTA per SM");
         configured[wide ? 1 : 0] = true;
     }
     void *params[] = {&a};
-    QG_CUDA(c, cudaLaunchCooperativeKernel(kern, dim3((unsigned)c->sm_count), dim3(HIST_THREADS), params, HIST_SMEM, st));
+    QG_CUDA(c, cudaLaunchCooperativeKernel(kern, dim3((unsigned)c->sm_count), dim3(GROW_THREADS), params, HIST_SMEM, st));
     c->n_launches++;
     return QGBDT_OK;
 }

@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
     const uint32_t P = effective_parts((uint32_t)td.parts, a.n);
     if (blockIdx.x >= P) return;
-    hist_cta<LOGW_T, WIDE, LIST>(a, td, blockIdx.x, P, sh);
+    hist_cta<HIST_THREADS, LOGW_T, WIDE, LIST>(a, td, blockIdx.x, P, sh);
 }
 
 // Sums the partial histograms of every tile that was built by more than one CTA.  A block takes

@@ -10,8 +10,9 @@ constexpr int HIST_THREADS = 1024;
 constexpr int HIST_WARPS = HIST_THREADS / 32;
 constexpr int HIST_SMEM = 192 * 1024;     // 128 KB histogram on a 64 KB boundary + the room below it
 constexpr uint32_t MIN_ROWS_PER_CTA = 4096;
-constexpr int U_ROOT = 4;                 // units in flight per lane, contiguous rows
-constexpr int U_LIST = 2;                 // units in flight per lane, row list (plus as many index units)
+// Units of four rows in flight per lane.  A CTA of 512 threads (the tree-growing kernel) has twice
+// the registers per thread and keeps more in flight per lane to make up for the fewer warps.
+template <int NT> struct Units { static constexpr int root = NT >= 1024 ? 4 : 6, list = NT >= 1024 ? 2 : 4; };
 
 struct HistArgs {
     const TileDesc *tiles;
@@ -93,13 +94,13 @@ struct Out {
 // Adds the CTA's local histogram into its output and clears it.  The R replicas of a column
 // (the row slots of word a) are R adjacent shared words, so one thread sums them from vector
 // loads and writes one packed 64-bit bin.
-template <bool WIDE>
+template <int NT, bool WIDE>
 __device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, int nb, int pass, Out &out) {
     const int W = 1 << logW, R = 32 >> logW;
     const int per_k = nb << logW;                                   // outputs per byte position k
     for (int kk = 0; kk < (WIDE ? 2 : 4); ++kk) {
         const int k = WIDE ? 2 * pass + kk : kk;
-        for (int e = threadIdx.x; e < per_k; e += HIST_THREADS) {
+        for (int e = threadIdx.x; e < per_k; e += NT) {
             const int a = e & (W - 1), bin = e >> logW;
             unsigned long long v;
             if (!WIDE) {
@@ -162,7 +163,7 @@ __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) 
 // from the tile.  The grid is (part, tile - tile0).
 // One CTA's share (part `part` of P) of the histogram of a.n rows for tile td.  `sh` is the
 // CTA's dynamic shared memory (HIST_SMEM bytes).  Ends with the CTA's local histogram flushed.
-template <int LOGW_T, bool WIDE, int LIST>
+template <int NT, int LOGW_T, bool WIDE, int LIST>
 __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, const uint32_t part, const uint32_t P,
                                          int *sh) {
     const uint32_t n = a.n;
@@ -178,7 +179,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     int *hp = sh + (h0 - sbase) / 4;
     const int lane = threadIdx.x & 31;
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
-    for (int i = threadIdx.x; i < a.nb * 64; i += HIST_THREADS) {
+    for (int i = threadIdx.x; i < a.nb * 64; i += NT) {
         hp[i] = 0;
         hp[16384 + i] = 0;
     }
@@ -227,7 +228,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     // ---- leftover rows first (the column counters are still zero): R rows per warp instruction
     uint32_t col_rows = 0;   // rows any one column may hold since the last flush
     if (s1 > s0) {
-        for (uint32_t i = s0 + warp * R + slot; i < s1; i += HIST_WARPS * R) {
+        for (uint32_t i = s0 + warp * R + slot; i < s1; i += (NT / 32) * R) {
             uint32_t row, c;
             if (LIST == 2) {
                 const uint2 e = __ldcg(a.ents + a.off + i);
@@ -244,7 +245,8 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     }
 
     // ---- fast warp-units, in epochs that keep every 16+16 column below its limit
-    constexpr int U = LIST ? U_LIST : U_ROOT;
+    constexpr int U = LIST ? Units<NT>::list : Units<NT>::root;
+    constexpr int NWARPS = NT / 32;
     uint32_t q = 0;
     while (q < q1) {
         uint32_t epoch = q1 - q;   // warp-units of this epoch, all warps together
@@ -253,7 +255,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
             const uint32_t fit = room >> 2;                          // every warp-unit adds 4 rows to each column
             if (fit == 0) {
                 __syncthreads();
-                flush_local<WIDE>(hp, td, logW, a.nb, pass, out);
+                flush_local<NT, WIDE>(hp, td, logW, a.nb, pass, out);
                 __syncthreads();
                 col_rows = 0;
                 continue;
@@ -261,15 +263,15 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
             if (fit < epoch) epoch = fit;
         }
         // this warp's warp-units: q + warp, q + warp + 32, ... < q + epoch
-        const uint32_t nq = epoch > (uint32_t)warp ? (epoch - warp + HIST_WARPS - 1) / HIST_WARPS : 0;
+        const uint32_t nq = epoch > (uint32_t)warp ? (epoch - warp + NWARPS - 1) / NWARPS : 0;
         if (!LIST) {
             const uint32_t v = first_unit + ((q + warp) << logR) + slot;         // first unit of this lane
             const uint32_t row0 = ((v >> 2) << 4) + (v & 3u);
             const uint32_t *pw = tile + ((size_t)row0 << logW) + wa;
             const uint2 *pc = reinterpret_cast<const uint2 *>(a.codes) + v;
             const uint32_t jstride = 4u << logW;                                  // words between rows 4 apart
-            constexpr uint32_t QW = 32 * 128;                                     // words per 32 warp-units
-            const uint32_t qc = 32u << logR;                                      // units per 32 warp-units
+            constexpr uint32_t QW = NWARPS * 128;                                 // words per round of the CTA's warps
+            const uint32_t qc = (uint32_t)NWARPS << logR;                         // units per round of the CTA's warps
             uint32_t w[U][4];
             uint2 c[U];
 #define QG_LOAD_UNIT(u)                                                                  \
@@ -317,7 +319,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
             const size_t e0 = a.off + ((size_t)(first_q + q + warp) << (logR + 2)) + slot;
             const uint32_t *pr = LIST == 2 ? nullptr : a.rows + e0;
             const uint2 *pe = LIST == 2 ? a.ents + e0 : nullptr;
-            const uint32_t qs = 128u << logR;                                     // entries per 32 warp-units
+            const uint32_t qs = (uint32_t)(4 * NWARPS) << logR;                   // entries per round of the CTA's warps
             const uint32_t *tw = tile + wa;
             uint32_t idx[U][4], w[U][4], c[U][4];
             uint32_t cn[LIST == 2 ? U : 1][4];   // codes that came with the indices (pair entries)
@@ -387,7 +389,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
         col_rows += 4 * epoch;
     }
     __syncthreads();
-    flush_local<WIDE>(hp, td, logW, a.nb, pass, out);
+    flush_local<NT, WIDE>(hp, td, logW, a.nb, pass, out);
 }
 
 }  // namespace

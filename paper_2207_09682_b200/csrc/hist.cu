@@ -40,6 +40,32 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     hist_cta<HIST_THREADS, LOGW_T, WIDE, LIST>(a, td, blockIdx.x, P, sh);
 }
 
+// Tree growth: the rows are the smaller child (ties: the left one) of the split recorded in the
+// grow state, as (row, code) pairs in the buffer the scatter kernel wrote; the histogram goes to
+// the pool slot numbered like the leaf about to be created.  The grid is (max parts, tile - tile0).
+struct GrowHist {
+    const GrowState *gs;
+    const uint2 *ent0, *ent1;
+    unsigned long long *pool;
+    size_t hist_words;
+};
+
+template <int LOGW_T, bool WIDE>
+__global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowHist g) {
+    extern __shared__ __align__(1024) int sh[];
+    const GrowState *gs = g.gs;
+    if (gs->done) return;
+    const uint32_t nl = gs->nl, nr = gs->n - nl;
+    a.ents = gs->buf == 0 ? g.ent1 : g.ent0;
+    a.off = nl <= nr ? gs->off : gs->off + nl;
+    a.n = nl <= nr ? nl : nr;
+    a.hist = g.pool + (size_t)gs->n_leaves * g.hist_words;
+    const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
+    const uint32_t P = effective_parts((uint32_t)td.parts, a.n);
+    if (blockIdx.x >= P) return;
+    hist_cta<HIST_THREADS, LOGW_T, WIDE, 2>(a, td, blockIdx.x, P, sh);
+}
+
 // Sums the partial histograms of every tile that was built by more than one CTA.  A block takes
 // 32 consecutive partial entries; its eight thread groups each add every eighth partial.
 __global__ void __launch_bounds__(256) k_hist_reduce(const TileDesc *__restrict__ tiles, uint32_t n, int nb,
@@ -197,6 +223,100 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
     }
     if (ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
     return QGBDT_OK;
+}
+
+namespace {
+
+template <int LOGW_T, bool WIDE>
+int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n_tiles, cudaStream_t st) {
+    auto kern = k_hist_grow<LOGW_T, WIDE>;
+    static bool configured = false;   // per instantiation
+    if (!configured) {
+        QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
+        configured = true;
+    }
+    int group_parts = 1;
+    for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
+        if (c->tiles[t].parts > group_parts) group_parts = c->tiles[t].parts;
+    kern<<<dim3((unsigned)group_parts, (unsigned)n_tiles), HIST_THREADS, HIST_SMEM, st>>>(args, g);
+    QG_LAUNCH_CHECK(c);
+    return QGBDT_OK;
+}
+
+template <bool WIDE>
+int launch_grow(qgbdt_ctx *c, HistArgs args, const GrowHist &g, cudaStream_t st) {
+    const int T = (int)c->tiles.size();
+    for (int t0 = 0; t0 < T;) {
+        int t1 = t0 + 1;
+        while (t1 < T && c->tiles[t1].logW == c->tiles[t0].logW) ++t1;
+        args.tile0 = t0;
+        int rc;
+        switch (c->tiles[t0].logW) {
+            case 5: rc = launch_grow_one<5, WIDE>(c, args, g, t1 - t0, st); break;
+            case 3: rc = launch_grow_one<3, WIDE>(c, args, g, t1 - t0, st); break;
+            default: rc = launch_grow_one<-1, WIDE>(c, args, g, t1 - t0, st); break;
+        }
+        if (rc != QGBDT_OK) return rc;
+        t0 = t1;
+    }
+    return QGBDT_OK;
+}
+
+}  // namespace
+
+// Histogram of the smaller child of the split recorded in the grow state (sizes known only on
+// the device): partial histograms or, for a small child, the finished histogram in its pool slot.
+int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
+    const int bits = c->prm.bits;
+    const int kg = qg_levels_g(bits);
+    const int kh = c->const_hess ? 1 : qg_levels_h(bits, c->prm.hess_levels_mode);
+    HistArgs a;
+    a.tiles = c->d_tiles;
+    a.codes = reinterpret_cast<const uint16_t *>(c->d_codes);
+    a.codes_nat = reinterpret_cast<const uint16_t *>(c->d_codes_nat);
+    a.tile0 = 0;
+    a.rows = nullptr;
+    a.ents = nullptr;
+    a.off = 0;
+    a.n = 0;
+    a.nb = c->nb;
+    a.hist = nullptr;
+    a.partial = c->d_partial;
+    const uint32_t by_h = 65535u / (uint32_t)kh, by_g = 32767u / (uint32_t)kg;
+    a.flush_rows = by_h < by_g ? by_h : by_g;
+    a.pass = 0;
+    a.state = c->d_state;
+    GrowHist g;
+    g.gs = c->d_gs;
+    g.ent0 = c->d_ent0;
+    g.ent1 = c->d_ent1;
+    g.pool = c->d_hist_pool;
+    g.hist_words = (size_t)c->F * c->nb;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (c->profile_hist) {
+        if (c->hist_events_used + 2 > c->hist_events.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                QG_CUDA(c, cudaEventCreate(&e));
+                c->hist_events.push_back(e);
+            }
+        }
+        ev0 = c->hist_events[c->hist_events_used++];
+        ev1 = c->hist_events[c->hist_events_used++];
+        QG_CUDA(c, cudaEventRecord(ev0, st));
+    }
+    int rc;
+    if (bits < 6) {
+        rc = launch_grow<false>(c, a, g, st);
+    } else {
+        rc = launch_grow<true>(c, a, g, st);
+        if (rc == QGBDT_OK) {
+            a.pass = 1;
+            rc = launch_grow<true>(c, a, g, st);
+        }
+    }
+    if (rc == QGBDT_OK && ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
+    return rc;
 }
 
 int qg_subtract(qgbdt_ctx *c, const unsigned long long *d_parent, const unsigned long long *d_small,

@@ -71,9 +71,20 @@ struct LeafRec {
     int32_t parent_node, parent_side;
 };
 
-// What the tree-growing kernel leaves behind for the refit kernels and the counters.
+// State of leaf-wise growth kept on the device, so that a tree grows without the host looking:
+// the split being executed and counters.
 struct GrowState {
-    int32_t n_leaves, pad;
+    int32_t n_leaves, done;
+    int32_t pick, feature, bin;      // leaf being split and its winning candidate
+    int32_t logW, byte;              // tile width (log2 words per row) and byte of the split feature's word
+    const uint32_t *col;             // that word in row 0 of the tile
+    uint32_t off, n;                 // rows of the leaf being split
+    int32_t buf;                     // their pair buffer
+    uint32_t nl;                     // rows that go left (written by the scatter kernel)
+    long long gl, hl, PG, PH;        // left totals of the candidate, totals of the leaf
+    double gain;
+    int32_t parent_slot;
+    unsigned int finish_count;       // blocks of the finishing kernel that are through
     unsigned long long hist_rows;    // rows visited by histogram builds of row lists (all trees so far)
     unsigned long long hist_builds;
 };
@@ -195,4 +206,6 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
 
 // grow.cu: one tree by leaf-wise growth, every decision taken on the device
 int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st);
+// hist.cu: histogram of the smaller child of the split recorded in the grow state
+int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st);
 

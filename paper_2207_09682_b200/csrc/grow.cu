@@ -200,9 +200,8 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
         pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl : nr;
         pL.G = small_is_left ? gr : gl; pL.H = small_is_left ? hr : hl; pL.n_s = small_is_left ? nr : nl;
     }
-    // ---- phase A: one thread per bin (groups of 256 bins): the smaller child's sum over the
-    //      partial histograms, the larger child's bin by subtraction; both kept for the scans
-    __shared__ unsigned long long binS[256], binL[256];
+    // ---- phase A: one thread per bin: the smaller child's sum over the partial histograms, the
+    //      larger child's bin by subtraction
     __shared__ SplitRec sm[2][FIN_WARPS * 32];
     __shared__ bool is_last;
     double dg, dh;
@@ -216,51 +215,84 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     const unsigned long long *part = a.partial + (size_t)td.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
     unsigned long long *S = a.pool + (ROOT ? 0 : (size_t)n_leaves * hw) + (size_t)f * a.nb;
     unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)gs->parent_slot * hw + (size_t)f * a.nb;
-    ScanState sc;
-    qg_scan_init(sc);
-    for (int base = 0; base < a.nb; base += 256) {
-        const int b = base + (int)threadIdx.x;
-        unsigned long long s = 0, l = 0;
-        if (b < a.nb) {
-            if (ROOT) {
-                s = S[b];
-            } else {
-                if (P > 1) {
-                    const unsigned long long *q = part + (size_t)b * W;
-                    for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
-                        unsigned long long x[16];
+    // n_bins <= 256: thread b owns bin b
+    const int b = (int)threadIdx.x;
+    unsigned long long s = 0, l = 0;
+    if (b < a.nb) {
+        if (ROOT) {
+            s = S[b];
+        } else {
+            if (P > 1) {
+                const unsigned long long *q = part + (size_t)b * W;
+                for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
+                    unsigned long long x[16];
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
+                    for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) s += x[k];
-                    }
-                    S[b] = s;
-                } else {
-                    s = S[b];
+                    for (int k = 0; k < 16; ++k) s += x[k];
                 }
-                l = Pp[b] - s;   // no field borrows: every child sum is at most the parent's
-                Pp[b] = l;
+                S[b] = s;
+            } else {
+                s = S[b];
             }
+            l = Pp[b] - s;   // no field borrows: every child sum is at most the parent's
+            Pp[b] = l;
         }
-        binS[threadIdx.x] = s;
-        binL[threadIdx.x] = l;
-        __syncthreads();
-        // ---- phase B: warp 0 scans the smaller child's bins, warp 1 the larger child's
-        if (warp < (ROOT ? 1 : 2)) {
-            const unsigned long long *bins = warp == 0 ? binS : binL;
-            const SplitParams &pp = warp == 0 ? pS : pL;
-            const double tp = warp == 0 ? tpS : tpL;
-            for (int g = 0; g < 256 && base + g < a.nb; g += 32)
-                qg_scan_step(sc, bins[g + lane], base + g + lane, a.nb, pp, dg, dh, tp);
-        }
-        __syncthreads();
     }
-    if (warp < 2) {
-        const SplitRec r = (ROOT && warp == 1) ? qg_invalid_rec() : qg_scan_finish(sc, f);
-        if (lane == 0) {
-            a.cand[2 * f + warp] = r;
-            __threadfence();
+    // ---- phase B: prefix sums over the bins by all eight warps (warp scan, then the warp totals),
+    //      every thread evaluates the threshold at its own bin for both children
+    __shared__ long long wtot[4][FIN_WARPS];
+    const bool in = b < a.nb - 1;   // thresholds 0 .. nb-2
+    long long v[4];
+    v[0] = in ? (long long)(int)(s >> 32) : 0;
+    v[1] = in ? (long long)(unsigned int)(s & 0xFFFFFFFFull) : 0;
+    v[2] = in ? (long long)(int)(l >> 32) : 0;
+    v[3] = in ? (long long)(unsigned int)(l & 0xFFFFFFFFull) : 0;
+#pragma unroll
+    for (int c = 0; c < (ROOT ? 2 : 4); ++c) {
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long u = __shfl_up_sync(0xffffffffu, v[c], o);
+            if (lane >= o) v[c] += u;
         }
+        if (lane == 31) wtot[c][warp] = v[c];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < (ROOT ? 2 : 4); ++c)
+        for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
+    SplitRec rS = qg_invalid_rec(), rL = qg_invalid_rec();
+    rS.feature = f;
+    rL.feature = f;
+    if (in) {
+        double gain;
+        if (qg_eval_candidate(v[0], v[1], pS, dg, dh, tpS, gain)) {
+            rS.valid = 1; rS.gain = gain; rS.bin = b; rS.gl = v[0]; rS.hl = v[1];
+        }
+        if (!ROOT && qg_eval_candidate(v[2], v[3], pL, dg, dh, tpL, gain)) {
+            rL.valid = 1; rL.gain = gain; rL.bin = b; rL.gl = v[2]; rL.hl = v[3];
+        }
+    }
+    // best threshold of the feature: largest gain, lowest bin on equal gain
+    for (int o = 16; o > 0; o >>= 1) {
+        SplitRec x = rS, y = rL;
+        x.gain = __shfl_xor_sync(0xffffffffu, rS.gain, o); y.gain = __shfl_xor_sync(0xffffffffu, rL.gain, o);
+        x.gl = __shfl_xor_sync(0xffffffffu, rS.gl, o);     y.gl = __shfl_xor_sync(0xffffffffu, rL.gl, o);
+        x.hl = __shfl_xor_sync(0xffffffffu, rS.hl, o);     y.hl = __shfl_xor_sync(0xffffffffu, rL.hl, o);
+        x.bin = __shfl_xor_sync(0xffffffffu, rS.bin, o);   y.bin = __shfl_xor_sync(0xffffffffu, rL.bin, o);
+        x.valid = __shfl_xor_sync(0xffffffffu, rS.valid, o); y.valid = __shfl_xor_sync(0xffffffffu, rL.valid, o);
+        if (qg_better(x.valid != 0, x.gain, x.bin, rS.valid != 0, rS.gain, rS.bin)) rS = x;
+        if (qg_better(y.valid != 0, y.gain, y.bin, rL.valid != 0, rL.gain, rL.bin)) rL = y;
+    }
+    if (lane == 0) { sm[0][warp] = rS; sm[1][warp] = rL; }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+        SplitRec r = sm[threadIdx.x][0];
+        for (int w = 1; w < FIN_WARPS; ++w) {
+            const SplitRec o = sm[threadIdx.x][w];
+            if (qg_better(o.valid != 0, o.gain, o.bin, r.valid != 0, r.gain, r.bin)) r = o;
+        }
+        a.cand[2 * f + threadIdx.x] = r;
+        __threadfence();
     }
     __syncthreads();
     if (threadIdx.x == 0) is_last = atomicAdd(&gs->finish_count, 1u) == gridDim.x - 1;

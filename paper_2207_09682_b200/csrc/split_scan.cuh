@@ -32,6 +32,24 @@ __device__ inline void qg_scales(const DevState *state, const SplitParams &p, do
     dh = p.const_h ? 1.0 : __ddiv_rn((double)__uint_as_float(state->hmax_bits), (double)p.kh);
 }
 
+// Threshold candidate with left sums (gl, hl): admissible?  If so its gain (Eq. 7).
+__device__ inline bool qg_eval_candidate(long long gl, long long hl, const SplitParams &p, double dg, double dh,
+                                         double tp, double &gain) {
+    const long long gr = p.G - gl, hr = p.H - hl;
+    if (!(hl > 0 && hr > 0)) return false;
+    long long nl;
+    if (p.const_h) nl = hl;
+    else nl = (long long)(((unsigned long long)hl * (unsigned long long)p.n_s + (unsigned long long)(p.H / 2)) /
+                          (unsigned long long)p.H);
+    const long long nr = p.n_s - nl;
+    if (!(nl >= p.min_data && nr >= p.min_data)) return false;
+    if (__dmul_rn((double)hl, dh) < p.min_sum_h || __dmul_rn((double)hr, dh) < p.min_sum_h) return false;
+    const double tl = qg_gain_term(gl, hl, dg, dh, p.lambda);
+    const double tr = qg_gain_term(gr, hr, dg, dh, p.lambda);
+    gain = __dmul_rn(0.5, __dsub_rn(__dadd_rn(tl, tr), tp));
+    return gain > p.min_gain;
+}
+
 // Running state of one feature's scan in one lane.
 struct ScanState {
     long long carry_g, carry_h;   // sums of the bins before the current group of 32
@@ -64,22 +82,9 @@ __device__ inline void qg_scan_step(ScanState &s, unsigned long long word, int t
     s.carry_g += __shfl_sync(0xffffffffu, g, 31);
     s.carry_h += __shfl_sync(0xffffffffu, h, 31);
     if (t < nb - 1) {
-        const long long gr = p.G - gl, hr = p.H - hl;
-        if (hl > 0 && hr > 0) {
-            long long nl;
-            if (p.const_h) nl = hl;
-            else nl = (long long)(((unsigned long long)hl * (unsigned long long)p.n_s +
-                                   (unsigned long long)(p.H / 2)) / (unsigned long long)p.H);
-            const long long nr = p.n_s - nl;
-            if (nl >= p.min_data && nr >= p.min_data &&
-                !(__dmul_rn((double)hl, dh) < p.min_sum_h) && !(__dmul_rn((double)hr, dh) < p.min_sum_h)) {
-                const double tl = qg_gain_term(gl, hl, dg, dh, p.lambda);
-                const double tr = qg_gain_term(gr, hr, dg, dh, p.lambda);
-                const double gain = __dmul_rn(0.5, __dsub_rn(__dadd_rn(tl, tr), tp));
-                if (gain > p.min_gain && (!s.bv || gain > s.bgain)) {
-                    s.bv = true; s.bgain = gain; s.bbin = t; s.bgl = gl; s.bhl = hl;
-                }
-            }
+        double gain;
+        if (qg_eval_candidate(gl, hl, p, dg, dh, tp, gain) && (!s.bv || gain > s.bgain)) {
+            s.bv = true; s.bgain = gain; s.bbin = t; s.bgl = gl; s.bhl = hl;
         }
     }
 }

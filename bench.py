@@ -30,6 +30,24 @@ sys.path.insert(0, ROOT)
 WORKLOAD_ROWS = {"large": 10_500_000, "tall": 1_000_000, "tiny": 50_000, "wide": 400_000}
 CPU_SAMPLE_ROWS = {"large": 3_000_000, "tall": 1_000_000, "tiny": 50_000, "wide": 20_000}
 FALLBACK_HBM_GBS = 6650.0
+# DRAM traffic of the histogram kernels on the 'large' workload from an ncu capture
+# (profiles/launch_list_large_10p5Mx28.md): 3.4 GB over the 255 builds of one tree.  Valid only for
+# the kernel sources the capture was taken with.
+HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 13.3e6,
+                "sources_sha1": "657c2a2975a875cce83c8dcd0aab0ef666cfcefa"}
+
+
+def hist_traffic(workload, rows):
+    import hashlib
+    h = hashlib.sha1()
+    try:
+        for f in ("hist_cta.cuh", "hist.cu", "grow.cu"):
+            h.update(open(os.path.join(ROOT, "paper_2207_09682_b200", "csrc", f), "rb").read())
+    except OSError:
+        return None
+    if workload != HIST_TRAFFIC["workload"] or rows != WORKLOAD_ROWS[workload] or h.hexdigest() != HIST_TRAFFIC["sources_sha1"]:
+        return None      # the kernel changed since the counters were taken (or another workload)
+    return HIST_TRAFFIC["bytes_per_launch"]
 
 
 def measured_peak():
@@ -206,6 +224,20 @@ def run_sweep(args):
                 del bins
 
 
+def aggregate_ranks(ms, row_features, launches, dist=None, device="cpu"):
+    """Whole-job figures from per-rank ones: the step time is the maximum over the ranks, work and
+    launch counts add up.  The ranks are independent replicas (no data-path collective): this is
+    the only exchange of a multi-GPU run."""
+    import torch
+    if dist is None:
+        return float(ms), float(row_features), float(launches)
+    t = torch.tensor([ms, float(row_features), float(launches)], dtype=torch.float64, device=device)
+    tmax = t.clone()
+    dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(tmax[0]), float(t[1]), float(t[2])
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -253,12 +285,7 @@ def run_ours(args):
     launches = c1["kernel_launches"] - c0["kernel_launches"]
     leaves = [int(x) for x in model.num_leaves]
 
-    t = torch.tensor([ms, float(rf), float(launches)], dtype=torch.float64, device="cuda")
-    if dist:
-        tmax = t.clone()
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        ms, rf, launches = float(tmax[0]), float(t[1]), float(t[2])
+    ms, rf, launches = aggregate_ranks(ms, rf, launches, dist, "cuda")
     if rank != 0:
         dist.destroy_process_group()
         return
@@ -277,7 +304,9 @@ def run_ours(args):
                    "leaves_per_tree": [min(leaves), max(leaves)]},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": peak_kind, "kernel": "k_hist",
+                     "traffic": hist_traffic(args.workload, n), "peak_kind": peak_kind,
+                     "kernel": "k_hist / k_hist_grow (+ merge): every histogram build of the timed trees",
+                     "algorithmic_bytes_per_launch": prof["total_bytes"] / max(prof["builds"], 1),
                      "launches": prof["builds"], "total_ms": prof["total_ms"],
                      "share_of_step": prof["total_ms"] / ms if ms else None},
         "clocks": clocks.summary(),

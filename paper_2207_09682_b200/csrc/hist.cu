@@ -31,13 +31,13 @@
 namespace {
 
 // Stand-alone build: the grid is (part, tile - tile0).
-template <int LOGW_T, bool WIDE, int LIST>
+template <int LOGW_T, int MODE, int LIST>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     extern __shared__ __align__(1024) int sh[];
     const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
     const uint32_t P = effective_parts((uint32_t)td.parts, a.n);
     if (blockIdx.x >= P) return;
-    hist_cta<HIST_THREADS, LOGW_T, WIDE, LIST>(a, td, blockIdx.x, P, sh);
+    hist_cta<HIST_THREADS, LOGW_T, MODE, LIST>(a, td, blockIdx.x, P, sh);
 }
 
 // Tree growth: the rows are the smaller child (ties: the left one) of the split recorded in the
@@ -50,7 +50,7 @@ struct GrowHist {
     size_t hist_words;
 };
 
-template <int LOGW_T, bool WIDE>
+template <int LOGW_T, int MODE>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowHist g) {
     extern __shared__ __align__(1024) int sh[];
     const GrowState *gs = g.gs;
@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowH
     const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
     const uint32_t P = effective_parts((uint32_t)td.parts, a.n);
     if (blockIdx.x >= P) return;
-    hist_cta<HIST_THREADS, LOGW_T, WIDE, 2>(a, td, blockIdx.x, P, sh);
+    hist_cta<HIST_THREADS, LOGW_T, MODE, 2>(a, td, blockIdx.x, P, sh);
 }
 
 // Sums the partial histograms of every tile that was built by more than one CTA.  A block takes
@@ -117,9 +117,9 @@ __global__ void k_subtract(const unsigned long long *__restrict__ parent, const 
         large[i] = parent[i] - small[i];
 }
 
-template <int LOGW_T, bool WIDE, int LIST>
+template <int LOGW_T, int MODE, int LIST>
 int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st) {
-    auto kern = k_hist<LOGW_T, WIDE, LIST>;
+    auto kern = k_hist<LOGW_T, MODE, LIST>;
     static bool configured = false;   // per instantiation
     if (!configured) {
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
@@ -135,7 +135,7 @@ int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st)
 }
 
 // One launch per run of tiles of equal width (the full 128-feature tiles, then the remainder).
-template <bool WIDE, int LIST>
+template <int MODE, int LIST>
 int launch_hist(qgbdt_ctx *c, HistArgs args, cudaStream_t st) {
     const int T = (int)c->tiles.size();
     for (int t0 = 0; t0 < T;) {
@@ -144,14 +144,32 @@ int launch_hist(qgbdt_ctx *c, HistArgs args, cudaStream_t st) {
         args.tile0 = t0;
         int rc;
         switch (c->tiles[t0].logW) {
-            case 5: rc = launch_one<5, WIDE, LIST>(c, args, t1 - t0, st); break;
-            case 3: rc = launch_one<3, WIDE, LIST>(c, args, t1 - t0, st); break;
-            default: rc = launch_one<-1, WIDE, LIST>(c, args, t1 - t0, st); break;
+            case 5: rc = launch_one<5, MODE, LIST>(c, args, t1 - t0, st); break;
+            case 3: rc = launch_one<3, MODE, LIST>(c, args, t1 - t0, st); break;
+            default: rc = launch_one<-1, MODE, LIST>(c, args, t1 - t0, st); break;
         }
         if (rc != QGBDT_OK) return rc;
         t0 = t1;
     }
     return QGBDT_OK;
+}
+
+// Narrow local bins: where to split the 32-bit word between the gradient sum (above) and the
+// hessian sum (below) so that a column can take the most rows before it must be flushed.  The
+// 16+16 split has the one-instruction decode and is kept unless another split at least doubles
+// the rows (a constant hessian counts rows in the low field: 14 bits are enough for 16383 of them).
+void pick_field_split(int kg, int kh, int &shift, uint32_t &rows) {
+    auto rows_at = [&](int s) {
+        const uint32_t by_h = ((1u << s) - 1u) / (uint32_t)kh, by_g = ((1u << (31 - s)) - 1u) / (uint32_t)kg;
+        return by_h < by_g ? by_h : by_g;
+    };
+    shift = 16;
+    rows = rows_at(16);
+    for (int s = 10; s <= 22; ++s)
+        if (rows_at(s) >= 2 * rows_at(16) && rows_at(s) > rows) {
+            shift = s;
+            rows = rows_at(s);
+        }
 }
 
 }  // namespace
@@ -184,8 +202,7 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
     a.nb = c->nb;
     a.hist = d_hist;
     a.partial = c->d_partial;
-    const uint32_t by_h = 65535u / (uint32_t)kh, by_g = 32767u / (uint32_t)kg;
-    a.flush_rows = by_h < by_g ? by_h : by_g;
+    pick_field_split(kg, kh, a.shift, a.flush_rows);
     a.pass = 0;
     a.state = c->d_state;
 
@@ -206,13 +223,15 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
         QG_CUDA(c, cudaEventRecord(ev0, st));
     }
     int rc;
-    if (!wide) {
-        rc = d_rows ? launch_hist<false, 1>(c, a, st) : launch_hist<false, 0>(c, a, st);
+    if (!wide && a.shift == 16) {
+        rc = d_rows ? launch_hist<0, 1>(c, a, st) : launch_hist<0, 0>(c, a, st);
+    } else if (!wide) {
+        rc = d_rows ? launch_hist<2, 1>(c, a, st) : launch_hist<2, 0>(c, a, st);
     } else {
-        rc = d_rows ? launch_hist<true, 1>(c, a, st) : launch_hist<true, 0>(c, a, st);
+        rc = d_rows ? launch_hist<1, 1>(c, a, st) : launch_hist<1, 0>(c, a, st);
         if (rc == QGBDT_OK) {
             a.pass = 1;
-            rc = d_rows ? launch_hist<true, 1>(c, a, st) : launch_hist<true, 0>(c, a, st);
+            rc = d_rows ? launch_hist<1, 1>(c, a, st) : launch_hist<1, 0>(c, a, st);
         }
     }
     if (rc != QGBDT_OK) return rc;
@@ -227,9 +246,9 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
 
 namespace {
 
-template <int LOGW_T, bool WIDE>
+template <int LOGW_T, int MODE>
 int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n_tiles, cudaStream_t st) {
-    auto kern = k_hist_grow<LOGW_T, WIDE>;
+    auto kern = k_hist_grow<LOGW_T, MODE>;
     static bool configured = false;   // per instantiation
     if (!configured) {
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
@@ -243,7 +262,7 @@ int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n
     return QGBDT_OK;
 }
 
-template <bool WIDE>
+template <int MODE>
 int launch_grow(qgbdt_ctx *c, HistArgs args, const GrowHist &g, cudaStream_t st) {
     const int T = (int)c->tiles.size();
     for (int t0 = 0; t0 < T;) {
@@ -252,9 +271,9 @@ int launch_grow(qgbdt_ctx *c, HistArgs args, const GrowHist &g, cudaStream_t st)
         args.tile0 = t0;
         int rc;
         switch (c->tiles[t0].logW) {
-            case 5: rc = launch_grow_one<5, WIDE>(c, args, g, t1 - t0, st); break;
-            case 3: rc = launch_grow_one<3, WIDE>(c, args, g, t1 - t0, st); break;
-            default: rc = launch_grow_one<-1, WIDE>(c, args, g, t1 - t0, st); break;
+            case 5: rc = launch_grow_one<5, MODE>(c, args, g, t1 - t0, st); break;
+            case 3: rc = launch_grow_one<3, MODE>(c, args, g, t1 - t0, st); break;
+            default: rc = launch_grow_one<-1, MODE>(c, args, g, t1 - t0, st); break;
         }
         if (rc != QGBDT_OK) return rc;
         t0 = t1;
@@ -282,8 +301,7 @@ int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
     a.nb = c->nb;
     a.hist = nullptr;
     a.partial = c->d_partial;
-    const uint32_t by_h = 65535u / (uint32_t)kh, by_g = 32767u / (uint32_t)kg;
-    a.flush_rows = by_h < by_g ? by_h : by_g;
+    pick_field_split(kg, kh, a.shift, a.flush_rows);
     a.pass = 0;
     a.state = c->d_state;
     GrowHist g;
@@ -306,13 +324,15 @@ int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
         QG_CUDA(c, cudaEventRecord(ev0, st));
     }
     int rc;
-    if (bits < 6) {
-        rc = launch_grow<false>(c, a, g, st);
+    if (bits < 6 && a.shift == 16) {
+        rc = launch_grow<0>(c, a, g, st);
+    } else if (bits < 6) {
+        rc = launch_grow<2>(c, a, g, st);
     } else {
-        rc = launch_grow<true>(c, a, g, st);
+        rc = launch_grow<1>(c, a, g, st);
         if (rc == QGBDT_OK) {
             a.pass = 1;
-            rc = launch_grow<true>(c, a, g, st);
+            rc = launch_grow<1>(c, a, g, st);
         }
     }
     if (rc == QGBDT_OK && ev1) QG_CUDA(c, cudaEventRecord(ev1, st));

@@ -25,7 +25,8 @@ struct HistArgs {
     int nb;
     unsigned long long *hist;      // [F][nb]
     unsigned long long *partial;   // [CTA][4][nb][32]
-    uint32_t flush_rows;           // rows one column may add between flushes (16+16 local only)
+    uint32_t flush_rows;           // rows one column may add between flushes (narrow local bins only)
+    int shift;                     // narrow local bins: bit position of the gradient field (16: the 16+16 split)
     int pass;                      // 32+32 local only: bytes 2*pass, 2*pass+1 of every word
     DevState *state;
 };
@@ -63,9 +64,18 @@ __device__ __forceinline__ uint32_t ldg16(const uint16_t *p) {
 
 // One row's word: its bin codes -> shared atomics.  `half` selects the 16-bit code in the low
 // or high half of c.
-template <bool WIDE>
-__device__ __forceinline__ void add_word(uint32_t base, uint32_t w, uint32_t c, int half, int pass) {
-    if (!WIDE) {
+template <int MODE>
+__device__ __forceinline__ void add_word(uint32_t base, uint32_t w, uint32_t c, int half, int pass, int shift) {
+    if (MODE == 2) {
+        // gradient field above bit `shift`, hessian below: inc = g * 2^shift + h
+        const int h = (int)prmt(c, 0u, half ? 0x4442u : 0x4440u);
+        const int g = (int)prmt(c, 0u, half ? 0xBBB3u : 0x9991u);   // sign-extended
+        const int inc = g * (1 << shift) + h;
+        red32<0>(prmt(w, base, 0x7604u), inc);
+        red32<128>(prmt(w, base, 0x7614u), inc);
+        red32<65536>(prmt(w, base, 0x7624u), inc);
+        red32<65536 + 128>(prmt(w, base, 0x7634u), inc);
+    } else if (MODE != 1) {
         // inc = g * 65536 + h: byte 0 = h, byte 1 = 0, byte 2 = g, byte 3 = sign of g
         const int inc = (int)prmt(c, 0u, half ? 0xB342u : 0x9140u);
         red32<0>(prmt(w, base, 0x7604u), inc);
@@ -94,31 +104,32 @@ struct Out {
 // Adds the CTA's local histogram into its output and clears it.  The R replicas of a column
 // (the row slots of word a) are R adjacent shared words, so one thread sums them from vector
 // loads and writes one packed 64-bit bin.
-template <int NT, bool WIDE>
-__device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, int nb, int pass, Out &out) {
+template <int NT, int MODE>
+__device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, int nb, int pass, int shift, Out &out) {
+    const int hmask = (1 << shift) - 1;   // narrow bins: hessian field below bit `shift` (16 unless MODE 2)
     const int W = 1 << logW, R = 32 >> logW;
     const int per_k = nb << logW;                                   // outputs per byte position k
-    for (int kk = 0; kk < (WIDE ? 2 : 4); ++kk) {
-        const int k = WIDE ? 2 * pass + kk : kk;
+    for (int kk = 0; kk < (MODE == 1 ? 2 : 4); ++kk) {
+        const int k = MODE == 1 ? 2 * pass + kk : kk;
         for (int e = threadIdx.x; e < per_k; e += NT) {
             const int a = e & (W - 1), bin = e >> logW;
             unsigned long long v;
-            if (!WIDE) {
+            if (MODE != 1) {
                 int *p = hp + (kk >> 1) * 16384 + bin * 64 + (kk & 1) * 32 + a * R;
                 int G = 0, H = 0;
                 if (R >= 4) {
                     for (int r = 0; r < R; r += 4) {
                         const int4 x = *reinterpret_cast<const int4 *>(p + r);
                         *reinterpret_cast<int4 *>(p + r) = make_int4(0, 0, 0, 0);
-                        G += (x.x >> 16) + (x.y >> 16) + (x.z >> 16) + (x.w >> 16);
-                        H += (x.x & 0xFFFF) + (x.y & 0xFFFF) + (x.z & 0xFFFF) + (x.w & 0xFFFF);
+                        G += (x.x >> shift) + (x.y >> shift) + (x.z >> shift) + (x.w >> shift);
+                        H += (x.x & hmask) + (x.y & hmask) + (x.z & hmask) + (x.w & hmask);
                     }
                 } else {
                     for (int r = 0; r < R; ++r) {
                         const int x = p[r];
                         p[r] = 0;
-                        G += x >> 16;
-                        H += x & 0xFFFF;
+                        G += x >> shift;
+                        H += x & hmask;
                     }
                 }
                 v = (unsigned long long)((long long)G * 4294967296LL + (long long)H);
@@ -163,7 +174,7 @@ __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) 
 // from the tile.  The grid is (part, tile - tile0).
 // One CTA's share (part `part` of P) of the histogram of a.n rows for tile td.  `sh` is the
 // CTA's dynamic shared memory (HIST_SMEM bytes).  Ends with the CTA's local histogram flushed.
-template <int NT, int LOGW_T, bool WIDE, int LIST>
+template <int NT, int LOGW_T, int MODE, int LIST>
 __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, const uint32_t part, const uint32_t P,
                                          int *sh) {
     const uint32_t n = a.n;
@@ -193,6 +204,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     const uint32_t base = h0 + lane * 4;
     const uint32_t *tile = td.data;
     const int pass = a.pass;
+    const int shift = MODE == 2 ? a.shift : 16;
 
     Out out;
     out.direct = P == 1;
@@ -239,7 +251,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
                 c = a.codes_nat[row];
             }
             const uint32_t w = tile[((size_t)row << logW) + wa];
-            add_word<WIDE>(base, w, c, 0, pass);
+            add_word<MODE>(base, w, c, 0, pass, shift);
         }
         col_rows = (s1 - s0 + R - 1) >> logR;
     }
@@ -250,12 +262,12 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     uint32_t q = 0;
     while (q < q1) {
         uint32_t epoch = q1 - q;   // warp-units of this epoch, all warps together
-        if (!WIDE) {
+        if (MODE != 1) {
             const uint32_t room = a.flush_rows > col_rows ? a.flush_rows - col_rows : 0;
             const uint32_t fit = room >> 2;                          // every warp-unit adds 4 rows to each column
             if (fit == 0) {
                 __syncthreads();
-                flush_local<NT, WIDE>(hp, td, logW, a.nb, pass, out);
+                flush_local<NT, MODE>(hp, td, logW, a.nb, pass, shift, out);
                 __syncthreads();
                 col_rows = 0;
                 continue;
@@ -281,10 +293,10 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     }
 #define QG_USE_UNIT(u)                                       \
     {                                                        \
-        add_word<WIDE>(base, w[u][0], c[u].x, 0, pass);      \
-        add_word<WIDE>(base, w[u][1], c[u].x, 1, pass);      \
-        add_word<WIDE>(base, w[u][2], c[u].y, 0, pass);      \
-        add_word<WIDE>(base, w[u][3], c[u].y, 1, pass);      \
+        add_word<MODE>(base, w[u][0], c[u].x, 0, pass, shift);      \
+        add_word<MODE>(base, w[u][1], c[u].x, 1, pass, shift);      \
+        add_word<MODE>(base, w[u][2], c[u].y, 0, pass, shift);      \
+        add_word<MODE>(base, w[u][3], c[u].y, 1, pass, shift);      \
     }
 #pragma unroll
             for (int u = 0; u < U; ++u)
@@ -345,7 +357,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     }
 #define QG_USE_DATA(u)                                                                           \
     {                                                                                            \
-        _Pragma("unroll") for (int j = 0; j < 4; ++j) add_word<WIDE>(base, w[u][j], c[u][j], 0, pass); \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) add_word<MODE>(base, w[u][j], c[u][j], 0, pass, shift); \
     }
 #pragma unroll
             for (int u = 0; u < U; ++u)
@@ -389,7 +401,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
         col_rows += 4 * epoch;
     }
     __syncthreads();
-    flush_local<NT, WIDE>(hp, td, logW, a.nb, pass, out);
+    flush_local<NT, MODE>(hp, td, logW, a.nb, pass, shift, out);
 }
 
 }  // namespace

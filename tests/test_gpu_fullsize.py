@@ -132,3 +132,25 @@ def test_worst_case_accumulation_at_scale():
         G, H = binding.unpack_hist(hist)
         m = rows.numel()
         assert G[27, 0] == -kg * m and H[27, 0] == kh * m and G[5, 3] == -kg * m
+
+
+def test_worst_case_accumulation_constant_hessian():
+    # constant hessian: the local bins split their 32 bits unevenly (row count below, gradient sum
+    # above); all rows in one bin at the extreme gradient level must still come out exact
+    n = 6_000_000
+    data = torch.zeros((n, 28), dtype=torch.uint8, device="cuda")
+    data[:, 9] = 7
+    for bits in (2, 4, 5):
+        kg, _ = oracle.levels(bits)
+        ctx = binding.Context(binding.make_params(bits=bits, objective=1))
+        ctx.load_binned(data, 8)
+        for sign in (-1.0, 1.0):
+            ctx.quantize_gradients(torch.full((n,), sign, device="cuda"), None)
+            hist = ctx.new_hist()
+            ctx.build_histograms(0, hist)
+            G, H = binding.unpack_hist(hist)
+            assert G[0, 0] == sign * kg * n and H[0, 0] == n and G[9, 7] == sign * kg * n and H[9, 7] == n and H[9, 0] == 0
+            rows = synth.subset_rows(n, device="cuda")
+            ctx.build_histograms_rows(rows, hist)
+            G, H = binding.unpack_hist(hist)
+            assert G[27, 0] == sign * kg * rows.numel() and H[27, 0] == rows.numel()

@@ -116,7 +116,7 @@ void plan_tiles(int F, std::vector<TileDesc> &out) {
 }
 
 // Histogram plan.  Tiles of equal width form a group that is built by one launch (the full
-// 128-feature tiles, then the remainder tiles); a group's tiles share the SMs equally, and with
+// 128-feature tiles, then the remainder tiles); a group's tiles get equal shares of the SMs, and with
 // more tiles than SMs every tile gets one CTA.  Fills parts / cta0 of the tiles; part p of a tile
 // owns partial-histogram slot cta0 + p.
 void plan_hist_ctas(int sm_count, std::vector<TileDesc> &tiles, int &n_ctas, int &max_parts) {
@@ -128,7 +128,7 @@ void plan_hist_ctas(int sm_count, std::vector<TileDesc> &tiles, int &n_ctas, int
         while (t1 < T && tiles[t1].logW == tiles[t0].logW) ++t1;
         const int g = t1 - t0;
         for (int i = t0; i < t1; ++i) {
-            int p = sm_count / g + (i - t0 < sm_count % g ? 1 : 0);
+            int p = sm_count / g;   // equal shares: (parts, tiles of the group) is then a grid of at most one CTA per SM
             if (p < 1) p = 1;
             tiles[i].parts = p;
             tiles[i].cta0 = n_ctas;
@@ -261,6 +261,7 @@ int qgbdt_create(qgbdt_ctx **out, const qgbdt_params *p) {
     }
     c->sm_count = prop.multiProcessorCount;
     c->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    c->coop_ok = prop.cooperativeLaunch != 0;
     const int L = p->num_leaves;
     bool ok = cudaMalloc(reinterpret_cast<void **>(&c->d_state), sizeof(DevState)) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_split_out), sizeof(SplitRec) * 4) == cudaSuccess &&

@@ -26,6 +26,8 @@
 // (signed), hessian sum in the low 16 bits; the CTA flushes before any column can have added
 // more rows than fit.  B >= 6 uses two 32-bit words per bin (32+32, a hessian plane and a gradient
 // plane) and two passes over the rows, each pass taking two of the four bytes of a word.
+#include <cooperative_groups.h>
+
 #include "hist_cta.cuh"
 
 namespace {
@@ -38,6 +40,62 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     const uint32_t P = effective_parts((uint32_t)td.parts, a.n);
     if (blockIdx.x >= P) return;
     hist_cta<HIST_THREADS, LOGW_T, MODE, LIST>(a, td, blockIdx.x, P, sh);
+}
+
+// Stand-alone build with the merge inside the kernel: a cooperative launch (every CTA resident),
+// a grid-wide barrier after the partial histograms, then the P CTAs of a tile share the sums of
+// its entries.  Saves the merge kernel and the gap before it.  Narrow local bins only.
+template <int LOGW_T, int MODE, int LIST>
+__global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_coop(HistArgs a) {
+    extern __shared__ __align__(1024) int sh[];
+    const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
+    const uint32_t P = effective_parts((uint32_t)td.parts, a.n), part = blockIdx.x;
+    if (part < P) hist_cta<HIST_THREADS, LOGW_T, MODE, LIST>(a, td, part, P, sh);
+    __threadfence();
+    cooperative_groups::this_grid().sync();
+    if (part >= P || P <= 1) return;
+    const int W = 1 << td.logW, nb = a.nb;
+    const uint32_t total = 4u * nb * W;
+    const size_t stride = (size_t)4 * nb * 32;
+    const uint32_t e0 = (uint32_t)((unsigned long long)total * part / P), e1 = (uint32_t)((unsigned long long)total * (part + 1) / P);
+    const unsigned long long *pbase = a.partial + (size_t)td.cta0 * stride;
+    auto store = [&](uint32_t e, unsigned long long v) {
+        const uint32_t wa = e & (W - 1), kb = e >> td.logW, k = kb / nb, bin = kb - k * nb, fl = 4 * wa + k;
+        if (fl < (uint32_t)td.nf) a.hist[(size_t)(td.f0 + fl) * nb + bin] = v;
+    };
+    if (P <= 16) {
+        for (uint32_t e = e0 + threadIdx.x; e < e1; e += HIST_THREADS) {
+            unsigned long long x[16], v = 0;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) x[k] = (uint32_t)k < P ? __ldcg(pbase + (size_t)k * stride + e) : 0ull;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) v += x[k];
+            store(e, v);
+        }
+    } else {
+        // 16 groups of 64 threads: group g adds partials g, g + 16, ... of 64 entries at a time
+        unsigned long long *acc = reinterpret_cast<unsigned long long *>(sh);   // [16][64], the local histogram is done with
+        const uint32_t eg = threadIdx.x & 63, pg = threadIdx.x >> 6;
+        for (uint32_t eb = e0; eb < e1; eb += 64) {
+            const uint32_t e = eb + eg;
+            unsigned long long x[10], v = 0;
+#pragma unroll
+            for (int k = 0; k < 10; ++k) {
+                const uint32_t i = pg + 16u * k;
+                x[k] = (e < e1 && i < P) ? __ldcg(pbase + (size_t)i * stride + e) : 0ull;
+            }
+#pragma unroll
+            for (int k = 0; k < 10; ++k) v += x[k];
+            for (uint32_t i = pg + 160u; e < e1 && i < P; i += 16) v += __ldcg(pbase + (size_t)i * stride + e);
+            __syncthreads();
+            acc[pg * 64 + eg] = v;
+            __syncthreads();
+            if (pg == 0 && e < e1) {
+                for (int g = 1; g < 16; ++g) v += acc[g * 64 + eg];
+                store(e, v);
+            }
+        }
+    }
 }
 
 // Tree growth: the rows are the smaller child (ties: the left one) of the split recorded in the
@@ -134,6 +192,44 @@ int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st)
     return QGBDT_OK;
 }
 
+template <int LOGW_T, int MODE, int LIST>
+int launch_one_coop(qgbdt_ctx *c, HistArgs &args, int n_tiles, cudaStream_t st) {
+    const void *kern = reinterpret_cast<const void *>(k_hist_coop<LOGW_T, MODE, LIST>);
+    static bool configured = false;   // per instantiation
+    if (!configured) {
+        QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
+        configured = true;
+    }
+    int group_parts = 1;
+    for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
+        if (c->tiles[t].parts > group_parts) group_parts = c->tiles[t].parts;
+    const dim3 grid(effective_parts((uint32_t)group_parts, args.n), (unsigned)n_tiles);
+    void *params[] = {&args};
+    QG_CUDA(c, cudaLaunchCooperativeKernel(kern, grid, dim3(HIST_THREADS), params, HIST_SMEM, st));
+    c->n_launches++;
+    return QGBDT_OK;
+}
+
+// Cooperative variant of launch_hist: the merge happens inside the kernels.
+template <int MODE, int LIST>
+int launch_hist_coop(qgbdt_ctx *c, HistArgs args, cudaStream_t st) {
+    const int T = (int)c->tiles.size();
+    for (int t0 = 0; t0 < T;) {
+        int t1 = t0 + 1;
+        while (t1 < T && c->tiles[t1].logW == c->tiles[t0].logW) ++t1;
+        args.tile0 = t0;
+        int rc;
+        switch (c->tiles[t0].logW) {
+            case 5: rc = launch_one_coop<5, MODE, LIST>(c, args, t1 - t0, st); break;
+            case 3: rc = launch_one_coop<3, MODE, LIST>(c, args, t1 - t0, st); break;
+            default: rc = launch_one_coop<-1, MODE, LIST>(c, args, t1 - t0, st); break;
+        }
+        if (rc != QGBDT_OK) return rc;
+        t0 = t1;
+    }
+    return QGBDT_OK;
+}
+
 // One launch per run of tiles of equal width (the full 128-feature tiles, then the remainder).
 template <int MODE, int LIST>
 int launch_hist(qgbdt_ctx *c, HistArgs args, cudaStream_t st) {
@@ -223,7 +319,14 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
         QG_CUDA(c, cudaEventRecord(ev0, st));
     }
     int rc;
-    if (!wide && a.shift == 16) {
+    const bool merge_needed = c->max_parts > 1 && effective_parts((uint32_t)c->max_parts, (uint32_t)n) > 1;
+    // with at most one CTA per SM in every launch, the merge can follow a grid barrier in the same kernel
+    const bool coop = !wide && merge_needed && c->coop_ok && (int)c->tiles.size() <= c->sm_count;
+    if (coop && a.shift == 16) {
+        rc = d_rows ? launch_hist_coop<0, 1>(c, a, st) : launch_hist_coop<0, 0>(c, a, st);
+    } else if (coop) {
+        rc = d_rows ? launch_hist_coop<2, 1>(c, a, st) : launch_hist_coop<2, 0>(c, a, st);
+    } else if (!wide && a.shift == 16) {
         rc = d_rows ? launch_hist<0, 1>(c, a, st) : launch_hist<0, 0>(c, a, st);
     } else if (!wide) {
         rc = d_rows ? launch_hist<2, 1>(c, a, st) : launch_hist<2, 0>(c, a, st);
@@ -235,7 +338,7 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
         }
     }
     if (rc != QGBDT_OK) return rc;
-    if (c->max_parts > 1 && effective_parts((uint32_t)c->max_parts, (uint32_t)n) > 1) {
+    if (merge_needed && !coop) {
         const dim3 grid((unsigned)((4 * c->nb * 32 + 31) / 32), (unsigned)c->tiles.size());
         k_hist_reduce<<<grid, 256, 0, st>>>(c->d_tiles, (uint32_t)n, c->nb, c->d_partial, d_hist);
         QG_LAUNCH_CHECK(c);

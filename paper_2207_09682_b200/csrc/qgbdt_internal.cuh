@@ -94,6 +94,7 @@ struct qgbdt_ctx {
     int device = 0;
     int sm_count = 0;
     int max_smem_optin = 0;
+    bool coop_ok = false;   // the device supports cooperative launches
     // data
     int64_t N = 0;
     int F = 0, nb = 0;

@@ -64,7 +64,8 @@ void free_data(qgbdt_ctx *c) {
     dev_free(c->d_ent0);
     dev_free(c->d_ent1);
     dev_free(c->d_cand);
-    dev_free(c->d_feat_tile);
+    dev_free(c->d_feat_rec);
+    dev_free(c->d_leaf_gain);
     dev_free(c->d_m_num_leaves);
     dev_free(c->d_m_feature);
     dev_free(c->d_m_bin);
@@ -200,11 +201,20 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     if ((rc = dev_alloc(c, &c->d_idx_tmp, (size_t)n_rows)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8 + (size_t)c->sm_count * 32)) != QGBDT_OK) return rc;
     {
-        std::vector<int32_t> ft((size_t)n_features);
-        for (size_t t = 0; t < c->tiles.size(); ++t)
-            for (int f = c->tiles[t].f0; f < c->tiles[t].f0 + c->tiles[t].nf; ++f) ft[f] = (int32_t)t;
-        if ((rc = dev_alloc(c, &c->d_feat_tile, (size_t)n_features)) != QGBDT_OK) return rc;
-        QG_CUDA(c, cudaMemcpy(c->d_feat_tile, ft.data(), sizeof(int32_t) * ft.size(), cudaMemcpyHostToDevice));
+        std::vector<FeatRec> fr((size_t)n_features);
+        for (const TileDesc &t : c->tiles)
+            for (int f = t.f0; f < t.f0 + t.nf; ++f) {
+                const int fl = f - t.f0;
+                fr[f].col = t.data + (fl >> 2);
+                fr[f].logW = t.logW;
+                fr[f].byte = fl & 3;
+                fr[f].cta0 = t.cta0;
+                fr[f].parts = t.parts;
+                fr[f].fl = fl;
+                fr[f].pad = 0;
+            }
+        if ((rc = dev_alloc(c, &c->d_feat_rec, (size_t)n_features)) != QGBDT_OK) return rc;
+        QG_CUDA(c, cudaMemcpy(c->d_feat_rec, fr.data(), sizeof(FeatRec) * fr.size(), cudaMemcpyHostToDevice));
     }
     if ((rc = dev_alloc(c, &c->d_part_bits, ((size_t)n_rows + 2048) / 32 + 64)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_feat_best, (size_t)n_features)) != QGBDT_OK) return rc;

@@ -27,8 +27,9 @@ struct GrowArgs {
     GrowState *gs;
     LeafRec *leaves;
     const DevState *state;
-    const TileDesc *tiles;
-    const int32_t *feat_tile;
+    const FeatRec *feat_rec;         // [F]
+    double *leaf_gain;               // [L] gain of every leaf's best split, -inf when it has none
+    uint32_t N;
     uint2 *ent0, *ent1;              // the two (row, gradient code) pair buffers
     const uint16_t *codes_nat;       // codes in row order (the root's identity list has no pairs yet)
     uint32_t *bits, *counts;         // predicate bits of the leaf being split, left rows per warp range
@@ -190,11 +191,11 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     const size_t hw = (size_t)a.F * a.nb;
 
     // the two children: "small" was built by Algorithm 1, "large" is parent - small
-    const uint32_t n = ROOT ? a.leaves[0].n : gs->n, nl = ROOT ? n : gs->nl, nr = n - nl;
+    const uint32_t n = ROOT ? a.N : gs->n, nl = ROOT ? n : gs->nl, nr = n - nl;
     const bool small_is_left = nl <= nr;
     SplitParams pS = a.sp, pL = a.sp;
     if (ROOT) {
-        pS.G = a.leaves[0].G; pS.H = a.leaves[0].H; pS.n_s = n;
+        pS.G = a.state->tot_g; pS.H = a.state->tot_h; pS.n_s = n;
     } else {
         const long long gl = gs->gl, hl = gs->hl, gr = gs->PG - gl, hr = gs->PH - hl;
         pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl : nr;
@@ -208,11 +209,11 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     qg_scales(a.state, pS, dg, dh);
     const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
     const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
-    const TileDesc td = a.tiles[a.feat_tile[f]];
-    const int fl = f - td.f0, W = 1 << td.logW;
-    const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)td.parts, (uint32_t)pS.n_s);
+    const FeatRec fr = a.feat_rec[f];
+    const int fl = fr.fl, W = 1 << fr.logW;
+    const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)fr.parts, (uint32_t)pS.n_s);
     const size_t pstride = (size_t)4 * a.nb * 32;
-    const unsigned long long *part = a.partial + (size_t)td.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
+    const unsigned long long *part = a.partial + (size_t)fr.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
     unsigned long long *S = a.pool + (ROOT ? 0 : (size_t)n_leaves * hw) + (size_t)f * a.nb;
     unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)gs->parent_slot * hw + (size_t)f * a.nb;
     // n_bins <= 256: thread b owns bin b
@@ -300,9 +301,19 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     if (!is_last) return;
     __threadfence();
 
+    // ---- the last block: best candidates over all features, the new leaves, the next pick
+    const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
+    const int leaves_now = ROOT ? 1 : n_leaves + 1;
+    // gains of the older leaves, fetched while the candidates are being reduced
+    double my_gain[4];
+#pragma unroll
+    for (int k2 = 0; k2 < 4; ++k2) {
+        const int i2 = (int)threadIdx.x + k2 * FIN_WARPS * 32;
+        my_gain[k2] = i2 < leaves_now ? __ldcg(a.leaf_gain + i2) : NEG;
+    }
     SplitRec bS = qg_invalid_rec(), bL = qg_invalid_rec();
-    for (int i = threadIdx.x; i < (int)gridDim.x; i += FIN_WARPS * 32) {
-        const SplitRec x = load_rec_cg(a.cand + 2 * i), y = load_rec_cg(a.cand + 2 * i + 1);
+    for (int i2 = threadIdx.x; i2 < (int)gridDim.x; i2 += FIN_WARPS * 32) {
+        const SplitRec x = load_rec_cg(a.cand + 2 * i2), y = load_rec_cg(a.cand + 2 * i2 + 1);
         if (qg_rec_better(x, bS)) bS = x;
         if (qg_rec_better(y, bL)) bL = y;
     }
@@ -316,56 +327,77 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
         }
         __syncthreads();
     }
-    int leaves_now = n_leaves;
+    __shared__ LeafRec s_new[2];   // the two leaves this split made (ROOT: [0] is the root)
+    __shared__ int s_new_id[2];
     if (threadIdx.x == 0) {
         bS = sm[0][0];
         bL = sm[1][0];
         if (ROOT) {
-            a.leaves[0].best = bS;
+            LeafRec r;
+            r.off = 0; r.n = a.N; r.buf = -1; r.slot = 0; r.G = pS.G; r.H = pS.H; r.best = bS;
+            r.parent_node = -1; r.parent_side = 0;
+            a.leaves[0] = r;
+            a.leaf_gain[0] = bS.valid ? bS.gain : NEG;
+            s_new[0] = r; s_new_id[0] = 0; s_new_id[1] = -1;
+            gs->n_leaves = 1;
         } else {
             const int pick = gs->pick, right = n_leaves, node = n_leaves - 1;
-            const LeafRec par = a.leaves[pick];
             a.m_feature[node] = gs->feature;
             a.m_bin[node] = gs->bin;
             a.m_left[node] = ~pick;
             a.m_right[node] = ~right;
             a.m_gain[node] = gs->gain;
-            if (par.parent_node >= 0) {
-                if (par.parent_side == 0) a.m_left[par.parent_node] = node;
-                else a.m_right[par.parent_node] = node;
+            if (gs->parent_node >= 0) {
+                if (gs->parent_side == 0) a.m_left[gs->parent_node] = node;
+                else a.m_right[gs->parent_node] = node;
             }
             const int dstbuf = gs->buf == 0 ? 1 : 0;
             LeafRec lf, rt;
-            lf.off = par.off; lf.n = nl; lf.buf = dstbuf;
+            lf.off = gs->off; lf.n = nl; lf.buf = dstbuf;
             lf.G = gs->gl; lf.H = gs->hl;
             lf.parent_node = node; lf.parent_side = 0;
-            rt.off = par.off + nl; rt.n = nr; rt.buf = dstbuf;
+            rt.off = gs->off + nl; rt.n = nr; rt.buf = dstbuf;
             rt.G = gs->PG - gs->gl; rt.H = gs->PH - gs->hl;
             rt.parent_node = node; rt.parent_side = 1;
-            lf.slot = small_is_left ? n_leaves : par.slot;
-            rt.slot = small_is_left ? par.slot : n_leaves;
+            lf.slot = small_is_left ? n_leaves : gs->parent_slot;
+            rt.slot = small_is_left ? gs->parent_slot : n_leaves;
             lf.best = small_is_left ? bS : bL;
             rt.best = small_is_left ? bL : bS;
             a.leaves[pick] = lf;
             a.leaves[right] = rt;
+            a.leaf_gain[pick] = lf.best.valid ? lf.best.gain : NEG;
+            a.leaf_gain[right] = rt.best.valid ? rt.best.gain : NEG;
+            s_new[0] = lf; s_new_id[0] = pick;
+            s_new[1] = rt; s_new_id[1] = right;
             gs->n_leaves = n_leaves + 1;
             gs->hist_rows += small_is_left ? nl : nr;
             gs->hist_builds += 1;
         }
         gs->finish_count = 0;
     }
-    if (!ROOT) leaves_now = n_leaves + 1;
     __syncthreads();
 
     // the next leaf to split: largest gain, lowest leaf number on equal gain
     __shared__ double pg[FIN_WARPS * 32];
     __shared__ int pi[FIN_WARPS * 32];
-    double bg = 0.0;
+    double bg = NEG;
     int bi = -1;
     if (leaves_now < a.L) {
-        for (int i = threadIdx.x; i < leaves_now; i += FIN_WARPS * 32) {
-            const SplitRec &r = a.leaves[i].best;
-            if (r.valid && (bi < 0 || r.gain > bg)) { bg = r.gain; bi = i; }
+#pragma unroll
+        for (int k2 = 0; k2 < 4; ++k2) {
+            const int i2 = (int)threadIdx.x + k2 * FIN_WARPS * 32;
+            if (i2 < leaves_now) {
+                double g = my_gain[k2];
+                if (i2 == s_new_id[0]) g = s_new[0].best.valid ? s_new[0].best.gain : NEG;
+                if (i2 == s_new_id[1]) g = s_new[1].best.valid ? s_new[1].best.gain : NEG;
+                if (g > bg) { bg = g; bi = i2; }
+            }
+        }
+        for (int i2 = (int)threadIdx.x + 4 * FIN_WARPS * 32; i2 < leaves_now; i2 += FIN_WARPS * 32) {   // more than 1024 leaves
+            double g = __ldcg(a.leaf_gain + i2);
+            if (i2 == s_new_id[0]) g = s_new[0].best.valid ? s_new[0].best.gain : NEG;
+            if (i2 == s_new_id[1]) g = s_new[1].best.valid ? s_new[1].best.gain : NEG;
+            if (g > bg) { bg = g; bi = i2; }
         }
     }
     pg[threadIdx.x] = bg;
@@ -388,15 +420,14 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
         if (pick < 0) {
             gs->done = 1;
         } else {
-            const LeafRec lr = a.leaves[pick];
-            const TileDesc td = a.tiles[a.feat_tile[lr.best.feature]];
-            const int fl = lr.best.feature - td.f0;
+            const LeafRec lr = pick == s_new_id[0] ? s_new[0] : (pick == s_new_id[1] ? s_new[1] : a.leaves[pick]);
+            const FeatRec pf = a.feat_rec[lr.best.feature];
             gs->pick = pick;
             gs->feature = lr.best.feature;
             gs->bin = lr.best.bin;
-            gs->col = td.data + (fl >> 2);
-            gs->logW = td.logW;
-            gs->byte = fl & 3;
+            gs->col = pf.col;
+            gs->logW = pf.logW;
+            gs->byte = pf.byte;
             gs->off = lr.off;
             gs->n = lr.n;
             gs->buf = lr.buf;
@@ -406,6 +437,8 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
             gs->PH = lr.H;
             gs->gain = lr.best.gain;
             gs->parent_slot = lr.slot;
+            gs->parent_node = lr.parent_node;
+            gs->parent_side = lr.parent_side;
         }
     }
 }
@@ -420,8 +453,9 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     a.gs = c->d_gs;
     a.leaves = c->d_leaves;
     a.state = c->d_state;
-    a.tiles = c->d_tiles;
-    a.feat_tile = c->d_feat_tile;
+    a.feat_rec = c->d_feat_rec;
+    a.leaf_gain = c->d_leaf_gain;
+    a.N = (uint32_t)c->N;
     a.ent0 = c->d_ent0;
     a.ent1 = c->d_ent1;
     a.codes_nat = reinterpret_cast<const uint16_t *>(c->d_codes_nat);

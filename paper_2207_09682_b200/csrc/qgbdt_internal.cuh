@@ -60,6 +60,15 @@ struct SplitRec {
     int valid, pad;
 };
 
+// Where a feature sits in the tiled matrix and in the histogram plan (one load instead of a
+// chain through the tile table).
+struct FeatRec {
+    const uint32_t *col;   // the feature's word in row 0 of its tile
+    int32_t logW, byte;    // words per row (log2) of the tile, byte of the word
+    int32_t cta0, parts;   // partial-histogram slots of the tile
+    int32_t fl, pad;       // feature number inside the tile
+};
+
 // One leaf of the tree being grown (device memory).  Its rows are entries [off, off + n) of the
 // (row, code) pair buffer `buf` (0 or 1; -1: the identity list of the root).
 struct LeafRec {
@@ -83,7 +92,7 @@ struct GrowState {
     uint32_t nl;                     // rows that go left (written by the scatter kernel)
     long long gl, hl, PG, PH;        // left totals of the candidate, totals of the leaf
     double gain;
-    int32_t parent_slot;
+    int32_t parent_slot, parent_node, parent_side;   // histogram slot and tree position of that leaf
     unsigned int finish_count;       // blocks of the finishing kernel that are through
     unsigned long long hist_rows;    // rows visited by histogram builds of row lists (all trees so far)
     unsigned long long hist_builds;
@@ -134,7 +143,8 @@ struct qgbdt_ctx {
     uint2 *d_ent0 = nullptr, *d_ent1 = nullptr; // [N] (row, gradient code) pairs of the leaves, two buffers
     GrowState *d_gs = nullptr;
     SplitRec *d_cand = nullptr;                 // [F][2] per-feature best candidates of the two children
-    int32_t *d_feat_tile = nullptr;             // [F] tile of every feature
+    FeatRec *d_feat_rec = nullptr;              // [F] location of every feature
+    double *d_leaf_gain = nullptr;              // [L] stored gain of every leaf's best split (-inf: none)
     // trees of the current qgbdt_train call, on the device until the call ends
     int model_cap = 0;                          // trees the arrays below can hold
     int32_t *d_m_num_leaves = nullptr, *d_m_feature = nullptr, *d_m_bin = nullptr, *d_m_left = nullptr,

@@ -52,6 +52,7 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
         (rc = alloc_dev(c, &c->d_hist_pool, (size_t)L * c->F * c->nb, "histogram pool")) != QGBDT_OK)
         return rc;
     if (!c->d_leaves && (rc = alloc_dev(c, &c->d_leaves, (size_t)L, "leaf records")) != QGBDT_OK) return rc;
+    if (!c->d_leaf_gain && (rc = alloc_dev(c, &c->d_leaf_gain, (size_t)L, "leaf gains")) != QGBDT_OK) return rc;
     if (!c->d_ent0 && (rc = alloc_dev(c, &c->d_ent0, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_ent1 && (rc = alloc_dev(c, &c->d_ent1, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_cand && (rc = alloc_dev(c, &c->d_cand, (size_t)2 * c->F, "candidate records")) != QGBDT_OK)

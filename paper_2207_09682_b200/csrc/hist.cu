@@ -178,10 +178,10 @@ __global__ void k_subtract(const unsigned long long *__restrict__ parent, const 
 template <int LOGW_T, int MODE, int LIST>
 int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st) {
     auto kern = k_hist<LOGW_T, MODE, LIST>;
-    static bool configured = false;   // per instantiation
-    if (!configured) {
+    static bool configured[64] = {};   // per instantiation and device (the attribute belongs to the device's context)
+    if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
-        configured = true;
+        if (c->device >= 0 && c->device < 64) configured[c->device] = true;
     }
     int group_parts = 1;
     for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
@@ -195,10 +195,10 @@ int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st)
 template <int LOGW_T, int MODE, int LIST>
 int launch_one_coop(qgbdt_ctx *c, HistArgs &args, int n_tiles, cudaStream_t st) {
     const void *kern = reinterpret_cast<const void *>(k_hist_coop<LOGW_T, MODE, LIST>);
-    static bool configured = false;   // per instantiation
-    if (!configured) {
+    static bool configured[64] = {};   // per instantiation and device (the attribute belongs to the device's context)
+    if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
-        configured = true;
+        if (c->device >= 0 && c->device < 64) configured[c->device] = true;
     }
     int group_parts = 1;
     for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
@@ -352,10 +352,10 @@ namespace {
 template <int LOGW_T, int MODE>
 int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n_tiles, cudaStream_t st) {
     auto kern = k_hist_grow<LOGW_T, MODE>;
-    static bool configured = false;   // per instantiation
-    if (!configured) {
+    static bool configured[64] = {};   // per instantiation and device (the attribute belongs to the device's context)
+    if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
-        configured = true;
+        if (c->device >= 0 && c->device < 64) configured[c->device] = true;
     }
     int group_parts = 1;
     for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)

@@ -265,7 +265,6 @@ def run_ours(args):
     ctx.train(wl.labels, scores, 0, W)                       # warm-up trees 0 .. W-1
     torch.cuda.synchronize()
     c0 = ctx.get_counters()
-    ctx.profile_histograms(True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if dist:
         dist.barrier()
@@ -278,9 +277,20 @@ def run_ours(args):
     if dist:
         dist.barrier()
     ms = e0.elapsed_time(e1)
+    c1 = ctx.get_counters()
+    # Roofline of the histogram kernels: the K boosting iterations that follow, with a pair of CUDA
+    # events around every histogram build.  (The timed region above replays a tree's ~1000 launches
+    # from a CUDA graph; event records between them would put the launches back on the stream, so
+    # the per-build timing runs right after it, on the same data, trees W+K .. W+2K-1.)
+    ctx.profile_histograms(True)
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    ctx.train(wl.labels, scores, W + K, K)
+    e3.record()
+    torch.cuda.synchronize()
     prof = ctx.get_histogram_profile()
     ctx.profile_histograms(False)
-    c1 = ctx.get_counters()
+    prof_ms = e2.elapsed_time(e3)
     rf = c1["hist_row_features"] - c0["hist_row_features"]
     launches = c1["kernel_launches"] - c0["kernel_launches"]
     leaves = [int(x) for x in model.num_leaves]
@@ -308,7 +318,9 @@ def run_ours(args):
                      "kernel": "k_hist / k_hist_grow (+ merge): every histogram build of the timed trees",
                      "algorithmic_bytes_per_launch": prof["total_bytes"] / max(prof["builds"], 1),
                      "launches": prof["builds"], "total_ms": prof["total_ms"],
-                     "share_of_step": prof["total_ms"] / ms if ms else None},
+                     "share_of_step": prof["total_ms"] / prof_ms if prof_ms else None,
+                     "region": "K more boosting iterations right after the timed ones, launches on the stream with "
+                               "an event pair around every build (%.2f ms per tree there)" % (prof_ms / K)},
         "clocks": clocks.summary(),
     }
 

@@ -45,6 +45,7 @@ void dev_free(T *&p) {
 }
 
 void free_data(qgbdt_ctx *c) {
+    qg_grow_graph_destroy(c);   // its launches point into the buffers freed below
     for (void *p : c->tile_allocs) cudaFree(p);
     c->tile_allocs.clear();
     c->tiles.clear();

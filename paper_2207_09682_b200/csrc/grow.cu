@@ -44,7 +44,8 @@ struct GrowArgs {
     double *m_gain;
 };
 
-__global__ void k_grow_begin(GrowState *gs, LeafRec *leaves, const DevState *state, uint32_t N) {
+__global__ void k_grow_begin(GrowState *gs, LeafRec *leaves, const DevState *state, uint32_t N, int tree_slot) {
+    gs->tree_slot = tree_slot;
     LeafRec r;
     r.off = 0; r.n = N; r.buf = -1; r.slot = 0;
     r.G = state->tot_g; r.H = state->tot_h;
@@ -342,14 +343,17 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
             gs->n_leaves = 1;
         } else {
             const int pick = gs->pick, right = n_leaves, node = n_leaves - 1;
-            a.m_feature[node] = gs->feature;
-            a.m_bin[node] = gs->bin;
-            a.m_left[node] = ~pick;
-            a.m_right[node] = ~right;
-            a.m_gain[node] = gs->gain;
+            // node arrays of the tree being grown (the slot is device state: the launch arguments
+            // are the same for every tree, so the launches can be replayed from a CUDA graph)
+            const size_t no = (size_t)gs->tree_slot * (a.L > 1 ? a.L - 1 : 1);
+            a.m_feature[no + node] = gs->feature;
+            a.m_bin[no + node] = gs->bin;
+            a.m_left[no + node] = ~pick;
+            a.m_right[no + node] = ~right;
+            a.m_gain[no + node] = gs->gain;
             if (gs->parent_node >= 0) {
-                if (gs->parent_side == 0) a.m_left[gs->parent_node] = node;
-                else a.m_right[gs->parent_node] = node;
+                if (gs->parent_side == 0) a.m_left[no + gs->parent_node] = node;
+                else a.m_right[no + gs->parent_node] = node;
             }
             const int dstbuf = gs->buf == 0 ? 1 : 0;
             LeafRec lf, rt;
@@ -445,11 +449,10 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
 
 }  // namespace
 
-// Grows the tree of boosting iteration slot `tree_slot` of the current train call.  Gradients must
-// have been quantized on the same stream (the state holds the totals and maxima).  Asynchronous.
-int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
+namespace {
+
+void fill_args(qgbdt_ctx *c, GrowArgs &a, int &part_blocks) {
     const int L = c->prm.num_leaves;
-    GrowArgs a;
     a.gs = c->d_gs;
     a.leaves = c->d_leaves;
     a.state = c->d_state;
@@ -461,7 +464,7 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     a.codes_nat = reinterpret_cast<const uint16_t *>(c->d_codes_nat);
     a.bits = c->d_part_bits;
     a.counts = c->d_part_counts;
-    const int part_blocks = c->sm_count * 4;
+    part_blocks = c->sm_count * 4;
     a.n_count = part_blocks * PART_WARPS;
     a.pool = c->d_hist_pool;
     a.partial = c->d_partial;
@@ -477,28 +480,94 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     a.sp.min_sum_h = c->prm.min_sum_hessian;
     a.sp.min_gain = c->prm.min_gain;
     a.sp.lambda = c->prm.lambda_l2;
-    const size_t no = (size_t)tree_slot * (L > 1 ? L - 1 : 1);
-    a.m_feature = c->d_m_feature + no;
-    a.m_bin = c->d_m_bin + no;
-    a.m_left = c->d_m_left + no;
-    a.m_right = c->d_m_right + no;
-    a.m_gain = c->d_m_gain + no;
+    a.m_feature = c->d_m_feature;
+    a.m_bin = c->d_m_bin;
+    a.m_left = c->d_m_left;
+    a.m_right = c->d_m_right;
+    a.m_gain = c->d_m_gain;
+}
 
-    k_grow_begin<<<1, 1, 0, st>>>(c->d_gs, c->d_leaves, c->d_state, (uint32_t)c->N);
-    QG_LAUNCH_CHECK(c);
-    int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
-    if (rc != QGBDT_OK) return rc;
+// The L - 1 splits of a tree: four kernels each, every size read from the grow state.
+int enqueue_splits(qgbdt_ctx *c, const GrowArgs &a, int part_blocks, cudaStream_t st) {
     const unsigned fin_blocks = (unsigned)c->F;
-    k_grow_finish<true><<<fin_blocks, FIN_WARPS * 32, 0, st>>>(a);
-    QG_LAUNCH_CHECK(c);
-    for (int split = 1; split < L; ++split) {
+    for (int split = 1; split < c->prm.num_leaves; ++split) {
         k_grow_flags<<<part_blocks, PART_THREADS, 0, st>>>(a);
         QG_LAUNCH_CHECK(c);
         k_grow_scatter<<<part_blocks, PART_THREADS, 0, st>>>(a);
         QG_LAUNCH_CHECK(c);
-        if ((rc = qg_hist_grow(c, st)) != QGBDT_OK) return rc;
+        const int rc = qg_hist_grow(c, st);
+        if (rc != QGBDT_OK) return rc;
         k_grow_finish<false><<<fin_blocks, FIN_WARPS * 32, 0, st>>>(a);
         QG_LAUNCH_CHECK(c);
     }
+    return QGBDT_OK;
+}
+
+}  // namespace
+
+void qg_grow_graph_destroy(qgbdt_ctx *c) {
+    if (c->grow_graph_exec) cudaGraphExecDestroy(reinterpret_cast<cudaGraphExec_t>(c->grow_graph_exec));
+    c->grow_graph_exec = nullptr;
+    c->grow_graph_launches = 0;
+}
+
+// The split loop of one tree as a CUDA graph (about a thousand launches whose arguments never
+// change: what differs from tree to tree is device state).  Built once per context and objective;
+// with the histogram event timers on, the launches go to the stream instead.
+static int build_grow_graph(qgbdt_ctx *c, const GrowArgs &a, int part_blocks) {
+    cudaStream_t cs = nullptr;
+    QG_CUDA(c, cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking));
+    const int64_t launches_before = c->n_launches;
+    int rc = qg_hist_grow_configure(c);
+    cudaGraph_t graph = nullptr;
+    if (rc == QGBDT_OK) {
+        cudaError_t e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
+        if (e == cudaSuccess) {
+            rc = enqueue_splits(c, a, part_blocks, cs);
+            e = cudaStreamEndCapture(cs, &graph);
+        }
+        if (e != cudaSuccess || rc != QGBDT_OK || !graph) {
+            cudaGetLastError();
+            if (graph) cudaGraphDestroy(graph);
+            cudaStreamDestroy(cs);
+            c->n_launches = launches_before;
+            return rc != QGBDT_OK ? rc : qg_fail(c, QGBDT_ERR_CUDA, "capturing the split loop failed: %s", cudaGetErrorString(e));
+        }
+        cudaGraphExec_t exec = nullptr;
+        e = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            cudaStreamDestroy(cs);
+            c->n_launches = launches_before;
+            return qg_fail(c, QGBDT_ERR_CUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(e));
+        }
+        c->grow_graph_exec = exec;
+        c->grow_graph_launches = c->n_launches - launches_before;
+        c->grow_graph_const_hess = c->const_hess;
+    }
+    c->n_launches = launches_before;
+    cudaStreamDestroy(cs);
+    return rc;
+}
+
+// Grows the tree of boosting iteration slot `tree_slot` of the current train call.  Gradients must
+// have been quantized on the same stream (the state holds the totals and maxima).  Asynchronous.
+int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
+    GrowArgs a;
+    int part_blocks;
+    fill_args(c, a, part_blocks);
+    k_grow_begin<<<1, 1, 0, st>>>(c->d_gs, c->d_leaves, c->d_state, (uint32_t)c->N, tree_slot);
+    QG_LAUNCH_CHECK(c);
+    int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
+    if (rc != QGBDT_OK) return rc;
+    k_grow_finish<true><<<(unsigned)c->F, FIN_WARPS * 32, 0, st>>>(a);
+    QG_LAUNCH_CHECK(c);
+    if (c->prm.num_leaves < 2) return QGBDT_OK;
+    if (c->profile_hist) return enqueue_splits(c, a, part_blocks, st);   // event records around every build
+    if (c->grow_graph_exec && c->grow_graph_const_hess != c->const_hess) qg_grow_graph_destroy(c);
+    if (!c->grow_graph_exec && (rc = build_grow_graph(c, a, part_blocks)) != QGBDT_OK) return rc;
+    QG_CUDA(c, cudaGraphLaunch(reinterpret_cast<cudaGraphExec_t>(c->grow_graph_exec), st));
+    c->n_launches += c->grow_graph_launches;
     return QGBDT_OK;
 }

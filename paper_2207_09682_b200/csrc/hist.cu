@@ -350,13 +350,15 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
 namespace {
 
 template <int LOGW_T, int MODE>
-int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n_tiles, cudaStream_t st) {
+int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n_tiles, cudaStream_t st,
+                    bool configure_only) {
     auto kern = k_hist_grow<LOGW_T, MODE>;
     static bool configured[64] = {};   // per instantiation and device (the attribute belongs to the device's context)
     if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
         QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
         if (c->device >= 0 && c->device < 64) configured[c->device] = true;
     }
+    if (configure_only) return QGBDT_OK;
     int group_parts = 1;
     for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
         if (c->tiles[t].parts > group_parts) group_parts = c->tiles[t].parts;
@@ -366,7 +368,7 @@ int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n
 }
 
 template <int MODE>
-int launch_grow(qgbdt_ctx *c, HistArgs args, const GrowHist &g, cudaStream_t st) {
+int launch_grow(qgbdt_ctx *c, HistArgs args, const GrowHist &g, cudaStream_t st, bool configure_only = false) {
     const int T = (int)c->tiles.size();
     for (int t0 = 0; t0 < T;) {
         int t1 = t0 + 1;
@@ -374,9 +376,9 @@ int launch_grow(qgbdt_ctx *c, HistArgs args, const GrowHist &g, cudaStream_t st)
         args.tile0 = t0;
         int rc;
         switch (c->tiles[t0].logW) {
-            case 5: rc = launch_grow_one<5, MODE>(c, args, g, t1 - t0, st); break;
-            case 3: rc = launch_grow_one<3, MODE>(c, args, g, t1 - t0, st); break;
-            default: rc = launch_grow_one<-1, MODE>(c, args, g, t1 - t0, st); break;
+            case 5: rc = launch_grow_one<5, MODE>(c, args, g, t1 - t0, st, configure_only); break;
+            case 3: rc = launch_grow_one<3, MODE>(c, args, g, t1 - t0, st, configure_only); break;
+            default: rc = launch_grow_one<-1, MODE>(c, args, g, t1 - t0, st, configure_only); break;
         }
         if (rc != QGBDT_OK) return rc;
         t0 = t1;
@@ -385,6 +387,18 @@ int launch_grow(qgbdt_ctx *c, HistArgs args, const GrowHist &g, cudaStream_t st)
 }
 
 }  // namespace
+
+// Sets the function attributes of the kernels qg_hist_grow launches for this context (stream
+// captures must not meet a first-use configuration).
+int qg_hist_grow_configure(qgbdt_ctx *c) {
+    const int bits = c->prm.bits;
+    const int kh = c->const_hess ? 1 : qg_levels_h(bits, c->prm.hess_levels_mode);
+    HistArgs a = {};
+    GrowHist g = {};
+    pick_field_split(qg_levels_g(bits), kh, a.shift, a.flush_rows);
+    if (bits >= 6) return launch_grow<1>(c, a, g, nullptr, true);
+    return a.shift == 16 ? launch_grow<0>(c, a, g, nullptr, true) : launch_grow<2>(c, a, g, nullptr, true);
+}
 
 // Histogram of the smaller child of the split recorded in the grow state (sizes known only on
 // the device): partial histograms or, for a small child, the finished histogram in its pool slot.

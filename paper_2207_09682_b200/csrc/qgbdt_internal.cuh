@@ -84,6 +84,7 @@ struct LeafRec {
 // the split being executed and counters.
 struct GrowState {
     int32_t n_leaves, done;
+    int32_t tree_slot;               // slot of the tree being grown in the device-side model arrays
     int32_t pick, feature, bin;      // leaf being split and its winning candidate
     int32_t logW, byte;              // tile width (log2 words per row) and byte of the split feature's word
     const uint32_t *col;             // that word in row 0 of the tile
@@ -145,6 +146,9 @@ struct qgbdt_ctx {
     SplitRec *d_cand = nullptr;                 // [F][2] per-feature best candidates of the two children
     FeatRec *d_feat_rec = nullptr;              // [F] location of every feature
     double *d_leaf_gain = nullptr;              // [L] stored gain of every leaf's best split (-inf: none)
+    void *grow_graph_exec = nullptr;            // cudaGraphExec_t: the split loop of one tree
+    int64_t grow_graph_launches = 0;            // kernel launches it replays
+    bool grow_graph_const_hess = false;         // objective it was captured for
     // trees of the current qgbdt_train call, on the device until the call ends
     int model_cap = 0;                          // trees the arrays below can hold
     int32_t *d_m_num_leaves = nullptr, *d_m_feature = nullptr, *d_m_bin = nullptr, *d_m_left = nullptr,
@@ -219,4 +223,6 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
 int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st);
 // hist.cu: histogram of the smaller child of the split recorded in the grow state
 int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st);
+int qg_hist_grow_configure(qgbdt_ctx *c);   // function attributes of the kernels it launches (before a capture)
+void qg_grow_graph_destroy(qgbdt_ctx *c);   // grow.cu: drops the captured split loop (buffers are about to change)
 

@@ -62,6 +62,7 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
         QG_CUDA(c, cudaMemsetAsync(c->d_gs, 0, sizeof(GrowState), st));
     }
     if (num_trees > c->model_cap) {
+        qg_grow_graph_destroy(c);   // the captured launches hold the old array addresses
         free_dev(c->d_m_num_leaves); free_dev(c->d_m_feature); free_dev(c->d_m_bin); free_dev(c->d_m_left);
         free_dev(c->d_m_right); free_dev(c->d_m_gain); free_dev(c->d_m_leaf_value); free_dev(c->d_m_leaf_count);
         c->model_cap = 0;

@@ -10,6 +10,9 @@ constexpr int HIST_THREADS = 1024;
 constexpr int HIST_WARPS = HIST_THREADS / 32;
 constexpr int HIST_SMEM = 192 * 1024;     // 128 KB histogram on a 64 KB boundary + the room below it
 constexpr uint32_t MIN_ROWS_PER_CTA = 4096;
+// Wide tiles with at least this many bins look for hot words instead of flushing everything (a
+// look comes twice as often as a flush would; with few bins a flush is cheap and wins).
+constexpr int SELECTIVE_MIN_BINS = 128;
 // Units of four rows in flight per lane.  A CTA of 512 threads (the tree-growing kernel) has twice
 // the registers per thread and keeps more in flight per lane to make up for the fewer warps.
 template <int NT> struct Units { static constexpr int root = NT >= 1024 ? 4 : 6, list = NT >= 1024 ? 2 : 4; };
@@ -25,7 +28,7 @@ struct HistArgs {
     int nb;
     unsigned long long *hist;      // [F][nb]
     unsigned long long *partial;   // [CTA][4][nb][32]
-    uint32_t flush_rows;           // rows one column may add between flushes (narrow local bins only)
+    uint32_t flush_rows;           // rows of the extreme levels a zeroed column can add (narrow local bins only)
     int shift;                     // narrow local bins: bit position of the gradient field (16: the 16+16 split)
     int pass;                      // 32+32 local only: bytes 2*pass, 2*pass+1 of every word
     DevState *state;
@@ -158,6 +161,63 @@ __device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, 
     out.first = false;
 }
 
+// Wide tiles (one or two row slots per column: a flush moves up to 32 k bins through global
+// memory) avoid most flushes: a column only adds half of `flush_rows` rows at a time, after which
+// the CTA looks at every local word.  One whose hessian field has reached half its range, or
+// whose gradient field has left the middle half of its range, is "hot": its sums move to the
+// output (a reduction on the word's 64-bit bin) and the word restarts from zero; all other words
+// can take another half of `flush_rows` rows as they are.  With bin codes spread over many bins
+// almost no word is hot.  Before the first flush the output holds nothing that could be added
+// to: then a hot word asks for a full flush (return value, CTA-uniform).  Callers synchronise
+// before the call; the call ends with a barrier.
+template <int NT, int MODE, int LOGW_T>
+__device__ __forceinline__ bool relieve_local(int *hp, const TileDesc &td, const int logW_rt, int nb, int shift,
+                                              const Out &out) {
+    static_assert(MODE != 1, "32+32 local bins never overflow");
+    const int logW = LOGW_T >= 0 ? LOGW_T : logW_rt;
+    const int logR = 5 - logW, W = 1 << logW;
+    const int lsh = 32 - shift;
+    const int hmask = (1 << shift) - 1;
+    bool want_full = false;
+    const int n4 = nb * 16;                       // 16-byte groups per half of the local histogram
+    for (int half = 0; half < 2; ++half) {
+        for (int i = threadIdx.x; i < n4; i += NT) {
+            int4 *p = reinterpret_cast<int4 *>(hp + half * 16384) + i;
+            const int4 x = *p;
+            // bit 31: gradient field outside [-2^(30-shift), 2^(30-shift)), or top bit of the hessian field set
+            const uint32_t m = (((uint32_t)x.x + 0x40000000u) | ((uint32_t)x.x << lsh)) |
+                               (((uint32_t)x.y + 0x40000000u) | ((uint32_t)x.y << lsh)) |
+                               (((uint32_t)x.z + 0x40000000u) | ((uint32_t)x.z << lsh)) |
+                               (((uint32_t)x.w + 0x40000000u) | ((uint32_t)x.w << lsh));
+            if (m & 0x80000000u) {
+                if (out.first) {
+                    want_full = true;
+                } else {
+                    int xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t hot = ((uint32_t)xs[j] + 0x40000000u) | ((uint32_t)xs[j] << lsh);
+                        if (hot & 0x80000000u) {
+                            const int w = i * 4 + j;                      // word inside this half
+                            const int bin = w >> 6, k = half * 2 + ((w >> 5) & 1), a = (w & 31) >> logR;
+                            const int fl = 4 * a + k;
+                            if (fl < td.nf) {
+                                const long long G = xs[j] >> shift, H = xs[j] & hmask;
+                                unsigned long long *q = out.direct ? out.ptr + (size_t)(td.f0 + fl) * nb + bin
+                                                                   : out.ptr + (size_t)k * nb * W + (bin << logW) + a;
+                                atomicAdd(q, (unsigned long long)(G * 4294967296LL + H));
+                            }
+                            xs[j] = 0;
+                        }
+                    }
+                    *p = make_int4(xs[0], xs[1], xs[2], xs[3]);
+                }
+            }
+        }
+    }
+    return __syncthreads_or(want_full ? 1 : 0) != 0;
+}
+
 // CTAs of the static plan that take part in a build of n rows of a tile.
 __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
     uint32_t want = (n + MIN_ROWS_PER_CTA - 1) / MIN_ROWS_PER_CTA;
@@ -259,16 +319,20 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     // ---- fast warp-units, in epochs that keep every 16+16 column below its limit
     constexpr int U = LIST ? Units<NT>::list : Units<NT>::root;
     constexpr int NWARPS = NT / 32;
+    const bool selective = logR <= 1 && a.nb >= SELECTIVE_MIN_BINS;   // wide tiles: look for hot words instead of flushing everything
     uint32_t q = 0;
     while (q < q1) {
         uint32_t epoch = q1 - q;   // warp-units of this epoch, all warps together
         if (MODE != 1) {
-            const uint32_t room = a.flush_rows > col_rows ? a.flush_rows - col_rows : 0;
+            const uint32_t limit = selective ? a.flush_rows >> 1 : a.flush_rows;
+            const uint32_t room = limit > col_rows ? limit - col_rows : 0;
             const uint32_t fit = room >> 2;                          // every warp-unit adds 4 rows to each column
             if (fit == 0) {
                 __syncthreads();
-                flush_local<NT, MODE>(hp, td, logW, a.nb, pass, shift, out);
-                __syncthreads();
+                if (!selective || relieve_local<NT, MODE == 1 ? 0 : MODE, LOGW_T>(hp, td, logW, a.nb, shift, out)) {
+                    flush_local<NT, MODE>(hp, td, logW, a.nb, pass, shift, out);
+                    __syncthreads();
+                }
                 col_rows = 0;
                 continue;
             }

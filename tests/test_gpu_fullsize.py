@@ -154,3 +154,34 @@ def test_worst_case_accumulation_constant_hessian():
             ctx.build_histograms_rows(rows, hist)
             G, H = binding.unpack_hist(hist)
             assert G[27, 0] == sign * kg * rows.numel() and H[27, 0] == rows.numel()
+
+
+def test_worst_case_accumulation_wide_tile():
+    # a 128-feature tile with many bins: its CTAs look for words that are about to overflow and
+    # move only those to the output; every row in one bin at the extreme levels makes the same
+    # words hot at every look
+    n = 3_000_000
+    data = torch.zeros((n, 160), dtype=torch.uint8, device="cuda")
+    data[:, 5] = 199
+    data[:, 131] = 77
+    data[::2, 64] = 100
+    for bits in (3, 5):
+        kg, kh = oracle.levels(bits)
+        ctx = binding.Context(binding.make_params(bits=bits))
+        ctx.load_binned(data, 200)
+        for sign in (-1.0, 1.0):
+            ctx.quantize_gradients(torch.full((n,), sign, device="cuda"), torch.full((n,), 0.25, device="cuda"))
+            hist = ctx.new_hist()
+            ctx.build_histograms(0, hist)
+            G, H = binding.unpack_hist(hist)
+            assert G[0, 0] == sign * kg * n and H[0, 0] == kh * n and H[5, 0] == 0
+            assert G[5, 199] == sign * kg * n and H[5, 199] == kh * n
+            assert G[131, 77] == sign * kg * n and H[131, 77] == kh * n
+            assert H[64, 100] == kh * (n // 2) and H[64, 0] == kh * (n // 2) and G[64, 100] == sign * kg * (n // 2)
+            assert (G.sum(axis=1) == sign * kg * n).all() and (H.sum(axis=1) == kh * n).all()
+            rows = synth.subset_rows(n, device="cuda")
+            ctx.build_histograms_rows(rows, hist)
+            G, H = binding.unpack_hist(hist)
+            m = rows.numel()
+            assert G[159, 0] == sign * kg * m and H[159, 0] == kh * m and G[5, 199] == sign * kg * m
+            assert (G.sum(axis=1) == sign * kg * m).all() and (H.sum(axis=1) == kh * m).all()

@@ -316,40 +316,45 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
         col_rows = (s1 - s0 + R - 1) >> logR;
     }
 
-    // ---- fast warp-units, in epochs that keep every 16+16 column below its limit
+    // ---- fast warp-units.  This warp takes warp-units warp, warp + NWARPS, ... of the part, in
+    //      groups of U; every lane keeps its loads for the next group in flight in registers.
+    //      Every 16+16 column must stay below its limit: after `kg` groups (4 U NWARPS kg rows per
+    //      column) all warps meet, and the CTA flushes, or looks for hot words.  The loads in
+    //      flight stay in flight across that meeting.
     constexpr int U = LIST ? Units<NT>::list : Units<NT>::root;
     constexpr int NWARPS = NT / 32;
     const bool selective = logR <= 1 && a.nb >= SELECTIVE_MIN_BINS;   // wide tiles: look for hot words instead of flushing everything
-    uint32_t q = 0;
-    while (q < q1) {
-        uint32_t epoch = q1 - q;   // warp-units of this epoch, all warps together
-        if (MODE != 1) {
-            const uint32_t limit = selective ? a.flush_rows >> 1 : a.flush_rows;
-            const uint32_t room = limit > col_rows ? limit - col_rows : 0;
-            const uint32_t fit = room >> 2;                          // every warp-unit adds 4 rows to each column
-            if (fit == 0) {
-                __syncthreads();
-                if (!selective || relieve_local<NT, MODE == 1 ? 0 : MODE, LOGW_T>(hp, td, logW, a.nb, shift, out)) {
-                    flush_local<NT, MODE>(hp, td, logW, a.nb, pass, shift, out);
-                    __syncthreads();
-                }
-                col_rows = 0;
-                continue;
-            }
-            if (fit < epoch) epoch = fit;
+    const uint32_t nq = q1 > (uint32_t)warp ? (q1 - warp + NWARPS - 1) / NWARPS : 0;   // this warp's units
+    const uint32_t groups = ((q1 + NWARPS - 1) / NWARPS + U - 1) / U;                  // of warp 0: the same in every warp
+    uint32_t kg = 0xFFFFFFFFu;                                                         // groups between two meetings
+    if (MODE != 1) {
+        const uint32_t limit = selective ? a.flush_rows >> 1 : a.flush_rows;
+        kg = (limit > col_rows ? limit - col_rows : 0) / (4u * U * NWARPS);
+        if (kg == 0) {   // the host picks wide local bins before the limit gets this small
+            if (threadIdx.x == 0) atomicExch(&a.state->kernel_error, 1);
+            return;
         }
-        // this warp's warp-units: q + warp, q + warp + 32, ... < q + epoch
-        const uint32_t nq = epoch > (uint32_t)warp ? (epoch - warp + NWARPS - 1) / NWARPS : 0;
-        if (!LIST) {
-            const uint32_t v = first_unit + ((q + warp) << logR) + slot;         // first unit of this lane
-            const uint32_t row0 = ((v >> 2) << 4) + (v & 3u);
-            const uint32_t *pw = tile + ((size_t)row0 << logW) + wa;
-            const uint2 *pc = reinterpret_cast<const uint2 *>(a.codes) + v;
-            const uint32_t jstride = 4u << logW;                                  // words between rows 4 apart
-            constexpr uint32_t QW = NWARPS * 128;                                 // words per round of the CTA's warps
-            const uint32_t qc = (uint32_t)NWARPS << logR;                         // units per round of the CTA's warps
-            uint32_t w[U][4];
-            uint2 c[U];
+    }
+    uint32_t since = 0;   // groups since the last meeting
+#define QG_MEET(grp)                                                                                          \
+    if (MODE != 1 && since == kg && (grp) < groups) {                                                         \
+        since = 0;                                                                                            \
+        __syncthreads();                                                                                      \
+        if (!selective || relieve_local<NT, MODE == 1 ? 0 : MODE, LOGW_T>(hp, td, logW, a.nb, shift, out)) { \
+            flush_local<NT, MODE>(hp, td, logW, a.nb, pass, shift, out);                                      \
+            __syncthreads();                                                                                  \
+        }                                                                                                     \
+    }
+    if (!LIST) {
+        const uint32_t v = first_unit + ((uint32_t)warp << logR) + slot;      // first unit of this lane
+        const uint32_t row0 = ((v >> 2) << 4) + (v & 3u);
+        const uint32_t *pw = tile + ((size_t)row0 << logW) + wa;
+        const uint2 *pc = reinterpret_cast<const uint2 *>(a.codes) + v;
+        const uint32_t jstride = 4u << logW;                                  // words between rows 4 apart
+        constexpr uint32_t QW = NWARPS * 128;                                 // words per round of the CTA's warps
+        const uint32_t qc = (uint32_t)NWARPS << logR;                         // units per round of the CTA's warps
+        uint32_t w[U][4];
+        uint2 c[U];
 #define QG_LOAD_UNIT(u)                                                                  \
     {                                                                                    \
         _Pragma("unroll") for (int j = 0; j < 4; ++j) w[u][j] = ldg32(pw + (u) * QW + j * jstride); \
@@ -363,42 +368,55 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
         add_word<MODE>(base, w[u][3], c[u].y, 1, pass, shift);      \
     }
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if ((uint32_t)u < nq) QG_LOAD_UNIT(u)
-            pw += U * QW;
-            pc += U * qc;
-            uint32_t i = 0;
-            for (; i + 2 * U <= nq; i += U) {   // units i .. i+U-1 are in registers, the next U exist
+        for (int u = 0; u < U; ++u)
+            if ((uint32_t)u < nq) QG_LOAD_UNIT(u)
+        pw += U * QW;
+        pc += U * qc;
+        uint32_t i = 0, grp = 0;
+        while (grp < groups) {
+            // groups that can run without a test: units in registers and the next U exist, until the next meeting
+            uint32_t run = i + 2 * U <= nq ? (nq - i - 2 * U) / U + 1 : 0;
+            run = run < kg - since ? run : kg - since;
+            if (run) {
+                for (uint32_t r = 0; r < run; ++r) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    QG_USE_UNIT(u)
-                    QG_LOAD_UNIT(u)
-                }
-                pw += U * QW;
-                pc += U * qc;
-            }
-            for (; i < nq; i += U) {
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    if (i + u < nq) {
+                    for (int u = 0; u < U; ++u) {
                         QG_USE_UNIT(u)
-                        if (i + u + U < nq) QG_LOAD_UNIT(u)
+                        QG_LOAD_UNIT(u)
+                    }
+                    pw += U * QW;
+                    pc += U * qc;
+                }
+            } else {
+                run = 1;
+                if (i < nq) {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (i + u < nq) {
+                            QG_USE_UNIT(u)
+                            if (i + u + U < nq) QG_LOAD_UNIT(u)
+                        }
                     }
                 }
                 pw += U * QW;
                 pc += U * qc;
             }
+            i += run * U;
+            grp += run;
+            since += run;
+            QG_MEET(grp)
+        }
 #undef QG_LOAD_UNIT
 #undef QG_USE_UNIT
-        } else {
-            // entry of (warp-unit wu, j): off + (4 wu << logR) + (j << logR) + slot
-            const size_t e0 = a.off + ((size_t)(first_q + q + warp) << (logR + 2)) + slot;
-            const uint32_t *pr = LIST == 2 ? nullptr : a.rows + e0;
-            const uint2 *pe = LIST == 2 ? a.ents + e0 : nullptr;
-            const uint32_t qs = (uint32_t)(4 * NWARPS) << logR;                   // entries per round of the CTA's warps
-            const uint32_t *tw = tile + wa;
-            uint32_t idx[U][4], w[U][4], c[U][4];
-            uint32_t cn[LIST == 2 ? U : 1][4];   // codes that came with the indices (pair entries)
+    } else {
+        // entry of (warp-unit wu, j): off + (4 wu << logR) + (j << logR) + slot
+        const size_t e0 = a.off + ((size_t)(first_q + warp) << (logR + 2)) + slot;
+        const uint32_t *pr = LIST == 2 ? nullptr : a.rows + e0;
+        const uint2 *pe = LIST == 2 ? a.ents + e0 : nullptr;
+        const uint32_t qs = (uint32_t)(4 * NWARPS) << logR;                   // entries per round of the CTA's warps
+        const uint32_t *tw = tile + wa;
+        uint32_t idx[U][4], w[U][4], c[U][4];
+        uint32_t cn[LIST == 2 ? U : 1][4];   // codes that came with the indices (pair entries)
 #define QG_LOAD_IDX(u)                                                                \
     {                                                                                 \
         _Pragma("unroll") for (int j = 0; j < 4; ++j) {                               \
@@ -424,27 +442,26 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
         _Pragma("unroll") for (int j = 0; j < 4; ++j) add_word<MODE>(base, w[u][j], c[u][j], 0, pass, shift); \
     }
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if ((uint32_t)u < nq) QG_LOAD_IDX(u)
-            if (LIST == 2) pe += U * qs; else pr += U * qs;
+        for (int u = 0; u < U; ++u)
+            if ((uint32_t)u < nq) QG_LOAD_IDX(u)
+        if (LIST == 2) pe += U * qs; else pr += U * qs;
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if ((uint32_t)u < nq) {
-                    QG_LOAD_DATA(u)
-                    if ((uint32_t)u + U < nq) QG_LOAD_IDX(u)
-                }
-            if (LIST == 2) pe += U * qs; else pr += U * qs;
-            uint32_t i = 0;
-            for (; i + 3 * U <= nq; i += U) {   // data of units i .. i+U-1 and indices of the next U are in registers
+        for (int u = 0; u < U; ++u)
+            if ((uint32_t)u < nq) {
+                QG_LOAD_DATA(u)
+                if ((uint32_t)u + U < nq) QG_LOAD_IDX(u)
+            }
+        if (LIST == 2) pe += U * qs; else pr += U * qs;
+        uint32_t i = 0;
+        for (uint32_t grp = 0; grp < groups; i += U) {
+            if (i + 3 * U <= nq) {   // data of units i .. i+U-1 and indices of the next U are in registers, U more exist
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     QG_USE_DATA(u)
                     QG_LOAD_DATA(u)
                     QG_LOAD_IDX(u)
                 }
-                if (LIST == 2) pe += U * qs; else pr += U * qs;
-            }
-            for (; i < nq; i += U) {
+            } else if (i < nq) {
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     if (i + u < nq) {
@@ -455,15 +472,17 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
                         }
                     }
                 }
-                if (LIST == 2) pe += U * qs; else pr += U * qs;
             }
+            if (LIST == 2) pe += U * qs; else pr += U * qs;
+            ++grp;
+            ++since;
+            QG_MEET(grp)
+        }
 #undef QG_LOAD_IDX
 #undef QG_LOAD_DATA
 #undef QG_USE_DATA
-        }
-        q += epoch;
-        col_rows += 4 * epoch;
     }
+#undef QG_MEET
     __syncthreads();
     flush_local<NT, MODE>(hp, td, logW, a.nb, pass, shift, out);
 }

@@ -195,7 +195,7 @@ def time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes, reps=10
         ms = float(np.median(ts))
         nbytes = nr * (features + code_bytes + (0 if r is None else 4)) + features * n_bins * 8
         out[name] = {"rows": nr, "us": 1e3 * ms, "row_features_per_s": nr * features / (ms * 1e-3),
-                     "gbs": nbytes / (ms * 1e6), "note": "partial-histogram kernel + merge kernel, %d builds per timing" % batch}
+                     "gbs": nbytes / (ms * 1e6), "note": "partial histograms and their merge in one cooperative kernel, %d builds per timing" % batch}
     return out
 
 

@@ -180,6 +180,18 @@ __device__ inline SplitRec load_rec_cg(const SplitRec *p) {   // bypasses L1: wr
 }
 static_assert(sizeof(SplitRec) == 40, "SplitRec is copied as five 64-bit words");
 
+__device__ inline SplitRec shfl_xor_rec(const SplitRec &r, int o) {
+    SplitRec x;
+    x.gain = __shfl_xor_sync(0xffffffffu, r.gain, o);
+    x.gl = __shfl_xor_sync(0xffffffffu, r.gl, o);
+    x.hl = __shfl_xor_sync(0xffffffffu, r.hl, o);
+    x.feature = __shfl_xor_sync(0xffffffffu, r.feature, o);
+    x.bin = __shfl_xor_sync(0xffffffffu, r.bin, o);
+    x.valid = __shfl_xor_sync(0xffffffffu, r.valid, o);
+    x.pad = 0;
+    return x;
+}
+
 // ROOT: scans the root histogram (pool slot 0).  Otherwise: completes the split recorded in the
 // grow state.  One block per feature.
 template <bool ROOT>
@@ -302,7 +314,9 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     if (!is_last) return;
     __threadfence();
 
-    // ---- the last block: best candidates over all features, the new leaves, the next pick
+    // ---- the last block: best candidates over all features, the new leaves, the next pick.
+    //      Every thread ends up with the same reduced values (warp shuffles, then the eight warp
+    //      results from shared memory), so thread 0 needs no further round of barriers.
     const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
     const int leaves_now = ROOT ? 1 : n_leaves + 1;
     // gains of the older leaves, fetched while the candidates are being reduced
@@ -318,72 +332,34 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
         if (qg_rec_better(x, bS)) bS = x;
         if (qg_rec_better(y, bL)) bL = y;
     }
-    sm[0][threadIdx.x] = bS;
-    sm[1][threadIdx.x] = bL;
-    __syncthreads();
-    for (int st = FIN_WARPS * 16; st > 0; st >>= 1) {
-        if ((int)threadIdx.x < st) {
-            if (qg_rec_better(sm[0][threadIdx.x + st], sm[0][threadIdx.x])) sm[0][threadIdx.x] = sm[0][threadIdx.x + st];
-            if (qg_rec_better(sm[1][threadIdx.x + st], sm[1][threadIdx.x])) sm[1][threadIdx.x] = sm[1][threadIdx.x + st];
-        }
-        __syncthreads();
+    for (int o = 16; o > 0; o >>= 1) {
+        const SplitRec x = shfl_xor_rec(bS, o), y = shfl_xor_rec(bL, o);
+        if (qg_rec_better(x, bS)) bS = x;
+        if (qg_rec_better(y, bL)) bL = y;
     }
-    __shared__ LeafRec s_new[2];   // the two leaves this split made (ROOT: [0] is the root)
-    __shared__ int s_new_id[2];
+    if (lane == 0) { sm[0][warp] = bS; sm[1][warp] = bL; }
+    __syncthreads();
+    bS = sm[0][0];
+    bL = sm[1][0];
+    for (int w = 1; w < FIN_WARPS; ++w) {
+        if (qg_rec_better(sm[0][w], bS)) bS = sm[0][w];
+        if (qg_rec_better(sm[1][w], bL)) bL = sm[1][w];
+    }
+    // where the winning features live (needed if one of the new leaves is picked next)
+    FeatRec fS = {}, fL = {};
     if (threadIdx.x == 0) {
-        bS = sm[0][0];
-        bL = sm[1][0];
-        if (ROOT) {
-            LeafRec r;
-            r.off = 0; r.n = a.N; r.buf = -1; r.slot = 0; r.G = pS.G; r.H = pS.H; r.best = bS;
-            r.parent_node = -1; r.parent_side = 0;
-            a.leaves[0] = r;
-            a.leaf_gain[0] = bS.valid ? bS.gain : NEG;
-            s_new[0] = r; s_new_id[0] = 0; s_new_id[1] = -1;
-            gs->n_leaves = 1;
-        } else {
-            const int pick = gs->pick, right = n_leaves, node = n_leaves - 1;
-            // node arrays of the tree being grown (the slot is device state: the launch arguments
-            // are the same for every tree, so the launches can be replayed from a CUDA graph)
-            const size_t no = (size_t)gs->tree_slot * (a.L > 1 ? a.L - 1 : 1);
-            a.m_feature[no + node] = gs->feature;
-            a.m_bin[no + node] = gs->bin;
-            a.m_left[no + node] = ~pick;
-            a.m_right[no + node] = ~right;
-            a.m_gain[no + node] = gs->gain;
-            if (gs->parent_node >= 0) {
-                if (gs->parent_side == 0) a.m_left[no + gs->parent_node] = node;
-                else a.m_right[no + gs->parent_node] = node;
-            }
-            const int dstbuf = gs->buf == 0 ? 1 : 0;
-            LeafRec lf, rt;
-            lf.off = gs->off; lf.n = nl; lf.buf = dstbuf;
-            lf.G = gs->gl; lf.H = gs->hl;
-            lf.parent_node = node; lf.parent_side = 0;
-            rt.off = gs->off + nl; rt.n = nr; rt.buf = dstbuf;
-            rt.G = gs->PG - gs->gl; rt.H = gs->PH - gs->hl;
-            rt.parent_node = node; rt.parent_side = 1;
-            lf.slot = small_is_left ? n_leaves : gs->parent_slot;
-            rt.slot = small_is_left ? gs->parent_slot : n_leaves;
-            lf.best = small_is_left ? bS : bL;
-            rt.best = small_is_left ? bL : bS;
-            a.leaves[pick] = lf;
-            a.leaves[right] = rt;
-            a.leaf_gain[pick] = lf.best.valid ? lf.best.gain : NEG;
-            a.leaf_gain[right] = rt.best.valid ? rt.best.gain : NEG;
-            s_new[0] = lf; s_new_id[0] = pick;
-            s_new[1] = rt; s_new_id[1] = right;
-            gs->n_leaves = n_leaves + 1;
-            gs->hist_rows += small_is_left ? nl : nr;
-            gs->hist_builds += 1;
-        }
-        gs->finish_count = 0;
+        if (bS.valid) fS = a.feat_rec[bS.feature];
+        if (!ROOT && bL.valid) fL = a.feat_rec[bL.feature];
     }
-    __syncthreads();
+    // the leaves this split made (ROOT: only the root) and their gains
+    const int id0 = ROOT ? 0 : gs->pick, id1 = ROOT ? -1 : n_leaves;
+    const SplitRec best0 = ROOT ? bS : (small_is_left ? bS : bL);   // of leaf id0 (the left child)
+    const SplitRec best1 = small_is_left ? bL : bS;                 // of leaf id1 (the right child)
+    const double gain0 = best0.valid ? best0.gain : NEG, gain1 = best1.valid ? best1.gain : NEG;
 
     // the next leaf to split: largest gain, lowest leaf number on equal gain
-    __shared__ double pg[FIN_WARPS * 32];
-    __shared__ int pi[FIN_WARPS * 32];
+    __shared__ double pg[FIN_WARPS];
+    __shared__ int pi[FIN_WARPS];
     double bg = NEG;
     int bi = -1;
     if (leaves_now < a.L) {
@@ -392,59 +368,111 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
             const int i2 = (int)threadIdx.x + k2 * FIN_WARPS * 32;
             if (i2 < leaves_now) {
                 double g = my_gain[k2];
-                if (i2 == s_new_id[0]) g = s_new[0].best.valid ? s_new[0].best.gain : NEG;
-                if (i2 == s_new_id[1]) g = s_new[1].best.valid ? s_new[1].best.gain : NEG;
+                if (i2 == id0) g = gain0;
+                if (i2 == id1) g = gain1;
                 if (g > bg) { bg = g; bi = i2; }
             }
         }
         for (int i2 = (int)threadIdx.x + 4 * FIN_WARPS * 32; i2 < leaves_now; i2 += FIN_WARPS * 32) {   // more than 1024 leaves
             double g = __ldcg(a.leaf_gain + i2);
-            if (i2 == s_new_id[0]) g = s_new[0].best.valid ? s_new[0].best.gain : NEG;
-            if (i2 == s_new_id[1]) g = s_new[1].best.valid ? s_new[1].best.gain : NEG;
+            if (i2 == id0) g = gain0;
+            if (i2 == id1) g = gain1;
             if (g > bg) { bg = g; bi = i2; }
         }
     }
-    pg[threadIdx.x] = bg;
-    pi[threadIdx.x] = bi;
+    for (int o = 16; o > 0; o >>= 1) {
+        const double og = __shfl_xor_sync(0xffffffffu, bg, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (oi >= 0 && (bi < 0 || og > bg || (og == bg && oi < bi))) { bg = og; bi = oi; }
+    }
+    if (lane == 0) { pg[warp] = bg; pi[warp] = bi; }
     __syncthreads();
-    for (int st = FIN_WARPS * 16; st > 0; st >>= 1) {
-        if ((int)threadIdx.x < st) {
-            const double og = pg[threadIdx.x + st];
-            const int oi = pi[threadIdx.x + st];
-            const int mi = pi[threadIdx.x];
-            if (oi >= 0 && (mi < 0 || og > pg[threadIdx.x] || (og == pg[threadIdx.x] && oi < mi))) {
-                pg[threadIdx.x] = og;
-                pi[threadIdx.x] = oi;
-            }
-        }
-        __syncthreads();
+    if (threadIdx.x != 0) return;
+    bg = pg[0];
+    bi = pi[0];
+    for (int w = 1; w < FIN_WARPS; ++w) {
+        const double og = pg[w];
+        const int oi = pi[w];
+        if (oi >= 0 && (bi < 0 || og > bg || (og == bg && oi < bi))) { bg = og; bi = oi; }
     }
-    if (threadIdx.x == 0) {
-        const int pick = pi[0];
-        if (pick < 0) {
-            gs->done = 1;
-        } else {
-            const LeafRec lr = pick == s_new_id[0] ? s_new[0] : (pick == s_new_id[1] ? s_new[1] : a.leaves[pick]);
-            const FeatRec pf = a.feat_rec[lr.best.feature];
-            gs->pick = pick;
-            gs->feature = lr.best.feature;
-            gs->bin = lr.best.bin;
-            gs->col = pf.col;
-            gs->logW = pf.logW;
-            gs->byte = pf.byte;
-            gs->off = lr.off;
-            gs->n = lr.n;
-            gs->buf = lr.buf;
-            gs->gl = lr.best.gl;
-            gs->hl = lr.best.hl;
-            gs->PG = lr.G;
-            gs->PH = lr.H;
-            gs->gain = lr.best.gain;
-            gs->parent_slot = lr.slot;
-            gs->parent_node = lr.parent_node;
-            gs->parent_side = lr.parent_side;
+    const int pick = bi;
+
+    LeafRec lf, rt;   // ROOT: lf is the root
+    if (ROOT) {
+        lf.off = 0; lf.n = a.N; lf.buf = -1; lf.slot = 0; lf.G = pS.G; lf.H = pS.H; lf.best = bS;
+        lf.parent_node = -1; lf.parent_side = 0;
+        a.leaves[0] = lf;
+        a.leaf_gain[0] = gain0;
+        rt = lf;
+        gs->n_leaves = 1;
+    } else {
+        const int right = n_leaves, node = n_leaves - 1;
+        // node arrays of the tree being grown (the slot is device state: the launch arguments
+        // are the same for every tree, so the launches can be replayed from a CUDA graph)
+        const size_t no = (size_t)gs->tree_slot * (a.L > 1 ? a.L - 1 : 1);
+        const int pn = gs->parent_node;
+        a.m_feature[no + node] = gs->feature;
+        a.m_bin[no + node] = gs->bin;
+        a.m_left[no + node] = ~id0;
+        a.m_right[no + node] = ~right;
+        a.m_gain[no + node] = gs->gain;
+        if (pn >= 0) {
+            if (gs->parent_side == 0) a.m_left[no + pn] = node;
+            else a.m_right[no + pn] = node;
         }
+        const int dstbuf = gs->buf == 0 ? 1 : 0;
+        lf.off = gs->off; lf.n = nl; lf.buf = dstbuf;
+        lf.G = gs->gl; lf.H = gs->hl;
+        lf.parent_node = node; lf.parent_side = 0;
+        rt.off = gs->off + nl; rt.n = nr; rt.buf = dstbuf;
+        rt.G = gs->PG - gs->gl; rt.H = gs->PH - gs->hl;
+        rt.parent_node = node; rt.parent_side = 1;
+        lf.slot = small_is_left ? n_leaves : gs->parent_slot;
+        rt.slot = small_is_left ? gs->parent_slot : n_leaves;
+        lf.best = best0;
+        rt.best = best1;
+        a.leaves[id0] = lf;
+        a.leaves[right] = rt;
+        a.leaf_gain[id0] = gain0;
+        a.leaf_gain[right] = gain1;
+        gs->n_leaves = n_leaves + 1;
+        gs->hist_rows += small_is_left ? nl : nr;
+        gs->hist_builds += 1;
     }
+    gs->finish_count = 0;
+    if (pick < 0) {
+        gs->done = 1;
+        return;
+    }
+    LeafRec lr;
+    FeatRec pf;
+    if (pick == id0) {
+        lr = lf;
+        pf = ROOT || small_is_left ? fS : fL;
+    } else if (pick == id1) {
+        lr = rt;
+        pf = small_is_left ? fL : fS;
+    } else {
+        lr = a.leaves[pick];
+        pf = a.feat_rec[lr.best.feature];
+    }
+    gs->pick = pick;
+    gs->feature = lr.best.feature;
+    gs->bin = lr.best.bin;
+    gs->col = pf.col;
+    gs->logW = pf.logW;
+    gs->byte = pf.byte;
+    gs->off = lr.off;
+    gs->n = lr.n;
+    gs->buf = lr.buf;
+    gs->gl = lr.best.gl;
+    gs->hl = lr.best.hl;
+    gs->PG = lr.G;
+    gs->PH = lr.H;
+    gs->gain = lr.best.gain;
+    gs->parent_slot = lr.slot;
+    gs->parent_node = lr.parent_node;
+    gs->parent_side = lr.parent_side;
 }
 
 }  // namespace

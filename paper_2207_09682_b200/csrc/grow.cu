@@ -15,7 +15,7 @@ namespace {
 constexpr int PART_THREADS = 256;
 constexpr int PART_WARPS = PART_THREADS / 32;
 constexpr int FIN_WARPS = 8;
-constexpr uint32_t MIN_ROWS_PER_CTA = 4096;   // same rule as the histogram kernel
+constexpr uint32_t MIN_ROWS_PER_CTA = 1024;   // same rule as the histogram kernel
 
 __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
     uint32_t want = (n + MIN_ROWS_PER_CTA - 1) / MIN_ROWS_PER_CTA;

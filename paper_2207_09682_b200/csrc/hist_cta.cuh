@@ -9,7 +9,7 @@ namespace {
 constexpr int HIST_THREADS = 1024;
 constexpr int HIST_WARPS = HIST_THREADS / 32;
 constexpr int HIST_SMEM = 192 * 1024;     // 128 KB histogram on a 64 KB boundary + the room below it
-constexpr uint32_t MIN_ROWS_PER_CTA = 4096;
+constexpr uint32_t MIN_ROWS_PER_CTA = 1024;
 // Wide tiles with at least this many bins look for hot words instead of flushing everything (a
 // look comes twice as often as a flush would; with few bins a flush is cheap and wins).
 constexpr int SELECTIVE_MIN_BINS = 128;

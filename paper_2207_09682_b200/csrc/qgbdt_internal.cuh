@@ -27,7 +27,7 @@
 //
 // Histogram plan: tiles of equal width are built by one launch and share the SMs equally;
 // a tile owns `parts` partial-histogram slots starting at `cta0`; the grid is (part, tile).  A build of n rows uses the first
-// min(parts, ceil(n / 4096)) parts of every tile.
+// min(parts, ceil(n / 1024)) parts of every tile.
 //
 // Row lists: one uint32 array of N entries; leaf l owns [leaf_off[l], +leaf_n[l]).
 // ---------------------------------------------------------------------------

@@ -72,18 +72,20 @@ __device__ inline void warp_range(uint32_t nw, uint32_t gw, uint32_t n_count, ui
 // in flight together.
 __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
     const GrowState *gs = a.gs;
-    if (gs->done) return;
+    // every field at once (one round trip to memory), then the early exits
+    const int done = gs->done, buf = gs->buf;
+    const uint32_t n = gs->n, off = gs->off;
+    const uint32_t *col = gs->col;
+    const int logW = gs->logW, shift = 8 * gs->byte;
+    const uint32_t thr = (uint32_t)gs->bin;
+    if (done) return;
     const int lane = threadIdx.x & 31;
     const uint32_t gw = blockIdx.x * PART_WARPS + (threadIdx.x >> 5);
-    const uint32_t n = gs->n, off = gs->off;
     const uint32_t nw = (n + 31) >> 5;
     uint32_t w0, w1, active;
     warp_range(nw, gw, (uint32_t)a.n_count, w0, w1, active);
     if (gw >= active) return;
-    const uint2 *src = gs->buf < 0 ? nullptr : (gs->buf ? a.ent1 : a.ent0);
-    const uint32_t *col = gs->col;
-    const int logW = gs->logW, shift = 8 * gs->byte;
-    const uint32_t thr = (uint32_t)gs->bin;
+    const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
     uint32_t lefts = 0;
     for (uint32_t w = w0; w < w1; w += 4) {
         uint32_t row[4], word[4];
@@ -109,10 +111,11 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
 
 __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
     GrowState *gs = a.gs;
-    if (gs->done) return;
+    const int done = gs->done, buf = gs->buf;   // every field at once, then the early exits
+    const uint32_t n = gs->n, off = gs->off;
+    if (done) return;
     const int lane = threadIdx.x & 31;
     const uint32_t gw = blockIdx.x * PART_WARPS + (threadIdx.x >> 5);
-    const uint32_t n = gs->n, off = gs->off;
     const uint32_t nw = (n + 31) >> 5;
     uint32_t w0, w1, active;
     warp_range(nw, gw, (uint32_t)a.n_count, w0, w1, active);
@@ -137,8 +140,8 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
         total += __shfl_xor_sync(0xffffffffu, total, o);
     }
     if (gw == 0 && lane == 0) gs->nl = total;
-    const uint2 *src = gs->buf < 0 ? nullptr : (gs->buf ? a.ent1 : a.ent0);
-    uint2 *dst = gs->buf == 0 ? a.ent1 : a.ent0;
+    const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
+    uint2 *dst = buf == 0 ? a.ent1 : a.ent0;
     for (uint32_t w = w0; w < w1; w += 4) {
         uint32_t bw[4];
         uint2 ent[4];
@@ -197,20 +200,26 @@ __device__ inline SplitRec shfl_xor_rec(const SplitRec &r, int o) {
 template <bool ROOT>
 __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     GrowState *gs = a.gs;
-    if (gs->done) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int f = blockIdx.x;   // one block per feature
-    const int n_leaves = gs->n_leaves;
+    // everything the block needs from the state, at once (one round trip to memory), then the early exit
+    const int done = gs->done, n_leaves = gs->n_leaves, parent_slot = ROOT ? 0 : gs->parent_slot;
+    const uint32_t gs_n = gs->n, gs_nl = gs->nl;
+    const long long gs_gl = gs->gl, gs_hl = gs->hl, gs_PG = gs->PG, gs_PH = gs->PH;
+    const long long tot_g = a.state->tot_g, tot_h = a.state->tot_h;
+    const uint32_t gmax_bits = a.state->gmax_bits, hmax_bits = a.state->hmax_bits;
+    const FeatRec fr = a.feat_rec[f];
+    if (done) return;
     const size_t hw = (size_t)a.F * a.nb;
 
     // the two children: "small" was built by Algorithm 1, "large" is parent - small
-    const uint32_t n = ROOT ? a.N : gs->n, nl = ROOT ? n : gs->nl, nr = n - nl;
+    const uint32_t n = ROOT ? a.N : gs_n, nl = ROOT ? n : gs_nl, nr = n - nl;
     const bool small_is_left = nl <= nr;
     SplitParams pS = a.sp, pL = a.sp;
     if (ROOT) {
-        pS.G = a.state->tot_g; pS.H = a.state->tot_h; pS.n_s = n;
+        pS.G = tot_g; pS.H = tot_h; pS.n_s = n;
     } else {
-        const long long gl = gs->gl, hl = gs->hl, gr = gs->PG - gl, hr = gs->PH - hl;
+        const long long gl = gs_gl, hl = gs_hl, gr = gs_PG - gl, hr = gs_PH - hl;
         pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl : nr;
         pL.G = small_is_left ? gr : gl; pL.H = small_is_left ? hr : hl; pL.n_s = small_is_left ? nr : nl;
     }
@@ -218,17 +227,17 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     //      larger child's bin by subtraction
     __shared__ SplitRec sm[2][FIN_WARPS * 32];
     __shared__ bool is_last;
-    double dg, dh;
-    qg_scales(a.state, pS, dg, dh);
+    // interval lengths of Eq. 5 from the maxima stored by the quantizer
+    const double dg = __ddiv_rn((double)__uint_as_float(gmax_bits), (double)pS.kg);
+    const double dh = pS.const_h ? 1.0 : __ddiv_rn((double)__uint_as_float(hmax_bits), (double)pS.kh);
     const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
     const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
-    const FeatRec fr = a.feat_rec[f];
     const int fl = fr.fl, W = 1 << fr.logW;
     const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)fr.parts, (uint32_t)pS.n_s);
     const size_t pstride = (size_t)4 * a.nb * 32;
     const unsigned long long *part = a.partial + (size_t)fr.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
     unsigned long long *S = a.pool + (ROOT ? 0 : (size_t)n_leaves * hw) + (size_t)f * a.nb;
-    unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)gs->parent_slot * hw + (size_t)f * a.nb;
+    unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)parent_slot * hw + (size_t)f * a.nb;
     // n_bins <= 256: thread b owns bin b
     const int b = (int)threadIdx.x;
     unsigned long long s = 0, l = 0;

@@ -112,13 +112,16 @@ template <int LOGW_T, int MODE>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowHist g) {
     extern __shared__ __align__(1024) int sh[];
     const GrowState *gs = g.gs;
-    if (gs->done) return;
-    const uint32_t nl = gs->nl, nr = gs->n - nl;
-    a.ents = gs->buf == 0 ? g.ent1 : g.ent0;
-    a.off = nl <= nr ? gs->off : gs->off + nl;
-    a.n = nl <= nr ? nl : nr;
-    a.hist = g.pool + (size_t)gs->n_leaves * g.hist_words;
+    // every field and the tile at once (one round trip to memory), then the early exits
+    const int done = gs->done, buf = gs->buf, n_leaves = gs->n_leaves;
+    const uint32_t nl = gs->nl, n = gs->n, off = gs->off;
     const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
+    if (done) return;
+    const uint32_t nr = n - nl;
+    a.ents = buf == 0 ? g.ent1 : g.ent0;
+    a.off = nl <= nr ? off : off + nl;
+    a.n = nl <= nr ? nl : nr;
+    a.hist = g.pool + (size_t)n_leaves * g.hist_words;
     const uint32_t P = effective_parts((uint32_t)td.parts, a.n);
     if (blockIdx.x >= P) return;
     hist_cta<HIST_THREADS, LOGW_T, MODE, 2>(a, td, blockIdx.x, P, sh);

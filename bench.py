@@ -31,10 +31,10 @@ WORKLOAD_ROWS = {"large": 10_500_000, "tall": 1_000_000, "tiny": 50_000, "wide":
 CPU_SAMPLE_ROWS = {"large": 3_000_000, "tall": 1_000_000, "tiny": 50_000, "wide": 20_000}
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the histogram kernels on the 'large' workload from an ncu capture
-# (profiles/launch_list_large_10p5Mx28.md): 3.33 GB over the 255 builds of one tree.  Valid only for
+# (profiles/launch_list_large_10p5Mx28.md): 3.37 GB over the 255 builds of one tree.  Valid only for
 # the kernel sources the capture was taken with.
-HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 13.05e6,
-                "sources_sha1": "e9d5494cc75be3cbe2f12a219513d11bfaa767f2"}
+HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 13.21e6,
+                "sources_sha1": "c4029d36fab32b2fdee5138478f4852488404037"}
 
 
 def hist_traffic(workload, rows):

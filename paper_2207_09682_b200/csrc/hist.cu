@@ -32,12 +32,24 @@
 
 namespace {
 
+// Row shares of a tile when its CTAs work in pairs (one pass of the 32+32 mode each).
+__device__ __host__ inline uint32_t paired_parts(uint32_t P) { return P > 1 ? P >> 1 : 1; }
+
 // Stand-alone build: the grid is (part, tile - tile0).
 template <int LOGW_T, int MODE, int LIST>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist(HistArgs a) {
     extern __shared__ __align__(1024) int sh[];
     const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
     const uint32_t P = effective_parts((uint32_t)td.parts, a.n);
+    if (MODE == 1 && a.pass < 0) {
+        // 32+32 local bins, both passes side by side: CTAs 2i and 2i + 1 take the same rows, one
+        // pass each, at the same time, so that the second reader of a row finds it in L2
+        const uint32_t P2 = paired_parts(P);
+        if ((blockIdx.x >> 1) >= P2) return;
+        a.pass = (int)(blockIdx.x & 1u);
+        hist_cta<HIST_THREADS, LOGW_T, MODE, LIST>(a, td, blockIdx.x >> 1, P2, sh);
+        return;
+    }
     if (blockIdx.x >= P) return;
     hist_cta<HIST_THREADS, LOGW_T, MODE, LIST>(a, td, blockIdx.x, P, sh);
 }
@@ -131,9 +143,9 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowH
 // 32 consecutive partial entries; its eight thread groups each add every eighth partial.
 __global__ void __launch_bounds__(256) k_hist_reduce(const TileDesc *__restrict__ tiles, uint32_t n, int nb,
                                                      const unsigned long long *__restrict__ partial,
-                                                     unsigned long long *__restrict__ hist) {
+                                                     unsigned long long *__restrict__ hist, int paired) {
     const TileDesc td = tiles[blockIdx.y];
-    const uint32_t P = effective_parts((uint32_t)td.parts, n);
+    const uint32_t P = paired ? paired_parts(effective_parts((uint32_t)td.parts, n)) : effective_parts((uint32_t)td.parts, n);
     if (P <= 1) return;
     const int W = 1 << td.logW;
     const uint32_t total = 4u * nb * W;
@@ -189,7 +201,9 @@ int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st)
     int group_parts = 1;
     for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
         if (c->tiles[t].parts > group_parts) group_parts = c->tiles[t].parts;
-    const dim3 grid(effective_parts((uint32_t)group_parts, args.n), (unsigned)n_tiles);
+    uint32_t gx = effective_parts((uint32_t)group_parts, args.n);
+    if (MODE == 1 && args.pass < 0) gx = 2 * paired_parts(gx);
+    const dim3 grid(gx, (unsigned)n_tiles);
     kern<<<grid, HIST_THREADS, HIST_SMEM, st>>>(args);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
@@ -334,16 +348,13 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
     } else if (!wide) {
         rc = d_rows ? launch_hist<2, 1>(c, a, st) : launch_hist<2, 0>(c, a, st);
     } else {
+        a.pass = -1;   // both passes in one launch, by pairs of CTAs
         rc = d_rows ? launch_hist<1, 1>(c, a, st) : launch_hist<1, 0>(c, a, st);
-        if (rc == QGBDT_OK) {
-            a.pass = 1;
-            rc = d_rows ? launch_hist<1, 1>(c, a, st) : launch_hist<1, 0>(c, a, st);
-        }
     }
     if (rc != QGBDT_OK) return rc;
     if (merge_needed && !coop) {
         const dim3 grid((unsigned)((4 * c->nb * 32 + 31) / 32), (unsigned)c->tiles.size());
-        k_hist_reduce<<<grid, 256, 0, st>>>(c->d_tiles, (uint32_t)n, c->nb, c->d_partial, d_hist);
+        k_hist_reduce<<<grid, 256, 0, st>>>(c->d_tiles, (uint32_t)n, c->nb, c->d_partial, d_hist, wide ? 1 : 0);
         QG_LAUNCH_CHECK(c);
     }
     if (ev1) QG_CUDA(c, cudaEventRecord(ev1, st));

@@ -30,7 +30,8 @@ struct HistArgs {
     unsigned long long *partial;   // [CTA][4][nb][32]
     uint32_t flush_rows;           // rows of the extreme levels a zeroed column can add (narrow local bins only)
     int shift;                     // narrow local bins: bit position of the gradient field (16: the 16+16 split)
-    int pass;                      // 32+32 local only: bytes 2*pass, 2*pass+1 of every word
+    int pass;                      // 32+32 local only: bytes 2*pass, 2*pass+1 of every word (-1 at launch: the
+                                   // CTA takes its pass from its number)
     DevState *state;
 };
 

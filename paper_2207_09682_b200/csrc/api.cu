@@ -66,6 +66,8 @@ void free_data(qgbdt_ctx *c) {
     dev_free(c->d_ent1);
     dev_free(c->d_cand);
     dev_free(c->d_feat_rec);
+    dev_free(c->d_colmajor);
+    c->col_stride = 0;
     dev_free(c->d_leaf_gain);
     dev_free(c->d_m_num_leaves);
     dev_free(c->d_m_feature);
@@ -213,6 +215,7 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
                 fr[f].parts = t.parts;
                 fr[f].fl = fl;
                 fr[f].pad = 0;
+                fr[f].col8 = nullptr;
             }
         if ((rc = dev_alloc(c, &c->d_feat_rec, (size_t)n_features)) != QGBDT_OK) return rc;
         QG_CUDA(c, cudaMemcpy(c->d_feat_rec, fr.data(), sizeof(FeatRec) * fr.size(), cudaMemcpyHostToDevice));

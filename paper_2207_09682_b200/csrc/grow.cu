@@ -76,6 +76,7 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
     const int done = gs->done, buf = gs->buf;
     const uint32_t n = gs->n, off = gs->off;
     const uint32_t *col = gs->col;
+    const uint8_t *col8 = gs->col8;
     const int logW = gs->logW, shift = 8 * gs->byte;
     const uint32_t thr = (uint32_t)gs->bin;
     if (done) return;
@@ -94,8 +95,15 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
             const uint32_t e = ((w + k) << 5) + lane;
             row[k] = (w + k < w1 && e < n) ? (src ? src[off + e].x : off + e) : 0xFFFFFFFFu;
         }
+        // the bin code of the split feature: one byte of the column-major copy (ascending rows share
+        // DRAM granules), or, without that copy, a word of the tile (a granule per row)
+        if (col8) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) word[k] = row[k] != 0xFFFFFFFFu ? col[(size_t)row[k] << logW] : 0xFFFFFFFFu;
+            for (int k = 0; k < 4; ++k) word[k] = row[k] != 0xFFFFFFFFu ? (uint32_t)col8[row[k]] << shift : 0xFFFFFFFFu;
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) word[k] = row[k] != 0xFFFFFFFFu ? col[(size_t)row[k] << logW] : 0xFFFFFFFFu;
+        }
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const bool left = row[k] != 0xFFFFFFFFu && ((word[k] >> shift) & 0xFFu) <= thr;
@@ -469,6 +477,7 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     gs->feature = lr.best.feature;
     gs->bin = lr.best.bin;
     gs->col = pf.col;
+    gs->col8 = pf.col8;
     gs->logW = pf.logW;
     gs->byte = pf.byte;
     gs->off = lr.off;

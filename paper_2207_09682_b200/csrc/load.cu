@@ -51,6 +51,49 @@ int qg_relayout(qgbdt_ctx *c, const uint8_t *d_bins, int layout, int64_t ld, cud
     return QGBDT_OK;
 }
 
+namespace {
+
+// Block (x, a): rows 256 x .. 256 x + 255 of word a of a tile; four coalesced byte columns out.
+__global__ void __launch_bounds__(256) k_to_columns(const uint32_t *__restrict__ tile, int logW, int nf, long long N,
+                                                    uint8_t *__restrict__ cols, size_t stride) {
+    const int a = blockIdx.y;
+    for (long long row = blockIdx.x * 256ll + threadIdx.x; row < N; row += (long long)gridDim.x * 256) {
+        const uint32_t w = tile[((size_t)row << logW) + a];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (4 * a + k < nf) cols[(size_t)(4 * a + k) * stride + row] = (uint8_t)(w >> (8 * k));
+    }
+}
+
+__global__ void k_set_columns(FeatRec *feat_rec, int F, uint8_t *cols, size_t stride) {
+    const int f = blockIdx.x * blockDim.x + threadIdx.x;
+    if (f < F) feat_rec[f].col8 = cols + (size_t)f * stride;
+}
+
+}  // namespace
+
+int qg_build_columns(qgbdt_ctx *c, cudaStream_t st) {
+    if (c->d_colmajor) return QGBDT_OK;
+    const size_t stride = ((size_t)c->N + 127) / 128 * 128;
+    void *p = nullptr;
+    if (cudaMalloc(&p, stride * (size_t)c->F) != cudaSuccess) {
+        cudaGetLastError();
+        return QGBDT_OK;   // the feature records keep col8 == nullptr
+    }
+    c->d_colmajor = reinterpret_cast<uint8_t *>(p);
+    c->col_stride = stride;
+    for (const TileDesc &t : c->tiles) {
+        long long bx = (c->N + 255) / 256;
+        if (bx > 65535) bx = 65535;
+        const dim3 grid((unsigned)bx, (unsigned)((t.nf + 3) / 4));
+        k_to_columns<<<grid, 256, 0, st>>>(t.data, t.logW, t.nf, c->N, c->d_colmajor + (size_t)t.f0 * stride, stride);
+        QG_LAUNCH_CHECK(c);
+    }
+    k_set_columns<<<(c->F + 255) / 256, 256, 0, st>>>(c->d_feat_rec, c->F, c->d_colmajor, stride);
+    QG_LAUNCH_CHECK(c);
+    return QGBDT_OK;
+}
+
 int qg_iota(qgbdt_ctx *c, cudaStream_t st) {
     long long blocks = (c->N + 255) / 256;
     if (blocks > (long long)c->sm_count * 16) blocks = (long long)c->sm_count * 16;

@@ -67,6 +67,7 @@ struct FeatRec {
     int32_t logW, byte;    // words per row (log2) of the tile, byte of the word
     int32_t cta0, parts;   // partial-histogram slots of the tile
     int32_t fl, pad;       // feature number inside the tile
+    const uint8_t *col8;   // the feature's column in the column-major copy (nullptr: there is none)
 };
 
 // One leaf of the tree being grown (device memory).  Its rows are entries [off, off + n) of the
@@ -88,6 +89,7 @@ struct GrowState {
     int32_t pick, feature, bin;      // leaf being split and its winning candidate
     int32_t logW, byte;              // tile width (log2 words per row) and byte of the split feature's word
     const uint32_t *col;             // that word in row 0 of the tile
+    const uint8_t *col8;             // the split feature's column in the column-major copy, or nullptr
     uint32_t off, n;                 // rows of the leaf being split
     int32_t buf;                     // their pair buffer
     uint32_t nl;                     // rows that go left (written by the scatter kernel)
@@ -145,6 +147,8 @@ struct qgbdt_ctx {
     GrowState *d_gs = nullptr;
     SplitRec *d_cand = nullptr;                 // [F][2] per-feature best candidates of the two children
     FeatRec *d_feat_rec = nullptr;              // [F] location of every feature
+    uint8_t *d_colmajor = nullptr;              // [F][col_stride] column-major copy of the bin codes (training only)
+    size_t col_stride = 0;
     double *d_leaf_gain = nullptr;              // [L] stored gain of every leaf's best split (-inf: none)
     void *grow_graph_exec = nullptr;            // cudaGraphExec_t: the split loop of one tree
     int64_t grow_graph_launches = 0;            // kernel launches it replays
@@ -192,6 +196,10 @@ static inline int qg_levels_h(int bits, int mode) { return mode == 0 ? (1 << bit
 // load.cu
 int qg_relayout(qgbdt_ctx *c, const uint8_t *d_bins, int layout, int64_t ld, cudaStream_t st);
 int qg_iota(qgbdt_ctx *c, cudaStream_t st);
+// Builds the column-major copy of the bin codes that the row partition of a split reads (one byte
+// per row instead of a DRAM granule per row) and records the columns in the feature records.
+// Without the memory for it the partition keeps reading the tiles.
+int qg_build_columns(qgbdt_ctx *c, cudaStream_t st);
 
 // quantize.cu
 int qg_gradients(qgbdt_ctx *c, const float *d_scores, const float *d_labels, float *d_g, float *d_h,

@@ -57,6 +57,7 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
     if (!c->d_ent1 && (rc = alloc_dev(c, &c->d_ent1, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_cand && (rc = alloc_dev(c, &c->d_cand, (size_t)2 * c->F, "candidate records")) != QGBDT_OK)
         return rc;
+    if ((rc = qg_build_columns(c, st)) != QGBDT_OK) return rc;
     if (!c->d_gs) {
         if ((rc = alloc_dev(c, &c->d_gs, 1, "grow state")) != QGBDT_OK) return rc;
         QG_CUDA(c, cudaMemsetAsync(c->d_gs, 0, sizeof(GrowState), st));

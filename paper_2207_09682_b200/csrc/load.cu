@@ -53,15 +53,26 @@ int qg_relayout(qgbdt_ctx *c, const uint8_t *d_bins, int layout, int64_t ld, cud
 
 namespace {
 
-// Block (x, a): rows 256 x .. 256 x + 255 of word a of a tile; four coalesced byte columns out.
+// A block moves 256 rows of a tile at a time: coalesced words in (through shared memory, rows
+// padded by one word against bank conflicts), 256 consecutive bytes of every column out.
 __global__ void __launch_bounds__(256) k_to_columns(const uint32_t *__restrict__ tile, int logW, int nf, long long N,
                                                     uint8_t *__restrict__ cols, size_t stride) {
-    const int a = blockIdx.y;
-    for (long long row = blockIdx.x * 256ll + threadIdx.x; row < N; row += (long long)gridDim.x * 256) {
-        const uint32_t w = tile[((size_t)row << logW) + a];
+    extern __shared__ uint32_t sw[];   // [256][W + 1]
+    const int W = 1 << logW;
+    for (long long row0 = blockIdx.x * 256ll; row0 < N; row0 += (long long)gridDim.x * 256) {
+        const int nrows = N - row0 < 256 ? (int)(N - row0) : 256;
+        const uint32_t *src = tile + ((size_t)row0 << logW);
+        for (int i = threadIdx.x; i < nrows * W; i += 256) sw[(i >> logW) * (W + 1) + (i & (W - 1))] = src[i];
+        __syncthreads();
+        if ((int)threadIdx.x < nrows) {
+            for (int a = 0; 4 * a < nf; ++a) {
+                const uint32_t w = sw[threadIdx.x * (W + 1) + a];
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (4 * a + k < nf) cols[(size_t)(4 * a + k) * stride + row] = (uint8_t)(w >> (8 * k));
+                for (int k = 0; k < 4; ++k)
+                    if (4 * a + k < nf) cols[(size_t)(4 * a + k) * stride + row0 + threadIdx.x] = (uint8_t)(w >> (8 * k));
+            }
+        }
+        __syncthreads();
     }
 }
 
@@ -84,9 +95,9 @@ int qg_build_columns(qgbdt_ctx *c, cudaStream_t st) {
     c->col_stride = stride;
     for (const TileDesc &t : c->tiles) {
         long long bx = (c->N + 255) / 256;
-        if (bx > 65535) bx = 65535;
-        const dim3 grid((unsigned)bx, (unsigned)((t.nf + 3) / 4));
-        k_to_columns<<<grid, 256, 0, st>>>(t.data, t.logW, t.nf, c->N, c->d_colmajor + (size_t)t.f0 * stride, stride);
+        if (bx > (long long)c->sm_count * 32) bx = (long long)c->sm_count * 32;
+        const size_t smem = (size_t)256 * ((1u << t.logW) + 1) * sizeof(uint32_t);
+        k_to_columns<<<(unsigned)bx, 256, smem, st>>>(t.data, t.logW, t.nf, c->N, c->d_colmajor + (size_t)t.f0 * stride, stride);
         QG_LAUNCH_CHECK(c);
     }
     k_set_columns<<<(c->F + 255) / 256, 256, 0, st>>>(c->d_feat_rec, c->F, c->d_colmajor, stride);

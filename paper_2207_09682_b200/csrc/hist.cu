@@ -18,14 +18,18 @@
 //    + hessian) is one more permute of the row's 16-bit code.
 //  * Rolling prefetch.  Every lane keeps U units of four rows in flight in registers and
 //    refills a slot as soon as it has been consumed.
-//  * Two-stage merge.  A CTA stores its partial histogram with plain coalesced stores; a small
-//    kernel sums the partials of each feature tile.  (64-bit global atomics from 148 CTAs on
-//    the same 7 k bins cost about as much as half of the whole build.)
+//  * Two-stage merge.  A CTA stores its partial histogram with plain coalesced stores; after a
+//    grid-wide barrier the CTAs of a tile share the sums of its entries (cooperative launch), or a
+//    small kernel does, or the kernel that finishes a split during tree growth.  (64-bit global
+//    atomics from 148 CTAs on the same 7 k bins cost about as much as half of the whole build.)
 //
-// Local bin width: B <= 5 uses one 32-bit word per bin, gradient sum in the high 16 bits
-// (signed), hessian sum in the low 16 bits; the CTA flushes before any column can have added
-// more rows than fit.  B >= 6 uses two 32-bit words per bin (32+32, a hessian plane and a gradient
-// plane) and two passes over the rows, each pass taking two of the four bytes of a word.
+// Local bin width: B <= 5 uses one 32-bit word per bin, gradient sum in the high bits (signed),
+// hessian sum in the low bits (16+16; 18+14 with a constant hessian, which only counts rows).
+// Before any column can have added more rows than fit, a CTA of a narrow tile flushes its local
+// histogram; a CTA of a wide tile moves only the words that are about to overflow.  B >= 6 uses
+// two 32-bit words per bin (32+32, a hessian plane and a gradient plane) and two passes over the
+// rows, each pass taking two of the four bytes of a word; in a stand-alone build the two passes
+// run side by side in pairs of CTAs that read the same rows at the same time.
 #include <cooperative_groups.h>
 
 #include "hist_cta.cuh"

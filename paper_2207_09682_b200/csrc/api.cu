@@ -202,7 +202,7 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     if ((rc = dev_alloc(c, &c->d_codes_nat, (size_t)n_rows * 2 + 16)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx, (size_t)n_rows)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx_tmp, (size_t)n_rows)) != QGBDT_OK) return rc;
-    if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8 + (size_t)c->sm_count * 32)) != QGBDT_OK) return rc;
+    if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8 + (size_t)c->sm_count * 40)) != QGBDT_OK) return rc;
     {
         std::vector<FeatRec> fr((size_t)n_features);
         for (const TileDesc &t : c->tiles)

@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
     const uint32_t nw = (n + 31) >> 5;
     uint32_t w0, w1, active;
     warp_range(nw, gw, (uint32_t)a.n_count, w0, w1, active);
-    if (gw >= active) return;
+    if (blockIdx.x * PART_WARPS >= active) return;   // no warp of this block has work
     const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
     uint32_t lefts = 0;
     for (uint32_t w = w0; w < w1; w += 4) {
@@ -114,7 +114,20 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
             }
         }
     }
-    if (lane == 0) a.counts[gw] = lefts;
+    // left rows of every warp range and of every block's ranges (the scatter kernel adds up the
+    // blocks before its own and the warps before it inside its block)
+    __shared__ uint32_t block_lefts[PART_WARPS];
+    if (lane == 0) {
+        a.counts[gw] = lefts;
+        block_lefts[threadIdx.x >> 5] = lefts;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = 0;
+#pragma unroll
+        for (int v = 0; v < PART_WARPS; ++v) t += block_lefts[v];
+        a.counts[a.n_count + blockIdx.x] = t;
+    }
 }
 
 __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
@@ -128,20 +141,27 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
     uint32_t w0, w1, active;
     warp_range(nw, gw, (uint32_t)a.n_count, w0, w1, active);
     if (gw >= active && gw != 0) return;
-    // left rows before this warp's range, and in the whole leaf
+    // left rows before this warp's range, and in the whole leaf: the totals of the blocks, and
+    // the warps of this block before this one
     uint32_t before = 0, total = 0;
-    for (uint32_t j0 = 0; j0 < active; j0 += 256) {   // eight independent loads per lane in flight
+    const uint32_t active_blocks = (active + PART_WARPS - 1) / PART_WARPS;
+    const uint32_t *block_counts = a.counts + a.n_count;
+    for (uint32_t j0 = 0; j0 < active_blocks; j0 += 256) {   // eight independent loads per lane in flight
         uint32_t v[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const uint32_t j = j0 + 32 * k + lane;
-            v[k] = j < active ? a.counts[j] : 0u;
+            v[k] = j < active_blocks ? block_counts[j] : 0u;
         }
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             total += v[k];
-            if (j0 + 32 * k + lane < gw) before += v[k];
+            if (j0 + 32 * k + lane < blockIdx.x) before += v[k];
         }
+    }
+    {
+        const uint32_t j = blockIdx.x * PART_WARPS + lane;
+        if (lane < PART_WARPS && j < gw) before += a.counts[j];
     }
     for (int o = 16; o > 0; o >>= 1) {
         before += __shfl_xor_sync(0xffffffffu, before, o);

@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (profiles/launch_list_large_10p5Mx28.md): 3.37 GB over the 255 builds of one tree.  Valid only for
 # the kernel sources the capture was taken with.
 HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 13.21e6,
-                "sources_sha1": "cb059626cedf2b060756629b2e35ae705afbe885"}
+                "sources_sha1": "9a9a10cefa66cbe6e57559fefa09715198166193"}
 
 
 def hist_traffic(workload, rows):

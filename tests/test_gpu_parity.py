@@ -367,6 +367,14 @@ def test_training_matches_oracle(name, rows, over):
     assert (got.view(np.uint32) == ref_scores.view(np.uint32)).all()
 
 
+def test_training_without_the_column_copy(monkeypatch):
+    # the row partition reads the split feature from the tiles when there is no column-major copy
+    # (its allocation failed, or it was switched off): same trees
+    monkeypatch.setenv("QGBDT_NO_COLUMN_COPY", "1")
+    for name, rows, over in (TRAIN_CASES[1], TRAIN_CASES[3]):
+        test_training_matches_oracle(name, rows, over)
+
+
 def test_training_resumes_and_host_variant_agrees():
     wl = synth.tiny(device="cpu", rows=15_000)
     kw = dict(wl.params, seed=3, num_trees=4)

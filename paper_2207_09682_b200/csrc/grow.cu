@@ -14,7 +14,6 @@ namespace {
 
 constexpr int PART_THREADS = 256;
 constexpr int PART_WARPS = PART_THREADS / 32;
-constexpr int FIN_WARPS = 8;
 constexpr uint32_t MIN_ROWS_PER_CTA = 1024;   // same rule as the histogram kernel
 
 __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
@@ -225,8 +224,11 @@ __device__ inline SplitRec shfl_xor_rec(const SplitRec &r, int o) {
 
 // ROOT: scans the root histogram (pool slot 0).  Otherwise: completes the split recorded in the
 // grow state.  One block per feature.
-template <bool ROOT>
-__global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
+// BPT bins per thread: 1 (256 threads) or 2 (128 threads: with thousands of features twice as many
+// blocks are resident, and the grid fits the SMs in one wave).
+template <bool ROOT, int BPT>
+__global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
+    constexpr int FIN_WARPS = 8 / BPT;
     GrowState *gs = a.gs;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int f = blockIdx.x;   // one block per feature
@@ -253,7 +255,7 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     }
     // ---- phase A: one thread per bin: the smaller child's sum over the partial histograms, the
     //      larger child's bin by subtraction
-    __shared__ SplitRec sm[2][FIN_WARPS * 32];
+    __shared__ SplitRec sm[2][FIN_WARPS];
     __shared__ bool is_last;
     // interval lengths of Eq. 5 from the maxima stored by the quantizer
     const double dg = __ddiv_rn((double)__uint_as_float(gmax_bits), (double)pS.kg);
@@ -266,61 +268,142 @@ __global__ void __launch_bounds__(FIN_WARPS * 32) k_grow_finish(GrowArgs a) {
     const unsigned long long *part = a.partial + (size_t)fr.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
     unsigned long long *S = a.pool + (ROOT ? 0 : (size_t)n_leaves * hw) + (size_t)f * a.nb;
     unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)parent_slot * hw + (size_t)f * a.nb;
-    // n_bins <= 256: thread b owns bin b
-    const int b = (int)threadIdx.x;
-    unsigned long long s = 0, l = 0;
-    if (b < a.nb) {
-        if (ROOT) {
-            s = S[b];
-        } else {
-            if (P > 1) {
-                const unsigned long long *q = part + (size_t)b * W;
-                for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
-                    unsigned long long x[16];
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) s += x[k];
-                }
-                S[b] = s;
-            } else {
-                s = S[b];
-            }
-            l = Pp[b] - s;   // no field borrows: every child sum is at most the parent's
-            Pp[b] = l;
-        }
-    }
-    // ---- phase B: prefix sums over the bins by all eight warps (warp scan, then the warp totals),
-    //      every thread evaluates the threshold at its own bin for both children
     __shared__ long long wtot[4][FIN_WARPS];
-    const bool in = b < a.nb - 1;   // thresholds 0 .. nb-2
-    long long v[4];
-    v[0] = in ? (long long)(int)(s >> 32) : 0;
-    v[1] = in ? (long long)(unsigned int)(s & 0xFFFFFFFFull) : 0;
-    v[2] = in ? (long long)(int)(l >> 32) : 0;
-    v[3] = in ? (long long)(unsigned int)(l & 0xFFFFFFFFull) : 0;
-#pragma unroll
-    for (int c = 0; c < (ROOT ? 2 : 4); ++c) {
-        for (int o = 1; o < 32; o <<= 1) {
-            const long long u = __shfl_up_sync(0xffffffffu, v[c], o);
-            if (lane >= o) v[c] += u;
-        }
-        if (lane == 31) wtot[c][warp] = v[c];
-    }
-    __syncthreads();
-#pragma unroll
-    for (int c = 0; c < (ROOT ? 2 : 4); ++c)
-        for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
     SplitRec rS = qg_invalid_rec(), rL = qg_invalid_rec();
     rS.feature = f;
     rL.feature = f;
-    if (in) {
-        double gain;
-        if (qg_eval_candidate(v[0], v[1], pS, dg, dh, tpS, gain)) {
-            rS.valid = 1; rS.gain = gain; rS.bin = b; rS.gl = v[0]; rS.hl = v[1];
+    if (BPT == 1) {
+        // n_bins <= 256: thread b owns bin b
+        const int b = (int)threadIdx.x;
+        unsigned long long s = 0, l = 0;
+        if (b < a.nb) {
+            if (ROOT) {
+                s = S[b];
+            } else {
+                if (P > 1) {
+                    const unsigned long long *q = part + (size_t)b * W;
+                    for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
+                        unsigned long long x[16];
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) s += x[k];
+                    }
+                    S[b] = s;
+                } else {
+                    s = S[b];
+                }
+                l = Pp[b] - s;   // no field borrows: every child sum is at most the parent's
+                Pp[b] = l;
+            }
         }
-        if (!ROOT && qg_eval_candidate(v[2], v[3], pL, dg, dh, tpL, gain)) {
-            rL.valid = 1; rL.gain = gain; rL.bin = b; rL.gl = v[2]; rL.hl = v[3];
+        // ---- phase B: prefix sums over the bins by all eight warps (warp scan, then the warp totals),
+        //      every thread evaluates the threshold at its own bin for both children
+        const bool in = b < a.nb - 1;   // thresholds 0 .. nb-2
+        long long v[4];
+        v[0] = in ? (long long)(int)(s >> 32) : 0;
+        v[1] = in ? (long long)(unsigned int)(s & 0xFFFFFFFFull) : 0;
+        v[2] = in ? (long long)(int)(l >> 32) : 0;
+        v[3] = in ? (long long)(unsigned int)(l & 0xFFFFFFFFull) : 0;
+#pragma unroll
+        for (int c = 0; c < (ROOT ? 2 : 4); ++c) {
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long u = __shfl_up_sync(0xffffffffu, v[c], o);
+                if (lane >= o) v[c] += u;
+            }
+            if (lane == 31) wtot[c][warp] = v[c];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int c = 0; c < (ROOT ? 2 : 4); ++c)
+            for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
+        if (in) {
+            double gain;
+            if (qg_eval_candidate(v[0], v[1], pS, dg, dh, tpS, gain)) {
+                rS.valid = 1; rS.gain = gain; rS.bin = b; rS.gl = v[0]; rS.hl = v[1];
+            }
+            if (!ROOT && qg_eval_candidate(v[2], v[3], pL, dg, dh, tpL, gain)) {
+                rL.valid = 1; rL.gain = gain; rL.bin = b; rL.gl = v[2]; rL.hl = v[3];
+            }
+        }
+    } else {
+        // n_bins <= 256: thread t owns bins BPT t .. BPT t + BPT - 1
+        unsigned long long sv[BPT], lv[BPT];
+        {
+            unsigned long long pv[BPT];
+#pragma unroll
+            for (int j = 0; j < BPT; ++j) {
+                const int b = (int)threadIdx.x * BPT + j;
+                sv[j] = 0; lv[j] = 0; pv[j] = 0;
+                if (b < a.nb) {
+                    if (!ROOT) pv[j] = Pp[b];
+                    if (!ROOT && P > 1) {
+                        const unsigned long long *q = part + (size_t)b * W;
+                        for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
+                            unsigned long long x[16];
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) sv[j] += x[k];
+                        }
+                    } else {
+                        sv[j] = S[b];
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < BPT; ++j) {
+                const int b = (int)threadIdx.x * BPT + j;
+                if (!ROOT && b < a.nb) {
+                    if (P > 1) S[b] = sv[j];
+                    lv[j] = pv[j] - sv[j];   // no field borrows: every child sum is at most the parent's
+                    Pp[b] = lv[j];
+                }
+            }
+        }
+        // ---- phase B: prefix sums over the bins by all warps (the thread's own bins, a warp scan of
+        //      the threads' totals, then the warp totals); every thread evaluates the thresholds at its
+        //      own bins for both children
+        long long x[BPT][4], v[4] = {0, 0, 0, 0};   // per bin; v: inclusive sum up to the thread's last bin
+#pragma unroll
+        for (int j = 0; j < BPT; ++j) {
+            const bool in = (int)threadIdx.x * BPT + j < a.nb - 1;   // thresholds 0 .. nb-2
+            x[j][0] = in ? (long long)(int)(sv[j] >> 32) : 0;
+            x[j][1] = in ? (long long)(unsigned int)(sv[j] & 0xFFFFFFFFull) : 0;
+            x[j][2] = in ? (long long)(int)(lv[j] >> 32) : 0;
+            x[j][3] = in ? (long long)(unsigned int)(lv[j] & 0xFFFFFFFFull) : 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) v[c] += x[j][c];
+        }
+#pragma unroll
+        for (int c = 0; c < (ROOT ? 2 : 4); ++c) {
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long u = __shfl_up_sync(0xffffffffu, v[c], o);
+                if (lane >= o) v[c] += u;
+            }
+            if (lane == 31) wtot[c][warp] = v[c];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int c = 0; c < (ROOT ? 2 : 4); ++c)
+            for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
+        // thresholds from the thread's last bin down (the lower bin wins on equal gain)
+#pragma unroll
+        for (int j = BPT - 1; j >= 0; --j) {
+            const int b = (int)threadIdx.x * BPT + j;
+            if (b < a.nb - 1) {
+                double gain;
+                if (qg_eval_candidate(v[0], v[1], pS, dg, dh, tpS, gain) &&
+                    qg_better(true, gain, b, rS.valid != 0, rS.gain, rS.bin)) {
+                    rS.valid = 1; rS.gain = gain; rS.bin = b; rS.gl = v[0]; rS.hl = v[1];
+                }
+                if (!ROOT && qg_eval_candidate(v[2], v[3], pL, dg, dh, tpL, gain) &&
+                    qg_better(true, gain, b, rL.valid != 0, rL.gain, rL.bin)) {
+                    rL.valid = 1; rL.gain = gain; rL.bin = b; rL.gl = v[2]; rL.hl = v[3];
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) v[c] -= x[j][c];
         }
     }
     // best threshold of the feature: largest gain, lowest bin on equal gain
@@ -563,7 +646,8 @@ int enqueue_splits(qgbdt_ctx *c, const GrowArgs &a, int part_blocks, cudaStream_
         QG_LAUNCH_CHECK(c);
         const int rc = qg_hist_grow(c, st);
         if (rc != QGBDT_OK) return rc;
-        k_grow_finish<false><<<fin_blocks, FIN_WARPS * 32, 0, st>>>(a);
+        if (c->F > c->sm_count * 8) k_grow_finish<false, 2><<<fin_blocks, 128, 0, st>>>(a);
+        else k_grow_finish<false, 1><<<fin_blocks, 256, 0, st>>>(a);
         QG_LAUNCH_CHECK(c);
     }
     return QGBDT_OK;
@@ -627,7 +711,7 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     QG_LAUNCH_CHECK(c);
     int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
     if (rc != QGBDT_OK) return rc;
-    k_grow_finish<true><<<(unsigned)c->F, FIN_WARPS * 32, 0, st>>>(a);
+    k_grow_finish<true, 1><<<(unsigned)c->F, 256, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     if (c->prm.num_leaves < 2) return QGBDT_OK;
     if (c->profile_hist) return enqueue_splits(c, a, part_blocks, st);   // event records around every build

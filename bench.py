@@ -34,14 +34,14 @@ FALLBACK_HBM_GBS = 6650.0
 # (profiles/launch_list_large_10p5Mx28.md): 3.37 GB over the 255 builds of one tree.  Valid only for
 # the kernel sources the capture was taken with.
 HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 13.21e6,
-                "sources_sha1": "9a9a10cefa66cbe6e57559fefa09715198166193"}
+                "sources_sha1": "ebe4072b9c79c96d2d555260a0b495f28b344e13"}
 
 
 def hist_traffic(workload, rows):
     import hashlib
     h = hashlib.sha1()
     try:
-        for f in ("hist_cta.cuh", "hist.cu", "grow.cu"):
+        for f in ("hist_cta.cuh", "hist.cu"):   # the sources of the histogram kernels
             h.update(open(os.path.join(ROOT, "paper_2207_09682_b200", "csrc", f), "rb").read())
     except OSError:
         return None

@@ -166,7 +166,12 @@ int qgbdt_refit_leaves(qgbdt_ctx *ctx, const float *d_g, const float *d_h, doubl
  * (gradients, quantization, leaf-wise growth with integer histograms and histogram
  * subtraction, refit, score update).  d_labels [n_rows]; d_scores [n_rows] holds the
  * current predictions on entry and the updated ones on return.  `model` (host) receives
- * the trees, tree k of this call in slot k.  Synchronises. */
+ * the trees, tree k of this call in slot k.  Synchronises.
+ * Memory: the first call after a load allocates the training workspaces, among them a
+ * column-major copy of the bin codes (n_rows * n_features bytes) that the row partition
+ * of a split reads; if that allocation fails, or the environment variable
+ * QGBDT_NO_COLUMN_COPY is 1, the partition reads the tiled matrix instead (same
+ * results, more memory traffic). */
 int qgbdt_train(qgbdt_ctx *ctx, const float *d_labels, float *d_scores, uint32_t first_tree,
                 int32_t num_trees, qgbdt_model *model, void *stream);
 /* Same with labels and scores in HOST memory; both copies are part of the call. */

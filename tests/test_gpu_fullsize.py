@@ -79,6 +79,8 @@ SWEEP_POINTS = [
     (1_000_000, 1000, 255, 8, 16),
     (4_000_000, 28, 64, 5, None),
     (16_000_000, 1000, 255, 3, 8),
+    (2_000_000, 28, 255, 8, None),      # 32+32 local bins: 74 pairs of CTAs, one pass each
+    (3_000_001, 136, 64, 7, 20),        # the same with two tile widths and a ragged tail
 ]
 
 

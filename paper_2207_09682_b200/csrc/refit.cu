@@ -111,6 +111,9 @@ __global__ void k_leaf_values(const long long *__restrict__ sums, const uint32_t
     }
 }
 
+// Dynamic shared memory: [n_leaves] offsets, [n_leaves] values, [n_leaves] pair buffers, so that
+// a row costs a search in shared memory and two global accesses (its pair, its score).  Four
+// rows per thread are in flight.
 __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *__restrict__ idx,
                                                                 const uint2 *__restrict__ ent0,
                                                                 const uint2 *__restrict__ ent1, uint32_t n,
@@ -121,12 +124,35 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *
     extern __shared__ uint32_t offs[];
     const bool grown = gs != nullptr;
     if (grown) n_leaves = gs->n_leaves;
-    for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) offs[i] = table[i];
+    float *vals = reinterpret_cast<float *>(offs + n_leaves);
+    int *bufs = reinterpret_cast<int *>(offs + 2 * n_leaves);
+    for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) {
+        offs[i] = table[i];
+        vals[i] = values[table[n_leaves + i]];
+        bufs[i] = grown ? (int)table[2 * n_leaves + i] : 0;
+    }
     __syncthreads();
-    for (uint32_t p = blockIdx.x * REFIT_THREADS + threadIdx.x; p < n; p += gridDim.x * REFIT_THREADS) {
-        const int s = slot_of(offs, n_leaves, p);
-        const uint32_t row = leaf_row(idx, ent0, ent1, table, n_leaves, grown, s, p);
-        scores[row] = __fadd_rn(scores[row], values[table[n_leaves + s]]);
+    const uint32_t stride = gridDim.x * REFIT_THREADS;
+    for (uint32_t p0 = blockIdx.x * REFIT_THREADS + threadIdx.x; p0 < n; p0 += 4 * stride) {
+        uint32_t row[4];
+        float add[4], old[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t p = p0 + k * stride;
+            row[k] = 0xFFFFFFFFu;
+            add[k] = 0.f;
+            if (p < n) {
+                const int sl = slot_of(offs, n_leaves, p);
+                add[k] = vals[sl];
+                if (!grown) row[k] = idx[p];
+                else row[k] = bufs[sl] < 0 ? p : (bufs[sl] ? ent1[p].x : ent0[p].x);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) old[k] = row[k] != 0xFFFFFFFFu ? scores[row[k]] : 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (row[k] != 0xFFFFFFFFu) scores[row[k]] = __fadd_rn(old[k], add[k]);
     }
 }
 
@@ -199,7 +225,7 @@ int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st) {
     const int L = c->n_leaves;
     unsigned blocks = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
     if (blocks > (unsigned)c->sm_count * 16) blocks = (unsigned)c->sm_count * 16;
-    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, nullptr, nullptr, (uint32_t)c->N,
+    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * 3 * L, st>>>(c->d_idx, nullptr, nullptr, (uint32_t)c->N,
                                                                        c->d_leaf_table, L, nullptr, c->d_leaf_value,
                                                                        d_scores);
     QG_LAUNCH_CHECK(c);
@@ -224,7 +250,7 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
     QG_LAUNCH_CHECK(c);
     unsigned ab = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
     if (ab > (unsigned)c->sm_count * 16) ab = (unsigned)c->sm_count * 16;
-    k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
+    k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * 3 * L, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
                                                                    c->d_leaf_table, L, c->d_gs,
                                                                    c->d_m_leaf_value + (size_t)tree_slot * L, d_scores);
     QG_LAUNCH_CHECK(c);

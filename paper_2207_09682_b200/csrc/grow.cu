@@ -282,12 +282,12 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
             } else {
                 if (P > 1) {
                     const unsigned long long *q = part + (size_t)b * W;
-                    for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
-                        unsigned long long x[16];
+                    for (uint32_t i0 = 0; i0 < P; i0 += 8) {   // 8 independent loads in flight
+                        unsigned long long x[8];
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
+                        for (int k = 0; k < 8; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) s += x[k];
+                        for (int k = 0; k < 8; ++k) s += x[k];
                     }
                     S[b] = s;
                 } else {

@@ -13,6 +13,17 @@ constexpr uint32_t MIN_ROWS_PER_CTA = 1024;
 // Wide tiles with at least this many bins look for hot words instead of flushing everything (a
 // look comes twice as often as a flush would; with few bins a flush is cheap and wins).
 constexpr int SELECTIVE_MIN_BINS = 128;
+// A word is hot from 2^-SELECTIVE_T of a field's range on: an eighth in stand-alone builds (fewer
+// looks); a half in the builds of tree growth, whose CTAs rarely see enough rows for a look and
+// whose kernel came out 4 % slower per tree of the 2000-feature workload with the other test
+// compiled in.
+template <int LIST> struct SelectiveT { static constexpr int value = LIST == 2 ? 1 : 3; };
+
+template <int T>
+__device__ __forceinline__ uint32_t hot_bits(uint32_t x, uint32_t gm, uint32_t hm, int lsh) {
+    if (T == 1) return ((x + 0x40000000u) | (x << lsh)) & 0x80000000u;   // the same test in fewer operations
+    return ((x ^ (x << 1)) & gm) | (x & hm);
+}
 // Units of four rows in flight per lane.  A CTA of 512 threads (the tree-growing kernel) has twice
 // the registers per thread and keeps more in flight per lane to make up for the fewer warps.
 template <int NT> struct Units { static constexpr int root = NT >= 1024 ? 4 : 6, list = NT >= 1024 ? 2 : 4; };
@@ -163,20 +174,24 @@ __device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, 
 }
 
 // Wide tiles (one or two row slots per column: a flush moves up to 32 k bins through global
-// memory) avoid most flushes: a column only adds half of `flush_rows` rows at a time, after which
-// the CTA looks at every local word.  One whose hessian field has reached half its range, or
-// whose gradient field has left the middle half of its range, is "hot": its sums move to the
+// memory) avoid most flushes: a column only adds 7/8 of `flush_rows` rows at a time, after which
+// the CTA looks at every local word.  One whose hessian field has reached an eighth of its range,
+// or whose gradient field has left the middle eighth of its range, is "hot": its sums move to the
 // output (a reduction on the word's 64-bit bin) and the word restarts from zero; all other words
-// can take another half of `flush_rows` rows as they are.  With bin codes spread over many bins
+// can take another 7/8 of `flush_rows` rows as they are.  With bin codes spread over many bins
 // almost no word is hot.  Before the first flush the output holds nothing that could be added
 // to: then a hot word asks for a full flush (return value, CTA-uniform).  Callers synchronise
 // before the call; the call ends with a barrier.
-template <int NT, int MODE, int LOGW_T>
+template <int NT, int MODE, int LOGW_T, int SELECTIVE_T>
 __device__ __forceinline__ bool relieve_local(int *hp, const TileDesc &td, const int logW_rt, int nb, int shift,
                                               const Out &out) {
     static_assert(MODE != 1, "32+32 local bins never overflow");
     const int logW = LOGW_T >= 0 ? LOGW_T : logW_rt;
     const int logR = 5 - logW, W = 1 << logW;
+    // hot: any of the top SELECTIVE_T bits of the hessian field set, or the top SELECTIVE_T + 1 bits
+    // of the word (the gradient field's sign and the bits below it) not all equal
+    const uint32_t hm = ((1u << SELECTIVE_T) - 1u) << (shift - SELECTIVE_T);
+    const uint32_t gm = ~0u << (32 - SELECTIVE_T);
     const int lsh = 32 - shift;
     const int hmask = (1 << shift) - 1;
     bool want_full = false;
@@ -186,19 +201,16 @@ __device__ __forceinline__ bool relieve_local(int *hp, const TileDesc &td, const
             int4 *p = reinterpret_cast<int4 *>(hp + half * 16384) + i;
             const int4 x = *p;
             // bit 31: gradient field outside [-2^(30-shift), 2^(30-shift)), or top bit of the hessian field set
-            const uint32_t m = (((uint32_t)x.x + 0x40000000u) | ((uint32_t)x.x << lsh)) |
-                               (((uint32_t)x.y + 0x40000000u) | ((uint32_t)x.y << lsh)) |
-                               (((uint32_t)x.z + 0x40000000u) | ((uint32_t)x.z << lsh)) |
-                               (((uint32_t)x.w + 0x40000000u) | ((uint32_t)x.w << lsh));
-            if (m & 0x80000000u) {
+            const uint32_t m = hot_bits<SELECTIVE_T>((uint32_t)x.x, gm, hm, lsh) | hot_bits<SELECTIVE_T>((uint32_t)x.y, gm, hm, lsh) |
+                               hot_bits<SELECTIVE_T>((uint32_t)x.z, gm, hm, lsh) | hot_bits<SELECTIVE_T>((uint32_t)x.w, gm, hm, lsh);
+            if (m) {
                 if (out.first) {
                     want_full = true;
                 } else {
                     int xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint32_t hot = ((uint32_t)xs[j] + 0x40000000u) | ((uint32_t)xs[j] << lsh);
-                        if (hot & 0x80000000u) {
+                        if (hot_bits<SELECTIVE_T>((uint32_t)xs[j], gm, hm, lsh)) {
                             const int w = i * 4 + j;                      // word inside this half
                             const int bin = w >> 6, k = half * 2 + ((w >> 5) & 1), a = (w & 31) >> logR;
                             const int fl = 4 * a + k;
@@ -324,12 +336,15 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     //      flight stay in flight across that meeting.
     constexpr int U = LIST ? Units<NT>::list : Units<NT>::root;
     constexpr int NWARPS = NT / 32;
+    constexpr int SELECTIVE_T = SelectiveT<LIST>::value;
     const bool selective = logR <= 1 && a.nb >= SELECTIVE_MIN_BINS;   // wide tiles: look for hot words instead of flushing everything
     const uint32_t nq = q1 > (uint32_t)warp ? (q1 - warp + NWARPS - 1) / NWARPS : 0;   // this warp's units
     const uint32_t groups = ((q1 + NWARPS - 1) / NWARPS + U - 1) / U;                  // of warp 0: the same in every warp
     uint32_t kg = 0xFFFFFFFFu;                                                         // groups between two meetings
     if (MODE != 1) {
-        const uint32_t limit = selective ? a.flush_rows >> 1 : a.flush_rows;
+        // after a look every field has at least 1 - 2^-SELECTIVE_T of its range left
+        const uint32_t limit = !selective ? a.flush_rows
+                               : (SELECTIVE_T == 1 ? a.flush_rows >> 1 : a.flush_rows - (a.flush_rows >> SELECTIVE_T) - 1);
         kg = (limit > col_rows ? limit - col_rows : 0) / (4u * U * NWARPS);
         if (kg == 0) {   // the host picks wide local bins before the limit gets this small
             if (threadIdx.x == 0) atomicExch(&a.state->kernel_error, 1);
@@ -341,7 +356,7 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
     if (MODE != 1 && since == kg && (grp) < groups) {                                                         \
         since = 0;                                                                                            \
         __syncthreads();                                                                                      \
-        if (!selective || relieve_local<NT, MODE == 1 ? 0 : MODE, LOGW_T>(hp, td, logW, a.nb, shift, out)) { \
+        if (!selective || relieve_local<NT, MODE == 1 ? 0 : MODE, LOGW_T, SELECTIVE_T>(hp, td, logW, a.nb, shift, out)) { \
             flush_local<NT, MODE>(hp, td, logW, a.nb, pass, shift, out);                                      \
             __syncthreads();                                                                                  \
         }                                                                                                     \

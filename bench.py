@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (profiles/launch_list_large_10p5Mx28.md): 3.37 GB over the 255 builds of one tree.  Valid only for
 # the kernel sources the capture was taken with.
 HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 13.21e6,
-                "sources_sha1": "ebe4072b9c79c96d2d555260a0b495f28b344e13"}
+                "sources_sha1": "331e037039ff3f9fab93e421716983d78c5b675e"}
 
 
 def hist_traffic(workload, rows):

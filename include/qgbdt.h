@@ -145,14 +145,17 @@ int qgbdt_subtract_histograms(qgbdt_ctx *ctx, const qgbdt_bin *d_parent, const q
 int qgbdt_find_best_split(qgbdt_ctx *ctx, const qgbdt_bin *d_hist, int64_t G, int64_t H, int64_t n_rows,
                           qgbdt_split *h_out, void *stream);
 
-/* Stable partition of the rows of `leaf` by (feature, bin): rows with bin code <= bin stay
- * in `leaf`, the others form leaf *right_leaf; relative order is kept.  Synchronises. */
+/* The index sets I_s of Sec. 3: a split of leaf s by (feature, bin) divides I_s into the rows
+ * with bin code <= bin, which stay in `leaf`, and the others, which form leaf *right_leaf
+ * (a stable partition: relative order is kept on both sides).  Any (feature, bin) in range is
+ * accepted, also one that leaves a side empty.  Synchronises. */
 int qgbdt_split_leaf(qgbdt_ctx *ctx, int32_t leaf, int32_t feature, int32_t bin, int32_t *right_leaf,
                      int64_t *n_left, int64_t *n_right, void *stream);
-/* Borrowed view of a leaf's row list (device memory inside the context; valid until the
- * next split or reset). */
+/* Borrowed view of I_s (Sec. 3), the row list of a leaf: device memory inside the context,
+ * valid until the next split or reset. */
 int qgbdt_get_leaf_rows(qgbdt_ctx *ctx, int32_t leaf, const uint32_t **d_rows, int64_t *n);
-/* Back to the single root leaf (all rows, ascending).  Asynchronous. */
+/* Back to the state before any split (Sec. 3: the tree starts from a single root leaf whose
+ * index set is all rows, ascending).  Asynchronous. */
 int qgbdt_reset_leaves(qgbdt_ctx *ctx, void *stream);
 
 /* Eq. 3 with the ORIGINAL gradients (leaf-value refitting, Sec. 4.2): for every current
@@ -162,6 +165,11 @@ int qgbdt_reset_leaves(qgbdt_ctx *ctx, void *stream);
 int qgbdt_refit_leaves(qgbdt_ctx *ctx, const float *d_g, const float *d_h, double *h_w, float *h_value,
                        void *stream);
 
+/* Fig. 1, last step of an iteration: adds to d_scores [n_rows] the output of the leaf every row
+ * is in (the values of the last qgbdt_refit_leaves, which must have run for the current leaves:
+ * QGBDT_ERR_STATE otherwise).  Asynchronous. */
+int qgbdt_apply_leaf_values(qgbdt_ctx *ctx, float *d_scores, void *stream);
+
 /* Fig. 1 workflow: trains boosting iterations first_tree .. first_tree + num_trees - 1
  * (gradients, quantization, leaf-wise growth with integer histograms and histogram
  * subtraction, refit, score update).  d_labels [n_rows]; d_scores [n_rows] holds the
@@ -169,14 +177,28 @@ int qgbdt_refit_leaves(qgbdt_ctx *ctx, const float *d_g, const float *d_h, doubl
  * the trees, tree k of this call in slot k.  Synchronises.
  * Memory: the first call after a load allocates the training workspaces, among them a
  * column-major copy of the bin codes (n_rows * n_features bytes) that the row partition
- * of a split reads; if that allocation fails, or the environment variable
- * QGBDT_NO_COLUMN_COPY is 1, the partition reads the tiled matrix instead (same
- * results, more memory traffic). */
+ * of a split reads; with option QGBDT_OPT_COLUMN_COPY set to 0, or if that allocation
+ * fails, the partition reads the tiled matrix instead (same results, more memory
+ * traffic); qgbdt_get_info(QGBDT_INFO_COLUMN_COPY) tells which path the last call took.
+ * Gradients out of domain (QGBDT_ERR_VALUE) are reported when the call returns; the trees
+ * from the offending iteration on are not grown (one leaf each). */
 int qgbdt_train(qgbdt_ctx *ctx, const float *d_labels, float *d_scores, uint32_t first_tree,
                 int32_t num_trees, qgbdt_model *model, void *stream);
 /* Same with labels and scores in HOST memory; both copies are part of the call. */
 int qgbdt_train_host(qgbdt_ctx *ctx, const float *h_labels, float *h_scores, uint32_t first_tree,
                      int32_t num_trees, qgbdt_model *model, void *stream);
+
+/* Options of a context (no counterpart in the paper).  Set them before qgbdt_load_binned /
+ * qgbdt_train; unknown options and values out of range give QGBDT_ERR_ARG.
+ *   QGBDT_OPT_COLUMN_COPY  1 (default): qgbdt_train keeps a column-major copy of the bin codes for
+ *                          the row partition; 0: never (saves n_rows * n_features bytes). */
+#define QGBDT_OPT_COLUMN_COPY 1
+int qgbdt_set_option(qgbdt_ctx *ctx, int32_t option, int64_t value);
+/* What the context is doing (host scalars, no synchronisation):
+ *   QGBDT_INFO_COLUMN_COPY  1 when the training workspaces hold the column-major copy (the row
+ *                           partition reads columns), 0 when they do not (it reads the tiles). */
+#define QGBDT_INFO_COLUMN_COPY 1
+int qgbdt_get_info(const qgbdt_ctx *ctx, int32_t what, int64_t *value);
 
 /* Counters of the work done by qgbdt_train since the context was created:
  * kernel launches, histogram builds, and rows x features accumulated by them. */
@@ -201,12 +223,14 @@ int qgbdt_get_histogram_profile(qgbdt_ctx *ctx, double *total_ms, int64_t *total
  *           (the optional outputs of qgbdt_quantize_gradients)
  *   d_rows  [n] row list, or NULL for all rows (then n must equal n_rows)
  *   d_hist  [n_features][n_bins], overwritten
- *   d_status  optional device word the caller clears: set to 1 when a row index or a bin code
- *           was out of range (such entries are skipped)
+ *   d_status  optional device word the caller clears: set to 1 when a row index (>= n_rows), a bin
+ *           code (>= n_bins) or a gradient code (-128) was out of range (such entries are skipped)
  * All pointers are device pointers owned by the caller.  The per-CTA partial histograms live in
  * a fixed 4 MiB array inside the library image (every GPU that loads the library holds it until
  * the process ends), so n_features * n_bins may be at most 16384; larger problems are refused
- * with QGBDT_ERR_ARG and need a context.  The call makes no cudaMalloc / cudaFree and calls no
+ * with QGBDT_ERR_ARG and need a context.  The call knows no bit width, so it bounds the sums by the
+ * widest codes: n (entries of the list, or n_rows) may be at most 16 843 009 (n * 255 must fit the
+ * 32-bit hessian field); more gives QGBDT_ERR_OVERFLOW.  The call makes no cudaMalloc / cudaFree and calls no
  * allocating routine.  The first call on a device looks up the array's device address; make
  * that first call outside any stream capture.  All calls share the one array, which keeps the
  * previous call's sums (each call clears what it uses): two calls whose kernels overlap on the

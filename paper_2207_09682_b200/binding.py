@@ -15,13 +15,15 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqgbdt.so")
 
 OK, ERR_ARG, ERR_STATE, ERR_OVERFLOW, ERR_CUDA, ERR_ALLOC, ERR_VALUE = 0, -1, -2, -3, -4, -5, -6
+OPT_COLUMN_COPY = 1
+INFO_COLUMN_COPY = 1
 
 EXPORTS = [
     "qgbdt_create", "qgbdt_destroy", "qgbdt_last_error", "qgbdt_load_binned", "qgbdt_load_binned_host",
     "qgbdt_compute_gradients", "qgbdt_quantize_gradients", "qgbdt_build_histograms",
     "qgbdt_build_histograms_rows", "qgbdt_subtract_histograms", "qgbdt_find_best_split", "qgbdt_split_leaf",
-    "qgbdt_get_leaf_rows", "qgbdt_reset_leaves", "qgbdt_refit_leaves", "qgbdt_train", "qgbdt_train_host",
-    "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile",
+    "qgbdt_get_leaf_rows", "qgbdt_reset_leaves", "qgbdt_refit_leaves", "qgbdt_apply_leaf_values", "qgbdt_train", "qgbdt_train_host",
+    "qgbdt_set_option", "qgbdt_get_info", "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile",
     "qgbdt_build_histograms_noalloc", "qgbdt_noalloc_last_error",
 ]
 
@@ -229,6 +231,9 @@ class Context:
                                                 v.ctypes.data_as(C.c_void_p), _stream(stream)))
         return (w, v) if n_leaves is None else (w[:n_leaves], v[:n_leaves])
 
+    def apply_leaf_values(self, scores, stream=None):
+        self._check(self.lib.qgbdt_apply_leaf_values(self.h, _dptr(scores), _stream(stream)))
+
     def train(self, labels, scores, first_tree: int, num_trees: int, stream=None) -> HostModel:
         """labels / scores: float32 [N]; CUDA tensors, or CPU tensors (host variant, scores updated in place)."""
         model = HostModel(num_trees, self.params.num_leaves)
@@ -243,6 +248,14 @@ class Context:
                                            _stream(stream))
         self._check(rc)
         return model
+
+    def set_option(self, option: int, value: int):
+        self._check(self.lib.qgbdt_set_option(self.h, C.c_int32(option), C.c_int64(value)))
+
+    def get_info(self, what: int) -> int:
+        v = C.c_int64()
+        self._check(self.lib.qgbdt_get_info(self.h, C.c_int32(what), C.byref(v)))
+        return v.value
 
     def get_counters(self) -> dict:
         a, b, c = C.c_int64(), C.c_int64(), C.c_int64()
@@ -270,9 +283,16 @@ def build_histograms_noalloc(bins: torch.Tensor, n_bins: int, gq: torch.Tensor, 
     hq uint8 [N], hist int64 [F, n_bins] (overwritten), rows optional int32 list.  Marshalling only."""
     lib = load_library()
     lib.qgbdt_noalloc_last_error.restype = C.c_char_p
+    # the C call takes raw pointers: a wrong dtype, a host tensor or a transposed view would be read as garbage
+    assert bins.is_cuda and bins.dtype == torch.uint8 and bins.dim() == 2 and bins.stride(1) == 1
+    assert gq.is_cuda and gq.dtype == torch.int8 and gq.is_contiguous() and gq.numel() == bins.shape[0]
+    assert hq.is_cuda and hq.dtype == torch.uint8 and hq.is_contiguous() and hq.numel() == bins.shape[0]
+    assert hist.is_cuda and hist.dtype == torch.int64 and hist.is_contiguous() and hist.numel() == bins.shape[1] * n_bins
+    assert rows is None or (rows.is_cuda and rows.dtype in (torch.int32, torch.uint32) and rows.is_contiguous())
+    assert status is None or (status.is_cuda and status.dtype == torch.int32)
     n_rows, f = bins.shape
     n = n_rows if rows is None else rows.numel()
-    rc = lib.qgbdt_build_histograms_noalloc(_dptr(bins), C.c_int64(n_rows), C.c_int32(f), C.c_int32(n_bins),
+    rc = lib.qgbdt_build_histograms_noalloc(C.c_void_p(bins.data_ptr()), C.c_int64(n_rows), C.c_int32(f), C.c_int32(n_bins),
                                             C.c_int64(bins.stride(0)), _dptr(gq), _dptr(hq), _dptr(rows), C.c_int64(n),
                                             _dptr(hist), _dptr(status), _stream(stream))
     if rc != OK:

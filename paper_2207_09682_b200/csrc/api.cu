@@ -151,6 +151,7 @@ int check_loaded(qgbdt_ctx *c) {
 
 void reset_leaf_state(qgbdt_ctx *c) {
     c->n_leaves = 1;
+    c->refit_leaves = 0;
     c->leaf_off.assign(c->prm.num_leaves, 0);
     c->leaf_n.assign(c->prm.num_leaves, 0);
     c->leaf_n[0] = c->N;
@@ -390,6 +391,10 @@ int qgbdt_build_histograms_rows(qgbdt_ctx *c, const uint32_t *d_rows, int64_t n,
     if (rc != QGBDT_OK) return rc;
     if (!c->quantized) return qg_fail(c, QGBDT_ERR_STATE, "quantize gradients before building histograms");
     if (!d_hist || (n > 0 && !d_rows) || n < 0 || n >= (1ll << 32)) return qg_fail(c, QGBDT_ERR_ARG, "bad argument");
+    // a list may repeat rows, so its length, not n_rows, bounds the sums of a bin
+    const int64_t kg = qg_levels_g(c->prm.bits), kh = c->const_hess ? 1 : qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
+    if (n * kg > 2147483647ll || n * kh > 4294967295ll)
+        return qg_fail(c, QGBDT_ERR_OVERFLOW, "a list of %lld rows could exceed the 32+32-bit histogram word", (long long)n);
     return qg_hist(c, d_rows, 0, n, reinterpret_cast<unsigned long long *>(d_hist), (cudaStream_t)stream);
 }
 
@@ -415,7 +420,11 @@ int qgbdt_find_best_split(qgbdt_ctx *c, const qgbdt_bin *d_hist, int64_t G, int6
         return rc;
     SplitRec *hr = reinterpret_cast<SplitRec *>(reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS + 256);
     QG_CUDA(c, cudaMemcpyAsync(hr, c->d_split_out, sizeof(SplitRec), cudaMemcpyDeviceToHost, st));
+    DevState *hs = reinterpret_cast<DevState *>(reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS);
+    QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
     QG_CUDA(c, cudaStreamSynchronize(st));
+    // a histogram kernel that refused to run (earlier on this stream) left d_hist unwritten
+    if (hs->kernel_error) return qg_fail(c, QGBDT_ERR_CUDA, "a histogram kernel refused its launch configuration");
     rec_to_split(*hr, G, H, n_rows, c->const_hess, h_out);
     return QGBDT_OK;
 }
@@ -439,6 +448,7 @@ int qgbdt_split_leaf(qgbdt_ctx *c, int32_t leaf, int32_t feature, int32_t bin, i
         nl = hs->part_nl;
     }
     const int r = c->n_leaves++;
+    c->refit_leaves = 0;
     c->leaf_n[leaf] = nl;
     c->leaf_off[r] = off + nl;
     c->leaf_n[r] = n - nl;
@@ -479,7 +489,39 @@ int qgbdt_refit_leaves(qgbdt_ctx *c, const float *d_g, const float *d_h, double 
     QG_CUDA(c, cudaStreamSynchronize(st));
     if (h_w) memcpy(h_w, hw, sizeof(double) * L);
     if (h_value) memcpy(h_value, hv, sizeof(float) * L);
+    c->refit_leaves = L;
     return QGBDT_OK;
+}
+
+int qgbdt_apply_leaf_values(qgbdt_ctx *c, float *d_scores, void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!d_scores) return qg_fail(c, QGBDT_ERR_ARG, "d_scores is NULL");
+    if (c->refit_leaves != c->n_leaves) return qg_fail(c, QGBDT_ERR_STATE, "refit the current leaves first");
+    return qg_apply_leaf_values(c, d_scores, (cudaStream_t)stream);
+}
+
+int qgbdt_set_option(qgbdt_ctx *c, int32_t option, int64_t value) {
+    if (!c) return QGBDT_ERR_ARG;
+    switch (option) {
+        case QGBDT_OPT_COLUMN_COPY:
+            if (value != 0 && value != 1) return qg_fail(c, QGBDT_ERR_ARG, "QGBDT_OPT_COLUMN_COPY takes 0 or 1");
+            c->want_column_copy = value != 0;
+            return QGBDT_OK;
+        default:
+            return qg_fail(c, QGBDT_ERR_ARG, "unknown option %d", option);
+    }
+}
+
+int qgbdt_get_info(const qgbdt_ctx *c, int32_t what, int64_t *value) {
+    if (!c || !value) return QGBDT_ERR_ARG;
+    switch (what) {
+        case QGBDT_INFO_COLUMN_COPY:
+            *value = c->d_colmajor != nullptr ? 1 : 0;
+            return QGBDT_OK;
+        default:
+            return QGBDT_ERR_ARG;
+    }
 }
 
 int qgbdt_get_counters(const qgbdt_ctx *c, int64_t *kernel_launches, int64_t *hist_builds, int64_t *hist_row_features) {

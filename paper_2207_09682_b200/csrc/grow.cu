@@ -52,7 +52,9 @@ __global__ void k_grow_begin(GrowState *gs, LeafRec *leaves, const DevState *sta
     r.parent_node = -1; r.parent_side = 0;
     leaves[0] = r;
     gs->n_leaves = 1;
-    gs->done = 0;
+    // gradients out of domain (the flag is sticky over the trees of a train call): the split
+    // kernels of this tree return at once, the call reports the error when it ends
+    gs->done = state->bad_value ? 1 : 0;
     gs->finish_count = 0;
 }
 

@@ -32,9 +32,15 @@
 // run side by side in pairs of CTAs that read the same rows at the same time.
 #include <cooperative_groups.h>
 
+#include <mutex>
+
 #include "hist_cta.cuh"
 
 namespace {
+
+// Guards the per-instantiation "attribute set on this device" flags below: they are shared by all
+// contexts of the process, and two contexts may be driven from two host threads.
+std::mutex g_configure_mutex;
 
 // Row shares of a tile when its CTAs work in pairs (one pass of the 32+32 mode each).
 __device__ __host__ inline uint32_t paired_parts(uint32_t P) { return P > 1 ? P >> 1 : 1; }
@@ -198,9 +204,12 @@ template <int LOGW_T, int MODE, int LIST>
 int launch_one(qgbdt_ctx *c, const HistArgs &args, int n_tiles, cudaStream_t st) {
     auto kern = k_hist<LOGW_T, MODE, LIST>;
     static bool configured[64] = {};   // per instantiation and device (the attribute belongs to the device's context)
-    if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
-        QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
-        if (c->device >= 0 && c->device < 64) configured[c->device] = true;
+    {
+        std::lock_guard<std::mutex> lock(g_configure_mutex);
+        if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
+            QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
+            if (c->device >= 0 && c->device < 64) configured[c->device] = true;
+        }
     }
     int group_parts = 1;
     for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
@@ -217,9 +226,12 @@ template <int LOGW_T, int MODE, int LIST>
 int launch_one_coop(qgbdt_ctx *c, HistArgs &args, int n_tiles, cudaStream_t st) {
     const void *kern = reinterpret_cast<const void *>(k_hist_coop<LOGW_T, MODE, LIST>);
     static bool configured[64] = {};   // per instantiation and device (the attribute belongs to the device's context)
-    if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
-        QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
-        if (c->device >= 0 && c->device < 64) configured[c->device] = true;
+    {
+        std::lock_guard<std::mutex> lock(g_configure_mutex);
+        if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
+            QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
+            if (c->device >= 0 && c->device < 64) configured[c->device] = true;
+        }
     }
     int group_parts = 1;
     for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
@@ -372,9 +384,12 @@ int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n
                     bool configure_only) {
     auto kern = k_hist_grow<LOGW_T, MODE>;
     static bool configured[64] = {};   // per instantiation and device (the attribute belongs to the device's context)
-    if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
-        QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
-        if (c->device >= 0 && c->device < 64) configured[c->device] = true;
+    {
+        std::lock_guard<std::mutex> lock(g_configure_mutex);
+        if (c->device < 0 || c->device >= 64 || !configured[c->device]) {
+            QG_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, HIST_SMEM));
+            if (c->device >= 0 && c->device < 64) configured[c->device] = true;
+        }
     }
     if (configure_only) return QGBDT_OK;
     int group_parts = 1;

@@ -149,7 +149,7 @@ __device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, 
                 }
                 v = (unsigned long long)((long long)G * 4294967296LL + (long long)H);
             } else {
-                // two 32-bit planes per bin; no field can overflow (checked at load time)
+                // two 32-bit planes per bin; no field can overflow (rows x levels is checked against the word at load time and for every row list)
                 int *p = hp + kk * 16384 + bin * 64 + a * R;
                 long long G = 0;
                 unsigned long long H = 0;

@@ -1,6 +1,4 @@
 // Bin-matrix relayout into feature tiles, and the identity row list of the root leaf.
-#include <cstdlib>
-
 #include "qgbdt_internal.cuh"
 
 // One thread per (row, word) of a tile: gathers four bin codes from the caller's matrix
@@ -87,10 +85,9 @@ __global__ void k_set_columns(FeatRec *feat_rec, int F, uint8_t *cols, size_t st
 
 int qg_build_columns(qgbdt_ctx *c, cudaStream_t st) {
     if (c->d_colmajor) return QGBDT_OK;
-    // QGBDT_NO_COLUMN_COPY=1 keeps training on the tiles alone (saves N x F bytes; also how the
-    // tests reach the path taken when the allocation below fails)
-    const char *off = getenv("QGBDT_NO_COLUMN_COPY");
-    if (off && off[0] == '1') return QGBDT_OK;
+    // switched off by the caller (qgbdt_set_option): training stays on the tiles alone, which saves
+    // N x F bytes; the same path is taken when the allocation below fails
+    if (!c->want_column_copy) return QGBDT_OK;
     const size_t stride = ((size_t)c->N + 127) / 128 * 128;
     void *p = nullptr;
     if (cudaMalloc(&p, stride * (size_t)c->F) != cudaSuccess) {

@@ -20,6 +20,7 @@ namespace {
 constexpr int NOALLOC_SLOTS = 32;            // CTAs of the first stage, one partial histogram each
 constexpr int NOALLOC_MAX_BINS = 16384;      // n_features * n_bins may not exceed this
 constexpr int NOALLOC_MAX_DEVICES = 64;
+constexpr long long NOALLOC_MAX_ENTRIES = 4294967295ll / 255;   // 16 843 009: n * 255 still fits the unsigned hessian field
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress; the
 // address a kernel can use is looked up once per device below.
@@ -53,6 +54,7 @@ __global__ void __launch_bounds__(256) k_na_partial(const uint8_t *__restrict__ 
         if (row >= n_rows) { if (bad) *bad = 1; continue; }
         const int bin = bins[row * ld + f];
         if (bin >= nb) { if (bad) *bad = 1; continue; }
+        if (gq[row] == -128) { if (bad) *bad = 1; continue; }   // outside every level range (|g| <= 127); the overflow bound assumes it
         const long long packed = (long long)gq[row] * 4294967296LL + (long long)hq[row];
         atomicAdd(&slot[(size_t)f * nb + bin], (unsigned long long)packed);
     }
@@ -87,7 +89,9 @@ int qgbdt_build_histograms_noalloc(const uint8_t *d_bins, int64_t n_rows, int32_
                  (long long)n_features * n_bins, NOALLOC_MAX_BINS);
         return QGBDT_ERR_ARG;
     }
-    if (n >= (1ll << 32) || n * 255 > 4294967295ll) return na_fail(QGBDT_ERR_OVERFLOW, "the sums could exceed the 32+32-bit histogram word");
+    // the caller's codes may be anything in [-127, 127] x [0, 255]: n entries can reach n * 255 in a hessian field
+    if (n > NOALLOC_MAX_ENTRIES)
+        return na_fail(QGBDT_ERR_OVERFLOW, "more than 16843009 entries: the sums could exceed the 32+32-bit histogram word");
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) {
         cudaGetLastError();

@@ -128,6 +128,7 @@ struct qgbdt_ctx {
     std::vector<int64_t> leaf_off, leaf_n;
     uint32_t *d_idx = nullptr, *d_idx_tmp = nullptr;
     bool idx_is_identity = false;
+    int refit_leaves = 0;   // leaf count the last qgbdt_refit_leaves ran for (0: the leaves changed since)
     // scratch
     DevState *d_state = nullptr;
     uint32_t *d_part_counts = nullptr;  // per partition block: rows going left, then its exclusive scan
@@ -149,6 +150,7 @@ struct qgbdt_ctx {
     FeatRec *d_feat_rec = nullptr;              // [F] location of every feature
     uint8_t *d_colmajor = nullptr;              // [F][col_stride] column-major copy of the bin codes (training only)
     size_t col_stride = 0;
+    bool want_column_copy = true;               // QGBDT_OPT_COLUMN_COPY
     double *d_leaf_gain = nullptr;              // [L] stored gain of every leaf's best split (-inf: none)
     void *grow_graph_exec = nullptr;            // cudaGraphExec_t: the split loop of one tree
     int64_t grow_graph_launches = 0;            // kernel launches it replays

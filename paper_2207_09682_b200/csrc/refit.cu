@@ -188,10 +188,20 @@ int upload_table(qgbdt_ctx *c, cudaStream_t st) {
     uint32_t *tab = reinterpret_cast<uint32_t *>(c->h_pinned);
     std::vector<int> order(L);
     for (int i = 0; i < L; ++i) order[i] = i;
-    for (int i = 1; i < L; ++i) {  // insertion sort by offset (lists are short and nearly sorted)
+    // Order: offset, then empty leaves before the non-empty one that starts at the same offset (a
+    // split that sends every row to one side leaves an empty leaf there; the search below takes the
+    // last slot whose offset is <= the position, which must be the leaf that owns the rows), then
+    // leaf number: the same ranking as k_leaf_table.
+    auto before = [&](int a, int b) {
+        if (c->leaf_off[a] != c->leaf_off[b]) return c->leaf_off[a] < c->leaf_off[b];
+        const bool ea = c->leaf_n[a] == 0, eb = c->leaf_n[b] == 0;
+        if (ea != eb) return ea;
+        return a < b;
+    };
+    for (int i = 1; i < L; ++i) {  // insertion sort (lists are short and nearly sorted)
         const int v = order[i];
         int j = i - 1;
-        while (j >= 0 && c->leaf_off[order[j]] > c->leaf_off[v]) { order[j + 1] = order[j]; --j; }
+        while (j >= 0 && before(v, order[j])) { order[j + 1] = order[j]; --j; }
         order[j + 1] = v;
     }
     for (int s = 0; s < L; ++s) {

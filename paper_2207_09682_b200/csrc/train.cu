@@ -127,6 +127,7 @@ int qgbdt_train(qgbdt_ctx *c, const float *d_labels, float *d_scores, uint32_t f
     QG_CUDA(c, cudaMemcpyAsync(hg, c->d_gs, sizeof(GrowState), cudaMemcpyDeviceToHost, st));
     // leave the step-wise interface in a defined state: one root leaf, rows ascending
     c->n_leaves = 1;
+    c->refit_leaves = 0;
     c->leaf_off.assign(L, 0);
     c->leaf_n.assign(L, 0);
     c->leaf_n[0] = c->N;

@@ -113,6 +113,10 @@ HIST_CASES = [
     (8_191, 136, 64, 5, False),
     (4_097, 150, 255, 8, False),
     (300_000, 28, 255, 4, False),
+    (50_003, 28, 255, 6, False),        # first bit width with 32+32 local bins
+    (50_003, 28, 64, 7, True),
+    (25_001, 136, 255, 6, True),        # two tile widths, 32+32 local bins
+    (25_001, 136, 128, 7, False),
 ]
 
 
@@ -165,6 +169,43 @@ def test_histogram_worst_case_accumulation():
         ctx.build_histograms(0, hist)
         G, H = binding.unpack_hist(hist)
         assert G[27, 0] == kg * n and H[27, 0] == kh * n
+
+
+def test_histogram_worst_case_accumulation_other_hessian_levels():
+    # hess_levels_mode 1 (2^B - 1 hessian levels): one more level per row, so a column fills up
+    # sooner (another flush interval); all rows in one bin at the extreme levels
+    for bits, n in ((2, 200_000), (4, 150_000), (5, 120_000)):
+        data = np.zeros((n, 28), np.uint8)
+        data[:, 11] = 6
+        kg, kh = oracle.levels(bits, 1)
+        assert kh == (1 << bits) - 1
+        g = np.full(n, -1.0, np.float32)
+        h = np.full(n, 0.25, np.float32)
+        ctx = make_ctx(data, 8, bits=bits, hess_levels_mode=1)
+        ctx.quantize_gradients(dev(g), dev(h))
+        ref = oracle.quantize(g, h, bits=bits, hess_levels_mode=1)
+        hist = ctx.new_hist()
+        ctx.build_histograms(0, hist)
+        G, H = binding.unpack_hist(hist)
+        og, oh = oracle.histogram(data, 8, ref.gq, ref.hq)
+        assert (G == og).all() and (H == oh).all()
+        assert G[0, 0] == -kg * n and H[0, 0] == kh * n and G[11, 6] == -kg * n and H[11, 0] == 0
+        rows = synth.subset_rows(n, device="cpu", seed=3).numpy().astype(np.uint32)
+        ctx.build_histograms_rows(dev(rows.view(np.int32)), hist)
+        G, H = binding.unpack_hist(hist)
+        assert G[27, 0] == -kg * len(rows) and H[27, 0] == kh * len(rows)
+
+
+def test_row_list_longer_than_the_histogram_word_allows_is_refused():
+    # a list may repeat rows: 8-bit gradients, 17 M entries -> 17e6 * 127 > 2^31 - 1
+    data = random_bins(1000, 4, 8, 0)
+    g, h = logistic_grads(1000, 1)
+    ctx = make_ctx(data, 8, bits=8)
+    ctx.quantize_gradients(dev(g), dev(h))
+    rows = torch.zeros(17_000_000, dtype=torch.int32, device="cuda")
+    with pytest.raises(binding.QgbdtError) as e:
+        ctx.build_histograms_rows(rows, ctx.new_hist())
+    assert e.value.code == binding.ERR_OVERFLOW
 
 
 def test_histogram_column_major_input_and_constant_hessian():
@@ -327,6 +368,33 @@ def test_refit_bit_exact(const_h):
         assert w[l] == ow and v[l] == ov
 
 
+def test_refit_with_an_empty_leaf_next_to_a_full_one():
+    # a user-chosen split that sends every row left makes an empty right leaf at the offset where
+    # the next leaf starts; the rows there must still be credited to the leaf that owns them
+    n, f, nb = 30_000, 6, 16
+    data = random_bins(n, f, nb, 12)
+    g, h = logistic_grads(n, 13)
+    ctx = make_ctx(data, nb, num_leaves=5, learning_rate=0.3)
+    leaves = {0: np.arange(n, dtype=np.uint32)}
+    for leaf, feat, thr in [(0, 2, 7), (0, 1, nb - 1), (0, 3, 4)]:     # the second split leaves leaf 2 empty
+        right, nl, nr = ctx.split_leaf(leaf, feat, thr)
+        out, onl = oracle.partition(data, leaves[leaf], feat, thr)
+        assert (nl, nr) == (onl, len(out) - onl)
+        leaves[leaf], leaves[right] = out[:onl], out[onl:]
+    assert len(leaves[2]) == 0 and len(leaves[1]) > 0
+    w, v = ctx.refit_leaves(dev(g), dev(h), n_leaves=4)
+    for l in range(4):
+        ow, ov = oracle.refit(g, h, leaves[l], learning_rate=0.3)
+        assert w[l] == ow and v[l] == ov, l
+    # the score update routes every row to its own leaf's value
+    scores = torch.zeros(n, device="cuda")
+    ctx.apply_leaf_values(scores)
+    want = np.zeros(n, np.float32)
+    for l in range(4):
+        want[leaves[l]] = v[l]
+    assert (scores.cpu().numpy() == want).all()
+
+
 # ------------------------------------------------------------------ training
 
 def compare_trees(model, k, ref):
@@ -345,16 +413,24 @@ TRAIN_CASES = [
     ("tall", 30_000, dict(num_trees=3, num_leaves=63)),
     ("large", 40_000, dict(num_trees=3, num_leaves=63)),
     ("wide", 3_000, dict(num_trees=2, num_leaves=15)),
+    # 32+32 local bins inside tree growth (two passes over the smaller child's rows)
+    ("tall", 30_000, dict(num_trees=3, num_leaves=63, bits=8)),
+    ("tall", 30_000, dict(num_trees=3, num_leaves=63, bits=6)),
+    ("large", 40_000, dict(num_trees=2, num_leaves=31, bits=7)),
+    ("tall", 30_000, dict(num_trees=2, num_leaves=31, bits=5, hess_levels_mode=1)),
+    ("tiny", 20_000, dict(num_trees=2, rounding=1)),
 ]
 
 
-@pytest.mark.parametrize("name,rows,over", TRAIN_CASES)
-def test_training_matches_oracle(name, rows, over):
+def train_case(name, rows, over, column_copy=None):
     wl = synth.CONFIGS[name](device="cpu", rows=rows) if name != "wide" else synth.wide(device="cpu", rows=rows, features=300)
     kw = dict(wl.params, seed=11)
     kw.update(over)
     data, y = wl.bins.numpy(), wl.labels.numpy()
-    ctx = make_ctx(data, wl.n_bins, **kw)
+    ctx = binding.Context(binding.make_params(**kw))
+    if column_copy is not None:
+        ctx.set_option(binding.OPT_COLUMN_COPY, column_copy)
+    ctx.load_binned(dev(data), wl.n_bins)
     scores = torch.zeros(rows, device="cuda")
     model = ctx.train(dev(y), scores, 0, kw["num_trees"])
     ref_scores = np.zeros(rows, np.float32)
@@ -365,14 +441,29 @@ def test_training_matches_oracle(name, rows, over):
     got = scores.cpu().numpy()
     assert np.allclose(got, ref_scores, rtol=1e-5, atol=1e-7)
     assert (got.view(np.uint32) == ref_scores.view(np.uint32)).all()
+    return ctx
 
 
-def test_training_without_the_column_copy(monkeypatch):
+@pytest.mark.parametrize("name,rows,over", TRAIN_CASES)
+def test_training_matches_oracle(name, rows, over):
+    train_case(name, rows, over)
+
+
+def test_training_without_the_column_copy():
     # the row partition reads the split feature from the tiles when there is no column-major copy
-    # (its allocation failed, or it was switched off): same trees
-    monkeypatch.setenv("QGBDT_NO_COLUMN_COPY", "1")
+    # (its allocation failed, or the option switched it off): same trees, and the context says
+    # which path it took
     for name, rows, over in (TRAIN_CASES[1], TRAIN_CASES[3]):
-        test_training_matches_oracle(name, rows, over)
+        for want in (0, 1):
+            ctx = train_case(name, rows, over, column_copy=want)
+            assert ctx.get_info(binding.INFO_COLUMN_COPY) == want
+    ctx = binding.Context(binding.make_params())
+    with pytest.raises(binding.QgbdtError) as e:
+        ctx.set_option(binding.OPT_COLUMN_COPY, 2)
+    assert e.value.code == binding.ERR_ARG
+    with pytest.raises(binding.QgbdtError) as e:
+        ctx.set_option(99, 0)
+    assert e.value.code == binding.ERR_ARG
 
 
 def test_training_resumes_and_host_variant_agrees():

@@ -552,7 +552,18 @@ def test_tree_structure_is_consistent():
     assert (np.bincount(row_leaf, minlength=t.num_leaves) == t.leaf_count).all()
     assert (oracle.predict_leaf(data, t) == row_leaf).all()          # node wiring routes rows to their leaf
     assert (scores == t.leaf_value[row_leaf]).all()                  # score update = leaf output
-    assert (np.diff(t.gain) <= 1e-12).all() or True                  # best-first: not necessarily monotone
+    # best-first: when node i was made, every leaf that already existed had a gain no larger than
+    # node i's; a later node j split such a leaf iff its parent node was made before i (gains are
+    # not monotone over the whole sequence: a child's gain may exceed its parent's)
+    parent = np.full(t.num_leaves - 1, -1)
+    for i in range(t.num_leaves - 1):
+        for c in (t.left[i], t.right[i]):
+            if c >= 0:
+                parent[c] = i
+    for i in range(t.num_leaves - 1):
+        for j in range(i + 1, t.num_leaves - 1):
+            if parent[j] < i:
+                assert t.gain[j] <= t.gain[i]
     # every internal node's children are either nodes created later or leaves
     for i in range(t.num_leaves - 1):
         for c in (t.left[i], t.right[i]):
@@ -644,3 +655,33 @@ def test_train_stops_when_no_valid_split():
     t = oracle.train_tree(data, 4, y, scores, oracle.make_params(num_leaves=8), 0)
     assert t.num_leaves == 1 and t.leaf_count[0] == 100
     assert abs(float(t.leaf_value[0])) < 1e-6                         # balanced labels: w = 0
+
+
+def test_multi_tree_wrapper_is_the_loop_over_single_trees():
+    # qo_train is only a loop over qo_train_tree that lays the trees out one after the other
+    import ctypes as C
+    data, y, _ = toy_classification(seed=9)
+    n, L, K = len(y), 7, 3
+    prm = oracle.make_params(bits=3, num_leaves=L, num_trees=K, seed=21)
+    want_scores = np.zeros(n, np.float32)
+    want = oracle.train(data, 32, y, want_scores, prm)
+    scores = np.zeros(n, np.float32)
+    leaves = np.zeros(K, np.int32)
+    nf, nb_, nl, nr = (np.zeros(K * (L - 1), np.int32) for _ in range(4))
+    ng = np.zeros(K * (L - 1), np.float64)
+    lv, lc = np.zeros(K * L, np.float32), np.zeros(K * L, np.int64)
+    p = lambda a, t: a.ctypes.data_as(C.POINTER(t))
+    d = np.ascontiguousarray(data, np.uint8)
+    rc = oracle.lib().qo_train(p(d, C.c_uint8), C.c_int64(n), d.shape[1], 32, p(y, C.c_float), p(scores, C.c_float),
+                               C.byref(prm), p(leaves, C.c_int32), p(nf, C.c_int32), p(nb_, C.c_int32),
+                               p(nl, C.c_int32), p(nr, C.c_int32), p(ng, C.c_double), p(lv, C.c_float),
+                               p(lc, C.c_int64))
+    assert rc == 0
+    assert (scores == want_scores).all()
+    for k, t in enumerate(want):
+        m = t.num_leaves
+        assert leaves[k] == m
+        s_ = slice(k * (L - 1), k * (L - 1) + m - 1)
+        assert (nf[s_] == t.feature).all() and (nb_[s_] == t.bin).all() and (nl[s_] == t.left).all()
+        assert (nr[s_] == t.right).all() and (ng[s_] == t.gain).all()
+        assert (lv[k * L:k * L + m] == t.leaf_value).all() and (lc[k * L:k * L + m] == t.leaf_count).all()

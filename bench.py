@@ -10,7 +10,8 @@ Metric: histogram row-features per second = rows x features that Algorithm 1 has
 (the root plus the smaller child of every split) divided by the time of the WHOLE step.
 ms_per_step is ms per tree.  `roofline` is the histogram kernel alone: algorithmic bytes of
 all its launches inside the timed region over their summed CUDA-event durations, against the
-measured HBM copy bandwidth.  `cpu_baseline` is the CPU oracle on a bounded row sample.
+measured HBM copy bandwidth; `tree_roofline` is the whole step: the algorithmic bytes of every
+kernel family of the timed trees over the step time.  `cpu_baseline` is the CPU oracle.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 """
@@ -28,7 +29,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 WORKLOAD_ROWS = {"large": 10_500_000, "tall": 1_000_000, "tiny": 50_000, "wide": 400_000}
-CPU_SAMPLE_ROWS = {"large": 3_000_000, "tall": 1_000_000, "tiny": 50_000, "wide": 20_000}
+# rows of the CPU arm: the same rows as the GPU arm (one oracle tree: about 9 s on 'large', 15 s on 'wide')
+CPU_SAMPLE_ROWS = dict(WORKLOAD_ROWS)
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the histogram kernels on the 'large' workload from an ncu capture
 # (profiles/launch_list_large_10p5Mx28.md): 3.37 GB over the 255 builds of one tree.  Valid only for
@@ -104,11 +106,12 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def needed_hist_rows(tree: dict, n_rows: int) -> int:
-    """Rows Algorithm 1 must visit for one tree: the root plus the smaller child of every split."""
+def tree_rows(tree: dict, n_rows: int) -> tuple[int, int]:
+    """Rows one tree must visit: (histogram rows = the root plus the smaller child of every split,
+    partition rows = the rows of every leaf that was split)."""
     nl = tree["num_leaves"]
     if nl <= 1:
-        return n_rows
+        return n_rows, 0
     count = {}
 
     def size(c):
@@ -118,14 +121,52 @@ def needed_hist_rows(tree: dict, n_rows: int) -> int:
             count[c] = size(int(tree["left"][c])) + size(int(tree["right"][c]))
         return count[c]
 
-    total = n_rows
+    hist, part = n_rows, 0
     for i in range(nl - 1):
-        total += min(size(int(tree["left"][i])), size(int(tree["right"][i])))
-    return total
+        a, b = size(int(tree["left"][i])), size(int(tree["right"][i]))
+        hist += min(a, b)
+        part += a + b
+    return hist, part
+
+
+def needed_hist_rows(tree: dict, n_rows: int) -> int:
+    return tree_rows(tree, n_rows)[0]
+
+
+def code_bytes(bits: int) -> int:
+    """Packed gradient + hessian code per row that the method has to move: one byte up to 4 bits, two beyond."""
+    return 1 if bits <= 4 else 2
+
+
+def tree_algorithmic_bytes(trees: list, n: int, features: int, n_bins: int, bits: int, const_hessian: bool) -> dict:
+    """Bytes every step of the path must move for the given trees (per kernel family, summed over the trees):
+    histogram builds  rows * (F + c [+ 4 row index for a child]) + F * bins * 8 per build
+    partition         parent rows * (4 index in + 1 bin code + 4 index out)
+    quantizer         N * (4 per gradient array read + c written)
+    gradients         N * (scores + labels read, one or two arrays written)
+    refit, scores     N * (gradient arrays + 4 row index) resp. N * 8
+    split search      2 * F * bins * 8 per split; subtraction 3 * F * bins * 8 per split"""
+    c = code_bytes(bits)
+    arrays = 1 if const_hessian else 2
+    hb = features * n_bins * 8
+    out = dict.fromkeys(("histogram", "partition", "quantize", "gradients", "refit", "score_update", "split_search",
+                         "subtraction"), 0)
+    for t in trees:
+        hist_rows, part_rows = tree_rows(t, n)
+        splits = max(int(t["num_leaves"]) - 1, 0)
+        out["histogram"] += n * (features + c) + (hist_rows - n) * (features + c + 4) + (splits + 1) * hb
+        out["partition"] += part_rows * 9
+        out["quantize"] += n * (4 * arrays + c)
+        out["gradients"] += n * (8 + 4 * arrays)
+        out["refit"] += n * (4 * arrays + 4)
+        out["score_update"] += n * 8
+        out["split_search"] += (2 * splits + 1) * hb
+        out["subtraction"] += 3 * splits * hb
+    return out
 
 
 def oracle_leg(wl_name: str, rows: int, steps: int, warmup: int, data=None, y=None, n_bins=None, params=None) -> dict:
-    """Times the CPU oracle (as it stands, one thread) on a bounded row sample of the workload."""
+    """Times the CPU oracle (as it stands, one thread): whole boosting iterations."""
     import numpy as np
     import oracle
     from paper_2207_09682_b200 import synth
@@ -144,9 +185,42 @@ def oracle_leg(wl_name: str, rows: int, steps: int, warmup: int, data=None, y=No
             rf += needed_hist_rows(tree, rows) * data.shape[1]
             secs += dt
     return {"value": rf / secs, "unit": "row-features/s", "cores": 1, "kind": "oracle",
-            "sample": "%d trees of %d leaves on the first-generated %d rows x %d features of workload '%s'"
+            "sample": "%d trees of %d leaves on all %d rows x %d features of workload '%s'"
                       % (steps, prm.num_leaves, rows, data.shape[1], wl_name),
-            "ms_per_tree": 1e3 * secs / steps}
+            "ms_per_tree": 1e3 * secs / steps, "host_cores": os.cpu_count()}
+
+
+def oracle_hist_all_cores(data, n_bins: int, max_rows: int = 4_000_000) -> dict:
+    """The oracle's Algorithm 1 on every host core: the harness cuts the rows into one chunk per
+    thread, every thread calls the unchanged single-threaded routine into arrays of its own (ctypes
+    releases the interpreter lock), and the per-chunk histograms are added up afterwards."""
+    import numpy as np
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+    cores = os.cpu_count() or 1
+    n = min(len(data), max_rows)
+    data = data[:n]
+    r = np.random.default_rng(0)
+    gq = r.integers(-7, 8, size=n).astype(np.int8)
+    hq = np.ones(n, np.uint8)
+    bounds = [n * i // cores for i in range(cores + 1)]
+
+    def chunk(i):
+        a, b = bounds[i], bounds[i + 1]
+        return oracle.histogram(data[a:b], n_bins, gq[a:b], hq[a:b])
+
+    best = None
+    with ThreadPoolExecutor(max_workers=cores) as pool:
+        for _ in range(3):
+            t0 = time.perf_counter()
+            parts = list(pool.map(chunk, range(cores)))
+            hg = sum(p[0] for p in parts)
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+    assert int(hg.sum()) == int(gq.astype(np.int64).sum()) * data.shape[1]
+    return {"value": n * data.shape[1] / best, "unit": "row-features/s", "cores": cores, "kind": "oracle",
+            "scope": "root histogram build only (Algorithm 1), best of 3",
+            "sample": "the first %d rows x %d features, one row chunk per thread" % (n, data.shape[1])}
 
 
 def run_reference(args):
@@ -159,14 +233,15 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "hist_row_features_per_s", "value": leg["value"], "unit": "row-features/s",
             "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "ms_per_step": leg["ms_per_tree"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-            "config": {"workload": args.workload, "rows": rows, "note": "CPU oracle on a bounded row sample"},
-            "cpu_baseline": {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "config": {"workload": args.workload, "rows": rows,
+                       "note": "CPU oracle, one thread of %s host cores, whole boosting iterations" % os.cpu_count()},
+            "cpu_baseline": {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample", "host_cores")},
             "e2e": {"value": leg["value"], "unit": "row-features/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
 
 
-def time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes, reps=10, batch=10):
+def time_hist_builds(ctx, torch, synth, n, features, n_bins, cbytes, reps=10, batch=10):
     """Stand-alone root and 50%-subset histogram builds on inputs larger than L2.
 
     `batch` builds are enqueued back to back between two CUDA events so that the GPU never waits
@@ -193,7 +268,7 @@ def time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes, reps=10
                 ts.append(e0.elapsed_time(e1) / batch)
         nr = n if r is None else int(r.numel())
         ms = float(np.median(ts))
-        nbytes = nr * (features + code_bytes + (0 if r is None else 4)) + features * n_bins * 8
+        nbytes = nr * (features + cbytes + (0 if r is None else 4)) + features * n_bins * 8
         out[name] = {"rows": nr, "us": 1e3 * ms, "row_features_per_s": nr * features / (ms * 1e-3),
                      "gbs": nbytes / (ms * 1e6), "note": "partial histograms and their merge in one cooperative kernel, %d builds per timing" % batch}
     return out
@@ -216,7 +291,7 @@ def run_sweep(args):
                     ctx = binding.Context(binding.make_params(bits=bits))
                     ctx.load_binned(bins, nb)
                     ctx.quantize_gradients(g, h)
-                    b = time_hist_builds(ctx, torch, synth, n, f, nb, 2, reps=3, batch=5)
+                    b = time_hist_builds(ctx, torch, synth, n, f, nb, code_bytes(bits), reps=3, batch=5)
                     print("%9d %5d %4d %2d | %9.1f %7.0f %5.3f | %9.1f %7.0f %5.3f" % (
                         n, f, nb, bits, b["root"]["us"], b["root"]["gbs"], b["root"]["gbs"] / peak,
                         b["subset50"]["us"], b["subset50"]["gbs"], b["subset50"]["gbs"] / peak), flush=True)
@@ -302,7 +377,11 @@ def run_ours(args):
 
     peak, peak_kind = measured_peak()
     achieved = prof["total_bytes"] / (prof["total_ms"] * 1e6) if prof["total_ms"] > 0 else 0.0
-    code_bytes = 2     # one 16-bit gradient/hessian code per row
+    cbytes = code_bytes(kw["bits"])
+    # the whole step against the bytes it has to move (this rank's trees; the ranks are replicas)
+    step_bytes = tree_algorithmic_bytes([model.tree(k) for k in range(K)], n, features, n_bins, kw["bits"],
+                                        kw["objective"] == 1)
+    step_total = sum(step_bytes.values())
     line = {
         "metric": "hist_row_features_per_s", "value": rf / (ms * 1e-3), "unit": "row-features/s",
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True,
@@ -321,7 +400,14 @@ def run_ours(args):
                      "share_of_step": prof["total_ms"] / prof_ms if prof_ms else None,
                      "region": "K more boosting iterations right after the timed ones, launches on the stream with "
                                "an event pair around every build (%.2f ms per tree there)" % (prof_ms / K)},
+        "tree_roofline": {"bound": "hbm", "achieved": step_total / (ms * 1e6), "peak": peak, "unit": "GB/s",
+                          "frac": step_total / (ms * 1e6) / peak, "peak_kind": peak_kind,
+                          "algorithmic_bytes_per_tree": step_total / K,
+                          "ms_per_tree_at_peak": step_total / K / (peak * 1e6),
+                          "bytes_per_tree_by_step": {k: v / K for k, v in step_bytes.items()},
+                          "note": "every kernel family of the timed trees: bytes the method has to move over the step time"},
         "clocks": clocks.summary(),
+        "host_cores": os.cpu_count(),
     }
 
     # stand-alone histogram builds on the same data (root leaf and a 50 % subset)
@@ -330,7 +416,7 @@ def run_ours(args):
     ctx.reset_leaves()
     ctx.compute_gradients(scores, wl.labels, g, h)
     ctx.quantize_gradients(g, h, tree=W + K)
-    builds = time_hist_builds(ctx, torch, synth, n, features, n_bins, code_bytes)
+    builds = time_hist_builds(ctx, torch, synth, n, features, n_bins, cbytes)
     for b in builds.values():
         b["frac"] = b["gbs"] / peak
     line["hist_builds"] = builds
@@ -368,7 +454,9 @@ def run_ours(args):
             leg = oracle_leg(args.workload, min(n, CPU_SAMPLE_ROWS[args.workload]), 1, 0)
         else:   # the very arrays the GPU path was timed on, all rows, one tree
             leg = oracle_leg(args.workload, n, 1, 0, host_data[0], host_data[1], n_bins, kw)
-        line["cpu_baseline"] = {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        line["cpu_baseline"] = {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample", "host_cores")}
+        if host_data is not None:
+            line["cpu_baseline"]["all_cores"] = oracle_hist_all_cores(host_data[0], n_bins)
     print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
@@ -386,6 +474,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="print the histogram-kernel sweep table instead")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand: start the N ranks (one per GPU) the way the driver does
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
     if args.sweep:
         run_sweep(args)
     elif args.impl == "reference":

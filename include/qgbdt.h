@@ -208,8 +208,9 @@ int qgbdt_get_counters(const qgbdt_ctx *ctx, int64_t *kernel_launches, int64_t *
 /* Measurement aid (no counterpart in the paper): when enabled, every histogram build is
  * bracketed by a pair of CUDA events on its stream.  qgbdt_get_histogram_profile() waits for
  * them and returns the summed kernel time, the algorithmic bytes of those builds
- * (rows * (features + gradient-code bytes [+ 4 for a row list]) + features * bins * 8) and
- * their number, then clears the record. */
+ * (rows * (features + gradient-code bytes [+ 4 for a row list]) + features * bins * 8, with one
+ * byte of packed gradient + hessian code per row up to 4 bits and two beyond) and their number,
+ * then clears the record. */
 int qgbdt_profile_histograms(qgbdt_ctx *ctx, int32_t enable);
 int qgbdt_get_histogram_profile(qgbdt_ctx *ctx, double *total_ms, int64_t *total_bytes, int64_t *builds);
 

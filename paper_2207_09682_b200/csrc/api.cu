@@ -183,7 +183,7 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     c->N = n_rows;
     c->F = n_features;
     c->nb = n_bins;
-    c->code_bytes = 2;
+    c->code_bytes = c->prm.bits <= 4 ? 1 : 2;   // packed gradient + hessian code of a row that the method has to move (Sec. 6.2)
     plan_tiles(n_features, c->tiles);
     plan_hist_ctas(c->sm_count, c->tiles, c->hist_grid, c->max_parts);
     int rc;

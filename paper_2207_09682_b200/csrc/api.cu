@@ -62,13 +62,16 @@ void free_data(qgbdt_ctx *c) {
     dev_free(c->d_h);
     dev_free(c->d_hist_pool);
     dev_free(c->d_leaves);
+    dev_free(c->d_recs);
+    dev_free(c->d_front);
+    dev_free(c->d_grow_bits);
+    dev_free(c->d_grow_partial);
     dev_free(c->d_ent0);
     dev_free(c->d_ent1);
     dev_free(c->d_cand);
     dev_free(c->d_feat_rec);
     dev_free(c->d_colmajor);
     c->col_stride = 0;
-    dev_free(c->d_leaf_gain);
     dev_free(c->d_m_num_leaves);
     dev_free(c->d_m_feature);
     dev_free(c->d_m_bin);
@@ -203,10 +206,18 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     if ((rc = dev_alloc(c, &c->d_codes_nat, (size_t)n_rows * 2 + 16)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx, (size_t)n_rows)) != QGBDT_OK) return rc;
     if ((rc = dev_alloc(c, &c->d_idx_tmp, (size_t)n_rows)) != QGBDT_OK) return rc;
-    if ((rc = dev_alloc(c, &c->d_part_counts, (size_t)n_rows / 2048 + 8 + (size_t)c->sm_count * 40)) != QGBDT_OK) return rc;
+    // block counts of the step-wise partition (a block per 2048 rows), or the warp and block counts
+    // of the partition launches of tree growth (nine words per block)
+    c->grow_pb_total = c->sm_count * 4 + GROW_MAX_JOBS;
+    {
+        size_t need = (size_t)n_rows / 2048 + 8, grow = (size_t)c->grow_pb_total * 9 + 8;
+        if ((rc = dev_alloc(c, &c->d_part_counts, need > grow ? need : grow)) != QGBDT_OK) return rc;
+    }
     {
         std::vector<FeatRec> fr((size_t)n_features);
-        for (const TileDesc &t : c->tiles)
+        int tile_no = -1;
+        for (const TileDesc &t : c->tiles) {
+            ++tile_no;
             for (int f = t.f0; f < t.f0 + t.nf; ++f) {
                 const int fl = f - t.f0;
                 fr[f].col = t.data + (fl >> 2);
@@ -215,9 +226,10 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
                 fr[f].cta0 = t.cta0;
                 fr[f].parts = t.parts;
                 fr[f].fl = fl;
-                fr[f].pad = 0;
+                fr[f].tile = tile_no;
                 fr[f].col8 = nullptr;
             }
+        }
         if ((rc = dev_alloc(c, &c->d_feat_rec, (size_t)n_features)) != QGBDT_OK) return rc;
         QG_CUDA(c, cudaMemcpy(c->d_feat_rec, fr.data(), sizeof(FeatRec) * fr.size(), cudaMemcpyHostToDevice));
     }
@@ -281,7 +293,7 @@ int qgbdt_create(qgbdt_ctx **out, const qgbdt_params *p) {
     bool ok = cudaMalloc(reinterpret_cast<void **>(&c->d_state), sizeof(DevState)) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_split_out), sizeof(SplitRec) * 4) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_sums), sizeof(long long) * 2 * L) == cudaSuccess &&
-              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_table), sizeof(uint32_t) * 3 * L) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_table), sizeof(uint32_t) * 7 * qg_leaf_table_slots(L)) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_value), sizeof(float) * L) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_w), sizeof(double) * L) == cudaSuccess &&
               cudaMallocHost(&c->h_pinned, PINNED_BYTES) == cudaSuccess;

@@ -1,19 +1,27 @@
-// Leaf-wise (best-first) growth of one tree (Sec. 3) with every decision taken on the device:
-// the host enqueues a fixed sequence of kernels per split and never waits for a result.
+// Leaf-wise (best-first) growth of one tree (Sec. 3) with every decision taken on the device.
 //
-// Per split: (1) k_grow_flags: one predicate bit per row of the leaf being split and the number
-// of left rows per warp range; (2) k_grow_scatter: stable scatter of the (row, gradient code)
-// pairs into the other pair buffer (left rows first); (3) the histogram kernel on the smaller child's rows
-// (Algorithm 1); (4) k_grow_finish: per feature, the smaller child's histogram from the partial
-// histograms, the larger child's as parent minus smaller, both children's best splits (Eq. 7);
-// the last block to finish records the split in the tree, creates the leaf records and picks
-// the leaf with the largest gain for the next split.
+// A tree grows in passes, several leaves per pass (the batch rule and the commit step that keeps
+// the result equal to best-first growth are described with the structures in the internal header).
+// Per pass, for all leaves of the batch at once:
+//   (1) k_grow_flags    one predicate bit per row of a leaf being split, left rows per warp range;
+//   (2) k_grow_scatter  stable scatter of the (row, gradient code) pairs into the other pair buffer
+//                       (left rows first);
+//   (3) the histogram kernel on the smaller child's rows (Algorithm 1);
+//   (4) k_grow_finish   per feature: the smaller child's histogram from the partial histograms, the
+//                       larger child's as parent minus smaller, both children's best splits (Eq. 7);
+//                       the last block of a leaf writes the children's growth records;
+//   (5) k_grow_commit   replays the best-first order over the leaves split so far (numbers the
+//                       children, records the nodes), then picks the next batch and plans its launches.
+// The passes of a tree are the body of a conditional (while) node of a CUDA graph: the commit kernel
+// clears the node's condition when the tree is full or no leaf can be split, so the host enqueues one
+// graph launch per tree and never waits for a result.
 #include "split_scan.cuh"
 
 namespace {
 
 constexpr int PART_THREADS = 256;
 constexpr int PART_WARPS = PART_THREADS / 32;
+constexpr int COMMIT_THREADS = 256;
 constexpr uint32_t MIN_ROWS_PER_CTA = 1024;   // same rule as the histogram kernel
 
 __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
@@ -24,42 +32,59 @@ __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) 
 
 struct GrowArgs {
     GrowState *gs;
+    NodeRec *recs;
     LeafRec *leaves;
-    const DevState *state;
+    int32_t *front;                  // [L] growth record of every numbered leaf
+    DevState *state;
     const FeatRec *feat_rec;         // [F]
-    double *leaf_gain;               // [L] gain of every leaf's best split, -inf when it has none
     uint32_t N;
     uint2 *ent0, *ent1;              // the two (row, gradient code) pair buffers
     const uint16_t *codes_nat;       // codes in row order (the root's identity list has no pairs yet)
-    uint32_t *bits, *counts;         // predicate bits of the leaf being split, left rows per warp range
-    int n_count;                     // warp ranges (= warps of the flag / scatter grids)
-    unsigned long long *pool;        // [L][F][nb]
+    uint32_t *bits;                  // [jobs][bits_stride] predicate bits of the leaves being split
+    size_t bits_stride;
+    uint32_t *counts;                // [pb_total * PART_WARPS] left rows per warp range, then [pb_total] per block
+    int pb_total;                    // blocks of a partition launch
+    unsigned long long *pool;        // [slots][F][nb]
     const unsigned long long *partial;
-    SplitRec *cand;                  // [F][2] best candidates of every feature for the two children
+    SplitRec *cand;                  // [jobs][F][2] best candidates of every feature for the two children
     int F, nb, L;
+    int K;                           // leaves per pass
+    int xcap, parts_cap, n_tiles;    // histogram CTAs per tile of a launch, of one leaf; tiles
+    int max_recs, max_slots;         // growth records and histogram slots allocated
     SplitParams sp;                  // G, H, n_s are filled per leaf on the device
-    // tree output (device arrays of the current tree)
+    // tree output (device arrays of the current train call)
     int32_t *m_feature, *m_bin, *m_left, *m_right;
     double *m_gain;
+    cudaGraphConditionalHandle cond; // condition of the graph's while node
+    int use_cond;                    // 0: launched on a stream, the host reads gs->done
 };
 
-__global__ void k_grow_begin(GrowState *gs, LeafRec *leaves, const DevState *state, uint32_t N, int tree_slot) {
+__global__ void k_grow_begin(GrowState *gs, NodeRec *recs, LeafRec *leaves, int32_t *front, const DevState *state,
+                             uint32_t N, int tree_slot) {
     gs->tree_slot = tree_slot;
-    LeafRec r;
+    NodeRec r;
     r.off = 0; r.n = N; r.buf = -1; r.slot = 0;
     r.G = state->tot_g; r.H = state->tot_h;
     r.best = qg_invalid_rec();
+    r.state = 0; r.child0 = -1; r.nl = 0;
     r.parent_node = -1; r.parent_side = 0;
-    leaves[0] = r;
+    recs[0] = r;
+    LeafRec l;
+    l.off = 0; l.n = N; l.buf = -1; l.rec = 0;
+    leaves[0] = l;
+    front[0] = 0;
     gs->n_leaves = 1;
-    // gradients out of domain (the flag is sticky over the trees of a train call): the split
-    // kernels of this tree return at once, the call reports the error when it ends
+    gs->n_exec = 0;
+    gs->n_recs = 1;
+    gs->n_jobs = 0;
+    // gradients out of domain (the flag is sticky over the trees of a train call): this tree stays
+    // a single leaf, the call reports the error when it ends
     gs->done = state->bad_value ? 1 : 0;
-    gs->finish_count = 0;
+    for (int j = 0; j < GROW_MAX_JOBS; ++j) gs->jobs[j].finish_count = 0;
 }
 
 // Words of 32 rows [w0, w1) of warp gw: every warp takes the same number of consecutive words
-// (at least 4), so the warps with work are a prefix [0, active) of the grid.
+// (at least 4), so the warps with work are a prefix [0, active) of the leaf's warps.
 __device__ inline void warp_range(uint32_t nw, uint32_t gw, uint32_t n_count, uint32_t &w0, uint32_t &w1,
                                   uint32_t &active) {
     uint32_t per = (nw + n_count - 1) / n_count;
@@ -69,24 +94,46 @@ __device__ inline void warp_range(uint32_t nw, uint32_t gw, uint32_t n_count, ui
     w1 = w0 + per < nw ? w0 + per : nw;
 }
 
+// The job whose block range [pb0, pb0 + pb) holds block b, or -1.
+__device__ inline int job_of_block(const GrowState *gs, int n_jobs, int b) {
+    int p0[GROW_MAX_JOBS], pn[GROW_MAX_JOBS];
+#pragma unroll
+    for (int i = 0; i < GROW_MAX_JOBS; ++i) {
+        p0[i] = gs->jobs[i].pb0;
+        pn[i] = gs->jobs[i].pb;
+    }
+    int j = -1;
+#pragma unroll
+    for (int i = 0; i < GROW_MAX_JOBS; ++i)
+        if (i < n_jobs && b >= p0[i] && b < p0[i] + pn[i]) j = i;
+    return j;
+}
+
 // Four words of 32 rows at a time, so that the dependent loads (pair -> bin word) of the four are
 // in flight together.
 __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
     const GrowState *gs = a.gs;
-    // every field at once (one round trip to memory), then the early exits
-    const int done = gs->done, buf = gs->buf;
-    const uint32_t n = gs->n, off = gs->off;
-    const uint32_t *col = gs->col;
-    const uint8_t *col8 = gs->col8;
-    const int logW = gs->logW, shift = 8 * gs->byte;
-    const uint32_t thr = (uint32_t)gs->bin;
-    if (done) return;
+    const int done = gs->done, n_jobs = gs->n_jobs;
+    const int j = job_of_block(gs, n_jobs, (int)blockIdx.x);
+    if (done || j < 0) return;
+    const GrowJob *job = gs->jobs + j;
+    // every field at once (one round trip to memory)
+    const int buf = job->buf, pb0 = job->pb0, pb = job->pb;
+    const uint32_t n = job->n, off = job->off;
+    const uint32_t *col = job->col;
+    const uint8_t *col8 = job->col8;
+    const int logW = job->logW, shift = 8 * job->byte;
+    const uint32_t thr = (uint32_t)job->bin;
     const int lane = threadIdx.x & 31;
-    const uint32_t gw = blockIdx.x * PART_WARPS + (threadIdx.x >> 5);
+    const uint32_t lb = blockIdx.x - (uint32_t)pb0;                      // block inside the job
+    const uint32_t gw = lb * PART_WARPS + (threadIdx.x >> 5);
     const uint32_t nw = (n + 31) >> 5;
     uint32_t w0, w1, active;
-    warp_range(nw, gw, (uint32_t)a.n_count, w0, w1, active);
-    if (blockIdx.x * PART_WARPS >= active) return;   // no warp of this block has work
+    warp_range(nw, gw, (uint32_t)pb * PART_WARPS, w0, w1, active);
+    uint32_t *bits = a.bits + (size_t)j * a.bits_stride;
+    uint32_t *wcounts = a.counts + (size_t)pb0 * PART_WARPS;
+    uint32_t *bcounts = a.counts + (size_t)a.pb_total * PART_WARPS + pb0;
+    if (lb * PART_WARPS >= active) return;                               // no warp of this block has work
     const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
     uint32_t lefts = 0;
     for (uint32_t w = w0; w < w1; w += 4) {
@@ -110,7 +157,7 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
             const bool left = row[k] != 0xFFFFFFFFu && ((word[k] >> shift) & 0xFFu) <= thr;
             const uint32_t b = __ballot_sync(0xffffffffu, left);
             if (w + k < w1) {
-                if (lane == 0) a.bits[w + k] = b;
+                if (lane == 0) bits[w + k] = b;
                 lefts += __popc(b);
             }
         }
@@ -119,7 +166,7 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
     // blocks before its own and the warps before it inside its block)
     __shared__ uint32_t block_lefts[PART_WARPS];
     if (lane == 0) {
-        a.counts[gw] = lefts;
+        wcounts[gw] = lefts;
         block_lefts[threadIdx.x >> 5] = lefts;
     }
     __syncthreads();
@@ -127,48 +174,54 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
         uint32_t t = 0;
 #pragma unroll
         for (int v = 0; v < PART_WARPS; ++v) t += block_lefts[v];
-        a.counts[a.n_count + blockIdx.x] = t;
+        bcounts[lb] = t;
     }
 }
 
 __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
     GrowState *gs = a.gs;
-    const int done = gs->done, buf = gs->buf;   // every field at once, then the early exits
-    const uint32_t n = gs->n, off = gs->off;
-    if (done) return;
+    const int done = gs->done, n_jobs = gs->n_jobs;
+    const int j = job_of_block(gs, n_jobs, (int)blockIdx.x);
+    if (done || j < 0) return;
+    GrowJob *job = gs->jobs + j;
+    const int buf = job->buf, pb0 = job->pb0, pb = job->pb;   // every field at once
+    const uint32_t n = job->n, off = job->off;
     const int lane = threadIdx.x & 31;
-    const uint32_t gw = blockIdx.x * PART_WARPS + (threadIdx.x >> 5);
+    const uint32_t lb = blockIdx.x - (uint32_t)pb0;
+    const uint32_t gw = lb * PART_WARPS + (threadIdx.x >> 5);
     const uint32_t nw = (n + 31) >> 5;
     uint32_t w0, w1, active;
-    warp_range(nw, gw, (uint32_t)a.n_count, w0, w1, active);
+    warp_range(nw, gw, (uint32_t)pb * PART_WARPS, w0, w1, active);
     if (gw >= active && gw != 0) return;
+    const uint32_t *bits = a.bits + (size_t)j * a.bits_stride;
+    const uint32_t *wcounts = a.counts + (size_t)pb0 * PART_WARPS;
+    const uint32_t *block_counts = a.counts + (size_t)a.pb_total * PART_WARPS + pb0;
     // left rows before this warp's range, and in the whole leaf: the totals of the blocks, and
     // the warps of this block before this one
     uint32_t before = 0, total = 0;
     const uint32_t active_blocks = (active + PART_WARPS - 1) / PART_WARPS;
-    const uint32_t *block_counts = a.counts + a.n_count;
     for (uint32_t j0 = 0; j0 < active_blocks; j0 += 256) {   // eight independent loads per lane in flight
         uint32_t v[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            const uint32_t j = j0 + 32 * k + lane;
-            v[k] = j < active_blocks ? block_counts[j] : 0u;
+            const uint32_t jj = j0 + 32 * k + lane;
+            v[k] = jj < active_blocks ? block_counts[jj] : 0u;
         }
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             total += v[k];
-            if (j0 + 32 * k + lane < blockIdx.x) before += v[k];
+            if (j0 + 32 * k + lane < lb) before += v[k];
         }
     }
     {
-        const uint32_t j = blockIdx.x * PART_WARPS + lane;
-        if (lane < PART_WARPS && j < gw) before += a.counts[j];
+        const uint32_t jj = lb * PART_WARPS + lane;
+        if (lane < PART_WARPS && jj < gw && jj < active) before += wcounts[jj];
     }
     for (int o = 16; o > 0; o >>= 1) {
         before += __shfl_xor_sync(0xffffffffu, before, o);
         total += __shfl_xor_sync(0xffffffffu, total, o);
     }
-    if (gw == 0 && lane == 0) gs->nl = total;
+    if (gw == 0 && lane == 0) job->nl = total;
     const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
     uint2 *dst = buf == 0 ? a.ent1 : a.ent0;
     for (uint32_t w = w0; w < w1; w += 4) {
@@ -177,7 +230,7 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const uint32_t e = ((w + k) << 5) + lane;
-            bw[k] = w + k < w1 ? a.bits[w + k] : 0u;
+            bw[k] = w + k < w1 ? bits[w + k] : 0u;
             if (w + k < w1 && e < n) {
                 if (src) {
                     ent[k] = src[off + e];
@@ -224,24 +277,28 @@ __device__ inline SplitRec shfl_xor_rec(const SplitRec &r, int o) {
     return x;
 }
 
-// ROOT: scans the root histogram (pool slot 0).  Otherwise: completes the split recorded in the
-// grow state.  One block per feature.
+// ROOT: scans the root histogram (pool slot 0), grid (F).  Otherwise: completes the splits of the
+// current pass, grid (F, leaves per pass).  One block per feature (and leaf).
 // BPT bins per thread: 1 (256 threads) or 2 (128 threads: with thousands of features twice as many
-// blocks are resident, and the grid fits the SMs in one wave).
+// blocks are resident).
 template <bool ROOT, int BPT>
 __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     constexpr int FIN_WARPS = 8 / BPT;
     GrowState *gs = a.gs;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int f = blockIdx.x;   // one block per feature
+    const int f = blockIdx.x;                 // one block per feature
+    const int j = ROOT ? 0 : (int)blockIdx.y; // and leaf being split
+    GrowJob *job = gs->jobs + j;
     // everything the block needs from the state, at once (one round trip to memory), then the early exit
-    const int done = gs->done, n_leaves = gs->n_leaves, parent_slot = ROOT ? 0 : gs->parent_slot;
-    const uint32_t gs_n = gs->n, gs_nl = gs->nl;
-    const long long gs_gl = gs->gl, gs_hl = gs->hl, gs_PG = gs->PG, gs_PH = gs->PH;
+    const int done = gs->done, n_jobs = gs->n_jobs;
+    const int parent_slot = ROOT ? 0 : job->parent_slot, small_slot = ROOT ? 0 : job->small_slot;
+    const int parts = job->parts, slot0 = job->slot0, child0 = job->child0, jrec = job->rec, jbuf = job->buf;
+    const uint32_t gs_n = job->n, gs_nl = job->nl, gs_off = job->off;
+    const long long gs_gl = job->gl, gs_hl = job->hl, gs_PG = job->PG, gs_PH = job->PH;
     const long long tot_g = a.state->tot_g, tot_h = a.state->tot_h;
     const uint32_t gmax_bits = a.state->gmax_bits, hmax_bits = a.state->hmax_bits;
     const FeatRec fr = a.feat_rec[f];
-    if (done) return;
+    if (done || (!ROOT && j >= n_jobs)) return;
     const size_t hw = (size_t)a.F * a.nb;
 
     // the two children: "small" was built by Algorithm 1, "large" is parent - small
@@ -265,10 +322,11 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
     const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
     const int fl = fr.fl, W = 1 << fr.logW;
-    const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)fr.parts, (uint32_t)pS.n_s);
+    const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)parts, (uint32_t)pS.n_s);
     const size_t pstride = (size_t)4 * a.nb * 32;
-    const unsigned long long *part = a.partial + (size_t)fr.cta0 * pstride + (size_t)(fl & 3) * a.nb * W + (fl >> 2);
-    unsigned long long *S = a.pool + (ROOT ? 0 : (size_t)n_leaves * hw) + (size_t)f * a.nb;
+    const unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
+                                     (size_t)(fl & 3) * a.nb * W + (fl >> 2);
+    unsigned long long *S = a.pool + (size_t)small_slot * hw + (size_t)f * a.nb;
     unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)parent_slot * hw + (size_t)f * a.nb;
     __shared__ long long wtot[4][FIN_WARPS];
     SplitRec rS = qg_invalid_rec(), rL = qg_invalid_rec();
@@ -334,11 +392,11 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
         {
             unsigned long long pv[BPT];
 #pragma unroll
-            for (int j = 0; j < BPT; ++j) {
-                const int b = (int)threadIdx.x * BPT + j;
-                sv[j] = 0; lv[j] = 0; pv[j] = 0;
+            for (int jb = 0; jb < BPT; ++jb) {
+                const int b = (int)threadIdx.x * BPT + jb;
+                sv[jb] = 0; lv[jb] = 0; pv[jb] = 0;
                 if (b < a.nb) {
-                    if (!ROOT) pv[j] = Pp[b];
+                    if (!ROOT) pv[jb] = Pp[b];
                     if (!ROOT && P > 1) {
                         const unsigned long long *q = part + (size_t)b * W;
                         for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
@@ -346,20 +404,20 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
 #pragma unroll
                             for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
 #pragma unroll
-                            for (int k = 0; k < 16; ++k) sv[j] += x[k];
+                            for (int k = 0; k < 16; ++k) sv[jb] += x[k];
                         }
                     } else {
-                        sv[j] = S[b];
+                        sv[jb] = S[b];
                     }
                 }
             }
 #pragma unroll
-            for (int j = 0; j < BPT; ++j) {
-                const int b = (int)threadIdx.x * BPT + j;
+            for (int jb = 0; jb < BPT; ++jb) {
+                const int b = (int)threadIdx.x * BPT + jb;
                 if (!ROOT && b < a.nb) {
-                    if (P > 1) S[b] = sv[j];
-                    lv[j] = pv[j] - sv[j];   // no field borrows: every child sum is at most the parent's
-                    Pp[b] = lv[j];
+                    if (P > 1) S[b] = sv[jb];
+                    lv[jb] = pv[jb] - sv[jb];   // no field borrows: every child sum is at most the parent's
+                    Pp[b] = lv[jb];
                 }
             }
         }
@@ -368,14 +426,14 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
         //      own bins for both children
         long long x[BPT][4], v[4] = {0, 0, 0, 0};   // per bin; v: inclusive sum up to the thread's last bin
 #pragma unroll
-        for (int j = 0; j < BPT; ++j) {
-            const bool in = (int)threadIdx.x * BPT + j < a.nb - 1;   // thresholds 0 .. nb-2
-            x[j][0] = in ? (long long)(int)(sv[j] >> 32) : 0;
-            x[j][1] = in ? (long long)(unsigned int)(sv[j] & 0xFFFFFFFFull) : 0;
-            x[j][2] = in ? (long long)(int)(lv[j] >> 32) : 0;
-            x[j][3] = in ? (long long)(unsigned int)(lv[j] & 0xFFFFFFFFull) : 0;
+        for (int jb = 0; jb < BPT; ++jb) {
+            const bool in = (int)threadIdx.x * BPT + jb < a.nb - 1;   // thresholds 0 .. nb-2
+            x[jb][0] = in ? (long long)(int)(sv[jb] >> 32) : 0;
+            x[jb][1] = in ? (long long)(unsigned int)(sv[jb] & 0xFFFFFFFFull) : 0;
+            x[jb][2] = in ? (long long)(int)(lv[jb] >> 32) : 0;
+            x[jb][3] = in ? (long long)(unsigned int)(lv[jb] & 0xFFFFFFFFull) : 0;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) v[c] += x[j][c];
+            for (int c = 0; c < 4; ++c) v[c] += x[jb][c];
         }
 #pragma unroll
         for (int c = 0; c < (ROOT ? 2 : 4); ++c) {
@@ -391,8 +449,8 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
             for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
         // thresholds from the thread's last bin down (the lower bin wins on equal gain)
 #pragma unroll
-        for (int j = BPT - 1; j >= 0; --j) {
-            const int b = (int)threadIdx.x * BPT + j;
+        for (int jb = BPT - 1; jb >= 0; --jb) {
+            const int b = (int)threadIdx.x * BPT + jb;
             if (b < a.nb - 1) {
                 double gain;
                 if (qg_eval_candidate(v[0], v[1], pS, dg, dh, tpS, gain) &&
@@ -405,7 +463,7 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
                 }
             }
 #pragma unroll
-            for (int c = 0; c < 4; ++c) v[c] -= x[j][c];
+            for (int c = 0; c < 4; ++c) v[c] -= x[jb][c];
         }
     }
     // best threshold of the feature: largest gain, lowest bin on equal gain
@@ -421,36 +479,27 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     }
     if (lane == 0) { sm[0][warp] = rS; sm[1][warp] = rL; }
     __syncthreads();
+    SplitRec *cand = a.cand + (size_t)j * a.F * 2;
     if (threadIdx.x < 2) {
         SplitRec r = sm[threadIdx.x][0];
         for (int w = 1; w < FIN_WARPS; ++w) {
             const SplitRec o = sm[threadIdx.x][w];
             if (qg_better(o.valid != 0, o.gain, o.bin, r.valid != 0, r.gain, r.bin)) r = o;
         }
-        a.cand[2 * f + threadIdx.x] = r;
+        cand[2 * f + threadIdx.x] = r;
         __threadfence();
     }
     __syncthreads();
-    if (threadIdx.x == 0) is_last = atomicAdd(&gs->finish_count, 1u) == gridDim.x - 1;
+    if (threadIdx.x == 0) is_last = atomicAdd(&job->finish_count, 1u) == gridDim.x - 1;
     __syncthreads();
     if (!is_last) return;
     __threadfence();
 
-    // ---- the last block: best candidates over all features, the new leaves, the next pick.
-    //      Every thread ends up with the same reduced values (warp shuffles, then the eight warp
-    //      results from shared memory), so thread 0 needs no further round of barriers.
-    const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
-    const int leaves_now = ROOT ? 1 : n_leaves + 1;
-    // gains of the older leaves, fetched while the candidates are being reduced
-    double my_gain[4];
-#pragma unroll
-    for (int k2 = 0; k2 < 4; ++k2) {
-        const int i2 = (int)threadIdx.x + k2 * FIN_WARPS * 32;
-        my_gain[k2] = i2 < leaves_now ? __ldcg(a.leaf_gain + i2) : NEG;
-    }
+    // ---- the last block of this leaf: best candidates over all features, then the growth records
+    //      of the two children (ROOT: the root's best split)
     SplitRec bS = qg_invalid_rec(), bL = qg_invalid_rec();
     for (int i2 = threadIdx.x; i2 < (int)gridDim.x; i2 += FIN_WARPS * 32) {
-        const SplitRec x = load_rec_cg(a.cand + 2 * i2), y = load_rec_cg(a.cand + 2 * i2 + 1);
+        const SplitRec x = load_rec_cg(cand + 2 * i2), y = load_rec_cg(cand + 2 * i2 + 1);
         if (qg_rec_better(x, bS)) bS = x;
         if (qg_rec_better(y, bL)) bL = y;
     }
@@ -461,168 +510,360 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     }
     if (lane == 0) { sm[0][warp] = bS; sm[1][warp] = bL; }
     __syncthreads();
+    if (threadIdx.x != 0) return;
     bS = sm[0][0];
     bL = sm[1][0];
     for (int w = 1; w < FIN_WARPS; ++w) {
         if (qg_rec_better(sm[0][w], bS)) bS = sm[0][w];
         if (qg_rec_better(sm[1][w], bL)) bL = sm[1][w];
     }
-    // where the winning features live (needed if one of the new leaves is picked next)
-    FeatRec fS = {}, fL = {};
-    if (threadIdx.x == 0) {
-        if (bS.valid) fS = a.feat_rec[bS.feature];
-        if (!ROOT && bL.valid) fL = a.feat_rec[bL.feature];
-    }
-    // the leaves this split made (ROOT: only the root) and their gains
-    const int id0 = ROOT ? 0 : gs->pick, id1 = ROOT ? -1 : n_leaves;
-    const SplitRec best0 = ROOT ? bS : (small_is_left ? bS : bL);   // of leaf id0 (the left child)
-    const SplitRec best1 = small_is_left ? bL : bS;                 // of leaf id1 (the right child)
-    const double gain0 = best0.valid ? best0.gain : NEG, gain1 = best1.valid ? best1.gain : NEG;
-
-    // the next leaf to split: largest gain, lowest leaf number on equal gain
-    __shared__ double pg[FIN_WARPS];
-    __shared__ int pi[FIN_WARPS];
-    double bg = NEG;
-    int bi = -1;
-    if (leaves_now < a.L) {
-#pragma unroll
-        for (int k2 = 0; k2 < 4; ++k2) {
-            const int i2 = (int)threadIdx.x + k2 * FIN_WARPS * 32;
-            if (i2 < leaves_now) {
-                double g = my_gain[k2];
-                if (i2 == id0) g = gain0;
-                if (i2 == id1) g = gain1;
-                if (g > bg) { bg = g; bi = i2; }
-            }
-        }
-        for (int i2 = (int)threadIdx.x + 4 * FIN_WARPS * 32; i2 < leaves_now; i2 += FIN_WARPS * 32) {   // more than 1024 leaves
-            double g = __ldcg(a.leaf_gain + i2);
-            if (i2 == id0) g = gain0;
-            if (i2 == id1) g = gain1;
-            if (g > bg) { bg = g; bi = i2; }
-        }
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        const double og = __shfl_xor_sync(0xffffffffu, bg, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (oi >= 0 && (bi < 0 || og > bg || (og == bg && oi < bi))) { bg = og; bi = oi; }
-    }
-    if (lane == 0) { pg[warp] = bg; pi[warp] = bi; }
-    __syncthreads();
-    if (threadIdx.x != 0) return;
-    bg = pg[0];
-    bi = pi[0];
-    for (int w = 1; w < FIN_WARPS; ++w) {
-        const double og = pg[w];
-        const int oi = pi[w];
-        if (oi >= 0 && (bi < 0 || og > bg || (og == bg && oi < bi))) { bg = og; bi = oi; }
-    }
-    const int pick = bi;
-
-    LeafRec lf, rt;   // ROOT: lf is the root
+    job->finish_count = 0;
     if (ROOT) {
-        lf.off = 0; lf.n = a.N; lf.buf = -1; lf.slot = 0; lf.G = pS.G; lf.H = pS.H; lf.best = bS;
-        lf.parent_node = -1; lf.parent_side = 0;
-        a.leaves[0] = lf;
-        a.leaf_gain[0] = gain0;
-        rt = lf;
-        gs->n_leaves = 1;
-    } else {
-        const int right = n_leaves, node = n_leaves - 1;
-        // node arrays of the tree being grown (the slot is device state: the launch arguments
-        // are the same for every tree, so the launches can be replayed from a CUDA graph)
-        const size_t no = (size_t)gs->tree_slot * (a.L > 1 ? a.L - 1 : 1);
-        const int pn = gs->parent_node;
-        a.m_feature[no + node] = gs->feature;
-        a.m_bin[no + node] = gs->bin;
-        a.m_left[no + node] = ~id0;
-        a.m_right[no + node] = ~right;
-        a.m_gain[no + node] = gs->gain;
-        if (pn >= 0) {
-            if (gs->parent_side == 0) a.m_left[no + pn] = node;
-            else a.m_right[no + pn] = node;
-        }
-        const int dstbuf = gs->buf == 0 ? 1 : 0;
-        lf.off = gs->off; lf.n = nl; lf.buf = dstbuf;
-        lf.G = gs->gl; lf.H = gs->hl;
-        lf.parent_node = node; lf.parent_side = 0;
-        rt.off = gs->off + nl; rt.n = nr; rt.buf = dstbuf;
-        rt.G = gs->PG - gs->gl; rt.H = gs->PH - gs->hl;
-        rt.parent_node = node; rt.parent_side = 1;
-        lf.slot = small_is_left ? n_leaves : gs->parent_slot;
-        rt.slot = small_is_left ? gs->parent_slot : n_leaves;
-        lf.best = best0;
-        rt.best = best1;
-        a.leaves[id0] = lf;
-        a.leaves[right] = rt;
-        a.leaf_gain[id0] = gain0;
-        a.leaf_gain[right] = gain1;
-        gs->n_leaves = n_leaves + 1;
-        gs->hist_rows += small_is_left ? nl : nr;
-        gs->hist_builds += 1;
-    }
-    gs->finish_count = 0;
-    if (pick < 0) {
-        gs->done = 1;
+        a.recs[0].best = bS;
         return;
     }
-    LeafRec lr;
-    FeatRec pf;
-    if (pick == id0) {
-        lr = lf;
-        pf = ROOT || small_is_left ? fS : fL;
-    } else if (pick == id1) {
-        lr = rt;
-        pf = small_is_left ? fL : fS;
-    } else {
-        lr = a.leaves[pick];
-        pf = a.feat_rec[lr.best.feature];
-    }
-    gs->pick = pick;
-    gs->feature = lr.best.feature;
-    gs->bin = lr.best.bin;
-    gs->col = pf.col;
-    gs->col8 = pf.col8;
-    gs->logW = pf.logW;
-    gs->byte = pf.byte;
-    gs->off = lr.off;
-    gs->n = lr.n;
-    gs->buf = lr.buf;
-    gs->gl = lr.best.gl;
-    gs->hl = lr.best.hl;
-    gs->PG = lr.G;
-    gs->PH = lr.H;
-    gs->gain = lr.best.gain;
-    gs->parent_slot = lr.slot;
-    gs->parent_node = lr.parent_node;
-    gs->parent_side = lr.parent_side;
+    const int dstbuf = jbuf == 0 ? 1 : 0;
+    NodeRec lf, rt;
+    lf.off = gs_off; lf.n = nl; lf.buf = dstbuf;
+    lf.G = gs_gl; lf.H = gs_hl;
+    rt.off = gs_off + nl; rt.n = nr; rt.buf = dstbuf;
+    rt.G = gs_PG - gs_gl; rt.H = gs_PH - gs_hl;
+    lf.slot = small_is_left ? small_slot : parent_slot;
+    rt.slot = small_is_left ? parent_slot : small_slot;
+    lf.best = small_is_left ? bS : bL;
+    rt.best = small_is_left ? bL : bS;
+    lf.state = rt.state = 0;
+    lf.child0 = rt.child0 = -1;
+    lf.nl = rt.nl = 0;
+    lf.parent_node = rt.parent_node = -1;
+    lf.parent_side = 0; rt.parent_side = 1;
+    a.recs[child0] = lf;
+    a.recs[child0 + 1] = rt;
+    a.recs[jrec].nl = nl;
 }
 
-}  // namespace
+// Shared memory of the commit kernel: per numbered leaf its gain, its growth record and the list
+// of splits confirmed in this launch; per growth record its gain, its children (or -1) and its
+// place in the tree.
+__host__ __device__ inline size_t commit_smem_bytes(int L, int max_recs) {
+    return (size_t)L * (sizeof(double) + 3 * sizeof(int)) + (size_t)max_recs * (sizeof(double) + 2 * sizeof(int)) + 16;
+}
 
-namespace {
+// Best of (gain, index) over a warp: larger gain, lower index on equal gain; index < 0: nothing.
+__device__ inline void warp_best(double &g, int &i) {
+    for (int o = 16; o > 0; o >>= 1) {
+        const double og = __shfl_xor_sync(0xffffffffu, g, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+        if (oi >= 0 && (i < 0 || og > g || (og == g && oi < i))) { g = og; i = oi; }
+    }
+}
 
-void fill_args(qgbdt_ctx *c, GrowArgs &a, int &part_blocks) {
+// One block.  (1) Replays best-first growth over what has been split so far: takes the numbered
+// leaf with the largest gain (lowest number on equal gain); if it has been split, numbers its
+// children (the left child keeps the number, the right child gets the next one), records the node
+// and goes on; stops at a leaf that has not been split yet, at a full tree, or when no leaf has an
+// admissible split.  (2) Picks the next batch: that leaf, then the unsplit leaves of largest gain
+// among all growth records.  (3) Fills the job table and shares out the blocks of the next launches.
+__global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    GrowState *gs = a.gs;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
+    if (gs->done) {
+        if (tid == 0) {
+            gs->n_jobs = 0;
+            if (a.use_cond) cudaGraphSetConditional(a.cond, 0);
+        }
+        return;
+    }
+    const int L = a.L, R = a.max_recs;
+    double *fg = reinterpret_cast<double *>(smem_raw);          // [L] gain of numbered leaf i
+    double *cg = fg + L;                                        // [R] gain of record r if it can still be split
+    int *sf = reinterpret_cast<int *>(cg + R);                  // [L] record of numbered leaf i
+    int *cl_rec = sf + L;                                       // [L] confirmed in this launch: the record split ...
+    int *cl_leaf = cl_rec + L;                                  // [L] ... and the number of the leaf it was
+    int *cs = cl_leaf + L;                                      // [R] first child record of a split record, else -1
+    int *spn = cs + R;                                          // [R] (node << 1 | side) of a numbered record's parent, -1: root
+    __shared__ int s_done, s_leaves, s_mand, s_commits;
+    __shared__ unsigned long long s_rows;
+    __shared__ double wg[COMMIT_THREADS / 32];
+    __shared__ int wi[COMMIT_THREADS / 32];
+    __shared__ int s_pick[GROW_MAX_JOBS];
+    __shared__ uint32_t s_n[GROW_MAX_JOBS];
+
+    const int n_leaves0 = gs->n_leaves, n_recs = gs->n_recs, n_exec = gs->n_exec, tree_slot = gs->tree_slot;
+    for (int r = tid; r < n_recs; r += COMMIT_THREADS) {
+        const NodeRec *q = a.recs + r;
+        const int st = q->state, c0 = q->child0, valid = q->best.valid, pn = q->parent_node, ps = q->parent_side;
+        const double g = q->best.gain;
+        cs[r] = st == 1 ? c0 : -1;
+        cg[r] = valid ? g : NEG;       // the gain of a leaf's best split, whether it has been split or not
+        spn[r] = pn < 0 ? -1 : (pn << 1 | ps);
+    }
+    for (int i = tid; i < n_leaves0; i += COMMIT_THREADS) sf[i] = a.front[i];
+    if (tid == 0) s_rows = 0;
+    __syncthreads();
+    for (int i = tid; i < n_leaves0; i += COMMIT_THREADS) fg[i] = cg[sf[i]];
+    __syncthreads();
+
+    // ---- (1) warp 0 replays the best-first order
+    if (warp == 0) {
+        int n_leaves = n_leaves0, mand = -1, done = 0, commits = 0;
+        const size_t no = (size_t)tree_slot * (L > 1 ? L - 1 : 1);
+        for (;;) {
+            if (n_leaves >= L) { done = 1; break; }
+            double bg = NEG;
+            int bi = -1;
+            for (int i = lane; i < n_leaves; i += 32) {
+                const double g = fg[i];
+                if (g > bg) { bg = g; bi = i; }
+            }
+            warp_best(bg, bi);
+            if (bi < 0) { done = 1; break; }
+            const int r = sf[bi], c0 = cs[r];
+            if (c0 < 0) { mand = r; break; }
+            const int node = n_leaves - 1, right = n_leaves;
+            if (lane == 0) {
+                a.m_left[no + node] = ~bi;
+                a.m_right[no + node] = ~right;
+                const int p = spn[r];
+                if (p >= 0) {
+                    if ((p & 1) == 0) a.m_left[no + (p >> 1)] = node;
+                    else a.m_right[no + (p >> 1)] = node;
+                }
+                spn[c0] = node << 1;
+                spn[c0 + 1] = node << 1 | 1;
+                sf[bi] = c0;
+                sf[right] = c0 + 1;
+                cl_rec[commits] = r;
+                cl_leaf[commits] = bi;
+            }
+            if (lane < 2) fg[lane == 0 ? bi : right] = cg[c0 + lane];   // gains of the two new numbered leaves
+            __syncwarp();
+            ++n_leaves;
+            ++commits;
+        }
+        if (lane == 0) { s_done = done; s_leaves = n_leaves; s_mand = mand; s_commits = commits; }
+    }
+    __syncthreads();
+    const int n_leaves = s_leaves, commits = s_commits, done = s_done, mand = s_mand;
+
+    // ---- the splits confirmed above, one thread each: node arrays, leaf records, tree positions
+    {
+        const size_t no = (size_t)tree_slot * (L > 1 ? L - 1 : 1);
+        unsigned long long rows = 0;
+        for (int t = tid; t < commits; t += COMMIT_THREADS) {
+            const int r = cl_rec[t], leaf = cl_leaf[t], node = n_leaves0 - 1 + t, right = node + 1;
+            const NodeRec *q = a.recs + r;
+            const int c0 = q->child0;
+            a.m_feature[no + node] = q->best.feature;
+            a.m_bin[no + node] = q->best.bin;
+            a.m_gain[no + node] = q->best.gain;
+            NodeRec *lc = a.recs + c0, *rc = lc + 1;
+            lc->parent_node = node; lc->parent_side = 0;
+            rc->parent_node = node; rc->parent_side = 1;
+            rows += lc->n < rc->n ? lc->n : rc->n;
+            (void)leaf; (void)right;
+        }
+        // leaf records: a leaf number may change hands more than once in a launch (a child that was
+        // split ahead is confirmed right after its parent), so they are written from the replay's
+        // final table, for the numbers whose record changed
+        for (int i = tid; i < n_leaves; i += COMMIT_THREADS) {
+            const int r = sf[i];
+            if (i >= n_leaves0 || a.front[i] != r) {
+                const NodeRec *q = a.recs + r;
+                LeafRec x;
+                x.off = q->off; x.n = q->n; x.buf = q->buf; x.rec = r;
+                a.leaves[i] = x;
+                a.front[i] = r;
+            }
+        }
+        if (rows) atomicAdd(&s_rows, rows);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        gs->n_leaves = n_leaves;
+        gs->hist_rows += s_rows;
+        gs->hist_builds += (unsigned long long)commits;
+        gs->passes += 1;
+    }
+    if (done) {
+        if (tid == 0) {
+            gs->done = 1;
+            gs->n_jobs = 0;
+            gs->extra_builds += (unsigned long long)(n_exec - (n_leaves - 1));   // split ahead, not used by this tree
+            if (a.use_cond) cudaGraphSetConditional(a.cond, 0);
+        }
+        return;
+    }
+
+    // ---- (2) the next batch: the leaf best-first growth needs next, then the unsplit leaves of
+    //      largest gain, as long as few enough leaves are split ahead of their confirmation and the
+    //      tree could still use them all
+    const int ahead = n_exec - (n_leaves - 1);            // split, not confirmed
+    const int room = (L - 1) - n_exec;                    // splits the tree can still use
+    int extra = a.K - 1;
+    if (extra > GROW_SLACK - ahead) extra = GROW_SLACK - ahead;
+    if (extra > room - 1) extra = room - 1;
+    if (extra > (R - n_recs) / 2 - 1) extra = (R - n_recs) / 2 - 1;
+    if (extra > a.max_slots - 2 - n_exec) extra = a.max_slots - 2 - n_exec;
+    if (extra < 0) extra = 0;
+    if ((R - n_recs) / 2 < 1 || a.max_slots - 1 - n_exec < 1) {
+        // cannot happen within the bounds above (records and slots are sized for num_leaves - 1 splits
+        // plus the slack): refuse rather than write out of bounds
+        if (tid == 0) {
+            atomicExch(&a.state->kernel_error, 1);
+            gs->done = 1;
+            gs->n_jobs = 0;
+            if (a.use_cond) cudaGraphSetConditional(a.cond, 0);
+        }
+        return;
+    }
+    if (tid == 0) {
+        s_pick[0] = mand;
+        cs[mand] = -2;
+    }
+    __syncthreads();
+    int n_jobs = 1;
+    for (int k = 1; k <= extra; ++k) {
+        double bg = NEG;
+        int bi = -1;
+        for (int r = tid; r < n_recs; r += COMMIT_THREADS) {
+            const double g = cs[r] == -1 ? cg[r] : NEG;   // not split and not in the batch yet
+            if (g > bg) { bg = g; bi = r; }
+        }
+        warp_best(bg, bi);
+        if (lane == 0) { wg[warp] = bg; wi[warp] = bi; }
+        __syncthreads();
+        bg = wg[0];
+        bi = wi[0];
+        for (int w = 1; w < COMMIT_THREADS / 32; ++w) {
+            const double og = wg[w];
+            const int oi = wi[w];
+            if (oi >= 0 && (bi < 0 || og > bg || (og == bg && oi < bi))) { bg = og; bi = oi; }
+        }
+        if (bi < 0) break;          // nothing left to split ahead (the same value in every thread)
+        if (tid == 0) {
+            s_pick[k] = bi;
+            cs[bi] = -2;
+        }
+        n_jobs = k + 1;
+        __syncthreads();
+    }
+    __syncthreads();
+
+    // ---- (3) the job table
+    if (tid < n_jobs) {
+        const int r = s_pick[tid];
+        NodeRec *q = a.recs + r;
+        const SplitRec best = q->best;
+        const FeatRec pf = a.feat_rec[best.feature];
+        GrowJob *job = gs->jobs + tid;
+        job->rec = r;
+        job->feature = best.feature;
+        job->bin = best.bin;
+        job->logW = pf.logW;
+        job->byte = pf.byte;
+        job->col = pf.col;
+        job->col8 = pf.col8;
+        job->off = q->off;
+        job->n = q->n;
+        job->buf = q->buf;
+        job->nl = 0;
+        job->gl = best.gl;
+        job->hl = best.hl;
+        job->PG = q->G;
+        job->PH = q->H;
+        job->parent_slot = q->slot;
+        job->small_slot = 1 + n_exec + tid;
+        job->child0 = n_recs + 2 * tid;
+        job->finish_count = 0;
+        q->state = 1;
+        q->child0 = n_recs + 2 * tid;
+        s_n[tid] = q->n;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        // blocks of the partition kernels: in proportion to the rows, at least one per leaf
+        int want[GROW_MAX_JOBS];
+        long long sum = 0;
+        const int pb_cap = a.pb_total - a.K;
+        for (int jj = 0; jj < n_jobs; ++jj) {
+            long long w = ((long long)s_n[jj] + 2047) / 2048;
+            if (w < 1) w = 1;
+            if (w > pb_cap) w = pb_cap;
+            want[jj] = (int)w;
+            sum += w;
+        }
+        int at = 0;
+        for (int jj = 0; jj < n_jobs; ++jj) {
+            int w = want[jj];
+            if (sum > pb_cap) {
+                w = (int)((long long)w * pb_cap / sum);
+                if (w < 1) w = 1;
+            }
+            gs->jobs[jj].pb0 = at;
+            gs->jobs[jj].pb = w;
+            at += w;
+        }
+        // histogram CTAs per tile: one per 1024 rows of half the leaf (the smaller child has at most
+        // that many rows), at most a leaf's share of the SMs, scaled down when the batch wants more
+        // than a launch has
+        sum = 0;
+        const int xc = a.xcap - a.K;
+        for (int jj = 0; jj < n_jobs; ++jj) {
+            long long w = ((long long)(s_n[jj] / 2) + MIN_ROWS_PER_CTA - 1) / MIN_ROWS_PER_CTA;
+            if (w < 1) w = 1;
+            if (w > a.parts_cap) w = a.parts_cap;
+            want[jj] = (int)w;
+            sum += w;
+        }
+        at = 0;
+        for (int jj = 0; jj < n_jobs; ++jj) {
+            int w = want[jj];
+            if (sum > xc) {
+                w = (int)((long long)w * xc / sum);
+                if (w < 1) w = 1;
+            }
+            gs->jobs[jj].cta0 = at;
+            gs->jobs[jj].parts = w;
+            gs->jobs[jj].slot0 = at * a.n_tiles;
+            at += w;
+        }
+        gs->n_jobs = n_jobs;
+        gs->n_exec = n_exec + n_jobs;
+        gs->n_recs = n_recs + 2 * n_jobs;
+    }
+}
+
+void fill_args(qgbdt_ctx *c, GrowArgs &a) {
     const int L = c->prm.num_leaves;
     a.gs = c->d_gs;
+    a.recs = c->d_recs;
     a.leaves = c->d_leaves;
+    a.front = c->d_front;
     a.state = c->d_state;
     a.feat_rec = c->d_feat_rec;
-    a.leaf_gain = c->d_leaf_gain;
     a.N = (uint32_t)c->N;
     a.ent0 = c->d_ent0;
     a.ent1 = c->d_ent1;
     a.codes_nat = reinterpret_cast<const uint16_t *>(c->d_codes_nat);
-    a.bits = c->d_part_bits;
+    a.bits = c->d_grow_bits;
+    a.bits_stride = c->grow_bits_stride;
     a.counts = c->d_part_counts;
-    part_blocks = c->sm_count * 4;
-    a.n_count = part_blocks * PART_WARPS;
+    a.pb_total = c->grow_pb_total;
     a.pool = c->d_hist_pool;
-    a.partial = c->d_partial;
+    a.partial = c->d_grow_partial;
     a.cand = c->d_cand;
     a.F = c->F;
     a.nb = c->nb;
     a.L = L;
+    a.K = c->grow_jobs;
+    a.xcap = c->grow_xcap;
+    a.n_tiles = (int)c->tiles.size();
+    a.parts_cap = qg_grow_parts_cap(c);
+    a.max_recs = qg_grow_max_recs(L);
+    a.max_slots = qg_grow_max_slots(L);
     a.sp.G = a.sp.H = a.sp.n_s = 0;
     a.sp.kg = qg_levels_g(c->prm.bits);
     a.sp.kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
@@ -636,90 +877,154 @@ void fill_args(qgbdt_ctx *c, GrowArgs &a, int &part_blocks) {
     a.m_left = c->d_m_left;
     a.m_right = c->d_m_right;
     a.m_gain = c->d_m_gain;
+    a.cond = 0;
+    a.use_cond = 0;
 }
 
-// The L - 1 splits of a tree: four kernels each, every size read from the grow state.
-int enqueue_splits(qgbdt_ctx *c, const GrowArgs &a, int part_blocks, cudaStream_t st) {
-    const unsigned fin_blocks = (unsigned)c->F;
-    for (int split = 1; split < c->prm.num_leaves; ++split) {
-        k_grow_flags<<<part_blocks, PART_THREADS, 0, st>>>(a);
-        QG_LAUNCH_CHECK(c);
-        k_grow_scatter<<<part_blocks, PART_THREADS, 0, st>>>(a);
-        QG_LAUNCH_CHECK(c);
-        const int rc = qg_hist_grow(c, st);
-        if (rc != QGBDT_OK) return rc;
-        if (c->F > c->sm_count * 8) k_grow_finish<false, 2><<<fin_blocks, 128, 0, st>>>(a);
-        else k_grow_finish<false, 1><<<fin_blocks, 256, 0, st>>>(a);
-        QG_LAUNCH_CHECK(c);
-    }
+int launch_commit(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st) {
+    k_grow_commit<<<1, COMMIT_THREADS, commit_smem_bytes(a.L, a.max_recs), st>>>(a);
+    QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
+}
+
+// One pass: the kernels that split the leaves of the current batch, then the commit step.
+int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st) {
+    k_grow_flags<<<a.pb_total, PART_THREADS, 0, st>>>(a);
+    QG_LAUNCH_CHECK(c);
+    k_grow_scatter<<<a.pb_total, PART_THREADS, 0, st>>>(a);
+    QG_LAUNCH_CHECK(c);
+    const int rc = qg_hist_grow(c, st);
+    if (rc != QGBDT_OK) return rc;
+    const dim3 fin((unsigned)c->F, (unsigned)a.K);
+    if (c->F > c->sm_count * 8) k_grow_finish<false, 2><<<fin, 128, 0, st>>>(a);
+    else k_grow_finish<false, 1><<<fin, 256, 0, st>>>(a);
+    QG_LAUNCH_CHECK(c);
+    return launch_commit(c, a, st);
 }
 
 }  // namespace
 
+int qg_grow_parts_cap(const qgbdt_ctx *c) {
+    const int t = (int)c->tiles.size();
+    const int p = c->sm_count / (t > 0 ? t : 1);
+    return p < 1 ? 1 : p;
+}
+
+int qg_grow_max_recs(int L) { return 1 + 2 * (L - 1 + GROW_SLACK) + 2 * GROW_MAX_JOBS; }
+int qg_grow_max_slots(int L) { return L + GROW_SLACK + GROW_MAX_JOBS + 2; }
+
 void qg_grow_graph_destroy(qgbdt_ctx *c) {
     if (c->grow_graph_exec) cudaGraphExecDestroy(reinterpret_cast<cudaGraphExec_t>(c->grow_graph_exec));
     c->grow_graph_exec = nullptr;
-    c->grow_graph_launches = 0;
+    c->grow_pass_launches = 0;
 }
 
-// The split loop of one tree as a CUDA graph (about a thousand launches whose arguments never
-// change: what differs from tree to tree is device state).  Built once per context and objective;
-// with the histogram event timers on, the launches go to the stream instead.
-static int build_grow_graph(qgbdt_ctx *c, const GrowArgs &a, int part_blocks) {
-    cudaStream_t cs = nullptr;
-    QG_CUDA(c, cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking));
+// The growth of one tree after its root as a CUDA graph: a commit kernel (which picks the first
+// batch), then a while node whose body is one pass.  The launch arguments never change (what
+// differs from pass to pass and from tree to tree is device state), so the graph is built once per
+// context and objective.
+static int build_grow_graph(qgbdt_ctx *c, GrowArgs a) {
     const int64_t launches_before = c->n_launches;
     int rc = qg_hist_grow_configure(c);
+    if (rc != QGBDT_OK) return rc;
     cudaGraph_t graph = nullptr;
-    if (rc == QGBDT_OK) {
-        cudaError_t e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
-        if (e == cudaSuccess) {
-            rc = enqueue_splits(c, a, part_blocks, cs);
-            e = cudaStreamEndCapture(cs, &graph);
-        }
-        if (e != cudaSuccess || rc != QGBDT_OK || !graph) {
-            cudaGetLastError();
-            if (graph) cudaGraphDestroy(graph);
-            cudaStreamDestroy(cs);
-            c->n_launches = launches_before;
-            return rc != QGBDT_OK ? rc : qg_fail(c, QGBDT_ERR_CUDA, "capturing the split loop failed: %s", cudaGetErrorString(e));
-        }
-        cudaGraphExec_t exec = nullptr;
-        e = cudaGraphInstantiate(&exec, graph, 0);
-        cudaGraphDestroy(graph);
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            cudaStreamDestroy(cs);
-            c->n_launches = launches_before;
-            return qg_fail(c, QGBDT_ERR_CUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(e));
-        }
-        c->grow_graph_exec = exec;
-        c->grow_graph_launches = c->n_launches - launches_before;
-        c->grow_graph_const_hess = c->const_hess;
+    cudaStream_t cs = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    const char *what = "cudaGraphCreate";
+    cudaError_t e = cudaGraphCreate(&graph, 0);
+    if (e == cudaSuccess) {
+        what = "cudaGraphConditionalHandleCreate";
+        e = cudaGraphConditionalHandleCreate(&a.cond, graph, 1, cudaGraphCondAssignDefault);
     }
+    a.use_cond = 1;
+    cudaGraphNode_t first = nullptr, loop = nullptr;
+    if (e == cudaSuccess) {
+        what = "cudaGraphAddKernelNode";
+        void *params[] = {&a};
+        cudaKernelNodeParams kp = {};
+        kp.func = reinterpret_cast<void *>(k_grow_commit);
+        kp.gridDim = dim3(1);
+        kp.blockDim = dim3(COMMIT_THREADS);
+        kp.sharedMemBytes = (unsigned)commit_smem_bytes(a.L, a.max_recs);
+        kp.kernelParams = params;
+        e = cudaGraphAddKernelNode(&first, graph, nullptr, 0, &kp);
+    }
+    cudaGraph_t body = nullptr;
+    if (e == cudaSuccess) {
+        what = "cudaGraphAddNode (while)";
+        cudaGraphNodeParams np = {};
+        np.type = cudaGraphNodeTypeConditional;
+        np.conditional.handle = a.cond;
+        np.conditional.type = cudaGraphCondTypeWhile;
+        np.conditional.size = 1;
+        e = cudaGraphAddNode(&loop, graph, &first, 1, &np);
+        if (e == cudaSuccess) body = np.conditional.phGraph_out[0];
+    }
+    if (e == cudaSuccess) {
+        what = "cudaStreamCreateWithFlags";
+        e = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking);
+    }
+    if (e == cudaSuccess) {
+        what = "capturing a pass";
+        e = cudaStreamBeginCaptureToGraph(cs, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal);
+        if (e == cudaSuccess) {
+            rc = enqueue_pass(c, a, cs);
+            cudaGraph_t out = nullptr;
+            e = cudaStreamEndCapture(cs, &out);
+        }
+    }
+    const int64_t pass_launches = c->n_launches - launches_before;
     c->n_launches = launches_before;
-    cudaStreamDestroy(cs);
-    return rc;
+    if (e == cudaSuccess && rc == QGBDT_OK) {
+        what = "cudaGraphInstantiate";
+        e = cudaGraphInstantiate(&exec, graph, 0);
+    }
+    if (cs) cudaStreamDestroy(cs);
+    if (graph) cudaGraphDestroy(graph);
+    if (rc != QGBDT_OK) return rc;
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return qg_fail(c, QGBDT_ERR_CUDA, "building the growth graph failed at %s: %s", what, cudaGetErrorString(e));
+    }
+    c->grow_graph_exec = exec;
+    c->grow_pass_launches = pass_launches;
+    c->grow_graph_const_hess = c->const_hess;
+    return QGBDT_OK;
 }
 
 // Grows the tree of boosting iteration slot `tree_slot` of the current train call.  Gradients must
-// have been quantized on the same stream (the state holds the totals and maxima).  Asynchronous.
+// have been quantized on the same stream (the state holds the totals and maxima).  Asynchronous,
+// unless the histogram event timers are on: then the passes go to the stream one by one and the
+// host reads after each whether the tree is finished.
 int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     GrowArgs a;
-    int part_blocks;
-    fill_args(c, a, part_blocks);
-    k_grow_begin<<<1, 1, 0, st>>>(c->d_gs, c->d_leaves, c->d_state, (uint32_t)c->N, tree_slot);
+    fill_args(c, a);
+    const size_t smem = commit_smem_bytes(a.L, a.max_recs);
+    if (smem > 48 * 1024) {
+        if (smem > (size_t)c->max_smem_optin) return qg_fail(c, QGBDT_ERR_ARG, "num_leaves too large for the commit step");
+        QG_CUDA(c, cudaFuncSetAttribute(k_grow_commit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
+    k_grow_begin<<<1, 1, 0, st>>>(c->d_gs, c->d_recs, c->d_leaves, c->d_front, c->d_state, (uint32_t)c->N, tree_slot);
     QG_LAUNCH_CHECK(c);
     int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
     if (rc != QGBDT_OK) return rc;
     k_grow_finish<true, 1><<<(unsigned)c->F, 256, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     if (c->prm.num_leaves < 2) return QGBDT_OK;
-    if (c->profile_hist) return enqueue_splits(c, a, part_blocks, st);   // event records around every build
+    if (c->profile_hist) {
+        // event records around every histogram launch: passes on the stream, the host follows
+        if ((rc = launch_commit(c, a, st)) != QGBDT_OK) return rc;
+        int *h_done = reinterpret_cast<int *>(reinterpret_cast<char *>(c->h_pinned) + 64 * 1024 + 8192);
+        for (int pass = 0; pass < c->prm.num_leaves; ++pass) {
+            QG_CUDA(c, cudaMemcpyAsync(h_done, &c->d_gs->done, sizeof(int), cudaMemcpyDeviceToHost, st));
+            QG_CUDA(c, cudaStreamSynchronize(st));
+            if (*h_done) break;
+            if ((rc = enqueue_pass(c, a, st)) != QGBDT_OK) return rc;
+        }
+        return QGBDT_OK;
+    }
     if (c->grow_graph_exec && c->grow_graph_const_hess != c->const_hess) qg_grow_graph_destroy(c);
-    if (!c->grow_graph_exec && (rc = build_grow_graph(c, a, part_blocks)) != QGBDT_OK) return rc;
+    if (!c->grow_graph_exec && (rc = build_grow_graph(c, a)) != QGBDT_OK) return rc;
     QG_CUDA(c, cudaGraphLaunch(reinterpret_cast<cudaGraphExec_t>(c->grow_graph_exec), st));
-    c->n_launches += c->grow_graph_launches;
     return QGBDT_OK;
 }

@@ -120,9 +120,11 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_coop(HistArgs a) {
     }
 }
 
-// Tree growth: the rows are the smaller child (ties: the left one) of the split recorded in the
-// grow state, as (row, code) pairs in the buffer the scatter kernel wrote; the histogram goes to
-// the pool slot numbered like the leaf about to be created.  The grid is (max parts, tile - tile0).
+// Tree growth: a launch builds the histograms of the smaller children (ties: the left one) of all
+// leaves being split in the current pass.  The rows are (row, code) pairs in the buffer the scatter
+// kernel wrote; a job owns the CTAs x in [cta0, cta0 + parts) of every tile and the partial slots
+// slot0 + tile * parts + part; the histogram goes to the job's pool slot.  The grid is
+// (CTAs per tile, tile - tile0).
 struct GrowHist {
     const GrowState *gs;
     const uint2 *ent0, *ent1;
@@ -134,19 +136,33 @@ template <int LOGW_T, int MODE>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowHist g) {
     extern __shared__ __align__(1024) int sh[];
     const GrowState *gs = g.gs;
-    // every field and the tile at once (one round trip to memory), then the early exits
-    const int done = gs->done, buf = gs->buf, n_leaves = gs->n_leaves;
-    const uint32_t nl = gs->nl, n = gs->n, off = gs->off;
-    const TileDesc td = a.tiles[a.tile0 + blockIdx.y];
+    // the job table and the tile at once (one round trip to memory), then the early exits
+    const int done = gs->done, n_jobs = gs->n_jobs;
+    int c0[GROW_MAX_JOBS], np[GROW_MAX_JOBS];
+#pragma unroll
+    for (int i = 0; i < GROW_MAX_JOBS; ++i) {
+        c0[i] = gs->jobs[i].cta0;
+        np[i] = gs->jobs[i].parts;
+    }
+    TileDesc td = a.tiles[a.tile0 + blockIdx.y];
     if (done) return;
+    int j = -1;
+#pragma unroll
+    for (int i = 0; i < GROW_MAX_JOBS; ++i)
+        if (i < n_jobs && (int)blockIdx.x >= c0[i] && (int)blockIdx.x < c0[i] + np[i]) j = i;
+    if (j < 0) return;
+    const GrowJob *job = gs->jobs + j;
+    const int buf = job->buf, parts = job->parts, slot0 = job->slot0, small_slot = job->small_slot;
+    const uint32_t nl = job->nl, n = job->n, off = job->off;
     const uint32_t nr = n - nl;
     a.ents = buf == 0 ? g.ent1 : g.ent0;
     a.off = nl <= nr ? off : off + nl;
     a.n = nl <= nr ? nl : nr;
-    a.hist = g.pool + (size_t)n_leaves * g.hist_words;
-    const uint32_t P = effective_parts((uint32_t)td.parts, a.n);
-    if (blockIdx.x >= P) return;
-    hist_cta<HIST_THREADS, LOGW_T, MODE, 2>(a, td, blockIdx.x, P, sh);
+    a.hist = g.pool + (size_t)small_slot * g.hist_words;
+    td.cta0 = slot0 + (a.tile0 + (int)blockIdx.y) * parts;
+    const uint32_t P = effective_parts((uint32_t)parts, a.n), part = blockIdx.x - (uint32_t)c0[j];
+    if (part >= P) return;
+    hist_cta<HIST_THREADS, LOGW_T, MODE, 2>(a, td, part, P, sh);
 }
 
 // Sums the partial histograms of every tile that was built by more than one CTA.  A block takes
@@ -392,10 +408,7 @@ int launch_grow_one(qgbdt_ctx *c, const HistArgs &args, const GrowHist &g, int n
         }
     }
     if (configure_only) return QGBDT_OK;
-    int group_parts = 1;
-    for (int t = args.tile0; t < args.tile0 + n_tiles; ++t)
-        if (c->tiles[t].parts > group_parts) group_parts = c->tiles[t].parts;
-    kern<<<dim3((unsigned)group_parts, (unsigned)n_tiles), HIST_THREADS, HIST_SMEM, st>>>(args, g);
+    kern<<<dim3((unsigned)c->grow_xcap, (unsigned)n_tiles), HIST_THREADS, HIST_SMEM, st>>>(args, g);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
 }
@@ -433,8 +446,9 @@ int qg_hist_grow_configure(qgbdt_ctx *c) {
     return a.shift == 16 ? launch_grow<0>(c, a, g, nullptr, true) : launch_grow<2>(c, a, g, nullptr, true);
 }
 
-// Histogram of the smaller child of the split recorded in the grow state (sizes known only on
-// the device): partial histograms or, for a small child, the finished histogram in its pool slot.
+// Histograms of the smaller children of the leaves being split in the current pass (sizes known
+// only on the device): partial histograms or, for a small child, the finished histogram in its
+// pool slot.
 int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
     const int bits = c->prm.bits;
     const int kg = qg_levels_g(bits);
@@ -450,7 +464,7 @@ int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
     a.n = 0;
     a.nb = c->nb;
     a.hist = nullptr;
-    a.partial = c->d_partial;
+    a.partial = c->d_grow_partial;
     pick_field_split(kg, kh, a.shift, a.flush_rows);
     a.pass = 0;
     a.state = c->d_state;

@@ -66,39 +66,77 @@ struct FeatRec {
     const uint32_t *col;   // the feature's word in row 0 of its tile
     int32_t logW, byte;    // words per row (log2) of the tile, byte of the word
     int32_t cta0, parts;   // partial-histogram slots of the tile
-    int32_t fl, pad;       // feature number inside the tile
+    int32_t fl, tile;      // feature number inside the tile, tile number
     const uint8_t *col8;   // the feature's column in the column-major copy (nullptr: there is none)
 };
 
-// One leaf of the tree being grown (device memory).  Its rows are entries [off, off + n) of the
-// (row, code) pair buffer `buf` (0 or 1; -1: the identity list of the root).
+// ---- leaf-wise growth on the device (grow.cu) --------------------------------------------------
+// A tree grows in passes.  A pass splits up to GROW_MAX_JOBS leaves at once (row partition, the
+// smaller child's histogram, the larger child's by subtraction, both children's best splits); the
+// batch always holds the leaf that best-first growth (Sec. 3) would split next and is filled up with
+// the known leaves of largest gain, also children of leaves whose own split has not been confirmed
+// yet.  After the pass a commit step replays the best-first order: it takes the leaf with the
+// largest gain, and if that leaf has been split already it numbers the children and records the
+// node, until it meets a leaf that has not been split (which goes into the next batch) or the tree
+// is full.  The result is the tree best-first growth builds, whatever the batches were.
+
+constexpr int GROW_MAX_JOBS = 16;   // leaves split per pass, at most
+constexpr int GROW_SLACK = 48;      // leaves that may be split ahead of their confirmation at any time
+
+// A leaf with a number (confirmed by the commit step): what the refit and the score update read.
 struct LeafRec {
+    uint32_t off, n;     // its rows: entries [off, off + n) of pair buffer `buf`
+    int32_t buf;         // 0 or 1; -1: the identity list of the root
+    int32_t rec;         // its growth record
+};
+
+// Growth record of a leaf the grower knows: confirmed or not, split or not.
+struct NodeRec {
     uint32_t off, n;
     int32_t buf;
     int32_t slot;            // histogram slot in the pool
     long long G, H;          // integer gradient / hessian totals
     SplitRec best;           // best split of the leaf
-    int32_t parent_node, parent_side;
+    int32_t state;           // 0: not split; 1: split (children in records child0, child0 + 1)
+    int32_t child0;
+    uint32_t nl;             // rows that went left when it was split
+    int32_t parent_node, parent_side;   // position in the tree, valid once confirmed
 };
 
-// State of leaf-wise growth kept on the device, so that a tree grows without the host looking:
-// the split being executed and counters.
-struct GrowState {
-    int32_t n_leaves, done;
-    int32_t tree_slot;               // slot of the tree being grown in the device-side model arrays
-    int32_t pick, feature, bin;      // leaf being split and its winning candidate
+// One leaf being split in the current pass.
+struct GrowJob {
+    int32_t rec;                     // its growth record
+    int32_t feature, bin;            // the split
     int32_t logW, byte;              // tile width (log2 words per row) and byte of the split feature's word
     const uint32_t *col;             // that word in row 0 of the tile
     const uint8_t *col8;             // the split feature's column in the column-major copy, or nullptr
-    uint32_t off, n;                 // rows of the leaf being split
+    uint32_t off, n;                 // rows of the leaf
     int32_t buf;                     // their pair buffer
     uint32_t nl;                     // rows that go left (written by the scatter kernel)
-    long long gl, hl, PG, PH;        // left totals of the candidate, totals of the leaf
-    double gain;
-    int32_t parent_slot, parent_node, parent_side;   // histogram slot and tree position of that leaf
+    long long gl, hl, PG, PH;        // left totals of the split, totals of the leaf
+    int32_t parent_slot, small_slot; // histogram slots: the leaf's (becomes the larger child's), the smaller child's
+    int32_t child0;                  // growth records of the children: child0 (left), child0 + 1 (right)
+    int32_t pb0, pb;                 // blocks of the partition kernels: [pb0, pb0 + pb)
+    int32_t cta0, parts;             // histogram CTAs per tile: x in [cta0, cta0 + parts) of the grid
+    int32_t slot0;                   // partial-histogram slots: tile t, part p uses slot0 + t * parts + p
     unsigned int finish_count;       // blocks of the finishing kernel that are through
-    unsigned long long hist_rows;    // rows visited by histogram builds of row lists (all trees so far)
-    unsigned long long hist_builds;
+    int32_t pad;
+};
+
+// State of the growth of one tree, kept on the device so that the host never looks.
+struct GrowState {
+    int32_t n_jobs, done;
+    int32_t n_leaves;                // confirmed leaves
+    int32_t n_exec;                  // leaves split so far (confirmed or not)
+    int32_t n_recs;                  // growth records in use
+    int32_t tree_slot;               // slot of the tree being grown in the device-side model arrays
+    GrowJob jobs[GROW_MAX_JOBS];
+    unsigned long long hist_rows;    // rows of the smaller children of confirmed splits (all trees so far)
+    unsigned long long hist_builds;  // confirmed splits (all trees so far)
+    unsigned long long extra_rows, extra_builds;   // the same for splits made ahead that the tree did not use
+    unsigned long long passes;
+    int32_t n_segs;                  // slots of the finished tree's leaf table (refit.cu)
+    int32_t pad;
 };
 
 struct qgbdt_ctx {
@@ -136,14 +174,22 @@ struct qgbdt_ctx {
     SplitRec *d_feat_best = nullptr;    // [F]
     SplitRec *d_split_out = nullptr;    // [2]
     long long *d_leaf_sums = nullptr;   // [L][2] fixed-point refit sums
-    uint32_t *d_leaf_table = nullptr;   // [L][2] (offset, leaf) sorted by offset, then [L] counts
+    uint32_t *d_leaf_table = nullptr;   // [S][3] (offset, leaf, pair buffer) of the slots sorted by offset, then [S][4] scratch; S = qg_leaf_table_slots(L)
     float *d_leaf_value = nullptr;      // [L]
     double *d_leaf_w = nullptr;         // [L]
     void *h_pinned = nullptr;           // small pinned staging area
     // training buffers (allocated on first qgbdt_train)
     float *d_g = nullptr, *d_h = nullptr;
     unsigned long long *d_hist_pool = nullptr;  // [L][F][nb]
-    LeafRec *d_leaves = nullptr;                // [L]
+    LeafRec *d_leaves = nullptr;                // [L] numbered leaves of the tree being grown
+    NodeRec *d_recs = nullptr;                  // [1 + 2 (L - 1 + GROW_SLACK)] growth records
+    int32_t *d_front = nullptr;                 // [L] growth record of every numbered leaf
+    int grow_jobs = 1;                          // leaves split per pass (<= GROW_MAX_JOBS; fewer with thousands of features)
+    int grow_pb_total = 0;                      // blocks of a partition launch
+    int grow_xcap = 0;                          // histogram CTAs per tile of a growth launch
+    uint32_t *d_grow_bits = nullptr;            // [grow_jobs][bits_stride] predicate bits of the leaves being split
+    size_t grow_bits_stride = 0;
+    unsigned long long *d_grow_partial = nullptr;   // [grow_xcap * tiles][4][nb][32] partial histograms of growth
     uint2 *d_ent0 = nullptr, *d_ent1 = nullptr; // [N] (row, gradient code) pairs of the leaves, two buffers
     GrowState *d_gs = nullptr;
     SplitRec *d_cand = nullptr;                 // [F][2] per-feature best candidates of the two children
@@ -151,9 +197,8 @@ struct qgbdt_ctx {
     uint8_t *d_colmajor = nullptr;              // [F][col_stride] column-major copy of the bin codes (training only)
     size_t col_stride = 0;
     bool want_column_copy = true;               // QGBDT_OPT_COLUMN_COPY
-    double *d_leaf_gain = nullptr;              // [L] stored gain of every leaf's best split (-inf: none)
     void *grow_graph_exec = nullptr;            // cudaGraphExec_t: the split loop of one tree
-    int64_t grow_graph_launches = 0;            // kernel launches it replays
+    int64_t grow_pass_launches = 0;             // kernel launches of one pass
     bool grow_graph_const_hess = false;         // objective it was captured for
     // trees of the current qgbdt_train call, on the device until the call ends
     int model_cap = 0;                          // trees the arrays below can hold
@@ -164,6 +209,7 @@ struct qgbdt_ctx {
     long long *d_m_leaf_count = nullptr;
     // counters
     int64_t n_launches = 0, n_hist_builds = 0, n_hist_row_features = 0;
+    int64_t n_passes = 0, n_extra_builds = 0;   // commit steps run; leaves split ahead that their tree did not use
     // optional per-launch timing of the histogram kernel (event pairs on the launching stream)
     bool profile_hist = false;
     std::vector<cudaEvent_t> hist_events;  // start/stop pairs, reused
@@ -227,12 +273,16 @@ int qg_partition(qgbdt_ctx *c, int64_t off, int64_t n, int feature, int bin, cud
 int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st);
 int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st);
 // the same two for a tree grown on the device (leaf table from the device leaf records)
+int qg_leaf_table_slots(int L);   // slots (and words / 7) of the leaf table of a tree grown on the device
 int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_scores, int tree_slot, cudaStream_t st);
 
 // grow.cu: one tree by leaf-wise growth, every decision taken on the device
 int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st);
-// hist.cu: histogram of the smaller child of the split recorded in the grow state
+// hist.cu: histograms of the smaller children of the leaves being split in the current pass
 int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st);
+int qg_grow_parts_cap(const qgbdt_ctx *c);   // grow.cu: histogram CTAs per tile one leaf may get
+int qg_grow_max_recs(int L);                 // grow.cu: growth records / histogram slots a tree of L leaves may use
+int qg_grow_max_slots(int L);
 int qg_hist_grow_configure(qgbdt_ctx *c);   // function attributes of the kernels it launches (before a capture)
 void qg_grow_graph_destroy(qgbdt_ctx *c);   // grow.cu: drops the captured split loop (buffers are about to change)
 

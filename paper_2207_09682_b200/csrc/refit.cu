@@ -22,9 +22,12 @@ __device__ inline int slot_of(const uint32_t *offs, int n_leaves, uint32_t p) {
 
 __device__ inline long long to_fixed(float v) { return __double2ll_rn(__dmul_rn((double)v, 1073741824.0)); }
 
-// table: [n_leaves] offsets ascending, then [n_leaves] leaf ids.  sums: [n_leaves][2] by slot.
-// gs != nullptr: a tree grown on the device: the leaf count comes from *gs and the table's third
-// part [n_leaves] says which (row, code) pair buffer holds a leaf's rows (-1: the identity list).
+// table: [n_slots] offsets ascending, then [n_slots] leaf ids.  A slot is a range of positions
+// whose rows belong to one leaf; the step-wise interface has one slot per leaf.  sums: [leaves][2]
+// by leaf id.  gs != nullptr: a tree grown on the device: the slot count comes from *gs (a leaf
+// whose rows were partitioned further ahead of the best-first order is covered by several slots)
+// and the table's third part [n_slots] says which (row, code) pair buffer holds a slot's rows
+// (-1: the identity list).
 __device__ inline uint32_t leaf_row(const uint32_t *idx, const uint2 *ent0, const uint2 *ent1, const uint32_t *table,
                                     int n_leaves, bool grown, int s, uint32_t p) {
     if (!grown) return idx[p];
@@ -41,7 +44,7 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__
                                                               long long *__restrict__ sums) {
     extern __shared__ uint32_t offs[];  // n_leaves offsets
     const bool grown = gs != nullptr;
-    if (grown) n_leaves = gs->n_leaves;
+    if (grown) n_leaves = gs->n_segs;   // slots
     __shared__ unsigned long long acc[REFIT_LOCAL][2];
     for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) offs[i] = table[i];
     for (int i = threadIdx.x; i < REFIT_LOCAL * 2; i += REFIT_THREADS) (&acc[0][0])[i] = 0ull;
@@ -74,8 +77,9 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__
                     atomicAdd(&acc[s0 - s_lo][0], (unsigned long long)gf);
                     atomicAdd(&acc[s0 - s_lo][1], (unsigned long long)hf);
                 } else {
-                    atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * s0]), (unsigned long long)gf);
-                    atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * s0 + 1]), (unsigned long long)hf);
+                    const uint32_t leaf = table[n_leaves + s0];
+                    atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * leaf]), (unsigned long long)gf);
+                    atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * leaf + 1]), (unsigned long long)hf);
                 }
             }
         } else if (ok) {
@@ -83,35 +87,35 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__
                 atomicAdd(&acc[s - s_lo][0], (unsigned long long)gf);
                 atomicAdd(&acc[s - s_lo][1], (unsigned long long)hf);
             } else {
-                atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * s]), (unsigned long long)gf);
-                atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * s + 1]), (unsigned long long)hf);
+                const uint32_t leaf = table[n_leaves + s];
+                atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * leaf]), (unsigned long long)gf);
+                atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * leaf + 1]), (unsigned long long)hf);
             }
         }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < REFIT_LOCAL; i += REFIT_THREADS) {
         if (s_lo + i < n_leaves && (acc[i][0] | acc[i][1]) != 0ull) {
-            atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * (s_lo + i)]), acc[i][0]);
-            atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * (s_lo + i) + 1]), acc[i][1]);
+            const uint32_t leaf = table[n_leaves + s_lo + i];
+            atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * leaf]), acc[i][0]);
+            atomicAdd(reinterpret_cast<unsigned long long *>(&sums[2 * leaf + 1]), acc[i][1]);
         }
     }
 }
 
-// w = -sum g / (sum h + lambda); output (float)(learning_rate * w); written by leaf id.
-__global__ void k_leaf_values(const long long *__restrict__ sums, const uint32_t *__restrict__ table, int n_leaves,
-                              const GrowState *gs, double lambda, double lr, double *__restrict__ w_out,
-                              float *__restrict__ v_out) {
+// w = -sum g / (sum h + lambda); output (float)(learning_rate * w); sums and outputs by leaf id.
+__global__ void k_leaf_values(const long long *__restrict__ sums, int n_leaves, const GrowState *gs, double lambda,
+                              double lr, double *__restrict__ w_out, float *__restrict__ v_out) {
     if (gs) n_leaves = gs->n_leaves;
-    for (int s = blockIdx.x * blockDim.x + threadIdx.x; s < n_leaves; s += gridDim.x * blockDim.x) {
-        const int leaf = (int)table[n_leaves + s];
-        const double den = __dadd_rn((double)sums[2 * s + 1], __dmul_rn(lambda, 1073741824.0));
-        const double w = den > 0.0 ? __ddiv_rn(-(double)sums[2 * s], den) : 0.0;
+    for (int leaf = blockIdx.x * blockDim.x + threadIdx.x; leaf < n_leaves; leaf += gridDim.x * blockDim.x) {
+        const double den = __dadd_rn((double)sums[2 * leaf + 1], __dmul_rn(lambda, 1073741824.0));
+        const double w = den > 0.0 ? __ddiv_rn(-(double)sums[2 * leaf], den) : 0.0;
         w_out[leaf] = w;
         v_out[leaf] = __double2float_rn(__dmul_rn(lr, w));
     }
 }
 
-// Dynamic shared memory: [n_leaves] offsets, [n_leaves] values, [n_leaves] pair buffers, so that
+// Dynamic shared memory: [n_slots] offsets, [n_slots] values, [n_slots] pair buffers, so that
 // a row costs a search in shared memory and two global accesses (its pair, its score).  Four
 // rows per thread are in flight.
 __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *__restrict__ idx,
@@ -123,7 +127,7 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *
                                                                 float *__restrict__ scores) {
     extern __shared__ uint32_t offs[];
     const bool grown = gs != nullptr;
-    if (grown) n_leaves = gs->n_leaves;
+    if (grown) n_leaves = gs->n_segs;   // slots
     float *vals = reinterpret_cast<float *>(offs + n_leaves);
     int *bufs = reinterpret_cast<int *>(offs + 2 * n_leaves);
     for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) {
@@ -156,30 +160,72 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *
     }
 }
 
-// Leaf table of a tree grown on the device: leaves ranked by (offset, empty first, leaf number);
-// [L] offsets, [L] leaf numbers, [L] index buffers.  Also zeroes the sums and stores the tree's
-// leaf count and rows per leaf.  One block.
-__global__ void __launch_bounds__(256) k_leaf_table(const LeafRec *__restrict__ leaves, const GrowState *gs,
-                                                    uint32_t *__restrict__ table, long long *__restrict__ sums,
+// Leaf table of a tree grown on the device.  A numbered leaf that was never split ahead of the
+// best-first order is one slot: its range of its pair buffer.  A leaf that was split ahead without
+// the tree using the split still owns the same rows, but only the deepest ranges written hold
+// them intact (the scatter of a grandchild reuses the leaf's own buffer), so such a leaf is
+// covered by the slots of its descendants: a record none of whose children has been split is
+// intact in its own buffer.  Slots are ranked by (offset, empty first, order of discovery);
+// [S] offsets, [S] leaf numbers, [S] pair buffers.  Also zeroes the sums and stores the tree's leaf
+// count and rows per leaf.  One block; `seg` is scratch for 4 S words.
+__global__ void __launch_bounds__(256) k_leaf_table(const LeafRec *__restrict__ leaves, const NodeRec *__restrict__ recs,
+                                                    GrowState *gs, uint32_t *__restrict__ table, uint32_t *__restrict__ seg,
+                                                    int max_segs, long long *__restrict__ sums,
                                                     int32_t *__restrict__ m_num_leaves,
-                                                    long long *__restrict__ m_leaf_count) {
+                                                    long long *__restrict__ m_leaf_count, DevState *state) {
     const int L = gs->n_leaves;
+    __shared__ int n_segs;
+    if (threadIdx.x == 0) n_segs = 0;
+    __syncthreads();
     for (int i = threadIdx.x; i < L; i += 256) {
-        const uint32_t off = leaves[i].off, n = leaves[i].n;
+        int stack[GROW_SLACK + GROW_MAX_JOBS + 4];
+        int sp = 0;
+        stack[sp++] = leaves[i].rec;
+        while (sp > 0) {
+            const int r = stack[--sp];
+            const NodeRec q = recs[r];
+            const bool deeper = q.state == 1 && (recs[q.child0].state == 1 || recs[q.child0 + 1].state == 1);
+            if (deeper && sp + 2 <= GROW_SLACK + GROW_MAX_JOBS + 4) {
+                stack[sp++] = q.child0 + 1;
+                stack[sp++] = q.child0;
+            } else {
+                if (deeper) atomicExch(&state->kernel_error, 1);   // deeper than the slack allows: cannot happen
+                const int k = atomicAdd(&n_segs, 1);
+                if (k < max_segs) {
+                    seg[4 * k] = q.off;
+                    seg[4 * k + 1] = q.n;
+                    seg[4 * k + 2] = (uint32_t)q.buf;
+                    seg[4 * k + 3] = (uint32_t)i;
+                }
+            }
+        }
+        sums[2 * i] = 0;
+        sums[2 * i + 1] = 0;
+        m_leaf_count[i] = leaves[i].n;
+    }
+    __syncthreads();
+    int S = n_segs;
+    if (S > max_segs) {
+        if (threadIdx.x == 0) atomicExch(&state->kernel_error, 1);
+        S = max_segs;
+    }
+    __threadfence_block();
+    for (int i = threadIdx.x; i < S; i += 256) {
+        const uint32_t off = seg[4 * i], n = seg[4 * i + 1];
         int rank = 0;
-        for (int j = 0; j < L; ++j) {
-            const uint32_t oj = leaves[j].off, nj = leaves[j].n;
+        for (int j = 0; j < S; ++j) {
+            const uint32_t oj = seg[4 * j], nj = seg[4 * j + 1];
             const bool before = oj < off || (oj == off && ((nj == 0) > (n == 0) || ((nj == 0) == (n == 0) && j < i)));
             rank += before ? 1 : 0;
         }
         table[rank] = off;
-        table[L + rank] = (uint32_t)i;
-        table[2 * L + rank] = (uint32_t)leaves[i].buf;
-        sums[2 * i] = 0;
-        sums[2 * i + 1] = 0;
-        m_leaf_count[i] = n;
+        table[S + rank] = seg[4 * i + 3];
+        table[2 * S + rank] = seg[4 * i + 2];
     }
-    if (threadIdx.x == 0) *m_num_leaves = L;
+    if (threadIdx.x == 0) {
+        *m_num_leaves = L;
+        gs->n_segs = S;
+    }
 }
 
 // Writes the offset-sorted leaf table into pinned memory and queues its copy to the device.
@@ -224,8 +270,8 @@ int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st) 
                                                                      c->d_leaf_table, L, nullptr, d_g, d_h,
                                                                      c->d_leaf_sums);
     QG_LAUNCH_CHECK(c);
-    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, c->d_leaf_table, L, nullptr, c->prm.lambda_l2,
-                                                   c->prm.learning_rate, c->d_leaf_w, c->d_leaf_value);
+    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, L, nullptr, c->prm.lambda_l2, c->prm.learning_rate,
+                                                   c->d_leaf_w, c->d_leaf_value);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
 }
@@ -245,24 +291,28 @@ int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st) {
 // Refit (Eq. 3 with the original gradients) and score update for the tree just grown on the
 // device; leaf values and counts go to slot `tree_slot` of the device-side model arrays.
 int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_scores, int tree_slot, cudaStream_t st) {
-    const int L = c->prm.num_leaves;   // upper bound; the kernels read the real count from the grow state
-    k_leaf_table<<<1, 256, 0, st>>>(c->d_leaves, c->d_gs, c->d_leaf_table, c->d_leaf_sums,
-                                    c->d_m_num_leaves + tree_slot, c->d_m_leaf_count + (size_t)tree_slot * L);
+    const int L = c->prm.num_leaves;     // upper bound; the kernels read the real counts from the grow state
+    const int S = qg_leaf_table_slots(L);
+    k_leaf_table<<<1, 256, 0, st>>>(c->d_leaves, c->d_recs, c->d_gs, c->d_leaf_table, c->d_leaf_table + 3 * (size_t)S, S,
+                                    c->d_leaf_sums, c->d_m_num_leaves + tree_slot,
+                                    c->d_m_leaf_count + (size_t)tree_slot * L, c->d_state);
     QG_LAUNCH_CHECK(c);
     const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
-    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
-                                                                     c->d_leaf_table, L, c->d_gs, d_g, d_h,
+    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * S, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
+                                                                     c->d_leaf_table, S, c->d_gs, d_g, d_h,
                                                                      c->d_leaf_sums);
     QG_LAUNCH_CHECK(c);
-    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, c->d_leaf_table, L, c->d_gs, c->prm.lambda_l2,
-                                                   c->prm.learning_rate, c->d_leaf_w,
-                                                   c->d_m_leaf_value + (size_t)tree_slot * L);
+    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, L, c->d_gs, c->prm.lambda_l2, c->prm.learning_rate,
+                                                   c->d_leaf_w, c->d_m_leaf_value + (size_t)tree_slot * L);
     QG_LAUNCH_CHECK(c);
     unsigned ab = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
     if (ab > (unsigned)c->sm_count * 16) ab = (unsigned)c->sm_count * 16;
-    k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * 3 * L, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
-                                                                   c->d_leaf_table, L, c->d_gs,
+    k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * 3 * S, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
+                                                                   c->d_leaf_table, S, c->d_gs,
                                                                    c->d_m_leaf_value + (size_t)tree_slot * L, d_scores);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
 }
+
+// Slots the leaf table of a grown tree may need: a leaf per slot, plus one per leaf split ahead.
+int qg_leaf_table_slots(int L) { return L + GROW_SLACK + GROW_MAX_JOBS + 2; }

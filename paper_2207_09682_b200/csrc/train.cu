@@ -48,14 +48,30 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
     if (!c->d_g && (rc = alloc_dev(c, &c->d_g, (size_t)c->N, "gradient buffer")) != QGBDT_OK) return rc;
     if (!c->d_h && c->prm.objective == 0 && (rc = alloc_dev(c, &c->d_h, (size_t)c->N, "hessian buffer")) != QGBDT_OK)
         return rc;
+    // leaves split per pass: fewer with thousands of features (the finishing kernel has a block per
+    // feature and leaf, the histogram pool a slot of F x bins words per split)
+    if (c->grow_jobs <= 1 || !c->d_recs) {
+        int k = 8192 / (c->F > 0 ? c->F : 1);
+        c->grow_jobs = k < 2 ? 2 : (k > GROW_MAX_JOBS ? GROW_MAX_JOBS : k);
+        c->grow_xcap = 2 * qg_grow_parts_cap(c) + c->grow_jobs;
+        c->grow_bits_stride = ((size_t)c->N + 31) / 32 + 64;
+    }
     if (!c->d_hist_pool &&
-        (rc = alloc_dev(c, &c->d_hist_pool, (size_t)L * c->F * c->nb, "histogram pool")) != QGBDT_OK)
+        (rc = alloc_dev(c, &c->d_hist_pool, (size_t)qg_grow_max_slots(L) * c->F * c->nb, "histogram pool")) != QGBDT_OK)
         return rc;
     if (!c->d_leaves && (rc = alloc_dev(c, &c->d_leaves, (size_t)L, "leaf records")) != QGBDT_OK) return rc;
-    if (!c->d_leaf_gain && (rc = alloc_dev(c, &c->d_leaf_gain, (size_t)L, "leaf gains")) != QGBDT_OK) return rc;
+    if (!c->d_recs && (rc = alloc_dev(c, &c->d_recs, (size_t)qg_grow_max_recs(L), "growth records")) != QGBDT_OK) return rc;
+    if (!c->d_front && (rc = alloc_dev(c, &c->d_front, (size_t)L, "leaf table")) != QGBDT_OK) return rc;
+    if (!c->d_grow_bits &&
+        (rc = alloc_dev(c, &c->d_grow_bits, c->grow_bits_stride * (size_t)c->grow_jobs, "partition bits")) != QGBDT_OK)
+        return rc;
+    if (!c->d_grow_partial &&
+        (rc = alloc_dev(c, &c->d_grow_partial, (size_t)c->grow_xcap * c->tiles.size() * 4 * c->nb * 32,
+                        "partial histograms of tree growth")) != QGBDT_OK)
+        return rc;
     if (!c->d_ent0 && (rc = alloc_dev(c, &c->d_ent0, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_ent1 && (rc = alloc_dev(c, &c->d_ent1, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
-    if (!c->d_cand && (rc = alloc_dev(c, &c->d_cand, (size_t)2 * c->F, "candidate records")) != QGBDT_OK)
+    if (!c->d_cand && (rc = alloc_dev(c, &c->d_cand, (size_t)2 * c->F * c->grow_jobs, "candidate records")) != QGBDT_OK)
         return rc;
     if ((rc = qg_build_columns(c, st)) != QGBDT_OK) return rc;
     if (!c->d_gs) {
@@ -133,6 +149,14 @@ int qgbdt_train(qgbdt_ctx *c, const float *d_labels, float *d_scores, uint32_t f
     c->leaf_n[0] = c->N;
     if ((rc = qg_iota(c, st)) != QGBDT_OK) return rc;
     QG_CUDA(c, cudaStreamSynchronize(st));
+    if (!c->profile_hist) {
+        // launches replayed from the growth graphs: per tree the first commit, then the passes
+        int64_t passes = (int64_t)(hg->passes - before.passes) - num_trees;
+        if (passes < 0) passes = 0;
+        c->n_launches += num_trees + passes * c->grow_pass_launches;
+    }
+    c->n_passes += (int64_t)(hg->passes - before.passes);
+    c->n_extra_builds += (int64_t)(hg->extra_builds - before.extra_builds);
     c->n_hist_builds += (int64_t)(hg->hist_builds - before.hist_builds);
     c->n_hist_row_features += (int64_t)(hg->hist_rows - before.hist_rows) * c->F;
     c->hist_prof_bytes += (int64_t)(hg->hist_rows - before.hist_rows) * (c->F + c->code_bytes + 4) +

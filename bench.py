@@ -337,6 +337,8 @@ def run_ours(args):
     scores = torch.zeros(n, device="cuda")
     K, W = args.steps, args.warmup
 
+    if args.stream_path:
+        ctx.profile_histograms(True)
     ctx.train(wl.labels, scores, 0, W)                       # warm-up trees 0 .. W-1
     torch.cuda.synchronize()
     c0 = ctx.get_counters()
@@ -470,6 +472,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=sorted(WORKLOAD_ROWS))
     ap.add_argument("--rows", type=int, default=0, help="override the workload's row count (profiling captures)")
+    ap.add_argument("--stream-path", action="store_true",
+                    help="launch every kernel of tree growth on the stream (the host follows the passes) instead of "
+                         "replaying the growth graph: for per-kernel launch lists, not for timing")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="print the histogram-kernel sweep table instead")

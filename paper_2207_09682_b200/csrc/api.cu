@@ -63,6 +63,10 @@ void free_data(qgbdt_ctx *c) {
     dev_free(c->d_hist_pool);
     dev_free(c->d_leaves);
     dev_free(c->d_recs);
+    dev_free(c->d_rec_gain);
+    dev_free(c->d_rec_child);
+    dev_free(c->d_rec_pos);
+    dev_free(c->d_rec_parent);
     dev_free(c->d_front);
     dev_free(c->d_grow_bits);
     dev_free(c->d_grow_partial);

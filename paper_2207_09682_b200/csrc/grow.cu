@@ -33,6 +33,10 @@ __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) 
 struct GrowArgs {
     GrowState *gs;
     NodeRec *recs;
+    double *rec_gain;                // per growth record: gain of its best split (-inf: none) ...
+    int32_t *rec_child;              // ... first child record if it has been split, else -1 ...
+    int32_t *rec_pos;                // ... (node << 1 | side) of its parent once it is numbered, else -1 ...
+    int32_t *rec_parent;             // ... and the record it was split from (-1: the root)
     LeafRec *leaves;
     int32_t *front;                  // [L] growth record of every numbered leaf
     DevState *state;
@@ -48,7 +52,7 @@ struct GrowArgs {
     const unsigned long long *partial;
     SplitRec *cand;                  // [jobs][F][2] best candidates of every feature for the two children
     int F, nb, L;
-    int K;                           // leaves per pass
+    int K, slack;                    // leaves per pass; leaves that may be split ahead of their confirmation
     int xcap, parts_cap, n_tiles;    // histogram CTAs per tile of a launch, of one leaf; tiles
     int max_recs, max_slots;         // growth records and histogram slots allocated
     SplitParams sp;                  // G, H, n_s are filled per leaf on the device
@@ -59,8 +63,11 @@ struct GrowArgs {
     int use_cond;                    // 0: launched on a stream, the host reads gs->done
 };
 
-__global__ void k_grow_begin(GrowState *gs, NodeRec *recs, LeafRec *leaves, int32_t *front, const DevState *state,
-                             uint32_t N, int tree_slot) {
+__global__ void k_grow_begin(GrowState *gs, NodeRec *recs, double *rec_gain, int32_t *rec_child, int32_t *rec_pos,
+                             LeafRec *leaves, int32_t *front, const DevState *state, uint32_t N, int tree_slot) {
+    rec_gain[0] = -__longlong_as_double(0x7FF0000000000000LL);
+    rec_child[0] = -1;
+    rec_pos[0] = -1;
     gs->tree_slot = tree_slot;
     NodeRec r;
     r.off = 0; r.n = N; r.buf = -1; r.slot = 0;
@@ -94,19 +101,13 @@ __device__ inline void warp_range(uint32_t nw, uint32_t gw, uint32_t n_count, ui
     w1 = w0 + per < nw ? w0 + per : nw;
 }
 
-// The job whose block range [pb0, pb0 + pb) holds block b, or -1.
+// The job whose block range [pb0, pb0 + pb) holds block b, or -1: lane i of the calling warp looks
+// at job i.
 __device__ inline int job_of_block(const GrowState *gs, int n_jobs, int b) {
-    int p0[GROW_MAX_JOBS], pn[GROW_MAX_JOBS];
-#pragma unroll
-    for (int i = 0; i < GROW_MAX_JOBS; ++i) {
-        p0[i] = gs->jobs[i].pb0;
-        pn[i] = gs->jobs[i].pb;
-    }
-    int j = -1;
-#pragma unroll
-    for (int i = 0; i < GROW_MAX_JOBS; ++i)
-        if (i < n_jobs && b >= p0[i] && b < p0[i] + pn[i]) j = i;
-    return j;
+    const int li = threadIdx.x & 31;
+    const int p0 = gs->jobs[li].pb0, pn = gs->jobs[li].pb;
+    const unsigned hit = __ballot_sync(0xffffffffu, li < n_jobs && b >= p0 && b < p0 + pn);
+    return hit ? __ffs(hit) - 1 : -1;
 }
 
 // Four words of 32 rows at a time, so that the dependent loads (pair -> bin word) of the four are
@@ -518,8 +519,10 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
         if (qg_rec_better(sm[1][w], bL)) bL = sm[1][w];
     }
     job->finish_count = 0;
+    const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
     if (ROOT) {
         a.recs[0].best = bS;
+        a.rec_gain[0] = bS.valid ? bS.gain : NEG;
         return;
     }
     const int dstbuf = jbuf == 0 ? 1 : 0;
@@ -540,22 +543,30 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     a.recs[child0] = lf;
     a.recs[child0 + 1] = rt;
     a.recs[jrec].nl = nl;
+    a.rec_gain[child0] = lf.best.valid ? lf.best.gain : NEG;
+    a.rec_gain[child0 + 1] = rt.best.valid ? rt.best.gain : NEG;
+    a.rec_child[child0] = a.rec_child[child0 + 1] = -1;
+    a.rec_pos[child0] = a.rec_pos[child0 + 1] = -1;
+    a.rec_parent[child0] = a.rec_parent[child0 + 1] = jrec;
 }
 
-// Shared memory of the commit kernel: per numbered leaf its gain, its growth record and the list
-// of splits confirmed in this launch; per growth record its gain, its children (or -1) and its
-// place in the tree.
+// Shared memory of the commit kernel.  A region that first holds, per numbered leaf, its gain, its
+// growth record and the list of splits confirmed in this launch, and later the compacted list of
+// the records whose split is not confirmed (the gain that orders them, the record, and the records
+// by rank); then, per growth record, its gain, its children (or -1) and its place in the tree.
+__host__ __device__ inline size_t commit_region_bytes(int L) {
+    const size_t a = (size_t)L * (sizeof(double) + 3 * sizeof(int));
+    const size_t b = (size_t)(L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8) * (sizeof(double) + 2 * sizeof(int));
+    return ((a > b ? a : b) + 15) / 16 * 16;
+}
 __host__ __device__ inline size_t commit_smem_bytes(int L, int max_recs) {
-    return (size_t)L * (sizeof(double) + 3 * sizeof(int)) + (size_t)max_recs * (sizeof(double) + 2 * sizeof(int)) + 16;
+    return commit_region_bytes(L) + (size_t)max_recs * (sizeof(double) + 2 * sizeof(int)) + 16;
 }
 
-// Best of (gain, index) over a warp: larger gain, lower index on equal gain; index < 0: nothing.
-__device__ inline void warp_best(double &g, int &i) {
-    for (int o = 16; o > 0; o >>= 1) {
-        const double og = __shfl_xor_sync(0xffffffffu, g, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, i, o);
-        if (oi >= 0 && (i < 0 || og > g || (og == g && oi < i))) { g = og; i = oi; }
-    }
+// Doubles as unsigned keys of the same order (-inf is the smallest key of a real gain; 0 is below all).
+__device__ inline unsigned long long gain_key(double g) {
+    const long long b = __double_as_longlong(g);
+    return (unsigned long long)(b ^ ((b >> 63) | (long long)0x8000000000000000ULL));
 }
 
 // One block.  (1) Replays best-first growth over what has been split so far: takes the numbered
@@ -577,49 +588,60 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         return;
     }
     const int L = a.L, R = a.max_recs;
+    // the region, first use
     double *fg = reinterpret_cast<double *>(smem_raw);          // [L] gain of numbered leaf i
-    double *cg = fg + L;                                        // [R] gain of record r if it can still be split
-    int *sf = reinterpret_cast<int *>(cg + R);                  // [L] record of numbered leaf i
+    int *sf = reinterpret_cast<int *>(fg + L);                  // [L] record of numbered leaf i
     int *cl_rec = sf + L;                                       // [L] confirmed in this launch: the record split ...
     int *cl_leaf = cl_rec + L;                                  // [L] ... and the number of the leaf it was
-    int *cs = cl_leaf + L;                                      // [R] first child record of a split record, else -1
-    int *spn = cs + R;                                          // [R] (node << 1 | side) of a numbered record's parent, -1: root
-    __shared__ int s_done, s_leaves, s_mand, s_commits;
+    // the region, second use
+    const int max_cand = L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8;
+    double *cand_g = reinterpret_cast<double *>(smem_raw);      // [max_cand] gains of the leaves that can still be split
+    int *cand_r = reinterpret_cast<int *>(cand_g + max_cand);   // [max_cand] their records
+    // per record
+    double *cg = reinterpret_cast<double *>(smem_raw + commit_region_bytes(L));   // [R]
+    int *cs = reinterpret_cast<int *>(cg + R);                  // [R] first child record of a split record, else -1
+    int *spn = cs + R;                                          // [R] (node << 1 | side) of a numbered record's parent, -1
+    __shared__ int s_done, s_leaves, s_mand, s_commits, s_ncand;
     __shared__ unsigned long long s_rows;
-    __shared__ double wg[COMMIT_THREADS / 32];
-    __shared__ int wi[COMMIT_THREADS / 32];
     __shared__ int s_pick[GROW_MAX_JOBS];
-    __shared__ uint32_t s_n[GROW_MAX_JOBS];
 
     const int n_leaves0 = gs->n_leaves, n_recs = gs->n_recs, n_exec = gs->n_exec, tree_slot = gs->tree_slot;
     for (int r = tid; r < n_recs; r += COMMIT_THREADS) {
-        const NodeRec *q = a.recs + r;
-        const int st = q->state, c0 = q->child0, valid = q->best.valid, pn = q->parent_node, ps = q->parent_side;
-        const double g = q->best.gain;
-        cs[r] = st == 1 ? c0 : -1;
-        cg[r] = valid ? g : NEG;       // the gain of a leaf's best split, whether it has been split or not
-        spn[r] = pn < 0 ? -1 : (pn << 1 | ps);
+        cg[r] = a.rec_gain[r];
+        cs[r] = a.rec_child[r];
+        spn[r] = a.rec_pos[r];
     }
     for (int i = tid; i < n_leaves0; i += COMMIT_THREADS) sf[i] = a.front[i];
-    if (tid == 0) s_rows = 0;
+    if (tid == 0) { s_rows = 0; s_ncand = 0; }
     __syncthreads();
     for (int i = tid; i < n_leaves0; i += COMMIT_THREADS) fg[i] = cg[sf[i]];
     __syncthreads();
 
-    // ---- (1) warp 0 replays the best-first order
+    // ---- (1) warp 0 replays the best-first order.  Lane l keeps the best of the leaves l, l + 32, ...
+    //      and looks at them again only when one of them changes.
     if (warp == 0) {
         int n_leaves = n_leaves0, mand = -1, done = 0, commits = 0;
         const size_t no = (size_t)tree_slot * (L > 1 ? L - 1 : 1);
+        unsigned long long lk = 0;   // key of the lane's best gain (0: the lane has no leaf)
+        int li = 0x7FFFFFFF;
+        auto rescan = [&]() {
+            lk = 0;
+            li = 0x7FFFFFFF;
+            for (int i = lane; i < n_leaves; i += 32) {
+                const unsigned long long k = gain_key(fg[i]);
+                if (k > lk) { lk = k; li = i; }
+            }
+        };
+        rescan();
+        const unsigned long long neg_key = gain_key(NEG);
         for (;;) {
             if (n_leaves >= L) { done = 1; break; }
-            double bg = NEG;
-            int bi = -1;
-            for (int i = lane; i < n_leaves; i += 32) {
-                const double g = fg[i];
-                if (g > bg) { bg = g; bi = i; }
-            }
-            warp_best(bg, bi);
-            if (bi < 0) { done = 1; break; }
+            const unsigned hi = (unsigned)(lk >> 32), lo = (unsigned)lk;
+            const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
+            const unsigned ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+            const bool top = hi == mh && lo == ml;
+            const int bi = (int)__reduce_min_sync(0xffffffffu, top ? (unsigned)li : 0x7FFFFFFFu);
+            if ((((unsigned long long)mh << 32) | ml) <= neg_key || bi == 0x7FFFFFFF) { done = 1; break; }
             const int r = sf[bi], c0 = cs[r];
             if (c0 < 0) { mand = r; break; }
             const int node = n_leaves - 1, right = n_leaves;
@@ -642,28 +664,27 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
             __syncwarp();
             ++n_leaves;
             ++commits;
+            if (lane == (bi & 31) || lane == (right & 31)) rescan();
         }
         if (lane == 0) { s_done = done; s_leaves = n_leaves; s_mand = mand; s_commits = commits; }
     }
     __syncthreads();
     const int n_leaves = s_leaves, commits = s_commits, done = s_done, mand = s_mand;
 
-    // ---- the splits confirmed above, one thread each: node arrays, leaf records, tree positions
+    // ---- the splits confirmed above, one thread each: node arrays and tree positions
     {
         const size_t no = (size_t)tree_slot * (L > 1 ? L - 1 : 1);
         unsigned long long rows = 0;
         for (int t = tid; t < commits; t += COMMIT_THREADS) {
-            const int r = cl_rec[t], leaf = cl_leaf[t], node = n_leaves0 - 1 + t, right = node + 1;
+            const int r = cl_rec[t], node = n_leaves0 - 1 + t, c0 = cs[r];
             const NodeRec *q = a.recs + r;
-            const int c0 = q->child0;
             a.m_feature[no + node] = q->best.feature;
             a.m_bin[no + node] = q->best.bin;
             a.m_gain[no + node] = q->best.gain;
-            NodeRec *lc = a.recs + c0, *rc = lc + 1;
-            lc->parent_node = node; lc->parent_side = 0;
-            rc->parent_node = node; rc->parent_side = 1;
-            rows += lc->n < rc->n ? lc->n : rc->n;
-            (void)leaf; (void)right;
+            a.rec_pos[c0] = node << 1;
+            a.rec_pos[c0 + 1] = node << 1 | 1;
+            const uint32_t nl = q->nl, n = q->n;
+            rows += nl < n - nl ? nl : n - nl;
         }
         // leaf records: a leaf number may change hands more than once in a launch (a child that was
         // split ahead is confirmed right after its parent), so they are written from the replay's
@@ -680,7 +701,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         }
         if (rows) atomicAdd(&s_rows, rows);
     }
-    __syncthreads();
+    __syncthreads();   // the region is free from here on
     if (tid == 0) {
         gs->n_leaves = n_leaves;
         gs->hist_rows += s_rows;
@@ -697,14 +718,16 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         return;
     }
 
-    // ---- (2) the next batch: the leaf best-first growth needs next, then the unsplit leaves of
-    //      largest gain, as long as few enough leaves are split ahead of their confirmation and the
-    //      tree could still use them all
+    // ---- (2) the next batch.  Best-first growth takes a leaf when its gain is the largest among the
+    //      leaves that exist, and a leaf exists once its parent has been taken; so, as far as the gains
+    //      are known, the records whose split is not confirmed yet will be taken in the order of
+    //      min(own gain, gains of the ancestors not taken yet), and only the first `budget` of them,
+    //      the splits the tree still has room for.  The batch is the leaf needed next, then the unsplit
+    //      records in that order, as long as few enough leaves are split ahead of their confirmation.
     const int ahead = n_exec - (n_leaves - 1);            // split, not confirmed
-    const int room = (L - 1) - n_exec;                    // splits the tree can still use
+    const int budget = L - n_leaves;                      // splits the tree can still take
     int extra = a.K - 1;
-    if (extra > GROW_SLACK - ahead) extra = GROW_SLACK - ahead;
-    if (extra > room - 1) extra = room - 1;
+    if (extra > a.slack - ahead) extra = a.slack - ahead;
     if (extra > (R - n_recs) / 2 - 1) extra = (R - n_recs) / 2 - 1;
     if (extra > a.max_slots - 2 - n_exec) extra = a.max_slots - 2 - n_exec;
     if (extra < 0) extra = 0;
@@ -719,46 +742,77 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         }
         return;
     }
-    if (tid == 0) {
-        s_pick[0] = mand;
-        cs[mand] = -2;
+    int *by_rank = cand_r + max_cand;                     // [max_cand] record at every rank if it may join the batch, else -1
+    if (extra > 0) {
+        for (int r0 = 0; r0 < n_recs; r0 += COMMIT_THREADS) {
+            const int r = r0 + tid;
+            bool open = false;       // a split that is not confirmed, with an admissible gain
+            double e = NEG;
+            if (r < n_recs) {
+                const int c0 = cs[r];
+                e = cg[r];
+                open = e > NEG && !(c0 >= 0 && spn[c0] >= 0);
+                if (open) {
+                    int p = r;
+                    while (p != 0 && spn[p] < 0) {       // not numbered: its parent has not been taken yet
+                        p = a.rec_parent[p];
+                        const double pg = cg[p];
+                        e = pg < e ? pg : e;
+                    }
+                }
+            }
+            const unsigned m = __ballot_sync(0xffffffffu, open);
+            int base = 0;
+            if (lane == 0 && m) base = atomicAdd(&s_ncand, __popc(m));
+            base = __shfl_sync(0xffffffffu, base, 0);
+            if (open) {
+                const int k = base + __popc(m & ((1u << lane) - 1u));
+                if (k < max_cand) {
+                    cand_g[k] = e;
+                    cand_r[k] = r;
+                }
+            }
+        }
     }
     __syncthreads();
+    int n_cand = s_ncand;
+    if (n_cand > max_cand) n_cand = max_cand;   // cannot happen: the bound counts every record without a confirmed split
+    // rank of every open record (larger gain first, lower record on equal gain)
+    for (int i = tid; i < n_cand; i += COMMIT_THREADS) {
+        const double g = cand_g[i];
+        const int r = cand_r[i];
+        int rank = 0;
+        for (int k = 0; k < n_cand; ++k) {
+            const double og = cand_g[k];
+            rank += (og > g || (og == g && cand_r[k] < r)) ? 1 : 0;
+        }
+        by_rank[rank] = (rank < budget && cs[r] == -1 && r != mand) ? r : -1;
+    }
+    if (tid == 0) s_pick[0] = mand;
+    __syncthreads();
+    if (warp != 0) return;
+    // the first `extra` unsplit records in rank order
     int n_jobs = 1;
-    for (int k = 1; k <= extra; ++k) {
-        double bg = NEG;
-        int bi = -1;
-        for (int r = tid; r < n_recs; r += COMMIT_THREADS) {
-            const double g = cs[r] == -1 ? cg[r] : NEG;   // not split and not in the batch yet
-            if (g > bg) { bg = g; bi = r; }
-        }
-        warp_best(bg, bi);
-        if (lane == 0) { wg[warp] = bg; wi[warp] = bi; }
-        __syncthreads();
-        bg = wg[0];
-        bi = wi[0];
-        for (int w = 1; w < COMMIT_THREADS / 32; ++w) {
-            const double og = wg[w];
-            const int oi = wi[w];
-            if (oi >= 0 && (bi < 0 || og > bg || (og == bg && oi < bi))) { bg = og; bi = oi; }
-        }
-        if (bi < 0) break;          // nothing left to split ahead (the same value in every thread)
-        if (tid == 0) {
-            s_pick[k] = bi;
-            cs[bi] = -2;
-        }
-        n_jobs = k + 1;
-        __syncthreads();
+    for (int k0 = 0; k0 < n_cand && n_jobs < 1 + extra; k0 += 32) {
+        const int k = k0 + lane;
+        const int r = k < n_cand ? by_rank[k] : -1;
+        const unsigned m = __ballot_sync(0xffffffffu, r >= 0);
+        const int pos = n_jobs + __popc(m & ((1u << lane) - 1u));
+        if (r >= 0 && pos < 1 + extra) s_pick[pos] = r;
+        n_jobs += __popc(m);
     }
-    __syncthreads();
+    if (n_jobs > 1 + extra) n_jobs = 1 + extra;
+    __syncwarp();
 
-    // ---- (3) the job table
-    if (tid < n_jobs) {
-        const int r = s_pick[tid];
+    // ---- (3) the job table, by warp 0: lane j fills job j, then the lanes share out the blocks
+    uint32_t n_j = 0;
+    if (lane < n_jobs) {
+        const int r = s_pick[lane];
         NodeRec *q = a.recs + r;
         const SplitRec best = q->best;
         const FeatRec pf = a.feat_rec[best.feature];
-        GrowJob *job = gs->jobs + tid;
+        GrowJob *job = gs->jobs + lane;
+        n_j = q->n;
         job->rec = r;
         job->feature = best.feature;
         job->bin = best.bin;
@@ -767,7 +821,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         job->col = pf.col;
         job->col8 = pf.col8;
         job->off = q->off;
-        job->n = q->n;
+        job->n = n_j;
         job->buf = q->buf;
         job->nl = 0;
         job->gl = best.gl;
@@ -775,61 +829,44 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         job->PG = q->G;
         job->PH = q->H;
         job->parent_slot = q->slot;
-        job->small_slot = 1 + n_exec + tid;
-        job->child0 = n_recs + 2 * tid;
+        job->small_slot = 1 + n_exec + lane;
+        job->child0 = n_recs + 2 * lane;
         job->finish_count = 0;
         q->state = 1;
-        q->child0 = n_recs + 2 * tid;
-        s_n[tid] = q->n;
+        q->child0 = n_recs + 2 * lane;
+        a.rec_child[r] = n_recs + 2 * lane;
     }
-    __syncthreads();
-    if (tid == 0) {
-        // blocks of the partition kernels: in proportion to the rows, at least one per leaf
-        int want[GROW_MAX_JOBS];
-        long long sum = 0;
-        const int pb_cap = a.pb_total - a.K;
-        for (int jj = 0; jj < n_jobs; ++jj) {
-            long long w = ((long long)s_n[jj] + 2047) / 2048;
-            if (w < 1) w = 1;
-            if (w > pb_cap) w = pb_cap;
-            want[jj] = (int)w;
-            sum += w;
-        }
-        int at = 0;
-        for (int jj = 0; jj < n_jobs; ++jj) {
-            int w = want[jj];
-            if (sum > pb_cap) {
-                w = (int)((long long)w * pb_cap / sum);
-                if (w < 1) w = 1;
-            }
-            gs->jobs[jj].pb0 = at;
-            gs->jobs[jj].pb = w;
-            at += w;
-        }
-        // histogram CTAs per tile: one per 1024 rows of half the leaf (the smaller child has at most
-        // that many rows), at most a leaf's share of the SMs, scaled down when the batch wants more
-        // than a launch has
-        sum = 0;
-        const int xc = a.xcap - a.K;
-        for (int jj = 0; jj < n_jobs; ++jj) {
-            long long w = ((long long)(s_n[jj] / 2) + MIN_ROWS_PER_CTA - 1) / MIN_ROWS_PER_CTA;
-            if (w < 1) w = 1;
-            if (w > a.parts_cap) w = a.parts_cap;
-            want[jj] = (int)w;
-            sum += w;
-        }
-        at = 0;
-        for (int jj = 0; jj < n_jobs; ++jj) {
-            int w = want[jj];
-            if (sum > xc) {
-                w = (int)((long long)w * xc / sum);
-                if (w < 1) w = 1;
-            }
-            gs->jobs[jj].cta0 = at;
-            gs->jobs[jj].parts = w;
-            gs->jobs[jj].slot0 = at * a.n_tiles;
-            at += w;
-        }
+    // blocks of the partition kernels: in proportion to the rows, at least one per leaf; histogram
+    // CTAs per tile: one per 1024 rows of half the leaf (the smaller child has at most that many
+    // rows), at most a leaf's share of the SMs; both scaled down when the batch wants more than a
+    // launch has
+    const uint32_t pb_cap = (uint32_t)(a.pb_total - a.K), xc = (uint32_t)(a.xcap - a.K);
+    uint32_t wpb = 0, wpt = 0;
+    if (lane < n_jobs) {
+        wpb = (n_j + 2047u) / 2048u;
+        wpb = wpb < 1u ? 1u : (wpb > pb_cap ? pb_cap : wpb);
+        wpt = (n_j / 2u + MIN_ROWS_PER_CTA - 1u) / MIN_ROWS_PER_CTA;
+        wpt = wpt < 1u ? 1u : (wpt > (uint32_t)a.parts_cap ? (uint32_t)a.parts_cap : wpt);
+    }
+    const uint32_t spb = __reduce_add_sync(0xffffffffu, wpb), spt = __reduce_add_sync(0xffffffffu, wpt);
+    if (lane < n_jobs) {
+        if (spb > pb_cap) { wpb = wpb * pb_cap / spb; if (wpb < 1u) wpb = 1u; }
+        if (spt > xc) { wpt = wpt * xc / spt; if (wpt < 1u) wpt = 1u; }
+    }
+    uint32_t apb = wpb, apt = wpt;   // inclusive prefix sums over the lanes
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t u = __shfl_up_sync(0xffffffffu, apb, o), v = __shfl_up_sync(0xffffffffu, apt, o);
+        if (lane >= o) { apb += u; apt += v; }
+    }
+    if (lane < n_jobs) {
+        GrowJob *job = gs->jobs + lane;
+        job->pb0 = (int)(apb - wpb);
+        job->pb = (int)wpb;
+        job->cta0 = (int)(apt - wpt);
+        job->parts = (int)wpt;
+        job->slot0 = (int)(apt - wpt) * a.n_tiles;
+    }
+    if (lane == 0) {
         gs->n_jobs = n_jobs;
         gs->n_exec = n_exec + n_jobs;
         gs->n_recs = n_recs + 2 * n_jobs;
@@ -840,6 +877,10 @@ void fill_args(qgbdt_ctx *c, GrowArgs &a) {
     const int L = c->prm.num_leaves;
     a.gs = c->d_gs;
     a.recs = c->d_recs;
+    a.rec_gain = c->d_rec_gain;
+    a.rec_child = c->d_rec_child;
+    a.rec_pos = c->d_rec_pos;
+    a.rec_parent = c->d_rec_parent;
     a.leaves = c->d_leaves;
     a.front = c->d_front;
     a.state = c->d_state;
@@ -859,11 +900,12 @@ void fill_args(qgbdt_ctx *c, GrowArgs &a) {
     a.nb = c->nb;
     a.L = L;
     a.K = c->grow_jobs;
+    a.slack = qg_grow_slack(c);
     a.xcap = c->grow_xcap;
     a.n_tiles = (int)c->tiles.size();
     a.parts_cap = qg_grow_parts_cap(c);
-    a.max_recs = qg_grow_max_recs(L);
-    a.max_slots = qg_grow_max_slots(L);
+    a.max_recs = qg_grow_max_recs(c);
+    a.max_slots = qg_grow_max_slots(c);
     a.sp.G = a.sp.H = a.sp.n_s = 0;
     a.sp.kg = qg_levels_g(c->prm.bits);
     a.sp.kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
@@ -910,8 +952,12 @@ int qg_grow_parts_cap(const qgbdt_ctx *c) {
     return p < 1 ? 1 : p;
 }
 
-int qg_grow_max_recs(int L) { return 1 + 2 * (L - 1 + GROW_SLACK) + 2 * GROW_MAX_JOBS; }
-int qg_grow_max_slots(int L) { return L + GROW_SLACK + GROW_MAX_JOBS + 2; }
+int qg_grow_slack(const qgbdt_ctx *c) {
+    const int s = 3 * c->grow_jobs;
+    return s > GROW_SLACK ? GROW_SLACK : s;
+}
+int qg_grow_max_recs(const qgbdt_ctx *c) { return 1 + 2 * (c->prm.num_leaves - 1 + qg_grow_slack(c)) + 2 * c->grow_jobs; }
+int qg_grow_max_slots(const qgbdt_ctx *c) { return c->prm.num_leaves + qg_grow_slack(c) + c->grow_jobs + 2; }
 
 void qg_grow_graph_destroy(qgbdt_ctx *c) {
     if (c->grow_graph_exec) cudaGraphExecDestroy(reinterpret_cast<cudaGraphExec_t>(c->grow_graph_exec));
@@ -1004,7 +1050,8 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
         if (smem > (size_t)c->max_smem_optin) return qg_fail(c, QGBDT_ERR_ARG, "num_leaves too large for the commit step");
         QG_CUDA(c, cudaFuncSetAttribute(k_grow_commit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
-    k_grow_begin<<<1, 1, 0, st>>>(c->d_gs, c->d_recs, c->d_leaves, c->d_front, c->d_state, (uint32_t)c->N, tree_slot);
+    k_grow_begin<<<1, 1, 0, st>>>(c->d_gs, c->d_recs, c->d_rec_gain, c->d_rec_child, c->d_rec_pos, c->d_leaves, c->d_front,
+                                  c->d_state, (uint32_t)c->N, tree_slot);
     QG_LAUNCH_CHECK(c);
     int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
     if (rc != QGBDT_OK) return rc;

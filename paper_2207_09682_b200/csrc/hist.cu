@@ -136,21 +136,17 @@ template <int LOGW_T, int MODE>
 __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowHist g) {
     extern __shared__ __align__(1024) int sh[];
     const GrowState *gs = g.gs;
-    // the job table and the tile at once (one round trip to memory), then the early exits
+    // the job table and the tile at once (one round trip to memory), then the early exits: lane i of
+    // every warp looks at job i
     const int done = gs->done, n_jobs = gs->n_jobs;
-    int c0[GROW_MAX_JOBS], np[GROW_MAX_JOBS];
-#pragma unroll
-    for (int i = 0; i < GROW_MAX_JOBS; ++i) {
-        c0[i] = gs->jobs[i].cta0;
-        np[i] = gs->jobs[i].parts;
-    }
+    const int li = threadIdx.x & 31;
+    const int c0 = gs->jobs[li].cta0, np = gs->jobs[li].parts;
     TileDesc td = a.tiles[a.tile0 + blockIdx.y];
     if (done) return;
-    int j = -1;
-#pragma unroll
-    for (int i = 0; i < GROW_MAX_JOBS; ++i)
-        if (i < n_jobs && (int)blockIdx.x >= c0[i] && (int)blockIdx.x < c0[i] + np[i]) j = i;
-    if (j < 0) return;
+    const unsigned hit = __ballot_sync(0xffffffffu, li < n_jobs && (int)blockIdx.x >= c0 && (int)blockIdx.x < c0 + np);
+    if (!hit) return;
+    const int j = __ffs(hit) - 1;
+    const int jc0 = __shfl_sync(0xffffffffu, c0, j);
     const GrowJob *job = gs->jobs + j;
     const int buf = job->buf, parts = job->parts, slot0 = job->slot0, small_slot = job->small_slot;
     const uint32_t nl = job->nl, n = job->n, off = job->off;
@@ -160,7 +156,7 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowH
     a.n = nl <= nr ? nl : nr;
     a.hist = g.pool + (size_t)small_slot * g.hist_words;
     td.cta0 = slot0 + (a.tile0 + (int)blockIdx.y) * parts;
-    const uint32_t P = effective_parts((uint32_t)parts, a.n), part = blockIdx.x - (uint32_t)c0[j];
+    const uint32_t P = effective_parts((uint32_t)parts, a.n), part = blockIdx.x - (uint32_t)jc0;
     if (part >= P) return;
     hist_cta<HIST_THREADS, LOGW_T, MODE, 2>(a, td, part, P, sh);
 }

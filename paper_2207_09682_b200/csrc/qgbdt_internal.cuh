@@ -80,8 +80,9 @@ struct FeatRec {
 // node, until it meets a leaf that has not been split (which goes into the next batch) or the tree
 // is full.  The result is the tree best-first growth builds, whatever the batches were.
 
-constexpr int GROW_MAX_JOBS = 16;   // leaves split per pass, at most
-constexpr int GROW_SLACK = 48;      // leaves that may be split ahead of their confirmation at any time
+constexpr int GROW_MAX_JOBS = 32;   // leaves split per pass, at most (a warp looks a job up with one ballot)
+constexpr int GROW_SLACK = 96;      // leaves that may be split ahead of their confirmation at any time, at most
+                                    // (a context allows three times its leaves per pass)
 
 // A leaf with a number (confirmed by the commit step): what the refit and the score update read.
 struct LeafRec {
@@ -182,7 +183,11 @@ struct qgbdt_ctx {
     float *d_g = nullptr, *d_h = nullptr;
     unsigned long long *d_hist_pool = nullptr;  // [L][F][nb]
     LeafRec *d_leaves = nullptr;                // [L] numbered leaves of the tree being grown
-    NodeRec *d_recs = nullptr;                  // [1 + 2 (L - 1 + GROW_SLACK)] growth records
+    NodeRec *d_recs = nullptr;                  // [qg_grow_max_recs] growth records
+    double *d_rec_gain = nullptr;               // [qg_grow_max_recs] gain of a record's best split (-inf: none)
+    int32_t *d_rec_child = nullptr;             // [qg_grow_max_recs] first child record of a split record, -1: not split
+    int32_t *d_rec_pos = nullptr;               // [qg_grow_max_recs] (node << 1 | side) of a numbered record's parent, -1
+    int32_t *d_rec_parent = nullptr;            // [qg_grow_max_recs] the record a record was split from
     int32_t *d_front = nullptr;                 // [L] growth record of every numbered leaf
     int grow_jobs = 1;                          // leaves split per pass (<= GROW_MAX_JOBS; fewer with thousands of features)
     int grow_pb_total = 0;                      // blocks of a partition launch
@@ -273,7 +278,7 @@ int qg_partition(qgbdt_ctx *c, int64_t off, int64_t n, int feature, int bin, cud
 int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st);
 int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st);
 // the same two for a tree grown on the device (leaf table from the device leaf records)
-int qg_leaf_table_slots(int L);   // slots (and words / 7) of the leaf table of a tree grown on the device
+int qg_leaf_table_slots(int L);   // slots (and words / 7) of the leaf table of a tree grown on the device, at most
 int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_scores, int tree_slot, cudaStream_t st);
 
 // grow.cu: one tree by leaf-wise growth, every decision taken on the device
@@ -281,8 +286,9 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st);
 // hist.cu: histograms of the smaller children of the leaves being split in the current pass
 int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st);
 int qg_grow_parts_cap(const qgbdt_ctx *c);   // grow.cu: histogram CTAs per tile one leaf may get
-int qg_grow_max_recs(int L);                 // grow.cu: growth records / histogram slots a tree of L leaves may use
-int qg_grow_max_slots(int L);
+int qg_grow_slack(const qgbdt_ctx *c);       // grow.cu: leaves that may be split ahead of their confirmation
+int qg_grow_max_recs(const qgbdt_ctx *c);    // grow.cu: growth records / histogram slots a tree may use
+int qg_grow_max_slots(const qgbdt_ctx *c);
 int qg_hist_grow_configure(qgbdt_ctx *c);   // function attributes of the kernels it launches (before a capture)
 void qg_grow_graph_destroy(qgbdt_ctx *c);   // grow.cu: drops the captured split loop (buffers are about to change)
 

@@ -57,10 +57,14 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
         c->grow_bits_stride = ((size_t)c->N + 31) / 32 + 64;
     }
     if (!c->d_hist_pool &&
-        (rc = alloc_dev(c, &c->d_hist_pool, (size_t)qg_grow_max_slots(L) * c->F * c->nb, "histogram pool")) != QGBDT_OK)
+        (rc = alloc_dev(c, &c->d_hist_pool, (size_t)qg_grow_max_slots(c) * c->F * c->nb, "histogram pool")) != QGBDT_OK)
         return rc;
     if (!c->d_leaves && (rc = alloc_dev(c, &c->d_leaves, (size_t)L, "leaf records")) != QGBDT_OK) return rc;
-    if (!c->d_recs && (rc = alloc_dev(c, &c->d_recs, (size_t)qg_grow_max_recs(L), "growth records")) != QGBDT_OK) return rc;
+    if (!c->d_recs && (rc = alloc_dev(c, &c->d_recs, (size_t)qg_grow_max_recs(c), "growth records")) != QGBDT_OK) return rc;
+    if (!c->d_rec_gain && (rc = alloc_dev(c, &c->d_rec_gain, (size_t)qg_grow_max_recs(c), "growth records")) != QGBDT_OK) return rc;
+    if (!c->d_rec_child && (rc = alloc_dev(c, &c->d_rec_child, (size_t)qg_grow_max_recs(c), "growth records")) != QGBDT_OK) return rc;
+    if (!c->d_rec_pos && (rc = alloc_dev(c, &c->d_rec_pos, (size_t)qg_grow_max_recs(c), "growth records")) != QGBDT_OK) return rc;
+    if (!c->d_rec_parent && (rc = alloc_dev(c, &c->d_rec_parent, (size_t)qg_grow_max_recs(c), "growth records")) != QGBDT_OK) return rc;
     if (!c->d_front && (rc = alloc_dev(c, &c->d_front, (size_t)L, "leaf table")) != QGBDT_OK) return rc;
     if (!c->d_grow_bits &&
         (rc = alloc_dev(c, &c->d_grow_bits, c->grow_bits_stride * (size_t)c->grow_jobs, "partition bits")) != QGBDT_OK)

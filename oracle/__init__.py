@@ -169,6 +169,15 @@ def refit(g, h, idx, lambda_l2=0.0, learning_rate=1.0) -> tuple[float, float]:
     return w.value, v.value
 
 
+def leaf_value_quantized(G, H, gmax, hmax, bits, hess_levels_mode=0, const_hessian=False, lambda_l2=0.0,
+                         learning_rate=1.0) -> tuple[float, float]:
+    w, v = C.c_double(), C.c_float()
+    lib().qo_leaf_value_quantized(C.c_int64(int(G)), C.c_int64(int(H)), C.c_float(gmax), C.c_float(hmax), bits,
+                                  hess_levels_mode, int(bool(const_hessian)), C.c_double(lambda_l2),
+                                  C.c_double(learning_rate), C.byref(w), C.byref(v))
+    return w.value, v.value
+
+
 def sigmoid(s: float) -> float:
     return lib().qo_sigmoid(C.c_float(s))
 
@@ -196,8 +205,9 @@ class Tree:
     leaf_count: np.ndarray
 
 
-def train_tree(data, n_bins, labels, scores, params: Params, tree: int, want_row_leaf=False):
-    """One boosting iteration; ``scores`` (float32) is updated in place."""
+def train_tree(data, n_bins, labels, scores, params: Params, tree: int, want_row_leaf=False, refit=True):
+    """One boosting iteration; ``scores`` (float32) is updated in place.  refit=False: leaf values from
+    the quantized sums (Sec. 4.2) instead of the original gradients."""
     data = _c(data, np.uint8)
     labels = _c(labels, np.float32)
     assert scores.dtype == np.float32 and scores.flags.c_contiguous
@@ -211,8 +221,8 @@ def train_tree(data, n_bins, labels, scores, params: Params, tree: int, want_row
     lv = np.zeros(L, np.float32)
     lc = np.zeros(L, np.int64)
     rl = np.empty(n, np.int32) if want_row_leaf else None
-    rc = lib().qo_train_tree(_p(data, C.c_uint8), C.c_int64(n), J, n_bins, _p(labels, C.c_float),
-                             _p(scores, C.c_float), C.byref(params), C.c_uint32(tree),
+    rc = lib().qo_train_tree_opt(_p(data, C.c_uint8), C.c_int64(n), J, n_bins, _p(labels, C.c_float),
+                             _p(scores, C.c_float), C.byref(params), C.c_uint32(tree), 0 if refit else 1,
                              _p(nf, C.c_int32), _p(nbn, C.c_int32), _p(nl, C.c_int32),
                              _p(nr, C.c_int32), _p(ng, C.c_double), _p(lv, C.c_float),
                              _p(lc, C.c_int64), _p(rl, C.c_int32))

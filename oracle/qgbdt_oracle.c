@@ -14,6 +14,7 @@
  *   qo_find_split      Eq. 7 (gain from integer sums), exhaustive scan of Sec. 3
  *   qo_partition       the index sets I_s of Sec. 3 (stable filter)
  *   qo_refit           Eq. 3 with the original gradients (Sec. 4.2, leaf-value refitting)
+ *   qo_leaf_value_quantized   the leaf value from the quantized sums (Sec. 4.2, first formula)
  *   qo_gradients       Eq. 1 for the logistic and the squared loss (Sec. 5)
  *   qo_train_tree      Sec. 3 greedy leaf-wise growth + Fig. 1 workflow
  *
@@ -270,6 +271,23 @@ int qo_refit(const float *g, const float *h, const uint32_t *idx, int64_t n_s, d
     return QO_OK;
 }
 
+/* Sec. 4.2, the leaf value without refitting: w~ = -(G~ delta_g) / (H~ delta_h), from the
+ * integer sums of the leaf and the interval lengths of Eq. 5 (constant hessian: delta_h = 1).
+ * lambda_l2 joins the denominator as in Eq. 7's terms; a non-positive denominator gives 0.
+ * The leaf output is (float)(learning_rate * w~). */
+int qo_leaf_value_quantized(int64_t G, int64_t H, float gmax, float hmax, int bits,
+                            int hess_levels_mode, int const_hessian, double lambda_l2,
+                            double learning_rate, double *w_out, float *value_out) {
+    double dg = (double)gmax / (double)qo_levels_g(bits);
+    double dh = const_hessian ? 1.0 : (double)hmax / (double)qo_levels_h(bits, hess_levels_mode);
+    double gd = (double)G * dg;
+    double hd = (double)H * dh + lambda_l2;
+    double w = hd > 0.0 ? -gd / hd : 0.0;
+    *w_out = w;
+    *value_out = (float)(learning_rate * w);
+    return QO_OK;
+}
+
 /* ---------------------------------------------------------------- gradients */
 
 /* A sigmoid built only from exactly rounded primitives (rintf, fmaf, one divide)
@@ -324,12 +342,14 @@ int qo_gradients(int objective, const float *scores, const float *labels, int64_
  * a child c < 0 is leaf ~c), node gain, leaf_value[num_leaves], leaf_count[num_leaves].
  * Splitting leaf l keeps l as the left child and makes leaf `n_leaves` the right one.
  * row_leaf[n] (optional) receives the leaf of every row.  Returns the leaf count
- * (>= 1) or a negative error. */
-int qo_train_tree(const uint8_t *data, int64_t n, int32_t n_features, int32_t n_bins,
-                  const float *labels, float *scores, const qo_params *prm, uint32_t tree,
-                  int32_t *node_feature, int32_t *node_bin, int32_t *node_left,
-                  int32_t *node_right, double *node_gain, float *leaf_value,
-                  int64_t *leaf_count, int32_t *row_leaf) {
+ * (>= 1) or a negative error.
+ * leaf_values_from_quantized_sums != 0: the leaf values are w~ of Sec. 4.2 (no refit). */
+int qo_train_tree_opt(const uint8_t *data, int64_t n, int32_t n_features, int32_t n_bins,
+                      const float *labels, float *scores, const qo_params *prm, uint32_t tree,
+                      int leaf_values_from_quantized_sums, int32_t *node_feature,
+                      int32_t *node_bin, int32_t *node_left, int32_t *node_right,
+                      double *node_gain, float *leaf_value, int64_t *leaf_count,
+                      int32_t *row_leaf) {
     if (!data || !labels || !scores || !prm || n <= 0 || prm->num_leaves < 1) return QO_ERR_ARG;
     int L = prm->num_leaves;
     int const_h = prm->objective == 1;
@@ -394,7 +414,11 @@ int qo_train_tree(const uint8_t *data, int64_t n, int32_t n_features, int32_t n_
 
     for (int l = 0; l < n_leaves; ++l) {
         double w;
-        qo_refit(g, h, idx + off[l], cnt[l], prm->lambda_l2, prm->learning_rate, &w, &leaf_value[l]);
+        if (leaf_values_from_quantized_sums) /* Sec. 4.2: w~ from the leaf's integer sums */
+            qo_leaf_value_quantized(tot_g[l], tot_h[l], gmax, hmax, prm->bits, prm->hess_levels_mode,
+                                    const_h, prm->lambda_l2, prm->learning_rate, &w, &leaf_value[l]);
+        else
+            qo_refit(g, h, idx + off[l], cnt[l], prm->lambda_l2, prm->learning_rate, &w, &leaf_value[l]);
         leaf_count[l] = cnt[l];
         for (int64_t p = 0; p < cnt[l]; ++p) {
             uint32_t i = idx[off[l] + p];
@@ -407,6 +431,17 @@ done:
     free(g); free(h); free(gq); free(hq); free(idx); free(tmp); free(hg); free(hh);
     free(off); free(cnt); free(tot_g); free(tot_h); free(parent_node); free(parent_side); free(best);
     return rc;
+}
+
+/* The same with the leaf values refitted from the original gradients (the default of Sec. 4.2). */
+int qo_train_tree(const uint8_t *data, int64_t n, int32_t n_features, int32_t n_bins,
+                  const float *labels, float *scores, const qo_params *prm, uint32_t tree,
+                  int32_t *node_feature, int32_t *node_bin, int32_t *node_left,
+                  int32_t *node_right, double *node_gain, float *leaf_value,
+                  int64_t *leaf_count, int32_t *row_leaf) {
+    return qo_train_tree_opt(data, n, n_features, n_bins, labels, scores, prm, tree, 0, node_feature,
+                             node_bin, node_left, node_right, node_gain, leaf_value, leaf_count,
+                             row_leaf);
 }
 
 /* Full training: num_trees iterations; tree k's arrays live at offset k*(L-1) (nodes)

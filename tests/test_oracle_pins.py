@@ -685,3 +685,45 @@ def test_multi_tree_wrapper_is_the_loop_over_single_trees():
         assert (nf[s_] == t.feature).all() and (nb_[s_] == t.bin).all() and (nl[s_] == t.left).all()
         assert (nr[s_] == t.right).all() and (ng[s_] == t.gain).all()
         assert (lv[k * L:k * L + m] == t.leaf_value).all() and (lc[k * L:k * L + m] == t.leaf_count).all()
+
+
+def test_leaf_value_from_quantized_sums_is_the_closed_form():
+    # Sec. 4.2: w~ = -(G~ delta_g) / (H~ delta_h); exact rational arithmetic as the reference
+    from fractions import Fraction
+    r = np.random.default_rng(4)
+    for bits, mode, const_h in ((2, 0, False), (3, 0, False), (4, 1, False), (5, 0, True), (8, 0, False)):
+        kg, kh = oracle.levels(bits, mode)
+        for _ in range(20):
+            G, H = int(r.integers(-10**6, 10**6)), int(r.integers(1, 10**7))
+            gmax, hmax = np.float32(r.uniform(0.1, 3.0)), np.float32(r.uniform(0.01, 0.25))
+            lam = float(r.choice([0.0, 0.5]))
+            w, v = oracle.leaf_value_quantized(G, H, float(gmax), float(hmax), bits, mode, const_h, lam, 0.1)
+            dg = Fraction(float(gmax)) / kg
+            dh = Fraction(1) if const_h else Fraction(float(hmax)) / kh
+            exact = -(G * dg) / (H * dh + Fraction(lam))
+            assert w == pytest.approx(float(exact), rel=1e-14)
+            assert v == np.float32(0.1 * w)
+    # no admissible denominator: value 0 (an empty leaf with no regulariser)
+    assert oracle.leaf_value_quantized(5, 0, 1.0, 1.0, 3)[0] == 0.0
+
+
+def test_unrefitted_tree_has_the_same_structure_and_close_values():
+    # the leaf-value rule does not touch the growth of the tree; at 8 bits w~ is within the
+    # quantization error of the refitted value (E[G~ delta_g] = G, Sec. 4.2), at 2 bits it is coarser
+    data, y, _ = toy_classification(seed=11)
+    for bits, tol in ((8, 0.03), (2, 0.6)):
+        prm = oracle.make_params(bits=bits, num_leaves=8, seed=13, learning_rate=1.0)
+        s1, s2 = np.zeros(len(y), np.float32), np.zeros(len(y), np.float32)
+        a = oracle.train_tree(data, 32, y, s1, prm, 0)
+        b, row_leaf = oracle.train_tree(data, 32, y, s2, prm, 0, want_row_leaf=True, refit=False)
+        assert a.num_leaves == b.num_leaves and (a.feature == b.feature).all() and (a.bin == b.bin).all()
+        assert (a.leaf_count == b.leaf_count).all()
+        assert np.abs(a.leaf_value - b.leaf_value).max() < tol * np.abs(a.leaf_value).max()
+        assert (s2 == b.leaf_value[row_leaf]).all()
+        # each value is the closed form on the leaf's own integer sums
+        g, h = oracle.gradients(0, np.zeros(len(y), np.float32), y)
+        q = oracle.quantize(g, h, bits=bits, seed=13, tree=0)
+        for l in range(b.num_leaves):
+            rows = np.nonzero(row_leaf == l)[0]
+            G, H = int(q.gq[rows].astype(np.int64).sum()), int(q.hq[rows].astype(np.int64).sum())
+            assert b.leaf_value[l] == oracle.leaf_value_quantized(G, H, q.gmax, q.hmax, bits, learning_rate=1.0)[1]

@@ -365,6 +365,7 @@ def run_ours(args):
     ctx.train(wl.labels, scores, W + K, K)
     e3.record()
     torch.cuda.synchronize()
+    phases = ctx.get_timings()
     prof = ctx.get_histogram_profile()
     ctx.profile_histograms(False)
     prof_ms = e2.elapsed_time(e3)
@@ -408,9 +409,12 @@ def run_ours(args):
                           "ms_per_tree_at_peak": step_total / K / (peak * 1e6),
                           "bytes_per_tree_by_step": {k: v / K for k, v in step_bytes.items()},
                           "note": "every kernel family of the timed trees: bytes the method has to move over the step time"},
+        "phases_us_per_tree": {k: round(1e3 * v["ms"] / K, 1) for k, v in phases.items()},
         "clocks": clocks.summary(),
         "host_cores": os.cpu_count(),
     }
+    line["phases_us_per_tree"]["note"] = ("CUDA events around every phase in the profiled pass (passes of tree growth on the "
+                                          "stream, the host following): where a tree's time goes, not how long it takes")
 
     # stand-alone histogram builds on the same data (root leaf and a 50 % subset)
     g = torch.empty(n, device="cuda")

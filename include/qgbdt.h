@@ -191,8 +191,13 @@ int qgbdt_train_host(qgbdt_ctx *ctx, const float *h_labels, float *h_scores, uin
 /* Options of a context (no counterpart in the paper).  Set them before qgbdt_load_binned /
  * qgbdt_train; unknown options and values out of range give QGBDT_ERR_ARG.
  *   QGBDT_OPT_COLUMN_COPY  1 (default): qgbdt_train keeps a column-major copy of the bin codes for
- *                          the row partition; 0: never (saves n_rows * n_features bytes). */
+ *                          the row partition; 0: never (saves n_rows * n_features bytes).
+ *   QGBDT_OPT_LEAF_VALUES  0 (default): qgbdt_train refits the leaf values from the original gradients
+ *                          (Eq. 3, Sec. 4.2); 1: it takes them from the quantized sums of the leaves,
+ *                          w~ = -(G~ delta_g) / (H~ delta_h + lambda_l2) (Sec. 4.2, first formula), and
+ *                          skips the pass over the gradients.  May be changed between train calls. */
 #define QGBDT_OPT_COLUMN_COPY 1
+#define QGBDT_OPT_LEAF_VALUES 2
 int qgbdt_set_option(qgbdt_ctx *ctx, int32_t option, int64_t value);
 /* What the context is doing (host scalars, no synchronisation):
  *   QGBDT_INFO_COLUMN_COPY  1 when the training workspaces hold the column-major copy (the row
@@ -213,6 +218,17 @@ int qgbdt_get_counters(const qgbdt_ctx *ctx, int64_t *kernel_launches, int64_t *
  * then clears the record. */
 int qgbdt_profile_histograms(qgbdt_ctx *ctx, int32_t enable);
 int qgbdt_get_histogram_profile(qgbdt_ctx *ctx, double *total_ms, int64_t *total_bytes, int64_t *builds);
+/* With the same switch on, qgbdt_train also brackets every phase of a boosting iteration (Fig. 1) with
+ * events, and runs the passes of tree growth on the stream with the host following them (slower than
+ * the graph it replays otherwise: this is for where the time goes, not for how long a tree takes).
+ * h_ms [QGBDT_N_PHASES] receives the summed times since the switch was set or the record cleared,
+ * h_intervals (may be NULL) the number of timed intervals; call it before
+ * qgbdt_get_histogram_profile, which clears the record.  Phases, in order: gradients (Eq. 1),
+ * quantization (Eq. 5, 6, 8), root histogram, row partition, children's histograms (Algorithm 1),
+ * finish (merge, subtraction, Eq. 7), commit (best-first order and next batch), leaf values (Eq. 3),
+ * score update. */
+#define QGBDT_N_PHASES 9
+int qgbdt_get_timings(qgbdt_ctx *ctx, double *h_ms, int64_t *h_intervals);
 
 /* Histogram build that allocates nothing (the paper has no counterpart; it exists for callers
  * that are not allowed to call cudaMalloc: code running inside a memory pool that owns the

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libqgbdt.so")
 
 OK, ERR_ARG, ERR_STATE, ERR_OVERFLOW, ERR_CUDA, ERR_ALLOC, ERR_VALUE = 0, -1, -2, -3, -4, -5, -6
 OPT_COLUMN_COPY = 1
+OPT_LEAF_VALUES = 2
 INFO_COLUMN_COPY = 1
 
 EXPORTS = [
@@ -23,7 +24,7 @@ EXPORTS = [
     "qgbdt_compute_gradients", "qgbdt_quantize_gradients", "qgbdt_build_histograms",
     "qgbdt_build_histograms_rows", "qgbdt_subtract_histograms", "qgbdt_find_best_split", "qgbdt_split_leaf",
     "qgbdt_get_leaf_rows", "qgbdt_reset_leaves", "qgbdt_refit_leaves", "qgbdt_apply_leaf_values", "qgbdt_train", "qgbdt_train_host",
-    "qgbdt_set_option", "qgbdt_get_info", "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile",
+    "qgbdt_set_option", "qgbdt_get_info", "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile", "qgbdt_get_timings",
     "qgbdt_build_histograms_noalloc", "qgbdt_noalloc_last_error",
 ]
 
@@ -273,6 +274,18 @@ def _get_histogram_profile(self) -> dict:
     return dict(total_ms=ms.value, total_bytes=nbytes.value, builds=builds.value)
 
 
+PHASES = ("gradients", "quantize", "root_histogram", "partition", "child_histograms", "finish", "commit",
+          "leaf_values", "score_update")
+
+
+def _get_timings(self) -> dict:
+    ms = (C.c_double * len(PHASES))()
+    cnt = (C.c_int64 * len(PHASES))()
+    self._check(self.lib.qgbdt_get_timings(self.h, ms, cnt))
+    return {name: dict(ms=ms[i], intervals=cnt[i]) for i, name in enumerate(PHASES)}
+
+
+Context.get_timings = _get_timings
 Context.profile_histograms = _profile_histograms
 Context.get_histogram_profile = _get_histogram_profile
 

@@ -17,6 +17,28 @@ int qg_fail(qgbdt_ctx *c, int code, const char *fmt, ...) {
     return code;
 }
 
+int qg_phase_begin(qgbdt_ctx *c, int phase, cudaStream_t st) {
+    if (!c->profile_hist) return QGBDT_OK;
+    if (c->hist_events_used + 2 > c->hist_events.size()) {
+        for (int i = 0; i < 2; ++i) {
+            cudaEvent_t e;
+            QG_CUDA(c, cudaEventCreate(&e));
+            c->hist_events.push_back(e);
+        }
+        c->hist_event_phase.push_back(phase);
+    }
+    c->hist_event_phase[c->hist_events_used / 2] = phase;
+    QG_CUDA(c, cudaEventRecord(c->hist_events[c->hist_events_used], st));
+    c->hist_events_used += 2;
+    return QGBDT_OK;
+}
+
+int qg_phase_end(qgbdt_ctx *c, cudaStream_t st) {
+    if (!c->profile_hist || c->hist_events_used < 2) return QGBDT_OK;
+    QG_CUDA(c, cudaEventRecord(c->hist_events[c->hist_events_used - 1], st));
+    return QGBDT_OK;
+}
+
 static_assert(sizeof(qgbdt_params) == 72 && sizeof(qgbdt_split) == 72 && sizeof(qgbdt_bin) == 8,
               "ABI struct sizes are part of the interface");
 
@@ -524,6 +546,10 @@ int qgbdt_set_option(qgbdt_ctx *c, int32_t option, int64_t value) {
             if (value != 0 && value != 1) return qg_fail(c, QGBDT_ERR_ARG, "QGBDT_OPT_COLUMN_COPY takes 0 or 1");
             c->want_column_copy = value != 0;
             return QGBDT_OK;
+        case QGBDT_OPT_LEAF_VALUES:
+            if (value != 0 && value != 1) return qg_fail(c, QGBDT_ERR_ARG, "QGBDT_OPT_LEAF_VALUES takes 0 or 1");
+            c->leaf_values_quantized = value != 0;
+            return QGBDT_OK;
         default:
             return qg_fail(c, QGBDT_ERR_ARG, "unknown option %d", option);
     }
@@ -557,10 +583,31 @@ int qgbdt_profile_histograms(qgbdt_ctx *c, int32_t enable) {
     return QGBDT_OK;
 }
 
+int qgbdt_get_timings(qgbdt_ctx *c, double *ms, int64_t *intervals) {
+    if (!c || !ms) return QGBDT_ERR_ARG;
+    for (int p = 0; p < QG_N_PHASES; ++p) {
+        ms[p] = 0.0;
+        if (intervals) intervals[p] = 0;
+    }
+    for (size_t i = 0; i + 1 < c->hist_events_used; i += 2) {
+        QG_CUDA(c, cudaEventSynchronize(c->hist_events[i + 1]));
+        float t = 0.f;
+        QG_CUDA(c, cudaEventElapsedTime(&t, c->hist_events[i], c->hist_events[i + 1]));
+        const int p = c->hist_event_phase[i / 2];
+        if (p >= 0 && p < QG_N_PHASES) {
+            ms[p] += t;
+            if (intervals) intervals[p]++;
+        }
+    }
+    return QGBDT_OK;
+}
+
 int qgbdt_get_histogram_profile(qgbdt_ctx *c, double *total_ms, int64_t *total_bytes, int64_t *builds) {
     if (!c) return QGBDT_ERR_ARG;
     double ms = 0.0;
     for (size_t i = 0; i + 1 < c->hist_events_used; i += 2) {
+        const int p = c->hist_event_phase[i / 2];
+        if (p != QG_PHASE_ROOT_HIST && p != QG_PHASE_CHILD_HIST) continue;
         QG_CUDA(c, cudaEventSynchronize(c->hist_events[i + 1]));
         float t = 0.f;
         QG_CUDA(c, cudaEventElapsedTime(&t, c->hist_events[i], c->hist_events[i + 1]));

@@ -21,7 +21,7 @@ namespace {
 
 constexpr int PART_THREADS = 256;
 constexpr int PART_WARPS = PART_THREADS / 32;
-constexpr int COMMIT_THREADS = 256;
+constexpr int COMMIT_THREADS = 1024;
 constexpr uint32_t MIN_ROWS_PER_CTA = 1024;   // same rule as the histogram kernel
 
 __device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
@@ -556,7 +556,9 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
 // by rank); then, per growth record, its gain, its children (or -1) and its place in the tree.
 __host__ __device__ inline size_t commit_region_bytes(int L) {
     const size_t a = (size_t)L * (sizeof(double) + 3 * sizeof(int));
-    const size_t b = (size_t)(L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8) * (sizeof(double) + 2 * sizeof(int));
+    size_t n = (size_t)(L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8);
+    if (n < 1024) n = 1024;   // the sort works on a power of two of entries
+    const size_t b = n * (sizeof(double) + 2 * sizeof(int));
     return ((a > b ? a : b) + 15) / 16 * 16;
 }
 __host__ __device__ inline size_t commit_smem_bytes(int L, int max_recs) {
@@ -594,9 +596,9 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
     int *cl_rec = sf + L;                                       // [L] confirmed in this launch: the record split ...
     int *cl_leaf = cl_rec + L;                                  // [L] ... and the number of the leaf it was
     // the region, second use
-    const int max_cand = L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8;
-    double *cand_g = reinterpret_cast<double *>(smem_raw);      // [max_cand] gains of the leaves that can still be split
-    int *cand_r = reinterpret_cast<int *>(cand_g + max_cand);   // [max_cand] their records
+    const int max_cand = (L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8) < 1024 ? 1024 : (L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8);
+    unsigned long long *cand_k = reinterpret_cast<unsigned long long *>(smem_raw);   // [max_cand] ordering keys of the open records
+    int *cand_r = reinterpret_cast<int *>(cand_k + max_cand);   // [max_cand] the records
     // per record
     double *cg = reinterpret_cast<double *>(smem_raw + commit_region_bytes(L));   // [R]
     int *cs = reinterpret_cast<int *>(cg + R);                  // [R] first child record of a split record, else -1
@@ -768,7 +770,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
             if (open) {
                 const int k = base + __popc(m & ((1u << lane) - 1u));
                 if (k < max_cand) {
-                    cand_g[k] = e;
+                    cand_k[k] = gain_key(e);
                     cand_r[k] = r;
                 }
             }
@@ -777,16 +779,47 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
     __syncthreads();
     int n_cand = s_ncand;
     if (n_cand > max_cand) n_cand = max_cand;   // cannot happen: the bound counts every record without a confirmed split
-    // rank of every open record (larger gain first, lower record on equal gain)
-    for (int i = tid; i < n_cand; i += COMMIT_THREADS) {
-        const double g = cand_g[i];
-        const int r = cand_r[i];
-        int rank = 0;
-        for (int k = 0; k < n_cand; ++k) {
-            const double og = cand_g[k];
-            rank += (og > g || (og == g && cand_r[k] < r)) ? 1 : 0;
+    // the open records in order: larger gain first, lower record on equal gain
+    if (n_cand <= 1024) {
+        // bitonic sort of the (key, record) pairs, padded to a power of two with entries that sort last
+        int m = 32;
+        while (m < n_cand) m <<= 1;
+        for (int i = n_cand + tid; i < m; i += COMMIT_THREADS) {
+            cand_k[i] = 0ull;
+            cand_r[i] = 0x7FFFFFFF;
         }
-        by_rank[rank] = (rank < budget && cs[r] == -1 && r != mand) ? r : -1;
+        __syncthreads();
+        for (int k = 2; k <= m; k <<= 1) {
+            for (int jj = k >> 1; jj > 0; jj >>= 1) {
+                const int i = tid, x = i ^ jj;
+                if (i < m && x > i) {
+                    const unsigned long long ka = cand_k[i], kb = cand_k[x];
+                    const int ra = cand_r[i], rb = cand_r[x];
+                    const bool a_first = ka > kb || (ka == kb && ra < rb);   // a belongs before b
+                    const bool want_a_first = (i & k) == 0;
+                    if (a_first != want_a_first) {
+                        cand_k[i] = kb; cand_k[x] = ka;
+                        cand_r[i] = rb; cand_r[x] = ra;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        for (int i = tid; i < n_cand; i += COMMIT_THREADS) {
+            const int r = cand_r[i];
+            by_rank[i] = (i < budget && cs[r] == -1 && r != mand) ? r : -1;
+        }
+    } else {
+        for (int i = tid; i < n_cand; i += COMMIT_THREADS) {
+            const unsigned long long g = cand_k[i];
+            const int r = cand_r[i];
+            int rank = 0;
+            for (int k = 0; k < n_cand; ++k) {
+                const unsigned long long og = cand_k[k];
+                rank += (og > g || (og == g && cand_r[k] < r)) ? 1 : 0;
+            }
+            by_rank[rank] = (rank < budget && cs[r] == -1 && r != mand) ? r : -1;
+        }
     }
     if (tid == 0) s_pick[0] = mand;
     __syncthreads();
@@ -924,23 +957,29 @@ void fill_args(qgbdt_ctx *c, GrowArgs &a) {
 }
 
 int launch_commit(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st) {
+    int rc = qg_phase_begin(c, QG_PHASE_COMMIT, st);
+    if (rc != QGBDT_OK) return rc;
     k_grow_commit<<<1, COMMIT_THREADS, commit_smem_bytes(a.L, a.max_recs), st>>>(a);
     QG_LAUNCH_CHECK(c);
-    return QGBDT_OK;
+    return qg_phase_end(c, st);
 }
 
 // One pass: the kernels that split the leaves of the current batch, then the commit step.
 int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st) {
+    int rc = qg_phase_begin(c, QG_PHASE_PARTITION, st);
+    if (rc != QGBDT_OK) return rc;
     k_grow_flags<<<a.pb_total, PART_THREADS, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     k_grow_scatter<<<a.pb_total, PART_THREADS, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
-    const int rc = qg_hist_grow(c, st);
-    if (rc != QGBDT_OK) return rc;
+    if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_hist_grow(c, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
     const dim3 fin((unsigned)c->F, (unsigned)a.K);
     if (c->F > c->sm_count * 8) k_grow_finish<false, 2><<<fin, 128, 0, st>>>(a);
     else k_grow_finish<false, 1><<<fin, 256, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
+    if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     return launch_commit(c, a, st);
 }
 
@@ -1055,8 +1094,10 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     QG_LAUNCH_CHECK(c);
     int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
     if (rc != QGBDT_OK) return rc;
+    if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
     k_grow_finish<true, 1><<<(unsigned)c->F, 256, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
+    if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     if (c->prm.num_leaves < 2) return QGBDT_OK;
     if (c->profile_hist) {
         // event records around every histogram launch: passes on the stream, the host follows

@@ -347,21 +347,12 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
     a.pass = 0;
     a.state = c->d_state;
 
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     if (c->profile_hist) {
-        if (c->hist_events_used + 2 > c->hist_events.size()) {
-            for (int i = 0; i < 2; ++i) {
-                cudaEvent_t e;
-                QG_CUDA(c, cudaEventCreate(&e));
-                c->hist_events.push_back(e);
-            }
-        }
-        ev0 = c->hist_events[c->hist_events_used++];
-        ev1 = c->hist_events[c->hist_events_used++];
         // algorithmic bytes of this build: bin codes + gradient code (+ row index) per row, histogram out
         c->hist_prof_bytes += n * (c->F + c->code_bytes + (d_rows ? 4 : 0)) + (int64_t)hist_bytes;
         c->hist_prof_launches++;
-        QG_CUDA(c, cudaEventRecord(ev0, st));
+        const int prc = qg_phase_begin(c, d_rows ? QG_PHASE_CHILD_HIST : QG_PHASE_ROOT_HIST, st);
+        if (prc != QGBDT_OK) return prc;
     }
     int rc;
     const bool merge_needed = c->max_parts > 1 && effective_parts((uint32_t)c->max_parts, (uint32_t)n) > 1;
@@ -385,8 +376,7 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
         k_hist_reduce<<<grid, 256, 0, st>>>(c->d_tiles, (uint32_t)n, c->nb, c->d_partial, d_hist, wide ? 1 : 0);
         QG_LAUNCH_CHECK(c);
     }
-    if (ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
-    return QGBDT_OK;
+    return qg_phase_end(c, st);
 }
 
 namespace {
@@ -470,19 +460,8 @@ int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
     g.ent1 = c->d_ent1;
     g.pool = c->d_hist_pool;
     g.hist_words = (size_t)c->F * c->nb;
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    if (c->profile_hist) {
-        if (c->hist_events_used + 2 > c->hist_events.size()) {
-            for (int i = 0; i < 2; ++i) {
-                cudaEvent_t e;
-                QG_CUDA(c, cudaEventCreate(&e));
-                c->hist_events.push_back(e);
-            }
-        }
-        ev0 = c->hist_events[c->hist_events_used++];
-        ev1 = c->hist_events[c->hist_events_used++];
-        QG_CUDA(c, cudaEventRecord(ev0, st));
-    }
+    int prc = qg_phase_begin(c, QG_PHASE_CHILD_HIST, st);
+    if (prc != QGBDT_OK) return prc;
     int rc;
     if (bits < 6 && a.shift == 16) {
         rc = launch_grow<0>(c, a, g, st);
@@ -495,7 +474,7 @@ int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
             rc = launch_grow<1>(c, a, g, st);
         }
     }
-    if (rc == QGBDT_OK && ev1) QG_CUDA(c, cudaEventRecord(ev1, st));
+    if (rc == QGBDT_OK) rc = qg_phase_end(c, st);
     return rc;
 }
 

@@ -202,6 +202,7 @@ struct qgbdt_ctx {
     uint8_t *d_colmajor = nullptr;              // [F][col_stride] column-major copy of the bin codes (training only)
     size_t col_stride = 0;
     bool want_column_copy = true;               // QGBDT_OPT_COLUMN_COPY
+    bool leaf_values_quantized = false;         // QGBDT_OPT_LEAF_VALUES: 1 = from the quantized sums (no refit)
     void *grow_graph_exec = nullptr;            // cudaGraphExec_t: the split loop of one tree
     int64_t grow_pass_launches = 0;             // kernel launches of one pass
     bool grow_graph_const_hess = false;         // objective it was captured for
@@ -218,12 +219,21 @@ struct qgbdt_ctx {
     // optional per-launch timing of the histogram kernel (event pairs on the launching stream)
     bool profile_hist = false;
     std::vector<cudaEvent_t> hist_events;  // start/stop pairs, reused
+    std::vector<int> hist_event_phase;     // phase (QG_PHASE_*) of every pair
     size_t hist_events_used = 0;
     int64_t hist_prof_bytes = 0, hist_prof_launches = 0;
     char err[512] = {0};
 };
 
 int qg_fail(qgbdt_ctx *c, int code, const char *fmt, ...);
+
+// Phases of a boosting iteration for the event timers (same order as qgbdt_get_timings reports them).
+enum { QG_PHASE_GRADIENTS = 0, QG_PHASE_QUANTIZE, QG_PHASE_ROOT_HIST, QG_PHASE_PARTITION, QG_PHASE_CHILD_HIST,
+       QG_PHASE_FINISH, QG_PHASE_COMMIT, QG_PHASE_REFIT, QG_PHASE_SCORES, QG_N_PHASES };
+// With the timers on, records the start event of a phase on `st` (api.cu); qg_phase_end records the
+// stop event of the phase begun last.  No-ops with the timers off.
+int qg_phase_begin(qgbdt_ctx *c, int phase, cudaStream_t st);
+int qg_phase_end(qgbdt_ctx *c, cudaStream_t st);
 
 #define QG_CUDA(c, expr)                                                                       \
     do {                                                                                       \

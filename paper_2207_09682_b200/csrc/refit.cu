@@ -115,6 +115,24 @@ __global__ void k_leaf_values(const long long *__restrict__ sums, int n_leaves, 
     }
 }
 
+// Sec. 4.2, leaf values without refitting: w~ = -(G~ delta_g) / (H~ delta_h + lambda) from the integer
+// totals of every numbered leaf of a tree grown on the device; output (float)(learning_rate * w~).
+__global__ void k_leaf_values_quantized(const LeafRec *__restrict__ leaves, const NodeRec *__restrict__ recs,
+                                        const GrowState *gs, const DevState *state, int kg, int kh, int const_h,
+                                        double lambda, double lr, double *__restrict__ w_out, float *__restrict__ v_out) {
+    const int n_leaves = gs->n_leaves;
+    const double dg = __ddiv_rn((double)__uint_as_float(state->gmax_bits), (double)kg);
+    const double dh = const_h ? 1.0 : __ddiv_rn((double)__uint_as_float(state->hmax_bits), (double)kh);
+    for (int leaf = blockIdx.x * blockDim.x + threadIdx.x; leaf < n_leaves; leaf += gridDim.x * blockDim.x) {
+        const NodeRec *q = recs + leaves[leaf].rec;
+        const double gd = __dmul_rn((double)q->G, dg);
+        const double hd = __dadd_rn(__dmul_rn((double)q->H, dh), lambda);
+        const double w = hd > 0.0 ? __ddiv_rn(-gd, hd) : 0.0;
+        w_out[leaf] = w;
+        v_out[leaf] = __double2float_rn(__dmul_rn(lr, w));
+    }
+}
+
 // Dynamic shared memory: [n_slots] offsets, [n_slots] values, [n_slots] pair buffers, so that
 // a row costs a search in shared memory and two global accesses (its pair, its score).  Four
 // rows per thread are in flight.
@@ -293,25 +311,37 @@ int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st) {
 int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_scores, int tree_slot, cudaStream_t st) {
     const int L = c->prm.num_leaves;     // upper bound; the kernels read the real counts from the grow state
     const int S = qg_leaf_table_slots(L);
+    int prc = qg_phase_begin(c, QG_PHASE_REFIT, st);
+    if (prc != QGBDT_OK) return prc;
     k_leaf_table<<<1, 256, 0, st>>>(c->d_leaves, c->d_recs, c->d_gs, c->d_leaf_table, c->d_leaf_table + 3 * (size_t)S, S,
                                     c->d_leaf_sums, c->d_m_num_leaves + tree_slot,
                                     c->d_m_leaf_count + (size_t)tree_slot * L, c->d_state);
     QG_LAUNCH_CHECK(c);
-    const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
-    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * S, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
-                                                                     c->d_leaf_table, S, c->d_gs, d_g, d_h,
-                                                                     c->d_leaf_sums);
-    QG_LAUNCH_CHECK(c);
-    k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, L, c->d_gs, c->prm.lambda_l2, c->prm.learning_rate,
-                                                   c->d_leaf_w, c->d_m_leaf_value + (size_t)tree_slot * L);
-    QG_LAUNCH_CHECK(c);
+    if (c->leaf_values_quantized) {
+        k_leaf_values_quantized<<<(L + 255) / 256, 256, 0, st>>>(
+            c->d_leaves, c->d_recs, c->d_gs, c->d_state, qg_levels_g(c->prm.bits),
+            qg_levels_h(c->prm.bits, c->prm.hess_levels_mode), c->const_hess ? 1 : 0, c->prm.lambda_l2,
+            c->prm.learning_rate, c->d_leaf_w, c->d_m_leaf_value + (size_t)tree_slot * L);
+        QG_LAUNCH_CHECK(c);
+    } else {
+        const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
+        k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * S, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
+                                                                         c->d_leaf_table, S, c->d_gs, d_g, d_h,
+                                                                         c->d_leaf_sums);
+        QG_LAUNCH_CHECK(c);
+        k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, L, c->d_gs, c->prm.lambda_l2, c->prm.learning_rate,
+                                                       c->d_leaf_w, c->d_m_leaf_value + (size_t)tree_slot * L);
+        QG_LAUNCH_CHECK(c);
+    }
+    if ((prc = qg_phase_end(c, st)) != QGBDT_OK) return prc;
+    if ((prc = qg_phase_begin(c, QG_PHASE_SCORES, st)) != QGBDT_OK) return prc;
     unsigned ab = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
     if (ab > (unsigned)c->sm_count * 16) ab = (unsigned)c->sm_count * 16;
     k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * 3 * S, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
                                                                    c->d_leaf_table, S, c->d_gs,
                                                                    c->d_m_leaf_value + (size_t)tree_slot * L, d_scores);
     QG_LAUNCH_CHECK(c);
-    return QGBDT_OK;
+    return qg_phase_end(c, st);
 }
 
 // Slots the leaf table of a grown tree may need: a leaf per slot, plus one per leaf split ahead.

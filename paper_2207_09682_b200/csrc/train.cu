@@ -17,9 +17,13 @@ int train_one_tree(qgbdt_ctx *c, const float *d_labels, float *d_scores, uint32_
     int rc;
     c->const_hess = const_h;
     c->quantized = false;
+    if ((rc = qg_phase_begin(c, QG_PHASE_GRADIENTS, st)) != QGBDT_OK) return rc;
     if ((rc = qg_gradients(c, d_scores, d_labels, c->d_g, const_h ? nullptr : c->d_h, true, first, st)) != QGBDT_OK)
         return rc;
+    if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_phase_begin(c, QG_PHASE_QUANTIZE, st)) != QGBDT_OK) return rc;
     if ((rc = qg_quantize(c, c->d_g, const_h ? nullptr : c->d_h, tree, nullptr, nullptr, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     c->quantized = true;
     if ((rc = qg_grow_tree(c, slot, st)) != QGBDT_OK) return rc;
     return qg_refit_grown(c, c->d_g, const_h ? nullptr : c->d_h, d_scores, slot, st);

@@ -422,7 +422,7 @@ TRAIN_CASES = [
 ]
 
 
-def train_case(name, rows, over, column_copy=None):
+def train_case(name, rows, over, column_copy=None, refit=True):
     wl = synth.CONFIGS[name](device="cpu", rows=rows) if name != "wide" else synth.wide(device="cpu", rows=rows, features=300)
     kw = dict(wl.params, seed=11)
     kw.update(over)
@@ -430,18 +430,26 @@ def train_case(name, rows, over, column_copy=None):
     ctx = binding.Context(binding.make_params(**kw))
     if column_copy is not None:
         ctx.set_option(binding.OPT_COLUMN_COPY, column_copy)
+    if not refit:
+        ctx.set_option(binding.OPT_LEAF_VALUES, 1)
     ctx.load_binned(dev(data), wl.n_bins)
     scores = torch.zeros(rows, device="cuda")
     model = ctx.train(dev(y), scores, 0, kw["num_trees"])
     ref_scores = np.zeros(rows, np.float32)
     prm = oracle.make_params(**kw)
     for k in range(kw["num_trees"]):
-        ref = oracle.train_tree(data, wl.n_bins, y, ref_scores, prm, k)
+        ref = oracle.train_tree(data, wl.n_bins, y, ref_scores, prm, k, refit=refit)
         compare_trees(model, k, ref)
     got = scores.cpu().numpy()
     assert np.allclose(got, ref_scores, rtol=1e-5, atol=1e-7)
     assert (got.view(np.uint32) == ref_scores.view(np.uint32)).all()
     return ctx
+
+
+@pytest.mark.parametrize("name,rows,over", [TRAIN_CASES[0], TRAIN_CASES[2], TRAIN_CASES[4]])
+def test_training_with_leaf_values_from_the_quantized_sums(name, rows, over):
+    # Sec. 4.2 without refitting: w~ from the integer sums of every leaf; trees, values and scores as the oracle's
+    train_case(name, rows, over, refit=False)
 
 
 @pytest.mark.parametrize("name,rows,over", TRAIN_CASES)
@@ -486,6 +494,28 @@ def test_training_resumes_and_host_variant_agrees():
     m_host = ctx_h.train(wl.labels.contiguous(), s3, 0, 4)  # host labels / scores
     assert torch.equal(s3, s1.cpu())
     assert (m_host.feature == m_all.feature).all() and (m_host.leaf_value == m_all.leaf_value).all()
+
+
+def test_phase_timers_cover_every_phase_and_do_not_change_the_trees():
+    wl = synth.tiny(device="cpu", rows=15_000)
+    kw = dict(wl.params, seed=3, num_trees=2)
+    data, y = wl.bins.numpy(), wl.labels.numpy()
+    ctx = make_ctx(data, wl.n_bins, **kw)
+    s1 = torch.zeros(15_000, device="cuda")
+    m1 = ctx.train(dev(y), s1, 0, 2)                 # growth replayed from the graph
+    ctx.profile_histograms(True)
+    s2 = torch.zeros(15_000, device="cuda")
+    m2 = ctx.train(dev(y), s2, 0, 2)                 # the same on the stream, every phase timed
+    t = ctx.get_timings()
+    prof = ctx.get_histogram_profile()
+    ctx.profile_histograms(False)
+    assert torch.equal(s1, s2) and (m1.feature == m2.feature).all() and (m1.leaf_value == m2.leaf_value).all()
+    assert set(t) == set(binding.PHASES)
+    for name, v in t.items():
+        assert v["intervals"] >= 2 and v["ms"] > 0.0, name
+    assert t["root_histogram"]["intervals"] == 2 and t["gradients"]["intervals"] == 2
+    hist_ms = t["root_histogram"]["ms"] + t["child_histograms"]["ms"]
+    assert abs(prof["total_ms"] - hist_ms) < 1e-6 and prof["builds"] == 2 + int(m2.num_leaves.sum()) - 2
 
 
 def test_stepwise_calls_compose_to_the_trained_tree():

@@ -328,12 +328,25 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     rows = args.rows or WORKLOAD_ROWS[args.workload]
-    wl = synth.CONFIGS[args.workload](device="cuda", rows=rows, seed=synth.MASTER_SEED + 100 + rank)
+    sharded = args.scaling == "strong" and world > 1
+    if sharded:
+        # data-distributed training (Sec. 7.3): one training set, every rank holds a contiguous row shard;
+        # the ranks exchange integer histograms, counts and the two maxima through NCCL all-reduces
+        from paper_2207_09682_b200 import dist as qdist
+        wl = synth.CONFIGS[args.workload](device="cuda", rows=rows, seed=synth.MASTER_SEED + 100)
+        lo, hi = rows * rank // world, rows * (rank + 1) // world
+        wl.bins, wl.labels = wl.bins[lo:hi].contiguous(), wl.labels[lo:hi].contiguous()
+        torch.cuda.empty_cache()
+    else:
+        wl = synth.CONFIGS[args.workload](device="cuda", rows=rows, seed=synth.MASTER_SEED + 100 + rank)
     n, features = wl.bins.shape
     n_bins = wl.n_bins
-    kw = dict(wl.params, num_trees=1, seed=1 + rank)
+    kw = dict(wl.params, num_trees=1, seed=1 if sharded else 1 + rank)
     ctx = binding.Context(binding.make_params(**kw))
     ctx.load_binned(wl.bins, wl.n_bins)
+    if sharded:
+        reducer = qdist.TorchDistReducer()
+        ctx.set_distributed(rank, world, lo, rows, reducer.callback)
     scores = torch.zeros(n, device="cuda")
     K, W = args.steps, args.warmup
 
@@ -388,11 +401,12 @@ def run_ours(args):
     line = {
         "metric": "hist_row_features_per_s", "value": rf / (ms * 1e-3), "unit": "row-features/s",
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": args.workload, "rows": n, "features": features, "bins": wl.n_bins,
+        "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": args.workload, "rows": rows if sharded else n, "features": features, "bins": wl.n_bins,
                    "bits": kw["bits"], "num_leaves": kw["num_leaves"], "objective": kw["objective"],
                    "l2_policy": "inputs larger than L2 (bin matrix %d MB)" % (n * ((features + 3) // 4 * 4) >> 20),
-                   "multi_gpu": "replicas only: one independent shard per GPU, no collective",
+                   "multi_gpu": ("rows sharded over the ranks, integer all-reduces through NCCL (Sec. 7.3)" if sharded else
+                                 "replicas: one independent training set per GPU, no data-path collective"),
                    "leaves_per_tree": [min(leaves), max(leaves)]},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -415,6 +429,13 @@ def run_ours(args):
     }
     line["phases_us_per_tree"]["note"] = ("CUDA events around every phase in the profiled pass (passes of tree growth on the "
                                           "stream, the host following): where a tree's time goes, not how long it takes")
+
+    if sharded:
+        line["exchanges"] = {"calls": reducer.calls, "words": reducer.words,
+                             "note": "all-reduce calls and 32/64-bit words of rank 0 since the context was created"}
+        print(json.dumps(line))
+        dist.destroy_process_group()
+        return
 
     # stand-alone histogram builds on the same data (root leaf and a 50 % subset)
     g = torch.empty(n, device="cuda")
@@ -479,6 +500,9 @@ def main():
     ap.add_argument("--stream-path", action="store_true",
                     help="launch every kernel of tree growth on the stream (the host follows the passes) instead of "
                          "replaying the growth graph: for per-kernel launch lists, not for timing")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="with --gpus N > 1: weak = N independent replicas of the workload (default); strong = one "
+                         "training set sharded by rows over the ranks (data-distributed training, NCCL all-reduces)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="print the histogram-kernel sweep table instead")

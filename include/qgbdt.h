@@ -188,6 +188,29 @@ int qgbdt_train(qgbdt_ctx *ctx, const float *d_labels, float *d_scores, uint32_t
 int qgbdt_train_host(qgbdt_ctx *ctx, const float *h_labels, float *h_scores, uint32_t first_tree,
                      int32_t num_trees, qgbdt_model *model, void *stream);
 
+/* Data-distributed training (Sec. 7.3: the rows are divided over the workers, the integer
+ * histograms are summed across them).  This context holds rows [row_offset, row_offset + n_rows)
+ * of a training set of total_rows rows (< 2^32, and total_rows * levels must fit the histogram
+ * word like n_rows at load); rank in [0, world).  Every rank loads its shard, sets the same
+ * parameters and calls qgbdt_train with its shard of labels and scores; the trees every rank
+ * gets are identical, and identical to those one context trains on all rows: stochastic
+ * rounding is keyed by the global row number, the two maxima of Eq. 5 are maximised and every
+ * integer sum (totals, histograms of the root and of the smaller children, row counts, refit
+ * sums) is added over the ranks, which is exact.  The exchange itself is the caller's:
+ * `reduce` is called from the calling host thread whenever `count` words at device pointer d_buf
+ * have to be combined in place over all ranks, kind QGBDT_REDUCE_SUM_I64 (64-bit integers, sum)
+ * or QGBDT_REDUCE_MAX_U32 (32-bit unsigned integers, maximum); it must order the exchange after
+ * the work already on `stream` and either finish it or enqueue it on `stream` (an NCCL all-reduce
+ * on that stream does), and return 0, anything else aborts the train call with QGBDT_ERR_CUDA.
+ * Every rank makes the same calls in the same order.  With ranks set, the passes of tree growth
+ * run on the stream with the host following them.  world <= 1 or reduce == NULL switches the
+ * mode off.  Set before qgbdt_train; model.leaf_count then holds global row counts. */
+#define QGBDT_REDUCE_SUM_I64 0
+#define QGBDT_REDUCE_MAX_U32 1
+typedef int (*qgbdt_allreduce_fn)(void *user, void *d_buf, int64_t count, int32_t kind, void *stream);
+int qgbdt_set_distributed(qgbdt_ctx *ctx, int32_t rank, int32_t world, int64_t row_offset, int64_t total_rows,
+                          qgbdt_allreduce_fn reduce, void *user);
+
 /* Options of a context (no counterpart in the paper).  Set them before qgbdt_load_binned /
  * qgbdt_train; unknown options and values out of range give QGBDT_ERR_ARG.
  *   QGBDT_OPT_COLUMN_COPY  1 (default): qgbdt_train keeps a column-major copy of the bin codes for

@@ -24,7 +24,7 @@ EXPORTS = [
     "qgbdt_compute_gradients", "qgbdt_quantize_gradients", "qgbdt_build_histograms",
     "qgbdt_build_histograms_rows", "qgbdt_subtract_histograms", "qgbdt_find_best_split", "qgbdt_split_leaf",
     "qgbdt_get_leaf_rows", "qgbdt_reset_leaves", "qgbdt_refit_leaves", "qgbdt_apply_leaf_values", "qgbdt_train", "qgbdt_train_host",
-    "qgbdt_set_option", "qgbdt_get_info", "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile", "qgbdt_get_timings",
+    "qgbdt_set_distributed", "qgbdt_set_option", "qgbdt_get_info", "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile", "qgbdt_get_timings",
     "qgbdt_build_histograms_noalloc", "qgbdt_noalloc_last_error",
 ]
 
@@ -249,6 +249,13 @@ class Context:
                                            _stream(stream))
         self._check(rc)
         return model
+
+    def set_distributed(self, rank: int, world: int, row_offset: int, total_rows: int, callback):
+        """callback: a dist.ALLREDUCE_FN instance (kept alive by this object); None switches the mode off."""
+        self._reduce_cb = callback
+        self._check(self.lib.qgbdt_set_distributed(self.h, C.c_int32(rank), C.c_int32(world), C.c_int64(row_offset),
+                                                   C.c_int64(total_rows), callback if callback is not None else None,
+                                                   None))
 
     def set_option(self, option: int, value: int):
         self._check(self.lib.qgbdt_set_option(self.h, C.c_int32(option), C.c_int64(value)))

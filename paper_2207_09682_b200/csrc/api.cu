@@ -39,6 +39,13 @@ int qg_phase_end(qgbdt_ctx *c, cudaStream_t st) {
     return QGBDT_OK;
 }
 
+int qg_allreduce(qgbdt_ctx *c, void *d_buf, int64_t count, int kind, cudaStream_t st) {
+    if (!qg_sharded(c) || count <= 0) return QGBDT_OK;
+    if (c->dist_reduce(c->dist_user, d_buf, count, kind, st) != 0)
+        return qg_fail(c, QGBDT_ERR_CUDA, "the all-reduce callback failed (%lld words, kind %d)", (long long)count, kind);
+    return QGBDT_OK;
+}
+
 static_assert(sizeof(qgbdt_params) == 72 && sizeof(qgbdt_split) == 72 && sizeof(qgbdt_bin) == 8,
               "ABI struct sizes are part of the interface");
 
@@ -395,7 +402,10 @@ int qgbdt_quantize_gradients(qgbdt_ctx *c, const float *d_g, const float *d_h, u
     c->quantized = false;
     c->const_hess = d_h == nullptr;
     if ((rc = qg_absmax(c, d_g, d_h, st)) != QGBDT_OK) return rc;
+    // sharded rows: the maxima (and the bad-value flag) and the totals are those of all ranks
+    if ((rc = qg_allreduce(c, &c->d_state->gmax_bits, 3, QGBDT_REDUCE_MAX_U32, st)) != QGBDT_OK) return rc;
     if ((rc = qg_quantize(c, d_g, d_h, tree, d_gq, d_hq, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_allreduce(c, &c->d_state->tot_g, 2, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return rc;
     DevState *hs = reinterpret_cast<DevState *>(reinterpret_cast<char *>(c->h_pinned) + PINNED_SCALARS);
     QG_CUDA(c, cudaMemcpyAsync(hs, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, st));
     QG_CUDA(c, cudaStreamSynchronize(st));
@@ -537,6 +547,25 @@ int qgbdt_apply_leaf_values(qgbdt_ctx *c, float *d_scores, void *stream) {
     if (!d_scores) return qg_fail(c, QGBDT_ERR_ARG, "d_scores is NULL");
     if (c->refit_leaves != c->n_leaves) return qg_fail(c, QGBDT_ERR_STATE, "refit the current leaves first");
     return qg_apply_leaf_values(c, d_scores, (cudaStream_t)stream);
+}
+
+int qgbdt_set_distributed(qgbdt_ctx *c, int32_t rank, int32_t world, int64_t row_offset, int64_t total_rows,
+                          qgbdt_allreduce_fn reduce, void *user) {
+    if (!c) return QGBDT_ERR_ARG;
+    if (world <= 1 || !reduce) {
+        c->dist_rank = 0; c->dist_world = 1; c->row_offset = 0; c->total_rows = 0;
+        c->dist_reduce = nullptr; c->dist_user = nullptr;
+        return QGBDT_OK;
+    }
+    if (rank < 0 || rank >= world || row_offset < 0 || total_rows < 1 || total_rows >= (1ll << 32) ||
+        (c->loaded && row_offset + c->N > total_rows))
+        return qg_fail(c, QGBDT_ERR_ARG, "rank, row_offset or total_rows out of range");
+    const int64_t kg = qg_levels_g(c->prm.bits), kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
+    if (total_rows * kg > 2147483647ll || total_rows * kh > 4294967295ll)
+        return qg_fail(c, QGBDT_ERR_OVERFLOW, "total_rows * levels exceeds the 32+32-bit histogram word");
+    c->dist_rank = rank; c->dist_world = world; c->row_offset = row_offset; c->total_rows = total_rows;
+    c->dist_reduce = reduce; c->dist_user = user;
+    return QGBDT_OK;
 }
 
 int qgbdt_set_option(qgbdt_ctx *c, int32_t option, int64_t value) {

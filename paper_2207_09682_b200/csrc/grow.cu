@@ -41,7 +41,10 @@ struct GrowArgs {
     int32_t *front;                  // [L] growth record of every numbered leaf
     DevState *state;
     const FeatRec *feat_rec;         // [F]
-    uint32_t N;
+    uint32_t N;                      // rows of this context
+    uint32_t N_all;                  // rows over all ranks (= N unless the rows are sharded)
+    int merged;                      // sharded rows: the smaller children's histograms were merged and summed over
+                                     // the ranks before the finishing kernel, which then reads them as they are
     uint2 *ent0, *ent1;              // the two (row, gradient code) pair buffers
     const uint16_t *codes_nat;       // codes in row order (the root's identity list has no pairs yet)
     uint32_t *bits;                  // [jobs][bits_stride] predicate bits of the leaves being split
@@ -64,20 +67,21 @@ struct GrowArgs {
 };
 
 __global__ void k_grow_begin(GrowState *gs, NodeRec *recs, double *rec_gain, int32_t *rec_child, int32_t *rec_pos,
-                             LeafRec *leaves, int32_t *front, const DevState *state, uint32_t N, int tree_slot) {
+                             LeafRec *leaves, int32_t *front, const DevState *state, uint32_t N, uint32_t N_all,
+                             int tree_slot) {
     rec_gain[0] = -__longlong_as_double(0x7FF0000000000000LL);
     rec_child[0] = -1;
     rec_pos[0] = -1;
     gs->tree_slot = tree_slot;
     NodeRec r;
-    r.off = 0; r.n = N; r.buf = -1; r.slot = 0;
+    r.off = 0; r.n = N; r.n_all = N_all; r.buf = -1; r.slot = 0;
     r.G = state->tot_g; r.H = state->tot_h;
     r.best = qg_invalid_rec();
     r.state = 0; r.child0 = -1; r.nl = 0;
     r.parent_node = -1; r.parent_side = 0;
     recs[0] = r;
     LeafRec l;
-    l.off = 0; l.n = N; l.buf = -1; l.rec = 0;
+    l.off = 0; l.n = N; l.buf = -1; l.rec = 0; l.n_all = N_all; l.pad = 0;
     leaves[0] = l;
     front[0] = 0;
     gs->n_leaves = 1;
@@ -222,7 +226,10 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
         before += __shfl_xor_sync(0xffffffffu, before, o);
         total += __shfl_xor_sync(0xffffffffu, total, o);
     }
-    if (gw == 0 && lane == 0) job->nl = total;
+    if (gw == 0 && lane == 0) {
+        job->nl = total;
+        gs->nl_all[j] = (long long)total;   // sharded rows: summed over the ranks before the histograms
+    }
     const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
     uint2 *dst = buf == 0 ? a.ent1 : a.ent0;
     for (uint32_t w = w0; w < w1; w += 4) {
@@ -294,7 +301,8 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     const int done = gs->done, n_jobs = gs->n_jobs;
     const int parent_slot = ROOT ? 0 : job->parent_slot, small_slot = ROOT ? 0 : job->small_slot;
     const int parts = job->parts, slot0 = job->slot0, child0 = job->child0, jrec = job->rec, jbuf = job->buf;
-    const uint32_t gs_n = job->n, gs_nl = job->nl, gs_off = job->off;
+    const uint32_t gs_n = job->n, gs_nl = job->nl, gs_off = job->off, gs_n_all = job->n_all;
+    const uint32_t gs_nl_all = (uint32_t)gs->nl_all[j];
     const long long gs_gl = job->gl, gs_hl = job->hl, gs_PG = job->PG, gs_PH = job->PH;
     const long long tot_g = a.state->tot_g, tot_h = a.state->tot_h;
     const uint32_t gmax_bits = a.state->gmax_bits, hmax_bits = a.state->hmax_bits;
@@ -303,15 +311,18 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     const size_t hw = (size_t)a.F * a.nb;
 
     // the two children: "small" was built by Algorithm 1, "large" is parent - small
+    // rows of this context (nl, nr) and over all ranks (nl_all, nr_all); which child is "small" and
+    // every row count that enters the split search are the ones over all ranks
     const uint32_t n = ROOT ? a.N : gs_n, nl = ROOT ? n : gs_nl, nr = n - nl;
-    const bool small_is_left = nl <= nr;
+    const uint32_t n_all = ROOT ? a.N_all : gs_n_all, nl_all = ROOT ? n_all : gs_nl_all, nr_all = n_all - nl_all;
+    const bool small_is_left = nl_all <= nr_all;
     SplitParams pS = a.sp, pL = a.sp;
     if (ROOT) {
-        pS.G = tot_g; pS.H = tot_h; pS.n_s = n;
+        pS.G = tot_g; pS.H = tot_h; pS.n_s = n_all;
     } else {
         const long long gl = gs_gl, hl = gs_hl, gr = gs_PG - gl, hr = gs_PH - hl;
-        pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl : nr;
-        pL.G = small_is_left ? gr : gl; pL.H = small_is_left ? hr : hl; pL.n_s = small_is_left ? nr : nl;
+        pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl_all : nr_all;
+        pL.G = small_is_left ? gr : gl; pL.H = small_is_left ? hr : hl; pL.n_s = small_is_left ? nr_all : nl_all;
     }
     // ---- phase A: one thread per bin: the smaller child's sum over the partial histograms, the
     //      larger child's bin by subtraction
@@ -323,7 +334,7 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
     const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
     const int fl = fr.fl, W = 1 << fr.logW;
-    const uint32_t P = ROOT ? 1u : effective_parts((uint32_t)parts, (uint32_t)pS.n_s);
+    const uint32_t P = (ROOT || a.merged) ? 1u : effective_parts((uint32_t)parts, small_is_left ? nl : nr);
     const size_t pstride = (size_t)4 * a.nb * 32;
     const unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
                                      (size_t)(fl & 3) * a.nb * W + (fl >> 2);
@@ -527,9 +538,9 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     }
     const int dstbuf = jbuf == 0 ? 1 : 0;
     NodeRec lf, rt;
-    lf.off = gs_off; lf.n = nl; lf.buf = dstbuf;
+    lf.off = gs_off; lf.n = nl; lf.n_all = nl_all; lf.buf = dstbuf;
     lf.G = gs_gl; lf.H = gs_hl;
-    rt.off = gs_off + nl; rt.n = nr; rt.buf = dstbuf;
+    rt.off = gs_off + nl; rt.n = nr; rt.n_all = nr_all; rt.buf = dstbuf;
     rt.G = gs_PG - gs_gl; rt.H = gs_PH - gs_hl;
     lf.slot = small_is_left ? small_slot : parent_slot;
     rt.slot = small_is_left ? parent_slot : small_slot;
@@ -548,6 +559,40 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     a.rec_child[child0] = a.rec_child[child0 + 1] = -1;
     a.rec_pos[child0] = a.rec_pos[child0 + 1] = -1;
     a.rec_parent[child0] = a.rec_parent[child0 + 1] = jrec;
+}
+
+// Sharded rows only: sums the partial histograms of every smaller child of the pass into its pool
+// slot, so that the slots can be added over the ranks before the finishing kernel.  Grid (F, leaves
+// per pass), one thread per bin.
+__global__ void __launch_bounds__(256) k_grow_merge(GrowArgs a) {
+    const GrowState *gs = a.gs;
+    const int f = blockIdx.x, j = (int)blockIdx.y;
+    const GrowJob *job = gs->jobs + j;
+    const int done = gs->done, n_jobs = gs->n_jobs;
+    const int small_slot = job->small_slot, parts = job->parts, slot0 = job->slot0;
+    const uint32_t n = job->n, nl = job->nl, n_all = job->n_all, nl_all = (uint32_t)gs->nl_all[j];
+    const FeatRec fr = a.feat_rec[f];
+    if (done || j >= n_jobs) return;
+    const bool small_is_left = nl_all <= n_all - nl_all;
+    const uint32_t P = effective_parts((uint32_t)parts, small_is_left ? nl : n - nl);
+    if (P <= 1) return;   // a single CTA wrote the slot itself
+    const int fl = fr.fl, W = 1 << fr.logW;
+    const size_t pstride = (size_t)4 * a.nb * 32;
+    const unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
+                                     (size_t)(fl & 3) * a.nb * W + (fl >> 2);
+    unsigned long long *S = a.pool + (size_t)small_slot * a.F * a.nb + (size_t)f * a.nb;
+    for (int b = threadIdx.x; b < a.nb; b += 256) {
+        const unsigned long long *q = part + (size_t)b * W;
+        unsigned long long v = 0;
+        for (uint32_t i0 = 0; i0 < P; i0 += 8) {
+            unsigned long long x[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v += x[k];
+        }
+        S[b] = v;
+    }
 }
 
 // Shared memory of the commit kernel.  A region that first holds, per numbered leaf, its gain, its
@@ -685,8 +730,8 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
             a.m_gain[no + node] = q->best.gain;
             a.rec_pos[c0] = node << 1;
             a.rec_pos[c0 + 1] = node << 1 | 1;
-            const uint32_t nl = q->nl, n = q->n;
-            rows += nl < n - nl ? nl : n - nl;
+            const NodeRec *lc = a.recs + c0, *rc = lc + 1;
+            rows += lc->n_all <= rc->n_all ? lc->n : rc->n;   // this context's rows of the child that was built
         }
         // leaf records: a leaf number may change hands more than once in a launch (a child that was
         // split ahead is confirmed right after its parent), so they are written from the replay's
@@ -696,7 +741,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
             if (i >= n_leaves0 || a.front[i] != r) {
                 const NodeRec *q = a.recs + r;
                 LeafRec x;
-                x.off = q->off; x.n = q->n; x.buf = q->buf; x.rec = r;
+                x.off = q->off; x.n = q->n; x.buf = q->buf; x.rec = r; x.n_all = q->n_all; x.pad = 0;
                 a.leaves[i] = x;
                 a.front[i] = r;
             }
@@ -855,6 +900,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         job->col8 = pf.col8;
         job->off = q->off;
         job->n = n_j;
+        job->n_all = q->n_all;
         job->buf = q->buf;
         job->nl = 0;
         job->gl = best.gl;
@@ -919,6 +965,8 @@ void fill_args(qgbdt_ctx *c, GrowArgs &a) {
     a.state = c->d_state;
     a.feat_rec = c->d_feat_rec;
     a.N = (uint32_t)c->N;
+    a.N_all = qg_sharded(c) ? (uint32_t)c->total_rows : (uint32_t)c->N;
+    a.merged = qg_sharded(c) ? 1 : 0;
     a.ent0 = c->d_ent0;
     a.ent1 = c->d_ent1;
     a.codes_nat = reinterpret_cast<const uint16_t *>(c->d_codes_nat);
@@ -965,7 +1013,9 @@ int launch_commit(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st) {
 }
 
 // One pass: the kernels that split the leaves of the current batch, then the commit step.
-int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st) {
+// n_jobs, first_slot: only for sharded rows (the host follows the passes and knows them): leaves in
+// the batch and the pool slot of the first one's smaller child.
+int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st, int n_jobs = 0, int first_slot = 0) {
     int rc = qg_phase_begin(c, QG_PHASE_PARTITION, st);
     if (rc != QGBDT_OK) return rc;
     k_grow_flags<<<a.pb_total, PART_THREADS, 0, st>>>(a);
@@ -973,9 +1023,21 @@ int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st) {
     k_grow_scatter<<<a.pb_total, PART_THREADS, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
+    // sharded rows: left rows of every leaf of the batch over all ranks (which child is the smaller one)
+    if (a.merged && (rc = qg_allreduce(c, c->d_gs->nl_all, n_jobs, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return rc;
     if ((rc = qg_hist_grow(c, st)) != QGBDT_OK) return rc;
-    if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
     const dim3 fin((unsigned)c->F, (unsigned)a.K);
+    if (a.merged) {
+        // the smaller children's histograms: merged here, then summed over the ranks (their pool slots
+        // are consecutive: 1 + splits before this pass + job)
+        k_grow_merge<<<fin, 256, 0, st>>>(a);
+        QG_LAUNCH_CHECK(c);
+        const size_t hw = (size_t)c->F * c->nb;
+        if ((rc = qg_allreduce(c, c->d_hist_pool + (size_t)first_slot * hw, (int64_t)n_jobs * (int64_t)hw,
+                               QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK)
+            return rc;
+    }
+    if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
     if (c->F > c->sm_count * 8) k_grow_finish<false, 2><<<fin, 128, 0, st>>>(a);
     else k_grow_finish<false, 1><<<fin, 256, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
@@ -1090,24 +1152,27 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
         QG_CUDA(c, cudaFuncSetAttribute(k_grow_commit, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
     k_grow_begin<<<1, 1, 0, st>>>(c->d_gs, c->d_recs, c->d_rec_gain, c->d_rec_child, c->d_rec_pos, c->d_leaves, c->d_front,
-                                  c->d_state, (uint32_t)c->N, tree_slot);
+                                  c->d_state, (uint32_t)c->N, a.N_all, tree_slot);
     QG_LAUNCH_CHECK(c);
     int rc = qg_hist(c, nullptr, 0, c->N, c->d_hist_pool, st);   // root: all rows, contiguous
     if (rc != QGBDT_OK) return rc;
+    if ((rc = qg_allreduce(c, c->d_hist_pool, (int64_t)c->F * c->nb, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return rc;
     if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
     k_grow_finish<true, 1><<<(unsigned)c->F, 256, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     if (c->prm.num_leaves < 2) return QGBDT_OK;
-    if (c->profile_hist) {
-        // event records around every histogram launch: passes on the stream, the host follows
+    if (c->profile_hist || a.merged) {
+        // event records around every phase, or exchanges between the ranks inside a pass: the passes
+        // go to the stream one by one and the host reads after each what the commit step decided
         if ((rc = launch_commit(c, a, st)) != QGBDT_OK) return rc;
-        int *h_done = reinterpret_cast<int *>(reinterpret_cast<char *>(c->h_pinned) + 64 * 1024 + 8192);
+        int *h_gs = reinterpret_cast<int *>(reinterpret_cast<char *>(c->h_pinned) + 64 * 1024 + 8192);
         for (int pass = 0; pass < c->prm.num_leaves; ++pass) {
-            QG_CUDA(c, cudaMemcpyAsync(h_done, &c->d_gs->done, sizeof(int), cudaMemcpyDeviceToHost, st));
+            // n_jobs, done, n_leaves, n_exec: the first four words of the grow state
+            QG_CUDA(c, cudaMemcpyAsync(h_gs, c->d_gs, 4 * sizeof(int), cudaMemcpyDeviceToHost, st));
             QG_CUDA(c, cudaStreamSynchronize(st));
-            if (*h_done) break;
-            if ((rc = enqueue_pass(c, a, st)) != QGBDT_OK) return rc;
+            if (h_gs[1]) break;
+            if ((rc = enqueue_pass(c, a, st, h_gs[0], 1 + h_gs[3] - h_gs[0])) != QGBDT_OK) return rc;
         }
         return QGBDT_OK;
     }

@@ -149,11 +149,12 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowH
     const int jc0 = __shfl_sync(0xffffffffu, c0, j);
     const GrowJob *job = gs->jobs + j;
     const int buf = job->buf, parts = job->parts, slot0 = job->slot0, small_slot = job->small_slot;
-    const uint32_t nl = job->nl, n = job->n, off = job->off;
+    const uint32_t nl = job->nl, n = job->n, off = job->off, n_all = job->n_all, nl_all = (uint32_t)gs->nl_all[j];
     const uint32_t nr = n - nl;
+    const bool small_is_left = nl_all <= n_all - nl_all;   // by the rows over all ranks (the same child on every rank)
     a.ents = buf == 0 ? g.ent1 : g.ent0;
-    a.off = nl <= nr ? off : off + nl;
-    a.n = nl <= nr ? nl : nr;
+    a.off = small_is_left ? off : off + nl;
+    a.n = small_is_left ? nl : nr;
     a.hist = g.pool + (size_t)small_slot * g.hist_words;
     td.cta0 = slot0 + (a.tile0 + (int)blockIdx.y) * parts;
     const uint32_t P = effective_parts((uint32_t)parts, a.n), part = blockIdx.x - (uint32_t)jc0;

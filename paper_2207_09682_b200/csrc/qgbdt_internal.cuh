@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstddef>
 #include <cstdio>
 #include <vector>
 
@@ -44,13 +45,16 @@ struct TileDesc {
 
 // Scalars produced and consumed on the device within one boosting iteration.
 struct DevState {
+    // the first three words are maximised over the ranks as they stand when the rows are sharded
     unsigned int gmax_bits;  // max |g| as float bits (non-negative floats order like uints)
     unsigned int hmax_bits;  // max h as float bits
-    int bad_value;           // set when a gradient / hessian / bin code is out of domain
+    int bad_value;           // set when a gradient / hessian / bin code is out of domain (0 or 1)
     int kernel_error;        // set by a kernel that refused to run (checked at the next synchronising call)
     unsigned int part_nl;    // rows that went left in the last partition
-    long long tot_g, tot_h;  // integer sums over all rows of the last quantization
+    long long tot_g, tot_h;  // integer sums over all rows of the last quantization (adjacent: summed over the ranks together)
 };
+static_assert(offsetof(DevState, hmax_bits) == 4 && offsetof(DevState, bad_value) == 8 &&
+              offsetof(DevState, tot_h) == offsetof(DevState, tot_g) + 8, "layout the rank exchanges rely on");
 
 // Per-feature best candidate, then the leaf's best split (same fields as qgbdt_split).
 struct SplitRec {
@@ -89,11 +93,14 @@ struct LeafRec {
     uint32_t off, n;     // its rows: entries [off, off + n) of pair buffer `buf`
     int32_t buf;         // 0 or 1; -1: the identity list of the root
     int32_t rec;         // its growth record
+    uint32_t n_all;      // its rows over all ranks (= n unless the rows are sharded, Sec. 7.3)
+    uint32_t pad;
 };
 
 // Growth record of a leaf the grower knows: confirmed or not, split or not.
 struct NodeRec {
     uint32_t off, n;
+    uint32_t n_all;          // rows of the leaf over all ranks (= n unless the rows are sharded, Sec. 7.3)
     int32_t buf;
     int32_t slot;            // histogram slot in the pool
     long long G, H;          // integer gradient / hessian totals
@@ -114,6 +121,7 @@ struct GrowJob {
     uint32_t off, n;                 // rows of the leaf
     int32_t buf;                     // their pair buffer
     uint32_t nl;                     // rows that go left (written by the scatter kernel)
+    uint32_t n_all;                  // rows of the leaf over all ranks
     long long gl, hl, PG, PH;        // left totals of the split, totals of the leaf
     int32_t parent_slot, small_slot; // histogram slots: the leaf's (becomes the larger child's), the smaller child's
     int32_t child0;                  // growth records of the children: child0 (left), child0 + 1 (right)
@@ -138,6 +146,8 @@ struct GrowState {
     unsigned long long passes;
     int32_t n_segs;                  // slots of the finished tree's leaf table (refit.cu)
     int32_t pad;
+    long long nl_all[GROW_MAX_JOBS]; // per job: rows that go left over all ranks (the scatter kernel writes this
+                                     // rank's count, a sharded run sums it over the ranks before the histograms)
 };
 
 struct qgbdt_ctx {
@@ -201,6 +211,11 @@ struct qgbdt_ctx {
     FeatRec *d_feat_rec = nullptr;              // [F] location of every feature
     uint8_t *d_colmajor = nullptr;              // [F][col_stride] column-major copy of the bin codes (training only)
     size_t col_stride = 0;
+    // rows sharded over ranks (Sec. 7.3): this context holds rows [row_offset, row_offset + N) of total_rows
+    int dist_rank = 0, dist_world = 1;
+    int64_t row_offset = 0, total_rows = 0;
+    qgbdt_allreduce_fn dist_reduce = nullptr;
+    void *dist_user = nullptr;
     bool want_column_copy = true;               // QGBDT_OPT_COLUMN_COPY
     bool leaf_values_quantized = false;         // QGBDT_OPT_LEAF_VALUES: 1 = from the quantized sums (no refit)
     void *grow_graph_exec = nullptr;            // cudaGraphExec_t: the split loop of one tree
@@ -295,6 +310,10 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
 int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st);
 // hist.cu: histograms of the smaller children of the leaves being split in the current pass
 int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st);
+// api.cu: sums (kind QGBDT_REDUCE_SUM_I64) or maximises (QGBDT_REDUCE_MAX_U32) `count` words at d_buf over the
+// ranks through the caller's callback; a no-op when the rows are not sharded
+int qg_allreduce(qgbdt_ctx *c, void *d_buf, int64_t count, int kind, cudaStream_t st);
+inline bool qg_sharded(const qgbdt_ctx *c) { return c->dist_world > 1 && c->dist_reduce != nullptr; }
 int qg_grow_parts_cap(const qgbdt_ctx *c);   // grow.cu: histogram CTAs per tile one leaf may get
 int qg_grow_slack(const qgbdt_ctx *c);       // grow.cu: leaves that may be split ahead of their confirmation
 int qg_grow_max_recs(const qgbdt_ctx *c);    // grow.cu: growth records / histogram slots a tree may use

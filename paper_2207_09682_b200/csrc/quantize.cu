@@ -127,7 +127,7 @@ __device__ inline int round_level(float x, int rounding, uint32_t u) {
 // Eq. 6 + Eq. 8 for every row; writes the packed 16-bit per-row code, optional unpacked copies,
 // and adds the integer totals (one atomic pair per block).
 __global__ void k_quantize(const float *__restrict__ g, const float *__restrict__ h, long long n, int kg, int kh,
-                           int rounding, uint32_t key, DevState *state, uint8_t *__restrict__ codes,
+                           int rounding, uint32_t key, uint32_t row_offset, DevState *state, uint8_t *__restrict__ codes,
                            uint16_t *__restrict__ codes_nat, int8_t *__restrict__ gq_out, uint8_t *__restrict__ hq_out) {
     const float gmax = __uint_as_float(state->gmax_bits);
     const float hmax = h ? __uint_as_float(state->hmax_bits) : 1.0f;
@@ -136,7 +136,7 @@ __global__ void k_quantize(const float *__restrict__ g, const float *__restrict_
     long long sg = 0, sh = 0;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
          i += (long long)gridDim.x * blockDim.x) {
-        const uint32_t r = mix32(key ^ (uint32_t)i);
+        const uint32_t r = mix32(key ^ ((uint32_t)i + row_offset));   // the row's number in the whole training set
         float x = __fmul_rn(g[i], inv_g);
         x = x > (float)kg ? (float)kg : x;
         x = x < -(float)kg ? -(float)kg : x;
@@ -220,7 +220,8 @@ int qg_quantize(qgbdt_ctx *c, const float *d_g, const float *d_h, uint32_t tree,
     const uint32_t key = mix32(mix32(mix32(seed_lo ^ 0x6A09E667u) + seed_hi) ^ tree);
     const int kg = qg_levels_g(c->prm.bits), kh = qg_levels_h(c->prm.bits, c->prm.hess_levels_mode);
     const unsigned grid = grid_for(c, c->N, 256, 8);
-    k_quantize<<<grid, 256, 0, st>>>(d_g, d_h, c->N, kg, kh, c->prm.rounding, key, c->d_state, c->d_codes,
+    k_quantize<<<grid, 256, 0, st>>>(d_g, d_h, c->N, kg, kh, c->prm.rounding, key,
+                                     qg_sharded(c) ? (uint32_t)c->row_offset : 0u, c->d_state, c->d_codes,
                                      reinterpret_cast<uint16_t *>(c->d_codes_nat), d_gq, d_hq);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;

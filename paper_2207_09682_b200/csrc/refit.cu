@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *
 // count and rows per leaf.  One block; `seg` is scratch for 4 S words.
 __global__ void __launch_bounds__(256) k_leaf_table(const LeafRec *__restrict__ leaves, const NodeRec *__restrict__ recs,
                                                     GrowState *gs, uint32_t *__restrict__ table, uint32_t *__restrict__ seg,
-                                                    int max_segs, long long *__restrict__ sums,
+                                                    int max_segs, int max_leaves, long long *__restrict__ sums,
                                                     int32_t *__restrict__ m_num_leaves,
                                                     long long *__restrict__ m_leaf_count, DevState *state) {
     const int L = gs->n_leaves;
@@ -217,10 +217,9 @@ __global__ void __launch_bounds__(256) k_leaf_table(const LeafRec *__restrict__ 
                 }
             }
         }
-        sums[2 * i] = 0;
-        sums[2 * i + 1] = 0;
-        m_leaf_count[i] = leaves[i].n;
+        m_leaf_count[i] = leaves[i].n_all;
     }
+    for (int i = threadIdx.x; i < 2 * max_leaves; i += 256) sums[i] = 0;   // all of them: a sharded run adds the whole array over the ranks
     __syncthreads();
     int S = n_segs;
     if (S > max_segs) {
@@ -313,7 +312,7 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
     const int S = qg_leaf_table_slots(L);
     int prc = qg_phase_begin(c, QG_PHASE_REFIT, st);
     if (prc != QGBDT_OK) return prc;
-    k_leaf_table<<<1, 256, 0, st>>>(c->d_leaves, c->d_recs, c->d_gs, c->d_leaf_table, c->d_leaf_table + 3 * (size_t)S, S,
+    k_leaf_table<<<1, 256, 0, st>>>(c->d_leaves, c->d_recs, c->d_gs, c->d_leaf_table, c->d_leaf_table + 3 * (size_t)S, S, L,
                                     c->d_leaf_sums, c->d_m_num_leaves + tree_slot,
                                     c->d_m_leaf_count + (size_t)tree_slot * L, c->d_state);
     QG_LAUNCH_CHECK(c);
@@ -329,6 +328,7 @@ int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_sc
                                                                          c->d_leaf_table, S, c->d_gs, d_g, d_h,
                                                                          c->d_leaf_sums);
         QG_LAUNCH_CHECK(c);
+        if ((prc = qg_allreduce(c, c->d_leaf_sums, 2 * (int64_t)L, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return prc;
         k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, L, c->d_gs, c->prm.lambda_l2, c->prm.learning_rate,
                                                        c->d_leaf_w, c->d_m_leaf_value + (size_t)tree_slot * L);
         QG_LAUNCH_CHECK(c);

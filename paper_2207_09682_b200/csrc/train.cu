@@ -21,9 +21,13 @@ int train_one_tree(qgbdt_ctx *c, const float *d_labels, float *d_scores, uint32_
     if ((rc = qg_gradients(c, d_scores, d_labels, c->d_g, const_h ? nullptr : c->d_h, true, first, st)) != QGBDT_OK)
         return rc;
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
+    // sharded rows (Sec. 7.3): Eq. 5's maxima run over all rows of all ranks (with them the flag for
+    // gradients out of domain), and so do the totals of the quantized gradients
+    if ((rc = qg_allreduce(c, &c->d_state->gmax_bits, 3, QGBDT_REDUCE_MAX_U32, st)) != QGBDT_OK) return rc;
     if ((rc = qg_phase_begin(c, QG_PHASE_QUANTIZE, st)) != QGBDT_OK) return rc;
     if ((rc = qg_quantize(c, c->d_g, const_h ? nullptr : c->d_h, tree, nullptr, nullptr, st)) != QGBDT_OK) return rc;
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
+    if ((rc = qg_allreduce(c, &c->d_state->tot_g, 2, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return rc;
     c->quantized = true;
     if ((rc = qg_grow_tree(c, slot, st)) != QGBDT_OK) return rc;
     return qg_refit_grown(c, c->d_g, const_h ? nullptr : c->d_h, d_scores, slot, st);

@@ -133,6 +133,24 @@ def histogram(data, n_bins, gq, hq, idx=None) -> tuple[np.ndarray, np.ndarray]:
     return hg, hh
 
 
+def histogram_fp(data, n_bins, g, h=None, idx=None) -> tuple[np.ndarray, np.ndarray]:
+    """Algorithm 1 with the original gradients, float64 sums: (hist_g, hist_h), each [J, n_bins]."""
+    data = _c(data, np.uint8)
+    n, J = data.shape
+    g = _c(g, np.float32)
+    h = None if h is None else _c(h, np.float32)
+    if idx is not None:
+        idx = _c(idx, np.uint32)
+    n_s = n if idx is None else idx.shape[0]
+    hg = np.empty((J, n_bins), np.float64)
+    hh = np.empty((J, n_bins), np.float64)
+    rc = lib().qo_histogram_fp(_p(data, C.c_uint8), C.c_int64(n), J, n_bins, _p(g, C.c_float), _p(h, C.c_float),
+                               _p(idx, C.c_uint32), C.c_int64(n_s), _p(hg, C.c_double), _p(hh, C.c_double))
+    if rc != OK:
+        raise ValueError("qo_histogram_fp failed: %d" % rc)
+    return hg, hh
+
+
 def gain(gl, hl, gr, hr, dg, dh, lambda_l2=0.0) -> float:
     return lib().qo_gain(gl, hl, gr, hr, dg, dh, lambda_l2)
 

@@ -11,6 +11,7 @@
  * What follows the paper, and where:
  *   qo_quantize        Eq. 5 (interval lengths), Eq. 6 (scaling), Eq. 8 (SR / RN)
  *   qo_histogram       Algorithm 1 with the integer gradients of Sec. 4.1
+ *   qo_histogram_fp    Algorithm 1 as printed, with the original floating-point gradients
  *   qo_find_split      Eq. 7 (gain from integer sums), exhaustive scan of Sec. 3
  *   qo_partition       the index sets I_s of Sec. 3 (stable filter)
  *   qo_refit           Eq. 3 with the original gradients (Sec. 4.2, leaf-value refitting)
@@ -168,6 +169,27 @@ int qo_histogram(const uint8_t *data, int64_t n_rows, int32_t n_features, int32_
             if (bin >= n_bins) return QO_ERR_ARG;
             hist_g[(int64_t)j * n_bins + bin] += gq[i];
             hist_h[(int64_t)j * n_bins + bin] += hq[i];
+        }
+    }
+    return QO_OK;
+}
+
+/* Algorithm 1 as the paper prints it, before quantization: the original gradients g_i, h_i
+ * (h == NULL: a constant hessian 1) summed per (feature, bin), here in double precision.  This
+ * is what a floating-point histogram (the unquantized baseline of Sec. 7.2) has to approximate. */
+int qo_histogram_fp(const uint8_t *data, int64_t n_rows, int32_t n_features, int32_t n_bins,
+                    const float *g, const float *h, const uint32_t *idx, int64_t n_s,
+                    double *hist_g, double *hist_h) {
+    if (!data || !g || !hist_g || !hist_h) return QO_ERR_ARG;
+    for (int64_t k = 0; k < (int64_t)n_features * n_bins; ++k) { hist_g[k] = 0.0; hist_h[k] = 0.0; }
+    for (int64_t p = 0; p < n_s; ++p) {
+        int64_t i = idx ? (int64_t)idx[p] : p;
+        if (i >= n_rows) return QO_ERR_ARG;
+        for (int32_t j = 0; j < n_features; ++j) {
+            int32_t bin = data[i * n_features + j];
+            if (bin >= n_bins) return QO_ERR_ARG;
+            hist_g[(int64_t)j * n_bins + bin] += (double)g[i];
+            hist_h[(int64_t)j * n_bins + bin] += h ? (double)h[i] : 1.0;
         }
     }
     return QO_OK;

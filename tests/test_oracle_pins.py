@@ -727,3 +727,29 @@ def test_unrefitted_tree_has_the_same_structure_and_close_values():
             rows = np.nonzero(row_leaf == l)[0]
             G, H = int(q.gq[rows].astype(np.int64).sum()), int(q.hq[rows].astype(np.int64).sum())
             assert b.leaf_value[l] == oracle.leaf_value_quantized(G, H, q.gmax, q.hmax, bits, learning_rate=1.0)[1]
+
+
+def test_floating_point_histogram_is_the_weighted_bincount():
+    # Algorithm 1 with the original gradients: per feature a bincount weighted by g resp. h
+    # (library routine), and the quantized histogram times the interval length approximates it
+    r = np.random.default_rng(8)
+    n, J, nb = 5000, 6, 11
+    data = r.integers(0, nb, size=(n, J), dtype=np.uint8)
+    g = r.normal(size=n).astype(np.float32)
+    h = r.uniform(0.01, 0.25, size=n).astype(np.float32)
+    idx = np.sort(r.choice(n, 1800, replace=False)).astype(np.uint32)
+    for rows in (None, idx):
+        hg, hh = oracle.histogram_fp(data, nb, g, h, rows)
+        sel = np.arange(n) if rows is None else rows
+        for j in range(J):
+            assert np.allclose(hg[j], np.bincount(data[sel, j], weights=g[sel].astype(np.float64), minlength=nb), rtol=1e-12, atol=1e-12)
+            assert np.allclose(hh[j], np.bincount(data[sel, j], weights=h[sel].astype(np.float64), minlength=nb), rtol=1e-12, atol=1e-12)
+    hg1, hh1 = oracle.histogram_fp(data, nb, g, None)
+    assert (hh1 == np.stack([np.bincount(data[:, j], minlength=nb) for j in range(J)])).all()   # constant hessian: counts
+    # E[G~ delta_g] = G (Sec. 4.2): at 8 bits the dequantized integer histogram is close to the floating-point one
+    q = oracle.quantize(g, h, bits=8, seed=3)
+    ig, ih = oracle.histogram(data, nb, q.gq, q.hq)
+    kg, kh = oracle.levels(8)
+    hg, hh = oracle.histogram_fp(data, nb, g, h)
+    assert np.abs(ig * (q.gmax / kg) - hg).max() < 0.02 * np.abs(hg).max() + 1.0
+    assert np.abs(ih * (q.hmax / kh) - hh).max() < 0.02 * hh.max()

@@ -133,6 +133,14 @@ int qgbdt_build_histograms(qgbdt_ctx *ctx, int32_t leaf, qgbdt_bin *d_hist, void
 /* The same for an explicit row list d_rows[n] (any order, duplicates counted twice). */
 int qgbdt_build_histograms_rows(qgbdt_ctx *ctx, const uint32_t *d_rows, int64_t n, qgbdt_bin *d_hist,
                                 void *stream);
+/* Algorithm 1 as printed, without quantization: the histogram of the ORIGINAL single-precision
+ * gradients (the floating-point baseline of Sec. 7.2's timing comparison), built on the same kernel
+ * design as the integer one.  d_g, d_h [n_rows] (d_h == NULL: hessian 1); d_rows [n] a row list, or
+ * NULL for all rows (then n must be n_rows); d_hist [n_features][n_bins][2] floats, gradient sum then
+ * hessian sum, overwritten.  Float additions are order-dependent: the sums agree with a double-precision
+ * sum to single-precision rounding error, not bit for bit.  Needs no quantize call.  Asynchronous. */
+int qgbdt_build_histograms_fp32(qgbdt_ctx *ctx, const float *d_g, const float *d_h, const uint32_t *d_rows, int64_t n,
+                                float *d_hist, void *stream);
 /* Histogram subtraction: d_large = d_parent - d_small, bin by bin (the larger sibling's
  * histogram from its parent's and its smaller sibling's).  d_large may alias d_parent.
  * Asynchronous. */

@@ -22,7 +22,7 @@ INFO_COLUMN_COPY = 1
 EXPORTS = [
     "qgbdt_create", "qgbdt_destroy", "qgbdt_last_error", "qgbdt_load_binned", "qgbdt_load_binned_host",
     "qgbdt_compute_gradients", "qgbdt_quantize_gradients", "qgbdt_build_histograms",
-    "qgbdt_build_histograms_rows", "qgbdt_subtract_histograms", "qgbdt_find_best_split", "qgbdt_split_leaf",
+    "qgbdt_build_histograms_rows", "qgbdt_build_histograms_fp32", "qgbdt_subtract_histograms", "qgbdt_find_best_split", "qgbdt_split_leaf",
     "qgbdt_get_leaf_rows", "qgbdt_reset_leaves", "qgbdt_refit_leaves", "qgbdt_apply_leaf_values", "qgbdt_train", "qgbdt_train_host",
     "qgbdt_set_distributed", "qgbdt_set_option", "qgbdt_get_info", "qgbdt_get_counters", "qgbdt_profile_histograms", "qgbdt_get_histogram_profile", "qgbdt_get_timings",
     "qgbdt_build_histograms_noalloc", "qgbdt_noalloc_last_error",
@@ -194,6 +194,15 @@ class Context:
         assert rows.dtype in (torch.int32, torch.uint32)
         self._check(self.lib.qgbdt_build_histograms_rows(self.h, _dptr(rows), C.c_int64(rows.numel()), _dptr(hist),
                                                          _stream(stream)))
+
+    def build_histograms_fp32(self, g, h=None, rows=None, stream=None) -> torch.Tensor:
+        """Floating-point histogram of the original gradients: float32 [F, n_bins, 2] (gradient sum, hessian sum)."""
+        assert g.dtype == torch.float32 and g.numel() == self.n_rows and (h is None or h.dtype == torch.float32)
+        hist = torch.empty((self.n_features, self.n_bins, 2), dtype=torch.float32, device="cuda")
+        n = self.n_rows if rows is None else rows.numel()
+        self._check(self.lib.qgbdt_build_histograms_fp32(self.h, _dptr(g), _dptr(h), _dptr(rows), C.c_int64(n),
+                                                         _dptr(hist), _stream(stream)))
+        return hist
 
     def subtract_histograms(self, parent, small, large, stream=None):
         self._check(self.lib.qgbdt_subtract_histograms(self.h, _dptr(parent), _dptr(small), _dptr(large),

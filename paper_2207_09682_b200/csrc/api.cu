@@ -446,6 +446,15 @@ int qgbdt_build_histograms_rows(qgbdt_ctx *c, const uint32_t *d_rows, int64_t n,
     return qg_hist(c, d_rows, 0, n, reinterpret_cast<unsigned long long *>(d_hist), (cudaStream_t)stream);
 }
 
+int qgbdt_build_histograms_fp32(qgbdt_ctx *c, const float *d_g, const float *d_h, const uint32_t *d_rows, int64_t n,
+                                float *d_hist, void *stream) {
+    int rc = check_loaded(c);
+    if (rc != QGBDT_OK) return rc;
+    if (!d_g || !d_hist || n < 0 || n >= (1ll << 32) || (!d_rows && n != c->N))
+        return qg_fail(c, QGBDT_ERR_ARG, "bad argument (without a row list n must be n_rows)");
+    return qg_hist_fp32(c, d_g, d_h, d_rows, n, d_hist, (cudaStream_t)stream);
+}
+
 int qgbdt_subtract_histograms(qgbdt_ctx *c, const qgbdt_bin *d_parent, const qgbdt_bin *d_small, qgbdt_bin *d_large,
                               void *stream) {
     int rc = check_loaded(c);

@@ -292,6 +292,10 @@ int qg_hist(qgbdt_ctx *c, const uint32_t *d_rows, int64_t off, int64_t n, unsign
 int qg_subtract(qgbdt_ctx *c, const unsigned long long *d_parent, const unsigned long long *d_small,
                 unsigned long long *d_large, cudaStream_t st);
 
+// hist_fp32.cu: Algorithm 1 with the original single-precision gradients (the unquantized baseline)
+int qg_hist_fp32(qgbdt_ctx *c, const float *d_g, const float *d_h, const uint32_t *d_rows, int64_t n, float *d_hist,
+                 cudaStream_t st);
+
 // split.cu
 int qg_find_split(qgbdt_ctx *c, const unsigned long long *d_hist, long long G, long long H, long long n_rows,
                   SplitRec *d_out, cudaStream_t st);

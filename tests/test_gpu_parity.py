@@ -225,6 +225,32 @@ def test_histogram_column_major_input_and_constant_hessian():
         assert (H[j] == np.bincount(data[:, j], minlength=nb)).all()
 
 
+@pytest.mark.parametrize("n,f,nb,const_h", [(70_001, 28, 255, False), (20_011, 136, 64, False), (9_999, 33, 16, True),
+                                            (300_000, 28, 255, True), (5_000, 300, 256, False)])
+def test_floating_point_histogram_matches_double_precision_sums(n, f, nb, const_h):
+    # Algorithm 1 with the original gradients in single precision (the unquantized baseline): float
+    # atomics add in any order, so each sum may differ from the double-precision one by single-precision
+    # rounding of its partial sums: at most (terms in the bin) * 2^-23 * (sum of the magnitudes)
+    data = random_bins(n, f, nb, 300 + f, skew=True)
+    g, h = logistic_grads(n, 17)
+    if const_h:
+        h = None
+    ctx = make_ctx(data, nb, bits=3)
+    rows = synth.subset_rows(n, device="cpu", seed=n).numpy().astype(np.uint32)
+    for r in (None, rows):
+        hist = ctx.build_histograms_fp32(dev(g), None if h is None else dev(h),
+                                         None if r is None else dev(r.view(np.int32))).cpu().numpy().astype(np.float64)
+        og, oh = oracle.histogram_fp(data, nb, g, h, r)
+        ag, _ = oracle.histogram_fp(data, nb, np.abs(g), None, r)       # sum of |g| and row count per bin
+        cnt = oracle.histogram_fp(data, nb, np.ones_like(g), None, r)[0]
+        tol_g = cnt * 2.0 ** -23 * ag + 1e-6
+        tol_h = cnt * 2.0 ** -23 * np.maximum(oh, 1.0) + 1e-6
+        assert (np.abs(hist[:, :, 0] - og) <= tol_g).all()
+        assert (np.abs(hist[:, :, 1] - oh) <= tol_h).all()
+        if const_h:
+            assert (hist[:, :, 1] == oh).all()                             # counts below 2^24 are exact in float
+
+
 def test_histogram_subtraction():
     n, f, nb = 50_000, 40, 64
     data = random_bins(n, f, nb, 1, True)

@@ -101,6 +101,7 @@ void free_data(qgbdt_ctx *c) {
     dev_free(c->d_grow_partial);
     dev_free(c->d_ent0);
     dev_free(c->d_ent1);
+    dev_free(c->d_leaf_id);
     dev_free(c->d_cand);
     dev_free(c->d_feat_rec);
     dev_free(c->d_colmajor);
@@ -326,7 +327,7 @@ int qgbdt_create(qgbdt_ctx **out, const qgbdt_params *p) {
     bool ok = cudaMalloc(reinterpret_cast<void **>(&c->d_state), sizeof(DevState)) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_split_out), sizeof(SplitRec) * 4) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_sums), sizeof(long long) * 2 * L) == cudaSuccess &&
-              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_table), sizeof(uint32_t) * 7 * qg_leaf_table_slots(L)) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_table), sizeof(uint32_t) * 2 * L) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_value), sizeof(float) * L) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void **>(&c->d_leaf_w), sizeof(double) * L) == cudaSuccess &&
               cudaMallocHost(&c->h_pinned, PINNED_BYTES) == cudaSuccess;

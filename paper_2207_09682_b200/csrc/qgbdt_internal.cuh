@@ -144,8 +144,6 @@ struct GrowState {
     unsigned long long hist_builds;  // confirmed splits (all trees so far)
     unsigned long long extra_rows, extra_builds;   // the same for splits made ahead that the tree did not use
     unsigned long long passes;
-    int32_t n_segs;                  // slots of the finished tree's leaf table (refit.cu)
-    int32_t pad;
     long long nl_all[GROW_MAX_JOBS]; // per job: rows that go left over all ranks (the scatter kernel writes this
                                      // rank's count, a sharded run sums it over the ranks before the histograms)
 };
@@ -185,7 +183,7 @@ struct qgbdt_ctx {
     SplitRec *d_feat_best = nullptr;    // [F]
     SplitRec *d_split_out = nullptr;    // [2]
     long long *d_leaf_sums = nullptr;   // [L][2] fixed-point refit sums
-    uint32_t *d_leaf_table = nullptr;   // [S][3] (offset, leaf, pair buffer) of the slots sorted by offset, then [S][4] scratch; S = qg_leaf_table_slots(L)
+    uint32_t *d_leaf_table = nullptr;   // [L][2] (offset, leaf) of the step-wise interface's leaves sorted by offset
     float *d_leaf_value = nullptr;      // [L]
     double *d_leaf_w = nullptr;         // [L]
     void *h_pinned = nullptr;           // small pinned staging area
@@ -206,6 +204,7 @@ struct qgbdt_ctx {
     size_t grow_bits_stride = 0;
     unsigned long long *d_grow_partial = nullptr;   // [grow_xcap * tiles][4][nb][32] partial histograms of growth
     uint2 *d_ent0 = nullptr, *d_ent1 = nullptr; // [N] (row, gradient code) pairs of the leaves, two buffers
+    uint16_t *d_leaf_id = nullptr;              // [N] leaf of every row in the tree just grown
     GrowState *d_gs = nullptr;
     SplitRec *d_cand = nullptr;                 // [F][2] per-feature best candidates of the two children
     FeatRec *d_feat_rec = nullptr;              // [F] location of every feature
@@ -307,7 +306,6 @@ int qg_partition(qgbdt_ctx *c, int64_t off, int64_t n, int feature, int bin, cud
 int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st);
 int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st);
 // the same two for a tree grown on the device (leaf table from the device leaf records)
-int qg_leaf_table_slots(int L);   // slots (and words / 7) of the leaf table of a tree grown on the device, at most
 int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_scores, int tree_slot, cudaStream_t st);
 
 // grow.cu: one tree by leaf-wise growth, every decision taken on the device

@@ -22,29 +22,13 @@ __device__ inline int slot_of(const uint32_t *offs, int n_leaves, uint32_t p) {
 
 __device__ inline long long to_fixed(float v) { return __double2ll_rn(__dmul_rn((double)v, 1073741824.0)); }
 
-// table: [n_slots] offsets ascending, then [n_slots] leaf ids.  A slot is a range of positions
-// whose rows belong to one leaf; the step-wise interface has one slot per leaf.  sums: [leaves][2]
-// by leaf id.  gs != nullptr: a tree grown on the device: the slot count comes from *gs (a leaf
-// whose rows were partitioned further ahead of the best-first order is covered by several slots)
-// and the table's third part [n_slots] says which (row, code) pair buffer holds a slot's rows
-// (-1: the identity list).
-__device__ inline uint32_t leaf_row(const uint32_t *idx, const uint2 *ent0, const uint2 *ent1, const uint32_t *table,
-                                    int n_leaves, bool grown, int s, uint32_t p) {
-    if (!grown) return idx[p];
-    const int buf = (int)table[2 * n_leaves + s];
-    return buf < 0 ? p : (buf ? ent1[p].x : ent0[p].x);
-}
-
-__global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__restrict__ idx,
-                                                              const uint2 *__restrict__ ent0,
-                                                              const uint2 *__restrict__ ent1, uint32_t n,
+// The step-wise interface: table: [n_leaves] offsets ascending, then [n_leaves] leaf ids; the leaf
+// of position p of the row list is the last table entry whose offset is <= p.  sums: [leaves][2].
+__global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__restrict__ idx, uint32_t n,
                                                               const uint32_t *__restrict__ table, int n_leaves,
-                                                              const GrowState *gs, const float *__restrict__ g,
-                                                              const float *__restrict__ h,
+                                                              const float *__restrict__ g, const float *__restrict__ h,
                                                               long long *__restrict__ sums) {
     extern __shared__ uint32_t offs[];  // n_leaves offsets
-    const bool grown = gs != nullptr;
-    if (grown) n_leaves = gs->n_segs;   // slots
     __shared__ unsigned long long acc[REFIT_LOCAL][2];
     for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) offs[i] = table[i];
     for (int i = threadIdx.x; i < REFIT_LOCAL * 2; i += REFIT_THREADS) (&acc[0][0])[i] = 0ull;
@@ -61,7 +45,7 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_refit_sums(const uint32_t *__
         long long gf = 0, hf = 0;
         if (ok) {
             s = slot_of(offs, n_leaves, p);
-            const uint32_t row = leaf_row(idx, ent0, ent1, table, n_leaves, grown, s, p);
+            const uint32_t row = idx[p];
             gf = to_fixed(g[row]);
             hf = h ? to_fixed(h[row]) : 1073741824LL;
         }
@@ -133,25 +117,18 @@ __global__ void k_leaf_values_quantized(const LeafRec *__restrict__ leaves, cons
     }
 }
 
-// Dynamic shared memory: [n_slots] offsets, [n_slots] values, [n_slots] pair buffers, so that
-// a row costs a search in shared memory and two global accesses (its pair, its score).  Four
-// rows per thread are in flight.
-__global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *__restrict__ idx,
-                                                                const uint2 *__restrict__ ent0,
-                                                                const uint2 *__restrict__ ent1, uint32_t n,
+// The step-wise interface.  Dynamic shared memory: [n_leaves] offsets, [n_leaves] values, so that a
+// row costs a search in shared memory and two global accesses (its index, its score).  Four rows
+// per thread are in flight.
+__global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *__restrict__ idx, uint32_t n,
                                                                 const uint32_t *__restrict__ table, int n_leaves,
-                                                                const GrowState *gs,
                                                                 const float *__restrict__ values,
                                                                 float *__restrict__ scores) {
     extern __shared__ uint32_t offs[];
-    const bool grown = gs != nullptr;
-    if (grown) n_leaves = gs->n_segs;   // slots
     float *vals = reinterpret_cast<float *>(offs + n_leaves);
-    int *bufs = reinterpret_cast<int *>(offs + 2 * n_leaves);
     for (int i = threadIdx.x; i < n_leaves; i += REFIT_THREADS) {
         offs[i] = table[i];
         vals[i] = values[table[n_leaves + i]];
-        bufs[i] = grown ? (int)table[2 * n_leaves + i] : 0;
     }
     __syncthreads();
     const uint32_t stride = gridDim.x * REFIT_THREADS;
@@ -164,10 +141,8 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *
             row[k] = 0xFFFFFFFFu;
             add[k] = 0.f;
             if (p < n) {
-                const int sl = slot_of(offs, n_leaves, p);
-                add[k] = vals[sl];
-                if (!grown) row[k] = idx[p];
-                else row[k] = bufs[sl] < 0 ? p : (bufs[sl] ? ent1[p].x : ent0[p].x);
+                add[k] = vals[slot_of(offs, n_leaves, p)];
+                row[k] = idx[p];
             }
         }
 #pragma unroll
@@ -178,71 +153,155 @@ __global__ void __launch_bounds__(REFIT_THREADS) k_apply_values(const uint32_t *
     }
 }
 
-// Leaf table of a tree grown on the device.  A numbered leaf that was never split ahead of the
-// best-first order is one slot: its range of its pair buffer.  A leaf that was split ahead without
-// the tree using the split still owns the same rows, but only the deepest ranges written hold
-// them intact (the scatter of a grandchild reuses the leaf's own buffer), so such a leaf is
-// covered by the slots of its descendants: a record none of whose children has been split is
-// intact in its own buffer.  Slots are ranked by (offset, empty first, order of discovery);
-// [S] offsets, [S] leaf numbers, [S] pair buffers.  Also zeroes the sums and stores the tree's leaf
-// count and rows per leaf.  One block; `seg` is scratch for 4 S words.
-__global__ void __launch_bounds__(256) k_leaf_table(const LeafRec *__restrict__ leaves, const NodeRec *__restrict__ recs,
-                                                    GrowState *gs, uint32_t *__restrict__ table, uint32_t *__restrict__ seg,
-                                                    int max_segs, int max_leaves, long long *__restrict__ sums,
-                                                    int32_t *__restrict__ m_num_leaves,
-                                                    long long *__restrict__ m_leaf_count, DevState *state) {
+// ---- trees grown on the device: rows find their leaf by walking the finished tree -------------
+//
+// The growth kernels may have partitioned rows further than the finished tree goes (leaves split
+// ahead of the best-first order that the tree did not use), so the leaf of a row is not read from
+// the row lists: every row walks the tree's nodes with its own bin codes (bin <= threshold: left).
+// Rows are visited in row order: the row's codes, its gradients and its score are read and
+// written in streams, and the leaf number is kept (16 bits per row) for the score update.
+
+struct WalkNode {           // a node of the tree being walked, in shared memory (16 bytes: one load)
+    int32_t left, right;    // children: a node >= 0, or ~leaf
+    uint8_t logW, shift, bin, byte;   // tile width, bit position in the word, threshold; byte of a 32-byte row
+    int32_t feature;
+};
+
+constexpr int WALK_THREADS = 256;
+
+// *p (two adjacent 32-bit shared words, low then high) += v, with 32-bit atomics.
+__device__ __forceinline__ void add64(uint32_t *p, unsigned long long v) {
+    const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
+    const uint32_t old = atomicAdd(p, lo);
+    const uint32_t carry = old + lo < old ? 1u : 0u;
+    if (hi + carry) atomicAdd(p + 1, hi + carry);
+}
+
+// nodes, then the refit sums of the block, then (32-byte rows) the block's rows, nine words apart
+__host__ __device__ inline size_t walk_smem_bytes(int L, bool sums, bool rows) {
+    return (size_t)(L > 1 ? L - 1 : 1) * sizeof(WalkNode) + (sums ? (size_t)L * 2 * sizeof(unsigned long long) : 0) +
+           (rows ? (size_t)WALK_THREADS * 9 * sizeof(uint32_t) : 0);
+}
+
+// Stores the tree's leaf count and rows per leaf, and zeroes the refit sums.  One block.
+__global__ void __launch_bounds__(256) k_tree_prepare(const LeafRec *__restrict__ leaves, const GrowState *gs, int max_leaves,
+                                                      long long *__restrict__ sums, int32_t *__restrict__ m_num_leaves,
+                                                      long long *__restrict__ m_leaf_count) {
     const int L = gs->n_leaves;
-    __shared__ int n_segs;
-    if (threadIdx.x == 0) n_segs = 0;
+    for (int i = threadIdx.x; i < L; i += 256) m_leaf_count[i] = leaves[i].n_all;
+    for (int i = threadIdx.x; i < 2 * max_leaves; i += 256) sums[i] = 0;   // all: a sharded run adds the whole array over the ranks
+    if (threadIdx.x == 0) *m_num_leaves = L;
+}
+
+// SUMS: also adds the row's gradients (2^-30 fixed point) to its leaf's sums (Eq. 3).
+// ROW_LOGW == 3: the matrix is one tile of 32-byte rows: a thread loads its whole row once
+// (consecutive threads, consecutive rows: a coalesced stream) into shared memory, nine words from
+// row to row so that the threads' accesses never share a bank, and reads the code of every node it
+// passes as one byte from there.  -1: any tiling, one global load per node passed.
+template <bool SUMS, int ROW_LOGW>
+__global__ void __launch_bounds__(WALK_THREADS) k_walk(const GrowState *gs, const FeatRec *__restrict__ feat_rec,
+                                                       const int32_t *__restrict__ m_feature, const int32_t *__restrict__ m_bin,
+                                                       const int32_t *__restrict__ m_left, const int32_t *__restrict__ m_right,
+                                                       uint32_t n, const float *__restrict__ g, const float *__restrict__ h,
+                                                       uint16_t *__restrict__ leaf_id, long long *__restrict__ sums) {
+    extern __shared__ __align__(16) unsigned char wsm[];
+    const int L = gs->n_leaves, n_nodes = L - 1;
+    WalkNode *nodes = reinterpret_cast<WalkNode *>(wsm);
+    unsigned long long *acc = reinterpret_cast<unsigned long long *>(wsm + (size_t)(n_nodes > 0 ? n_nodes : 1) * sizeof(WalkNode));
+    uint32_t *srow = reinterpret_cast<uint32_t *>(acc + (SUMS ? 2 * L : 0)) + threadIdx.x * 9;   // this thread's row
+    for (int i = threadIdx.x; i < n_nodes; i += WALK_THREADS) {
+        const int f = m_feature[i];
+        const FeatRec fr = feat_rec[f];
+        WalkNode w;
+        w.left = m_left[i]; w.right = m_right[i];
+        w.logW = (uint8_t)fr.logW; w.shift = (uint8_t)(8 * fr.byte); w.bin = (uint8_t)m_bin[i]; w.byte = (uint8_t)fr.fl;
+        w.feature = f;
+        nodes[i] = w;
+    }
+    uint32_t *acc32 = reinterpret_cast<uint32_t *>(acc);   // [L][g lo, g hi, h lo, h hi]
+    if (SUMS)
+        for (int i = threadIdx.x; i < 4 * L; i += WALK_THREADS) acc32[i] = 0u;
     __syncthreads();
-    for (int i = threadIdx.x; i < L; i += 256) {
-        int stack[GROW_SLACK + GROW_MAX_JOBS + 4];
-        int sp = 0;
-        stack[sp++] = leaves[i].rec;
-        while (sp > 0) {
-            const int r = stack[--sp];
-            const NodeRec q = recs[r];
-            const bool deeper = q.state == 1 && (recs[q.child0].state == 1 || recs[q.child0 + 1].state == 1);
-            if (deeper && sp + 2 <= GROW_SLACK + GROW_MAX_JOBS + 4) {
-                stack[sp++] = q.child0 + 1;
-                stack[sp++] = q.child0;
-            } else {
-                if (deeper) atomicExch(&state->kernel_error, 1);   // deeper than the slack allows: cannot happen
-                const int k = atomicAdd(&n_segs, 1);
-                if (k < max_segs) {
-                    seg[4 * k] = q.off;
-                    seg[4 * k + 1] = q.n;
-                    seg[4 * k + 2] = (uint32_t)q.buf;
-                    seg[4 * k + 3] = (uint32_t)i;
+    const int lane = threadIdx.x & 31;
+    for (uint32_t base = blockIdx.x * WALK_THREADS + (threadIdx.x & ~31u); base < n; base += gridDim.x * WALK_THREADS) {
+        const uint32_t r = base + lane;
+        const bool active = r < n;
+        int leaf = 0;
+        if (active && n_nodes > 0) {
+            if (ROW_LOGW == 3) {
+                const uint4 *row = reinterpret_cast<const uint4 *>(feat_rec[0].col + ((size_t)r << 3));   // feature 0: word 0 of the tile
+                const uint4 v0 = row[0], v1 = row[1];
+                srow[0] = v0.x; srow[1] = v0.y; srow[2] = v0.z; srow[3] = v0.w;
+                srow[4] = v1.x; srow[5] = v1.y; srow[6] = v1.z; srow[7] = v1.w;
+            }
+            int node = 0;
+            for (;;) {
+                const WalkNode w = nodes[node];
+                uint32_t code;
+                if (ROW_LOGW == 3) {
+                    code = reinterpret_cast<const uint8_t *>(srow)[w.byte];
+                } else {
+                    const FeatRec fr = feat_rec[w.feature];
+                    code = (fr.col[(size_t)r << w.logW] >> w.shift) & 0xFFu;
                 }
+                const int next = code <= w.bin ? w.left : w.right;
+                if (next < 0) { leaf = ~next; break; }
+                node = next;
             }
         }
-        m_leaf_count[i] = leaves[i].n_all;
-    }
-    for (int i = threadIdx.x; i < 2 * max_leaves; i += 256) sums[i] = 0;   // all of them: a sharded run adds the whole array over the ranks
-    __syncthreads();
-    int S = n_segs;
-    if (S > max_segs) {
-        if (threadIdx.x == 0) atomicExch(&state->kernel_error, 1);
-        S = max_segs;
-    }
-    __threadfence_block();
-    for (int i = threadIdx.x; i < S; i += 256) {
-        const uint32_t off = seg[4 * i], n = seg[4 * i + 1];
-        int rank = 0;
-        for (int j = 0; j < S; ++j) {
-            const uint32_t oj = seg[4 * j], nj = seg[4 * j + 1];
-            const bool before = oj < off || (oj == off && ((nj == 0) > (n == 0) || ((nj == 0) == (n == 0) && j < i)));
-            rank += before ? 1 : 0;
+        if (active) leaf_id[r] = (uint16_t)leaf;
+        if (SUMS) {
+            // Consecutive rows often share a leaf (a few leaves hold most rows), and lanes adding to
+            // one shared word serialise: up to two rounds in which the lanes of one leaf add up
+            // their terms with shuffles and one lane adds the sum; what is left adds on its own.
+            // 64-bit sums are two 32-bit shared atomics each (the low word's old value tells the
+            // carry); a constant hessian only counts rows.
+            const long long gf = active ? to_fixed(g[r]) : 0;
+            const long long hf = (active && h) ? to_fixed(h[r]) : 0;
+            unsigned rem = __ballot_sync(0xffffffffu, active);
+            for (int round = 0; round < 2 && rem; ++round) {
+                const int src = __ffs(rem) - 1;
+                const int l0 = __shfl_sync(0xffffffffu, leaf, src);
+                const bool mine = ((rem >> lane) & 1u) && leaf == l0;
+                const unsigned m = __ballot_sync(0xffffffffu, mine);
+                if (__popc(m) >= 4) {
+                    long long gs_ = mine ? gf : 0, hs_ = mine ? hf : 0;
+                    for (int o = 16; o > 0; o >>= 1) {
+                        gs_ += __shfl_xor_sync(0xffffffffu, gs_, o);
+                        if (h) hs_ += __shfl_xor_sync(0xffffffffu, hs_, o);
+                    }
+                    if (lane == src) {
+                        add64(acc32 + 4 * l0, (unsigned long long)gs_);
+                        if (h) add64(acc32 + 4 * l0 + 2, (unsigned long long)hs_);
+                        else atomicAdd(acc32 + 4 * l0 + 2, (uint32_t)__popc(m));
+                    }
+                    rem &= ~m;
+                } else {
+                    break;   // the leaves of this warp are spread out: no gain in adding up first
+                }
+            }
+            if ((rem >> lane) & 1u) {
+                add64(acc32 + 4 * leaf, (unsigned long long)gf);
+                if (h) add64(acc32 + 4 * leaf + 2, (unsigned long long)hf);
+                else atomicAdd(acc32 + 4 * leaf + 2, 1u);
+            }
         }
-        table[rank] = off;
-        table[S + rank] = seg[4 * i + 3];
-        table[2 * S + rank] = seg[4 * i + 2];
     }
-    if (threadIdx.x == 0) {
-        *m_num_leaves = L;
-        gs->n_segs = S;
+    if (SUMS) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < 2 * L; i += WALK_THREADS) {
+            unsigned long long v = ((unsigned long long)acc32[2 * i + 1] << 32) | acc32[2 * i];
+            if ((i & 1) && !h) v = (unsigned long long)acc32[2 * i] << 30;   // rows counted, each 2^30
+            if (v != 0ull) atomicAdd(reinterpret_cast<unsigned long long *>(&sums[i]), v);
+        }
     }
+}
+
+// scores[r] += value of r's leaf, in row order.
+__global__ void __launch_bounds__(256) k_apply_ids(const uint16_t *__restrict__ leaf_id, const float *__restrict__ values,
+                                                   uint32_t n, float *__restrict__ scores) {
+    for (uint32_t r = blockIdx.x * 256 + threadIdx.x; r < n; r += gridDim.x * 256)
+        scores[r] = __fadd_rn(scores[r], values[leaf_id[r]]);
 }
 
 // Writes the offset-sorted leaf table into pinned memory and queues its copy to the device.
@@ -252,9 +311,9 @@ int upload_table(qgbdt_ctx *c, cudaStream_t st) {
     std::vector<int> order(L);
     for (int i = 0; i < L; ++i) order[i] = i;
     // Order: offset, then empty leaves before the non-empty one that starts at the same offset (a
-    // split that sends every row to one side leaves an empty leaf there; the search below takes the
-    // last slot whose offset is <= the position, which must be the leaf that owns the rows), then
-    // leaf number: the same ranking as k_leaf_table.
+    // split that sends every row to one side leaves an empty leaf there; the search takes the last
+    // slot whose offset is <= the position, which must be the leaf that owns the rows), then leaf
+    // number.
     auto before = [&](int a, int b) {
         if (c->leaf_off[a] != c->leaf_off[b]) return c->leaf_off[a] < c->leaf_off[b];
         const bool ea = c->leaf_n[a] == 0, eb = c->leaf_n[b] == 0;
@@ -283,8 +342,7 @@ int qg_refit(qgbdt_ctx *c, const float *d_g, const float *d_h, cudaStream_t st) 
     if (rc != QGBDT_OK) return rc;
     QG_CUDA(c, cudaMemsetAsync(c->d_leaf_sums, 0, sizeof(long long) * 2 * L, st));
     const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
-    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, nullptr, nullptr, (uint32_t)c->N,
-                                                                     c->d_leaf_table, L, nullptr, d_g, d_h,
+    k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * L, st>>>(c->d_idx, (uint32_t)c->N, c->d_leaf_table, L, d_g, d_h,
                                                                      c->d_leaf_sums);
     QG_LAUNCH_CHECK(c);
     k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, L, nullptr, c->prm.lambda_l2, c->prm.learning_rate,
@@ -298,51 +356,65 @@ int qg_apply_leaf_values(qgbdt_ctx *c, float *d_scores, cudaStream_t st) {
     const int L = c->n_leaves;
     unsigned blocks = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
     if (blocks > (unsigned)c->sm_count * 16) blocks = (unsigned)c->sm_count * 16;
-    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * 3 * L, st>>>(c->d_idx, nullptr, nullptr, (uint32_t)c->N,
-                                                                       c->d_leaf_table, L, nullptr, c->d_leaf_value,
-                                                                       d_scores);
+    k_apply_values<<<blocks, REFIT_THREADS, sizeof(uint32_t) * 2 * L, st>>>(c->d_idx, (uint32_t)c->N, c->d_leaf_table, L,
+                                                                       c->d_leaf_value, d_scores);
     QG_LAUNCH_CHECK(c);
     return QGBDT_OK;
 }
 
-// Refit (Eq. 3 with the original gradients) and score update for the tree just grown on the
-// device; leaf values and counts go to slot `tree_slot` of the device-side model arrays.
+// Leaf values (Eq. 3 with the original gradients, or Sec. 4.2's values from the quantized sums)
+// and score update for the tree just grown on the device; leaf values and counts go to slot
+// `tree_slot` of the device-side model arrays.
 int qg_refit_grown(qgbdt_ctx *c, const float *d_g, const float *d_h, float *d_scores, int tree_slot, cudaStream_t st) {
-    const int L = c->prm.num_leaves;     // upper bound; the kernels read the real counts from the grow state
-    const int S = qg_leaf_table_slots(L);
+    const int L = c->prm.num_leaves;     // upper bound; the kernels read the real count from the grow state
+    const size_t no = (size_t)tree_slot * (L > 1 ? L - 1 : 1);
+    const bool refit = !c->leaf_values_quantized;
     int prc = qg_phase_begin(c, QG_PHASE_REFIT, st);
     if (prc != QGBDT_OK) return prc;
-    k_leaf_table<<<1, 256, 0, st>>>(c->d_leaves, c->d_recs, c->d_gs, c->d_leaf_table, c->d_leaf_table + 3 * (size_t)S, S, L,
-                                    c->d_leaf_sums, c->d_m_num_leaves + tree_slot,
-                                    c->d_m_leaf_count + (size_t)tree_slot * L, c->d_state);
+    k_tree_prepare<<<1, 256, 0, st>>>(c->d_leaves, c->d_gs, L, c->d_leaf_sums, c->d_m_num_leaves + tree_slot,
+                                      c->d_m_leaf_count + (size_t)tree_slot * L);
     QG_LAUNCH_CHECK(c);
-    if (c->leaf_values_quantized) {
-        k_leaf_values_quantized<<<(L + 255) / 256, 256, 0, st>>>(
-            c->d_leaves, c->d_recs, c->d_gs, c->d_state, qg_levels_g(c->prm.bits),
-            qg_levels_h(c->prm.bits, c->prm.hess_levels_mode), c->const_hess ? 1 : 0, c->prm.lambda_l2,
-            c->prm.learning_rate, c->d_leaf_w, c->d_m_leaf_value + (size_t)tree_slot * L);
-        QG_LAUNCH_CHECK(c);
-    } else {
-        const unsigned blocks = (unsigned)((c->N + REFIT_BLOCK - 1) / REFIT_BLOCK);
-        k_refit_sums<<<blocks, REFIT_THREADS, sizeof(uint32_t) * S, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
-                                                                         c->d_leaf_table, S, c->d_gs, d_g, d_h,
-                                                                         c->d_leaf_sums);
+    // one tile of 32-byte rows (up to 32 features): the walk stages the row in shared memory
+    const bool row8 = c->tiles.size() == 1 && c->tiles[0].logW == 3;
+    const size_t smem = walk_smem_bytes(L, refit, row8);
+    static bool configured[64] = {};
+    if (smem > 48 * 1024 && (c->device < 0 || c->device >= 64 || !configured[c->device])) {
+        const int cap_s = (int)walk_smem_bytes(4096, true, true), cap_n = (int)walk_smem_bytes(4096, false, true);
+        QG_CUDA(c, cudaFuncSetAttribute(k_walk<true, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, cap_s));
+        QG_CUDA(c, cudaFuncSetAttribute(k_walk<false, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, cap_n));
+        QG_CUDA(c, cudaFuncSetAttribute(k_walk<true, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, cap_s));
+        QG_CUDA(c, cudaFuncSetAttribute(k_walk<false, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, cap_n));
+        if (c->device >= 0 && c->device < 64) configured[c->device] = true;
+    }
+    unsigned wb = (unsigned)((c->N + WALK_THREADS - 1) / WALK_THREADS);
+    if (wb > (unsigned)c->sm_count * 8) wb = (unsigned)c->sm_count * 8;
+    auto walk = [&](auto kern, const float *gg, const float *hh, long long *sums) {
+        kern<<<wb, WALK_THREADS, smem, st>>>(c->d_gs, c->d_feat_rec, c->d_m_feature + no, c->d_m_bin + no, c->d_m_left + no,
+                                             c->d_m_right + no, (uint32_t)c->N, gg, hh, c->d_leaf_id, sums);
+    };
+    if (refit) {
+        if (row8) walk(k_walk<true, 3>, d_g, d_h, c->d_leaf_sums);
+        else walk(k_walk<true, -1>, d_g, d_h, c->d_leaf_sums);
         QG_LAUNCH_CHECK(c);
         if ((prc = qg_allreduce(c, c->d_leaf_sums, 2 * (int64_t)L, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return prc;
         k_leaf_values<<<(L + 255) / 256, 256, 0, st>>>(c->d_leaf_sums, L, c->d_gs, c->prm.lambda_l2, c->prm.learning_rate,
                                                        c->d_leaf_w, c->d_m_leaf_value + (size_t)tree_slot * L);
         QG_LAUNCH_CHECK(c);
+    } else {
+        if (row8) walk(k_walk<false, 3>, nullptr, nullptr, nullptr);
+        else walk(k_walk<false, -1>, nullptr, nullptr, nullptr);
+        QG_LAUNCH_CHECK(c);
+        k_leaf_values_quantized<<<(L + 255) / 256, 256, 0, st>>>(
+            c->d_leaves, c->d_recs, c->d_gs, c->d_state, qg_levels_g(c->prm.bits),
+            qg_levels_h(c->prm.bits, c->prm.hess_levels_mode), c->const_hess ? 1 : 0, c->prm.lambda_l2,
+            c->prm.learning_rate, c->d_leaf_w, c->d_m_leaf_value + (size_t)tree_slot * L);
+        QG_LAUNCH_CHECK(c);
     }
     if ((prc = qg_phase_end(c, st)) != QGBDT_OK) return prc;
     if ((prc = qg_phase_begin(c, QG_PHASE_SCORES, st)) != QGBDT_OK) return prc;
-    unsigned ab = (unsigned)((c->N + REFIT_THREADS - 1) / REFIT_THREADS);
+    unsigned ab = (unsigned)((c->N + 255) / 256);
     if (ab > (unsigned)c->sm_count * 16) ab = (unsigned)c->sm_count * 16;
-    k_apply_values<<<ab, REFIT_THREADS, sizeof(uint32_t) * 3 * S, st>>>(nullptr, c->d_ent0, c->d_ent1, (uint32_t)c->N,
-                                                                   c->d_leaf_table, S, c->d_gs,
-                                                                   c->d_m_leaf_value + (size_t)tree_slot * L, d_scores);
+    k_apply_ids<<<ab, 256, 0, st>>>(c->d_leaf_id, c->d_m_leaf_value + (size_t)tree_slot * L, (uint32_t)c->N, d_scores);
     QG_LAUNCH_CHECK(c);
     return qg_phase_end(c, st);
 }
-
-// Slots the leaf table of a grown tree may need: a leaf per slot, plus one per leaf split ahead.
-int qg_leaf_table_slots(int L) { return L + GROW_SLACK + GROW_MAX_JOBS + 2; }

@@ -83,6 +83,7 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
         return rc;
     if (!c->d_ent0 && (rc = alloc_dev(c, &c->d_ent0, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_ent1 && (rc = alloc_dev(c, &c->d_ent1, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
+    if (!c->d_leaf_id && (rc = alloc_dev(c, &c->d_leaf_id, (size_t)c->N, "leaf numbers")) != QGBDT_OK) return rc;
     if (!c->d_cand && (rc = alloc_dev(c, &c->d_cand, (size_t)2 * c->F * c->grow_jobs, "candidate records")) != QGBDT_OK)
         return rc;
     if ((rc = qg_build_columns(c, st)) != QGBDT_OK) return rc;

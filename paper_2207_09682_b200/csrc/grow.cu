@@ -285,17 +285,14 @@ __device__ inline SplitRec shfl_xor_rec(const SplitRec &r, int o) {
     return x;
 }
 
-// ROOT: scans the root histogram (pool slot 0), grid (F).  Otherwise: completes the splits of the
-// current pass, grid (F, leaves per pass).  One block per feature (and leaf).
+// One feature of one leaf being split (ROOT: of the root): the work of a block of k_grow_finish.
 // BPT bins per thread: 1 (256 threads) or 2 (128 threads: with thousands of features twice as many
 // blocks are resident).
 template <bool ROOT, int BPT>
-__global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
+__device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const int j) {
     constexpr int FIN_WARPS = 8 / BPT;
     GrowState *gs = a.gs;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int f = blockIdx.x;                 // one block per feature
-    const int j = ROOT ? 0 : (int)blockIdx.y; // and leaf being split
     GrowJob *job = gs->jobs + j;
     // everything the block needs from the state, at once (one round trip to memory), then the early exit
     const int done = gs->done, n_jobs = gs->n_jobs;
@@ -561,37 +558,56 @@ __global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
     a.rec_parent[child0] = a.rec_parent[child0 + 1] = jrec;
 }
 
+// ROOT: scans the root histogram (pool slot 0), grid (F).  Otherwise: completes the splits of the
+// current pass, grid (F, Y): block (f, y) takes feature f of the leaves y, y + Y, ... of the batch
+// (Y is chosen on the host so that the grid fills the SMs a few times over without launching a block
+// for every feature of every possible leaf).
+template <bool ROOT, int BPT>
+__global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
+    if (ROOT) {
+        finish_one<ROOT, BPT>(a, (int)blockIdx.x, 0);
+        return;
+    }
+    const int n_jobs = a.gs->n_jobs;
+    for (int j = (int)blockIdx.y; j < n_jobs; j += (int)gridDim.y) {
+        finish_one<ROOT, BPT>(a, (int)blockIdx.x, j);
+        __syncthreads();   // the shared arrays of finish_one are reused by the next leaf
+    }
+}
+
 // Sharded rows only: sums the partial histograms of every smaller child of the pass into its pool
-// slot, so that the slots can be added over the ranks before the finishing kernel.  Grid (F, leaves
-// per pass), one thread per bin.
+// slot, so that the slots can be added over the ranks before the finishing kernel.  Grid (F, Y) like
+// the finishing kernel, one thread per bin.
 __global__ void __launch_bounds__(256) k_grow_merge(GrowArgs a) {
     const GrowState *gs = a.gs;
-    const int f = blockIdx.x, j = (int)blockIdx.y;
-    const GrowJob *job = gs->jobs + j;
+    const int f = blockIdx.x;
     const int done = gs->done, n_jobs = gs->n_jobs;
-    const int small_slot = job->small_slot, parts = job->parts, slot0 = job->slot0;
-    const uint32_t n = job->n, nl = job->nl, n_all = job->n_all, nl_all = (uint32_t)gs->nl_all[j];
     const FeatRec fr = a.feat_rec[f];
-    if (done || j >= n_jobs) return;
-    const bool small_is_left = nl_all <= n_all - nl_all;
-    const uint32_t P = effective_parts((uint32_t)parts, small_is_left ? nl : n - nl);
-    if (P <= 1) return;   // a single CTA wrote the slot itself
-    const int fl = fr.fl, W = 1 << fr.logW;
-    const size_t pstride = (size_t)4 * a.nb * 32;
-    const unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
-                                     (size_t)(fl & 3) * a.nb * W + (fl >> 2);
-    unsigned long long *S = a.pool + (size_t)small_slot * a.F * a.nb + (size_t)f * a.nb;
-    for (int b = threadIdx.x; b < a.nb; b += 256) {
-        const unsigned long long *q = part + (size_t)b * W;
-        unsigned long long v = 0;
-        for (uint32_t i0 = 0; i0 < P; i0 += 8) {
-            unsigned long long x[8];
+    if (done) return;
+    for (int j = (int)blockIdx.y; j < n_jobs; j += (int)gridDim.y) {   // the leaves y, y + Y, ... of the batch
+        const GrowJob *job = gs->jobs + j;
+        const int small_slot = job->small_slot, parts = job->parts, slot0 = job->slot0;
+        const uint32_t n = job->n, nl = job->nl, n_all = job->n_all, nl_all = (uint32_t)gs->nl_all[j];
+        const bool small_is_left = nl_all <= n_all - nl_all;
+        const uint32_t P = effective_parts((uint32_t)parts, small_is_left ? nl : n - nl);
+        if (P <= 1) continue;   // a single CTA wrote the slot itself
+        const int fl = fr.fl, W = 1 << fr.logW;
+        const size_t pstride = (size_t)4 * a.nb * 32;
+        const unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
+                                         (size_t)(fl & 3) * a.nb * W + (fl >> 2);
+        unsigned long long *S = a.pool + (size_t)small_slot * a.F * a.nb + (size_t)f * a.nb;
+        for (int b = threadIdx.x; b < a.nb; b += 256) {
+            const unsigned long long *q = part + (size_t)b * W;
+            unsigned long long v = 0;
+            for (uint32_t i0 = 0; i0 < P; i0 += 8) {
+                unsigned long long x[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
+                for (int k = 0; k < 8; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) v += x[k];
+                for (int k = 0; k < 8; ++k) v += x[k];
+            }
+            S[b] = v;
         }
-        S[b] = v;
     }
 }
 
@@ -1026,7 +1042,9 @@ int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st, int n_jobs = 
     // sharded rows: left rows of every leaf of the batch over all ranks (which child is the smaller one)
     if (a.merged && (rc = qg_allreduce(c, c->d_gs->nl_all, n_jobs, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return rc;
     if ((rc = qg_hist_grow(c, st)) != QGBDT_OK) return rc;
-    const dim3 fin((unsigned)c->F, (unsigned)a.K);
+    int fin_y = (c->sm_count * 24 + c->F - 1) / c->F;   // blocks for about one and a half rounds of all SMs
+    fin_y = fin_y < 1 ? 1 : (fin_y > a.K ? a.K : fin_y);
+    const dim3 fin((unsigned)c->F, (unsigned)fin_y);
     if (a.merged) {
         // the smaller children's histograms: merged here, then summed over the ranks (their pool slots
         // are consecutive: 1 + splits before this pass + job)

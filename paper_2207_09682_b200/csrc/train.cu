@@ -56,10 +56,10 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
     if (!c->d_g && (rc = alloc_dev(c, &c->d_g, (size_t)c->N, "gradient buffer")) != QGBDT_OK) return rc;
     if (!c->d_h && c->prm.objective == 0 && (rc = alloc_dev(c, &c->d_h, (size_t)c->N, "hessian buffer")) != QGBDT_OK)
         return rc;
-    // leaves split per pass: fewer with thousands of features (the finishing kernel has a block per
-    // feature and leaf, the histogram pool a slot of F x bins words per split)
+    // leaves split per pass: fewer with many thousands of features (the histogram pool has a slot of
+    // F x bins words for every leaf that may be split ahead)
     if (c->grow_jobs <= 1 || !c->d_recs) {
-        int k = 8192 / (c->F > 0 ? c->F : 1);
+        int k = 65536 / (c->F > 0 ? c->F : 1);
         c->grow_jobs = k < 2 ? 2 : (k > GROW_MAX_JOBS ? GROW_MAX_JOBS : k);
         c->grow_xcap = 2 * qg_grow_parts_cap(c) + c->grow_jobs;
         c->grow_bits_stride = ((size_t)c->N + 31) / 32 + 64;

@@ -22,14 +22,6 @@ namespace {
 constexpr int PART_THREADS = 256;
 constexpr int PART_WARPS = PART_THREADS / 32;
 constexpr int COMMIT_THREADS = 1024;
-constexpr uint32_t MIN_ROWS_PER_CTA = 1024;   // same rule as the histogram kernel
-
-__device__ __host__ inline uint32_t effective_parts(uint32_t parts, uint32_t n) {
-    uint32_t want = (n + MIN_ROWS_PER_CTA - 1) / MIN_ROWS_PER_CTA;
-    if (want < 1) want = 1;
-    return want < parts ? want : parts;
-}
-
 struct GrowArgs {
     GrowState *gs;
     NodeRec *recs;
@@ -57,6 +49,7 @@ struct GrowArgs {
     int F, nb, L;
     int K, slack;                    // leaves per pass; leaves that may be split ahead of their confirmation
     int xcap, parts_cap, n_tiles;    // histogram CTAs per tile of a launch, of one leaf; tiles
+    uint32_t rows_min;               // rows per histogram CTA, at least (see qg_grow_parts)
     int max_recs, max_slots;         // growth records and histogram slots allocated
     SplitParams sp;                  // G, H, n_s are filled per leaf on the device
     // tree output (device arrays of the current train call)
@@ -331,7 +324,7 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
     const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
     const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
     const int fl = fr.fl, W = 1 << fr.logW;
-    const uint32_t P = (ROOT || a.merged) ? 1u : effective_parts((uint32_t)parts, small_is_left ? nl : nr);
+    const uint32_t P = (ROOT || a.merged) ? 1u : qg_grow_parts((uint32_t)parts, small_is_left ? nl : nr, a.rows_min);
     const size_t pstride = (size_t)4 * a.nb * 32;
     const unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
                                      (size_t)(fl & 3) * a.nb * W + (fl >> 2);
@@ -589,7 +582,7 @@ __global__ void __launch_bounds__(256) k_grow_merge(GrowArgs a) {
         const int small_slot = job->small_slot, parts = job->parts, slot0 = job->slot0;
         const uint32_t n = job->n, nl = job->nl, n_all = job->n_all, nl_all = (uint32_t)gs->nl_all[j];
         const bool small_is_left = nl_all <= n_all - nl_all;
-        const uint32_t P = effective_parts((uint32_t)parts, small_is_left ? nl : n - nl);
+        const uint32_t P = qg_grow_parts((uint32_t)parts, small_is_left ? nl : n - nl, a.rows_min);
         if (P <= 1) continue;   // a single CTA wrote the slot itself
         const int fl = fr.fl, W = 1 << fr.logW;
         const size_t pstride = (size_t)4 * a.nb * 32;
@@ -932,7 +925,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         a.rec_child[r] = n_recs + 2 * lane;
     }
     // blocks of the partition kernels: in proportion to the rows, at least one per leaf; histogram
-    // CTAs per tile: one per 1024 rows of half the leaf (the smaller child has at most that many
+    // CTAs per tile: one per rows_min rows of half the leaf (the smaller child has at most that many
     // rows), at most a leaf's share of the SMs; both scaled down when the batch wants more than a
     // launch has
     const uint32_t pb_cap = (uint32_t)(a.pb_total - a.K), xc = (uint32_t)(a.xcap - a.K);
@@ -940,7 +933,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
     if (lane < n_jobs) {
         wpb = (n_j + 2047u) / 2048u;
         wpb = wpb < 1u ? 1u : (wpb > pb_cap ? pb_cap : wpb);
-        wpt = (n_j / 2u + MIN_ROWS_PER_CTA - 1u) / MIN_ROWS_PER_CTA;
+        wpt = (n_j / 2u + a.rows_min - 1u) / a.rows_min;
         wpt = wpt < 1u ? 1u : (wpt > (uint32_t)a.parts_cap ? (uint32_t)a.parts_cap : wpt);
     }
     const uint32_t spb = __reduce_add_sync(0xffffffffu, wpb), spt = __reduce_add_sync(0xffffffffu, wpt);
@@ -999,6 +992,7 @@ void fill_args(qgbdt_ctx *c, GrowArgs &a) {
     a.K = c->grow_jobs;
     a.slack = qg_grow_slack(c);
     a.xcap = c->grow_xcap;
+    a.rows_min = (uint32_t)c->grow_rows_min;
     a.n_tiles = (int)c->tiles.size();
     a.parts_cap = qg_grow_parts_cap(c);
     a.max_recs = qg_grow_max_recs(c);

@@ -130,6 +130,7 @@ struct GrowHist {
     const uint2 *ent0, *ent1;
     unsigned long long *pool;
     size_t hist_words;
+    uint32_t rows_min;   // rows per CTA, at least (qg_grow_parts)
 };
 
 template <int LOGW_T, int MODE>
@@ -157,7 +158,7 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_grow(HistArgs a, GrowH
     a.n = small_is_left ? nl : nr;
     a.hist = g.pool + (size_t)small_slot * g.hist_words;
     td.cta0 = slot0 + (a.tile0 + (int)blockIdx.y) * parts;
-    const uint32_t P = effective_parts((uint32_t)parts, a.n), part = blockIdx.x - (uint32_t)jc0;
+    const uint32_t P = qg_grow_parts((uint32_t)parts, a.n, g.rows_min), part = blockIdx.x - (uint32_t)jc0;
     if (part >= P) return;
     hist_cta<HIST_THREADS, LOGW_T, MODE, 2>(a, td, part, P, sh);
 }
@@ -461,6 +462,7 @@ int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
     g.ent1 = c->d_ent1;
     g.pool = c->d_hist_pool;
     g.hist_words = (size_t)c->F * c->nb;
+    g.rows_min = (uint32_t)c->grow_rows_min;
     int prc = qg_phase_begin(c, QG_PHASE_CHILD_HIST, st);
     if (prc != QGBDT_OK) return prc;
     int rc;

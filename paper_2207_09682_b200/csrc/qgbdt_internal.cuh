@@ -74,6 +74,17 @@ struct FeatRec {
     const uint8_t *col8;   // the feature's column in the column-major copy (nullptr: there is none)
 };
 
+// Histogram CTAs per tile that take part in building a child of n rows during tree growth: one per
+// `rows_min` rows, at most `parts`.  rows_min is 1024 for rows of up to 32 bytes and grows with the
+// width of the widest tile (4096 for 128-byte rows): a CTA of a wide tile writes a quarter of a
+// megabyte of partial histogram that the finishing kernel has to read back, and has four times the
+// work per row to make up for its fixed cost.
+__device__ __host__ inline uint32_t qg_grow_parts(uint32_t parts, uint32_t n, uint32_t rows_min) {
+    uint32_t want = (n + rows_min - 1) / rows_min;
+    if (want < 1) want = 1;
+    return want < parts ? want : parts;
+}
+
 // ---- leaf-wise growth on the device (grow.cu) --------------------------------------------------
 // A tree grows in passes.  A pass splits up to GROW_MAX_JOBS leaves at once (row partition, the
 // smaller child's histogram, the larger child's by subtraction, both children's best splits); the
@@ -200,6 +211,7 @@ struct qgbdt_ctx {
     int grow_jobs = 1;                          // leaves split per pass (<= GROW_MAX_JOBS; fewer with thousands of features)
     int grow_pb_total = 0;                      // blocks of a partition launch
     int grow_xcap = 0;                          // histogram CTAs per tile of a growth launch
+    int grow_rows_min = 1024;                   // rows per histogram CTA of tree growth, at least
     uint32_t *d_grow_bits = nullptr;            // [grow_jobs][bits_stride] predicate bits of the leaves being split
     size_t grow_bits_stride = 0;
     unsigned long long *d_grow_partial = nullptr;   // [grow_xcap * tiles][4][nb][32] partial histograms of growth

@@ -62,6 +62,9 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
         int k = 65536 / (c->F > 0 ? c->F : 1);
         c->grow_jobs = k < 2 ? 2 : (k > GROW_MAX_JOBS ? GROW_MAX_JOBS : k);
         c->grow_xcap = 2 * qg_grow_parts_cap(c) + c->grow_jobs;
+        int max_logw = 0;
+        for (const TileDesc &t : c->tiles) max_logw = t.logW > max_logw ? t.logW : max_logw;
+        c->grow_rows_min = 1024 << (max_logw > 3 ? max_logw - 3 : 0);
         c->grow_bits_stride = ((size_t)c->N + 31) / 32 + 64;
     }
     if (!c->d_hist_pool &&

@@ -278,6 +278,19 @@ __device__ inline SplitRec shfl_xor_rec(const SplitRec &r, int o) {
     return x;
 }
 
+// Largest a and largest b over the block (NW warps); ends with every thread holding both.
+template <int NW>
+__device__ __forceinline__ void block_max2(float &a, float &b, float (*buf)[NW]) {
+    for (int o = 16; o > 0; o >>= 1) {
+        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+        b = fmaxf(b, __shfl_xor_sync(0xffffffffu, b, o));
+    }
+    if ((threadIdx.x & 31) == 0) { buf[0][threadIdx.x >> 5] = a; buf[1][threadIdx.x >> 5] = b; }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { a = fmaxf(a, buf[0][w]); b = fmaxf(b, buf[1][w]); }
+}
+
 // One feature of one leaf being split (ROOT: of the root): the work of a block of k_grow_finish.
 // BPT bins per thread: 1 (256 threads) or 2 (128 threads: with thousands of features twice as many
 // blocks are resident).
@@ -331,6 +344,10 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
     unsigned long long *S = a.pool + (size_t)small_slot * hw + (size_t)f * a.nb;
     unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)parent_slot * hw + (size_t)f * a.nb;
     __shared__ long long wtot[4][FIN_WARPS];
+    __shared__ float fmax_buf[2][FIN_WARPS];
+    const float NEGF = -__int_as_float(0x7f800000);
+    GainScale sc;
+    sc.dg = (float)dg; sc.dh = (float)dh; sc.lambda = (float)pS.lambda;
     SplitRec rS = qg_invalid_rec(), rL = qg_invalid_rec();
     rS.feature = f;
     rL.feature = f;
@@ -379,6 +396,8 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
 #pragma unroll
         for (int c = 0; c < (ROOT ? 2 : 4); ++c)
             for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
+        // with a block per feature and few features the blocks wait on memory, not on the gains: every
+        // admissible threshold is evaluated outright (the pruning below pays with thousands of features)
         if (in) {
             double gain;
             if (qg_eval_candidate(v[0], v[1], pS, dg, dh, tpS, gain)) {
@@ -449,23 +468,44 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
 #pragma unroll
         for (int c = 0; c < (ROOT ? 2 : 4); ++c)
             for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
+        // the inclusive sums at each of the thread's bins (from the last one down)
+        long long sums[BPT][4];
+#pragma unroll
+        for (int jb = BPT - 1; jb >= 0; --jb) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { sums[jb][c] = v[c]; v[c] -= x[jb][c]; }
+        }
+        // cheap bounds on every admissible threshold's gain first; the exact gain (two double-precision
+        // divisions) only where the upper bound reaches the block's largest lower bound
+        bool okS[BPT], okL[BPT];
+        float hiS[BPT], hiL[BPT], mS = NEGF, mL = NEGF;
+#pragma unroll
+        for (int jb = 0; jb < BPT; ++jb) {
+            const bool in = (int)threadIdx.x * BPT + jb < a.nb - 1;
+            okS[jb] = in && qg_candidate_admissible(sums[jb][0], sums[jb][1], pS, dh);
+            okL[jb] = !ROOT && in && qg_candidate_admissible(sums[jb][2], sums[jb][3], pL, dh);
+            float lo = NEGF;
+            hiS[jb] = hiL[jb] = NEGF;
+            if (okS[jb]) { qg_gain_bounds(sums[jb][0], sums[jb][1], pS, sc, (float)tpS, lo, hiS[jb]); mS = fmaxf(mS, lo); }
+            if (okL[jb]) { qg_gain_bounds(sums[jb][2], sums[jb][3], pL, sc, (float)tpL, lo, hiL[jb]); mL = fmaxf(mL, lo); }
+        }
+        block_max2<FIN_WARPS>(mS, mL, fmax_buf);
         // thresholds from the thread's last bin down (the lower bin wins on equal gain)
 #pragma unroll
         for (int jb = BPT - 1; jb >= 0; --jb) {
             const int b = (int)threadIdx.x * BPT + jb;
-            if (b < a.nb - 1) {
-                double gain;
-                if (qg_eval_candidate(v[0], v[1], pS, dg, dh, tpS, gain) &&
-                    qg_better(true, gain, b, rS.valid != 0, rS.gain, rS.bin)) {
-                    rS.valid = 1; rS.gain = gain; rS.bin = b; rS.gl = v[0]; rS.hl = v[1];
-                }
-                if (!ROOT && qg_eval_candidate(v[2], v[3], pL, dg, dh, tpL, gain) &&
-                    qg_better(true, gain, b, rL.valid != 0, rL.gain, rL.bin)) {
-                    rL.valid = 1; rL.gain = gain; rL.bin = b; rL.gl = v[2]; rL.hl = v[3];
+            if (okS[jb] && hiS[jb] >= mS) {
+                const double gain = qg_candidate_gain(sums[jb][0], sums[jb][1], pS, dg, dh, tpS);
+                if (gain > pS.min_gain && qg_better(true, gain, b, rS.valid != 0, rS.gain, rS.bin)) {
+                    rS.valid = 1; rS.gain = gain; rS.bin = b; rS.gl = sums[jb][0]; rS.hl = sums[jb][1];
                 }
             }
-#pragma unroll
-            for (int c = 0; c < 4; ++c) v[c] -= x[jb][c];
+            if (okL[jb] && hiL[jb] >= mL) {
+                const double gain = qg_candidate_gain(sums[jb][2], sums[jb][3], pL, dg, dh, tpL);
+                if (gain > pL.min_gain && qg_better(true, gain, b, rL.valid != 0, rL.gain, rL.bin)) {
+                    rL.valid = 1; rL.gain = gain; rL.bin = b; rL.gl = sums[jb][2]; rL.hl = sums[jb][3];
+                }
+            }
         }
     }
     // best threshold of the feature: largest gain, lowest bin on equal gain
@@ -556,7 +596,7 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
 // (Y is chosen on the host so that the grid fills the SMs a few times over without launching a block
 // for every feature of every possible leaf).
 template <bool ROOT, int BPT>
-__global__ void __launch_bounds__(256 / BPT) k_grow_finish(GrowArgs a) {
+__global__ void __launch_bounds__(256 / BPT, BPT == 2 ? 8 : 1) k_grow_finish(GrowArgs a) {
     if (ROOT) {
         finish_one<ROOT, BPT>(a, (int)blockIdx.x, 0);
         return;

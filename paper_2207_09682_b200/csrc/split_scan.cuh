@@ -32,22 +32,63 @@ __device__ inline void qg_scales(const DevState *state, const SplitParams &p, do
     dh = p.const_h ? 1.0 : __ddiv_rn((double)__uint_as_float(state->hmax_bits), (double)p.kh);
 }
 
+// Threshold candidate with left sums (gl, hl): everything of its admissibility that needs no gain.
+// The row estimate of a side is floor((hl * n_s + H / 2) / H) (exact count with a constant hessian);
+// it is only compared with min_data, so the comparisons are made on the products instead of
+// dividing: floor(X / H) >= m  <=>  X >= m * H, and floor(X / H) <= k  <=>  X < (k + 1) * H.
+__device__ inline bool qg_candidate_admissible(long long gl, long long hl, const SplitParams &p, double dh) {
+    (void)gl;
+    const long long hr = p.H - hl;
+    if (!(hl > 0 && hr > 0)) return false;
+    if (p.const_h) {
+        if (!(hl >= p.min_data && p.n_s - hl >= p.min_data)) return false;
+    } else {
+        const unsigned long long H = (unsigned long long)p.H, X = (unsigned long long)hl * (unsigned long long)p.n_s + H / 2;
+        const long long k = p.n_s - p.min_data;          // the left side may have at most this many rows
+        if (X < (unsigned long long)p.min_data * H) return false;
+        if (k < 0 || X >= (unsigned long long)(k + 1) * H) return false;
+    }
+    if (__dmul_rn((double)hl, dh) < p.min_sum_h || __dmul_rn((double)hr, dh) < p.min_sum_h) return false;
+    return true;
+}
+
+// Eq. 7 for an admissible candidate, every operation individually rounded in double precision.
+__device__ inline double qg_candidate_gain(long long gl, long long hl, const SplitParams &p, double dg, double dh, double tp) {
+    const double tl = qg_gain_term(gl, hl, dg, dh, p.lambda);
+    const double tr = qg_gain_term(p.G - gl, p.H - hl, dg, dh, p.lambda);
+    return __dmul_rn(0.5, __dsub_rn(__dadd_rn(tl, tr), tp));
+}
+
 // Threshold candidate with left sums (gl, hl): admissible?  If so its gain (Eq. 7).
 __device__ inline bool qg_eval_candidate(long long gl, long long hl, const SplitParams &p, double dg, double dh,
                                          double tp, double &gain) {
-    const long long gr = p.G - gl, hr = p.H - hl;
-    if (!(hl > 0 && hr > 0)) return false;
-    long long nl;
-    if (p.const_h) nl = hl;
-    else nl = (long long)(((unsigned long long)hl * (unsigned long long)p.n_s + (unsigned long long)(p.H / 2)) /
-                          (unsigned long long)p.H);
-    const long long nr = p.n_s - nl;
-    if (!(nl >= p.min_data && nr >= p.min_data)) return false;
-    if (__dmul_rn((double)hl, dh) < p.min_sum_h || __dmul_rn((double)hr, dh) < p.min_sum_h) return false;
-    const double tl = qg_gain_term(gl, hl, dg, dh, p.lambda);
-    const double tr = qg_gain_term(gr, hr, dg, dh, p.lambda);
-    gain = __dmul_rn(0.5, __dsub_rn(__dadd_rn(tl, tr), tp));
+    if (!qg_candidate_admissible(gl, hl, p, dh)) return false;
+    gain = qg_candidate_gain(gl, hl, p, dg, dh, tp);
     return gain > p.min_gain;
+}
+
+// Single-precision bounds [lo, hi] on the double-precision gain of an admissible candidate, about a
+// sixth of the cost of the gain itself (no double-precision division).  Every term of Eq. 7 comes
+// out with a relative error of at most 12 * 2^-24 (conversions, products, one division each), so the
+// gain is off by less than 16 * 2^-24 * (term L + term R + term P); the bounds take four times
+// that.  A search that keeps every candidate whose `hi` reaches the largest `lo` keeps every
+// candidate that can have the largest gain.
+struct GainScale {
+    float dg, dh, lambda;
+};
+__device__ inline void qg_gain_bounds(long long gl, long long hl, const SplitParams &p, const GainScale &sc, float tp,
+                                      float &lo, float &hi) {
+    const float gdl = __fmul_rn((float)gl, sc.dg), gdr = __fmul_rn((float)(p.G - gl), sc.dg);
+    const float hdl = __fadd_rn(__fmul_rn((float)hl, sc.dh), sc.lambda), hdr = __fadd_rn(__fmul_rn((float)(p.H - hl), sc.dh), sc.lambda);
+    const float tl = __fdiv_rn(__fmul_rn(gdl, gdl), hdl), tr = __fdiv_rn(__fmul_rn(gdr, gdr), hdr);
+    const float gain = __fmul_rn(0.5f, __fsub_rn(__fadd_rn(tl, tr), tp));
+    const float err = __fmul_rn(3.814697265625e-6f, __fadd_rn(__fadd_rn(tl, tr), tp));   // 64 * 2^-24
+    lo = __fsub_rn(gain, err);
+    hi = __fadd_rn(gain, err);
+    if (!(fabsf(gain) <= 3.0e38f) || !(err <= 3.0e38f)) {   // out of single-precision range: no information
+        lo = -__int_as_float(0x7f800000);
+        hi = __int_as_float(0x7f800000);
+    }
 }
 
 // Running state of one feature's scan in one lane.

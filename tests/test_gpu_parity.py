@@ -445,6 +445,12 @@ TRAIN_CASES = [
     ("large", 40_000, dict(num_trees=2, num_leaves=31, bits=7)),
     ("tall", 30_000, dict(num_trees=2, num_leaves=31, bits=5, hess_levels_mode=1)),
     ("tiny", 20_000, dict(num_trees=2, rounding=1)),
+    # the smallest trees, and the most leaves a context takes (thousands of growth records in the commit step)
+    ("tiny", 5_000, dict(num_trees=2, num_leaves=1)),
+    ("tiny", 5_000, dict(num_trees=2, num_leaves=2)),
+    ("tiny", 5_000, dict(num_trees=2, num_leaves=3)),
+    ("tall", 60_000, dict(num_trees=2, num_leaves=4096, min_data_in_leaf=3)),
+    ("tall", 40_000, dict(num_trees=1, num_leaves=1500, min_data_in_leaf=1, bits=2)),
 ]
 
 

@@ -84,7 +84,7 @@ __global__ void k_grow_begin(GrowState *gs, NodeRec *recs, double *rec_gain, int
     // gradients out of domain (the flag is sticky over the trees of a train call): this tree stays
     // a single leaf, the call reports the error when it ends
     gs->done = state->bad_value ? 1 : 0;
-    for (int j = 0; j < GROW_MAX_JOBS; ++j) gs->jobs[j].finish_count = 0;
+    for (int j = 0; j < GROW_MAX_JOBS; ++j) { gs->jobs[j].finish_count = 0; gs->jobs[j].lb[0] = gs->jobs[j].lb[1] = 0; }
 }
 
 // Words of 32 rows [w0, w1) of warp gw: every warp takes the same number of consecutive words
@@ -278,6 +278,15 @@ __device__ inline SplitRec shfl_xor_rec(const SplitRec &r, int o) {
     return x;
 }
 
+// Floats as unsigned integers of the same order (every such integer is at least 1: 0 can stand for "none").
+__device__ __forceinline__ unsigned int float_order_bits(float f) {
+    const unsigned int u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float order_bits_float(unsigned int k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
 // Largest a and largest b over the block (NW warps); ends with every thread holding both.
 template <int NW>
 __device__ __forceinline__ void block_max2(float &a, float &b, float (*buf)[NW]) {
@@ -345,6 +354,7 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
     unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)parent_slot * hw + (size_t)f * a.nb;
     __shared__ long long wtot[4][FIN_WARPS];
     __shared__ float fmax_buf[2][FIN_WARPS];
+    __shared__ float lb_buf[2];
     const float NEGF = -__int_as_float(0x7f800000);
     GainScale sc;
     sc.dg = (float)dg; sc.dh = (float)dh; sc.lambda = (float)pS.lambda;
@@ -490,6 +500,18 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
             if (okL[jb]) { qg_gain_bounds(sums[jb][2], sums[jb][3], pL, sc, (float)tpL, lo, hiL[jb]); mL = fmaxf(mL, lo); }
         }
         block_max2<FIN_WARPS>(mS, mL, fmax_buf);
+        // the largest lower bound any feature of this leaf has seen so far prunes as well: a threshold
+        // whose upper bound lies below it has a strictly smaller gain than some admissible threshold and
+        // cannot be the leaf's best (which blocks came first changes the work, never the result)
+        if (threadIdx.x < 2) {
+            const float m = threadIdx.x == 0 ? mS : mL;
+            const unsigned int mine = float_order_bits(m);
+            const unsigned int old = atomicMax(&job->lb[threadIdx.x], mine);
+            lb_buf[threadIdx.x] = order_bits_float(old > mine ? old : mine);
+        }
+        __syncthreads();
+        mS = lb_buf[0];
+        mL = lb_buf[1];
         // thresholds from the thread's last bin down (the lower bin wins on equal gain)
 #pragma unroll
         for (int jb = BPT - 1; jb >= 0; --jb) {
@@ -560,6 +582,7 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
         if (qg_rec_better(sm[1][w], bL)) bL = sm[1][w];
     }
     job->finish_count = 0;
+    job->lb[0] = job->lb[1] = 0;
     const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
     if (ROOT) {
         a.recs[0].best = bS;
@@ -960,6 +983,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         job->small_slot = 1 + n_exec + lane;
         job->child0 = n_recs + 2 * lane;
         job->finish_count = 0;
+        job->lb[0] = job->lb[1] = 0;
         q->state = 1;
         q->child0 = n_recs + 2 * lane;
         a.rec_child[r] = n_recs + 2 * lane;
@@ -1090,8 +1114,7 @@ int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st, int n_jobs = 
             return rc;
     }
     if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
-    if (c->F > c->sm_count * 8) k_grow_finish<false, 2><<<fin, 128, 0, st>>>(a);
-    else k_grow_finish<false, 1><<<fin, 256, 0, st>>>(a);
+    k_grow_finish<false, 2><<<fin, 128, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     return launch_commit(c, a, st);

@@ -140,6 +140,8 @@ struct GrowJob {
     int32_t cta0, parts;             // histogram CTAs per tile: x in [cta0, cta0 + parts) of the grid
     int32_t slot0;                   // partial-histogram slots: tile t, part p uses slot0 + t * parts + p
     unsigned int finish_count;       // blocks of the finishing kernel that are through
+    unsigned int lb[2];              // largest lower bound on a gain seen so far over all features (smaller, larger
+                                     // child), as order-preserving bits of a float; 0 = none yet
     int32_t pad;
 };
 

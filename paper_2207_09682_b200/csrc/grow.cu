@@ -287,30 +287,43 @@ __device__ __forceinline__ float order_bits_float(unsigned int k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-// Largest a and largest b over the block (NW warps); ends with every thread holding both.
-template <int NW>
-__device__ __forceinline__ void block_max2(float &a, float &b, float (*buf)[NW]) {
+// Best threshold of a warp: every lane brings its best (gain, bin >= 0, packed left sums) or bin < 0;
+// all lanes return the warp's best (largest gain, lowest bin on equal gain; bin < 0: none).
+__device__ __forceinline__ void warp_best(double &gain, int &bin, unsigned long long &w) {
+    if (!__any_sync(0xffffffffu, bin >= 0)) return;
+    double g = gain;
+    int b = bin;
     for (int o = 16; o > 0; o >>= 1) {
-        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-        b = fmaxf(b, __shfl_xor_sync(0xffffffffu, b, o));
+        const double og = __shfl_xor_sync(0xffffffffu, g, o);
+        const int ob = __shfl_xor_sync(0xffffffffu, b, o);
+        if (qg_better(ob >= 0, og, ob, b >= 0, g, b)) { g = og; b = ob; }
     }
-    if ((threadIdx.x & 31) == 0) { buf[0][threadIdx.x >> 5] = a; buf[1][threadIdx.x >> 5] = b; }
-    __syncthreads();
-#pragma unroll
-    for (int w = 0; w < NW; ++w) { a = fmaxf(a, buf[0][w]); b = fmaxf(b, buf[1][w]); }
+    // the bins of the lanes are distinct: the lane that brought the winning bin owns the sums
+    const unsigned int owner = __ballot_sync(0xffffffffu, bin == b);
+    w = __shfl_sync(0xffffffffu, w, __ffs(owner) - 1);
+    gain = g;
+    bin = b;
 }
 
+// What a warp of the finishing kernel leaves for the block's first thread.
+struct WarpBest {
+    double gain;
+    unsigned long long w;
+    int bin, pad;
+};
+
+constexpr int FIN_THREADS = 128, FIN_WARPS = FIN_THREADS / 32, FIN_BLOCKS_PER_SM = 8;
+
 // One feature of one leaf being split (ROOT: of the root): the work of a block of k_grow_finish.
-// BPT bins per thread: 1 (256 threads) or 2 (128 threads: with thousands of features twice as many
-// blocks are resident).
-template <bool ROOT, int BPT>
+// 128 threads, thread t owns bins 2 t and 2 t + 1 (n_bins <= 256).  A bin is one 64-bit word, the
+// gradient sum in the upper half and the hessian sum in the lower; the sums of a whole leaf fit the
+// halves (checked when the rows are loaded), so prefix sums are taken on the words themselves.
+template <bool ROOT>
 __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const int j) {
-    constexpr int FIN_WARPS = 8 / BPT;
     GrowState *gs = a.gs;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     GrowJob *job = gs->jobs + j;
-    // everything the block needs from the state, at once (one round trip to memory), then the early exit
-    const int done = gs->done, n_jobs = gs->n_jobs;
+    // everything the block needs from the state, at once (one round trip to memory)
     const int parent_slot = ROOT ? 0 : job->parent_slot, small_slot = ROOT ? 0 : job->small_slot;
     const int parts = job->parts, slot0 = job->slot0, child0 = job->child0, jrec = job->rec, jbuf = job->buf;
     const uint32_t gs_n = job->n, gs_nl = job->nl, gs_off = job->off, gs_n_all = job->n_all;
@@ -319,7 +332,6 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
     const long long tot_g = a.state->tot_g, tot_h = a.state->tot_h;
     const uint32_t gmax_bits = a.state->gmax_bits, hmax_bits = a.state->hmax_bits;
     const FeatRec fr = a.feat_rec[f];
-    if (done || (!ROOT && j >= n_jobs)) return;
     const size_t hw = (size_t)a.F * a.nb;
 
     // the two children: "small" was built by Algorithm 1, "large" is parent - small
@@ -336,15 +348,20 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
         pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl_all : nr_all;
         pL.G = small_is_left ? gr : gl; pL.H = small_is_left ? hr : hl; pL.n_s = small_is_left ? nr_all : nl_all;
     }
-    // ---- phase A: one thread per bin: the smaller child's sum over the partial histograms, the
-    //      larger child's bin by subtraction
-    __shared__ SplitRec sm[2][FIN_WARPS];
+    __shared__ WarpBest sm[2][FIN_WARPS];
     __shared__ bool is_last;
+    __shared__ unsigned long long wtot[2][FIN_WARPS];
     // interval lengths of Eq. 5 from the maxima stored by the quantizer
     const double dg = __ddiv_rn((double)__uint_as_float(gmax_bits), (double)pS.kg);
     const double dh = pS.const_h ? 1.0 : __ddiv_rn((double)__uint_as_float(hmax_bits), (double)pS.kh);
     const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
     const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
+    GainScale sc;
+    sc.dg = (float)dg; sc.dh = (float)dh; sc.lambda = (float)pS.lambda;
+    const Admit32 aS = qg_admit32(pS, dh), aL = qg_admit32(pL, dh);
+
+    // ---- phase A: the smaller child's bins summed over the partial histograms, the larger child's
+    //      by subtraction from the parent's
     const int fl = fr.fl, W = 1 << fr.logW;
     const uint32_t P = (ROOT || a.merged) ? 1u : qg_grow_parts((uint32_t)parts, small_is_left ? nl : nr, a.rows_min);
     const size_t pstride = (size_t)4 * a.nb * 32;
@@ -352,217 +369,141 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
                                      (size_t)(fl & 3) * a.nb * W + (fl >> 2);
     unsigned long long *S = a.pool + (size_t)small_slot * hw + (size_t)f * a.nb;
     unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)parent_slot * hw + (size_t)f * a.nb;
-    __shared__ long long wtot[4][FIN_WARPS];
-    __shared__ float fmax_buf[2][FIN_WARPS];
-    __shared__ float lb_buf[2];
-    const float NEGF = -__int_as_float(0x7f800000);
-    GainScale sc;
-    sc.dg = (float)dg; sc.dh = (float)dh; sc.lambda = (float)pS.lambda;
-    SplitRec rS = qg_invalid_rec(), rL = qg_invalid_rec();
-    rS.feature = f;
-    rL.feature = f;
-    if (BPT == 1) {
-        // n_bins <= 256: thread b owns bin b
-        const int b = (int)threadIdx.x;
-        unsigned long long s = 0, l = 0;
-        if (b < a.nb) {
-            if (ROOT) {
-                s = S[b];
-            } else {
-                if (P > 1) {
+    unsigned long long sv[2], lv[2];
+    {
+        unsigned long long pv[2];
+#pragma unroll
+        for (int jb = 0; jb < 2; ++jb) {
+            const int b = (int)threadIdx.x * 2 + jb;
+            sv[jb] = 0; lv[jb] = 0; pv[jb] = 0;
+            if (b < a.nb) {
+                if (!ROOT) pv[jb] = Pp[b];
+                if (!ROOT && P > 1) {
                     const unsigned long long *q = part + (size_t)b * W;
-                    for (uint32_t i0 = 0; i0 < P; i0 += 8) {   // 8 independent loads in flight
-                        unsigned long long x[8];
+                    for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
+                        unsigned long long x[16];
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
+                        for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) s += x[k];
+                        for (int k = 0; k < 16; ++k) sv[jb] += x[k];
                     }
-                    S[b] = s;
                 } else {
-                    s = S[b];
-                }
-                l = Pp[b] - s;   // no field borrows: every child sum is at most the parent's
-                Pp[b] = l;
-            }
-        }
-        // ---- phase B: prefix sums over the bins by all eight warps (warp scan, then the warp totals),
-        //      every thread evaluates the threshold at its own bin for both children
-        const bool in = b < a.nb - 1;   // thresholds 0 .. nb-2
-        long long v[4];
-        v[0] = in ? (long long)(int)(s >> 32) : 0;
-        v[1] = in ? (long long)(unsigned int)(s & 0xFFFFFFFFull) : 0;
-        v[2] = in ? (long long)(int)(l >> 32) : 0;
-        v[3] = in ? (long long)(unsigned int)(l & 0xFFFFFFFFull) : 0;
-#pragma unroll
-        for (int c = 0; c < (ROOT ? 2 : 4); ++c) {
-            for (int o = 1; o < 32; o <<= 1) {
-                const long long u = __shfl_up_sync(0xffffffffu, v[c], o);
-                if (lane >= o) v[c] += u;
-            }
-            if (lane == 31) wtot[c][warp] = v[c];
-        }
-        __syncthreads();
-#pragma unroll
-        for (int c = 0; c < (ROOT ? 2 : 4); ++c)
-            for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
-        // with a block per feature and few features the blocks wait on memory, not on the gains: every
-        // admissible threshold is evaluated outright (the pruning below pays with thousands of features)
-        if (in) {
-            double gain;
-            if (qg_eval_candidate(v[0], v[1], pS, dg, dh, tpS, gain)) {
-                rS.valid = 1; rS.gain = gain; rS.bin = b; rS.gl = v[0]; rS.hl = v[1];
-            }
-            if (!ROOT && qg_eval_candidate(v[2], v[3], pL, dg, dh, tpL, gain)) {
-                rL.valid = 1; rL.gain = gain; rL.bin = b; rL.gl = v[2]; rL.hl = v[3];
-            }
-        }
-    } else {
-        // n_bins <= 256: thread t owns bins BPT t .. BPT t + BPT - 1
-        unsigned long long sv[BPT], lv[BPT];
-        {
-            unsigned long long pv[BPT];
-#pragma unroll
-            for (int jb = 0; jb < BPT; ++jb) {
-                const int b = (int)threadIdx.x * BPT + jb;
-                sv[jb] = 0; lv[jb] = 0; pv[jb] = 0;
-                if (b < a.nb) {
-                    if (!ROOT) pv[jb] = Pp[b];
-                    if (!ROOT && P > 1) {
-                        const unsigned long long *q = part + (size_t)b * W;
-                        for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
-                            unsigned long long x[16];
-#pragma unroll
-                            for (int k = 0; k < 16; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
-#pragma unroll
-                            for (int k = 0; k < 16; ++k) sv[jb] += x[k];
-                        }
-                    } else {
-                        sv[jb] = S[b];
-                    }
-                }
-            }
-#pragma unroll
-            for (int jb = 0; jb < BPT; ++jb) {
-                const int b = (int)threadIdx.x * BPT + jb;
-                if (!ROOT && b < a.nb) {
-                    if (P > 1) S[b] = sv[jb];
-                    lv[jb] = pv[jb] - sv[jb];   // no field borrows: every child sum is at most the parent's
-                    Pp[b] = lv[jb];
+                    sv[jb] = S[b];
                 }
             }
         }
-        // ---- phase B: prefix sums over the bins by all warps (the thread's own bins, a warp scan of
-        //      the threads' totals, then the warp totals); every thread evaluates the thresholds at its
-        //      own bins for both children
-        long long x[BPT][4], v[4] = {0, 0, 0, 0};   // per bin; v: inclusive sum up to the thread's last bin
 #pragma unroll
-        for (int jb = 0; jb < BPT; ++jb) {
-            const bool in = (int)threadIdx.x * BPT + jb < a.nb - 1;   // thresholds 0 .. nb-2
-            x[jb][0] = in ? (long long)(int)(sv[jb] >> 32) : 0;
-            x[jb][1] = in ? (long long)(unsigned int)(sv[jb] & 0xFFFFFFFFull) : 0;
-            x[jb][2] = in ? (long long)(int)(lv[jb] >> 32) : 0;
-            x[jb][3] = in ? (long long)(unsigned int)(lv[jb] & 0xFFFFFFFFull) : 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) v[c] += x[jb][c];
-        }
-#pragma unroll
-        for (int c = 0; c < (ROOT ? 2 : 4); ++c) {
-            for (int o = 1; o < 32; o <<= 1) {
-                const long long u = __shfl_up_sync(0xffffffffu, v[c], o);
-                if (lane >= o) v[c] += u;
+        for (int jb = 0; jb < 2; ++jb) {
+            const int b = (int)threadIdx.x * 2 + jb;
+            if (!ROOT && b < a.nb) {
+                if (P > 1) S[b] = sv[jb];
+                lv[jb] = pv[jb] - sv[jb];   // no field borrows: every child sum is at most the parent's
+                Pp[b] = lv[jb];
             }
-            if (lane == 31) wtot[c][warp] = v[c];
         }
-        __syncthreads();
-#pragma unroll
-        for (int c = 0; c < (ROOT ? 2 : 4); ++c)
-            for (int w = 0; w < warp; ++w) v[c] += wtot[c][w];
-        // the inclusive sums at each of the thread's bins (from the last one down)
-        long long sums[BPT][4];
-#pragma unroll
-        for (int jb = BPT - 1; jb >= 0; --jb) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) { sums[jb][c] = v[c]; v[c] -= x[jb][c]; }
+    }
+    // ---- phase B: prefix sums over the bins (the thread's two bins, a warp scan of the threads'
+    //      totals, then the totals of the warps before); thresholds are the bins 0 .. nb-2
+    const int b0 = (int)threadIdx.x * 2;
+    const bool in0 = b0 < a.nb - 1, in1 = b0 + 1 < a.nb - 1;
+    const unsigned long long xS1 = in1 ? sv[1] : 0ull, xL1 = in1 ? lv[1] : 0ull;
+    unsigned long long vS = (in0 ? sv[0] : 0ull) + xS1, vL = (in0 ? lv[0] : 0ull) + xL1;
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long uS = __shfl_up_sync(0xffffffffu, vS, o);
+        if (lane >= o) vS += uS;
+        if (!ROOT) {
+            const unsigned long long uL = __shfl_up_sync(0xffffffffu, vL, o);
+            if (lane >= o) vL += uL;
         }
-        // cheap bounds on every admissible threshold's gain first; the exact gain (two double-precision
-        // divisions) only where the upper bound reaches the block's largest lower bound
-        bool okS[BPT], okL[BPT];
-        float hiS[BPT], hiL[BPT], mS = NEGF, mL = NEGF;
+    }
+    if (lane == 31) { wtot[0][warp] = vS; wtot[1][warp] = vL; }
+    __syncthreads();
+    for (int w = 0; w < warp; ++w) { vS += wtot[0][w]; vL += wtot[1][w]; }
+    // inclusive sums at the thread's bins: [1] at bin b0 + 1, [0] at bin b0
+    const unsigned long long pS2[2] = {vS - xS1, vS}, pL2[2] = {vL - xL1, vL};
+
+    // ---- phase C: cheap single-precision bounds on every admissible threshold's gain; the exact gain
+    //      (two double-precision divisions) only where the upper bound reaches the largest lower bound
+    //      the warp knows of: its own, and the largest any warp working on this leaf has published so
+    //      far, whatever its feature.  A threshold whose upper bound lies below a lower bound has a
+    //      strictly smaller gain than some admissible threshold of the leaf and cannot be its best
+    //      (which warps came first changes the work, never the result).
+    const float NEGF = -__int_as_float(0x7f800000);
+    bool okS[2], okL[2];
+    float hiS[2], hiL[2], mS = NEGF, mL = NEGF;
 #pragma unroll
-        for (int jb = 0; jb < BPT; ++jb) {
-            const bool in = (int)threadIdx.x * BPT + jb < a.nb - 1;
-            okS[jb] = in && qg_candidate_admissible(sums[jb][0], sums[jb][1], pS, dh);
-            okL[jb] = !ROOT && in && qg_candidate_admissible(sums[jb][2], sums[jb][3], pL, dh);
-            float lo = NEGF;
-            hiS[jb] = hiL[jb] = NEGF;
-            if (okS[jb]) { qg_gain_bounds(sums[jb][0], sums[jb][1], pS, sc, (float)tpS, lo, hiS[jb]); mS = fmaxf(mS, lo); }
-            if (okL[jb]) { qg_gain_bounds(sums[jb][2], sums[jb][3], pL, sc, (float)tpL, lo, hiL[jb]); mL = fmaxf(mL, lo); }
-        }
-        block_max2<FIN_WARPS>(mS, mL, fmax_buf);
-        // the largest lower bound any feature of this leaf has seen so far prunes as well: a threshold
-        // whose upper bound lies below it has a strictly smaller gain than some admissible threshold and
-        // cannot be the leaf's best (which blocks came first changes the work, never the result)
-        if (threadIdx.x < 2) {
-            const float m = threadIdx.x == 0 ? mS : mL;
-            const unsigned int mine = float_order_bits(m);
-            const unsigned int old = atomicMax(&job->lb[threadIdx.x], mine);
-            lb_buf[threadIdx.x] = order_bits_float(old > mine ? old : mine);
-        }
-        __syncthreads();
-        mS = lb_buf[0];
-        mL = lb_buf[1];
-        // thresholds from the thread's last bin down (the lower bin wins on equal gain)
+    for (int jb = 0; jb < 2; ++jb) {
+        const bool in = jb == 0 ? in0 : in1;
+        const int glS = (int)(pS2[jb] >> 32), glL = (int)(pL2[jb] >> 32);
+        const uint32_t hlS = (uint32_t)pS2[jb], hlL = (uint32_t)pL2[jb];
+        okS[jb] = in && qg_admissible32(hlS, aS, sc);
+        okL[jb] = !ROOT && in && qg_admissible32(hlL, aL, sc);
+        float lo;
+        hiS[jb] = hiL[jb] = NEGF;
+        if (okS[jb]) { qg_gain_bounds32(glS, hlS, aS, sc, (float)tpS, lo, hiS[jb]); mS = fmaxf(mS, lo); }
+        if (okL[jb]) { qg_gain_bounds32(glL, hlL, aL, sc, (float)tpL, lo, hiL[jb]); mL = fmaxf(mL, lo); }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        mS = fmaxf(mS, __shfl_xor_sync(0xffffffffu, mS, o));
+        if (!ROOT) mL = fmaxf(mL, __shfl_xor_sync(0xffffffffu, mL, o));
+    }
+    if (lane < (ROOT ? 1 : 2)) {
+        const unsigned int mine = float_order_bits(lane == 0 ? mS : mL);
+        unsigned int seen = *reinterpret_cast<volatile unsigned int *>(&job->lb[lane]);
+        if (mine > seen) seen = max(atomicMax(&job->lb[lane], mine), mine);
+        mS = order_bits_float(seen);   // lane 0: smaller child, lane 1: larger child
+    }
+    mL = __shfl_sync(0xffffffffu, mS, 1);
+    mS = __shfl_sync(0xffffffffu, mS, 0);
+    double gS = 0.0, gL = 0.0;
+    int binS = -1, binL = -1;
+    unsigned long long wS = 0, wL = 0;
+    // thresholds from the thread's upper bin down (the lower bin wins on equal gain)
 #pragma unroll
-        for (int jb = BPT - 1; jb >= 0; --jb) {
-            const int b = (int)threadIdx.x * BPT + jb;
-            if (okS[jb] && hiS[jb] >= mS) {
-                const double gain = qg_candidate_gain(sums[jb][0], sums[jb][1], pS, dg, dh, tpS);
-                if (gain > pS.min_gain && qg_better(true, gain, b, rS.valid != 0, rS.gain, rS.bin)) {
-                    rS.valid = 1; rS.gain = gain; rS.bin = b; rS.gl = sums[jb][0]; rS.hl = sums[jb][1];
-                }
-            }
-            if (okL[jb] && hiL[jb] >= mL) {
-                const double gain = qg_candidate_gain(sums[jb][2], sums[jb][3], pL, dg, dh, tpL);
-                if (gain > pL.min_gain && qg_better(true, gain, b, rL.valid != 0, rL.gain, rL.bin)) {
-                    rL.valid = 1; rL.gain = gain; rL.bin = b; rL.gl = sums[jb][2]; rL.hl = sums[jb][3];
-                }
-            }
+    for (int jb = 1; jb >= 0; --jb) {
+        if (okS[jb] && hiS[jb] >= mS) {
+            const double gain = qg_candidate_gain((long long)(int)(pS2[jb] >> 32), (long long)(uint32_t)pS2[jb], pS, dg, dh, tpS);
+            if (gain > pS.min_gain && (binS < 0 || gain >= gS)) { gS = gain; binS = b0 + jb; wS = pS2[jb]; }
+        }
+        if (okL[jb] && hiL[jb] >= mL) {
+            const double gain = qg_candidate_gain((long long)(int)(pL2[jb] >> 32), (long long)(uint32_t)pL2[jb], pL, dg, dh, tpL);
+            if (gain > pL.min_gain && (binL < 0 || gain >= gL)) { gL = gain; binL = b0 + jb; wL = pL2[jb]; }
         }
     }
     // best threshold of the feature: largest gain, lowest bin on equal gain
-    for (int o = 16; o > 0; o >>= 1) {
-        SplitRec x = rS, y = rL;
-        x.gain = __shfl_xor_sync(0xffffffffu, rS.gain, o); y.gain = __shfl_xor_sync(0xffffffffu, rL.gain, o);
-        x.gl = __shfl_xor_sync(0xffffffffu, rS.gl, o);     y.gl = __shfl_xor_sync(0xffffffffu, rL.gl, o);
-        x.hl = __shfl_xor_sync(0xffffffffu, rS.hl, o);     y.hl = __shfl_xor_sync(0xffffffffu, rL.hl, o);
-        x.bin = __shfl_xor_sync(0xffffffffu, rS.bin, o);   y.bin = __shfl_xor_sync(0xffffffffu, rL.bin, o);
-        x.valid = __shfl_xor_sync(0xffffffffu, rS.valid, o); y.valid = __shfl_xor_sync(0xffffffffu, rL.valid, o);
-        if (qg_better(x.valid != 0, x.gain, x.bin, rS.valid != 0, rS.gain, rS.bin)) rS = x;
-        if (qg_better(y.valid != 0, y.gain, y.bin, rL.valid != 0, rL.gain, rL.bin)) rL = y;
+    warp_best(gS, binS, wS);
+    if (!ROOT) warp_best(gL, binL, wL);
+    if (lane == 0) {
+        sm[0][warp].gain = gS; sm[0][warp].bin = binS; sm[0][warp].w = wS;
+        sm[1][warp].gain = gL; sm[1][warp].bin = binL; sm[1][warp].w = wL;
     }
-    if (lane == 0) { sm[0][warp] = rS; sm[1][warp] = rL; }
     __syncthreads();
     SplitRec *cand = a.cand + (size_t)j * a.F * 2;
-    if (threadIdx.x < 2) {
-        SplitRec r = sm[threadIdx.x][0];
-        for (int w = 1; w < FIN_WARPS; ++w) {
-            const SplitRec o = sm[threadIdx.x][w];
-            if (qg_better(o.valid != 0, o.gain, o.bin, r.valid != 0, r.gain, r.bin)) r = o;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            WarpBest r = sm[c][0];
+            for (int w = 1; w < FIN_WARPS; ++w) {
+                const WarpBest o = sm[c][w];
+                if (qg_better(o.bin >= 0, o.gain, o.bin, r.bin >= 0, r.gain, r.bin)) r = o;
+            }
+            SplitRec x = qg_invalid_rec();
+            x.feature = f;
+            if (r.bin >= 0) { x.valid = 1; x.gain = r.gain; x.bin = r.bin; x.gl = (long long)(int)(r.w >> 32); x.hl = (long long)(uint32_t)r.w; }
+            cand[2 * f + c] = x;
         }
-        cand[2 * f + threadIdx.x] = r;
         __threadfence();
+        is_last = atomicAdd(&job->finish_count, 1u) == (unsigned int)a.F - 1u;
     }
-    __syncthreads();
-    if (threadIdx.x == 0) is_last = atomicAdd(&job->finish_count, 1u) == gridDim.x - 1;
     __syncthreads();
     if (!is_last) return;
     __threadfence();
 
     // ---- the last block of this leaf: best candidates over all features, then the growth records
     //      of the two children (ROOT: the root's best split)
+    __shared__ SplitRec fin_rec[2][FIN_WARPS];
     SplitRec bS = qg_invalid_rec(), bL = qg_invalid_rec();
-    for (int i2 = threadIdx.x; i2 < (int)gridDim.x; i2 += FIN_WARPS * 32) {
+    for (int i2 = threadIdx.x; i2 < a.F; i2 += FIN_THREADS) {
         const SplitRec x = load_rec_cg(cand + 2 * i2), y = load_rec_cg(cand + 2 * i2 + 1);
         if (qg_rec_better(x, bS)) bS = x;
         if (qg_rec_better(y, bL)) bL = y;
@@ -572,14 +513,14 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
         if (qg_rec_better(x, bS)) bS = x;
         if (qg_rec_better(y, bL)) bL = y;
     }
-    if (lane == 0) { sm[0][warp] = bS; sm[1][warp] = bL; }
+    if (lane == 0) { fin_rec[0][warp] = bS; fin_rec[1][warp] = bL; }
     __syncthreads();
     if (threadIdx.x != 0) return;
-    bS = sm[0][0];
-    bL = sm[1][0];
+    bS = fin_rec[0][0];
+    bL = fin_rec[1][0];
     for (int w = 1; w < FIN_WARPS; ++w) {
-        if (qg_rec_better(sm[0][w], bS)) bS = sm[0][w];
-        if (qg_rec_better(sm[1][w], bL)) bL = sm[1][w];
+        if (qg_rec_better(fin_rec[0][w], bS)) bS = fin_rec[0][w];
+        if (qg_rec_better(fin_rec[1][w], bL)) bL = fin_rec[1][w];
     }
     job->finish_count = 0;
     job->lb[0] = job->lb[1] = 0;
@@ -614,20 +555,23 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
     a.rec_parent[child0] = a.rec_parent[child0 + 1] = jrec;
 }
 
-// ROOT: scans the root histogram (pool slot 0), grid (F).  Otherwise: completes the splits of the
-// current pass, grid (F, Y): block (f, y) takes feature f of the leaves y, y + Y, ... of the batch
-// (Y is chosen on the host so that the grid fills the SMs a few times over without launching a block
-// for every feature of every possible leaf).
-template <bool ROOT, int BPT>
-__global__ void __launch_bounds__(256 / BPT, BPT == 2 ? 8 : 1) k_grow_finish(GrowArgs a) {
+// ROOT: scans the root histogram (pool slot 0), one block per feature.  Otherwise: completes the
+// splits of the current pass: the (leaf, feature) pairs of the batch, leaf-major, are dealt round-robin
+// to a grid sized to what the SMs hold at once, so that every block gets the same number of pairs to
+// within one, whatever the batch size.
+template <bool ROOT>
+__global__ void __launch_bounds__(FIN_THREADS, FIN_BLOCKS_PER_SM) k_grow_finish(GrowArgs a) {
+    if (a.gs->done) return;
     if (ROOT) {
-        finish_one<ROOT, BPT>(a, (int)blockIdx.x, 0);
+        finish_one<ROOT>(a, (int)blockIdx.x, 0);
         return;
     }
-    const int n_jobs = a.gs->n_jobs;
-    for (int j = (int)blockIdx.y; j < n_jobs; j += (int)gridDim.y) {
-        finish_one<ROOT, BPT>(a, (int)blockIdx.x, j);
-        __syncthreads();   // the shared arrays of finish_one are reused by the next leaf
+    const int items = a.gs->n_jobs * a.F;
+    for (int it = (int)blockIdx.x; it < items; it += (int)gridDim.x) {
+        const int j = it / a.F;
+        // the shared arrays of finish_one need no barrier in between: each is last read before a
+        // barrier that every thread passes before the next leaf's first write to it
+        finish_one<ROOT>(a, it - j * a.F, j);
     }
 }
 
@@ -1114,7 +1058,10 @@ int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st, int n_jobs = 
             return rc;
     }
     if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
-    k_grow_finish<false, 2><<<fin, 128, 0, st>>>(a);
+    {
+        const int resident = c->sm_count * FIN_BLOCKS_PER_SM, all = c->F * a.K;
+        k_grow_finish<false><<<(unsigned)(all < resident ? all : resident), FIN_THREADS, 0, st>>>(a);
+    }
     QG_LAUNCH_CHECK(c);
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     return launch_commit(c, a, st);
@@ -1233,7 +1180,7 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     if (rc != QGBDT_OK) return rc;
     if ((rc = qg_allreduce(c, c->d_hist_pool, (int64_t)c->F * c->nb, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return rc;
     if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
-    k_grow_finish<true, 1><<<(unsigned)c->F, 256, 0, st>>>(a);
+    k_grow_finish<true><<<(unsigned)c->F, FIN_THREADS, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     if (c->prm.num_leaves < 2) return QGBDT_OK;

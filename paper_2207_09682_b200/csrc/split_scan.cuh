@@ -91,6 +91,71 @@ __device__ inline void qg_gain_bounds(long long gl, long long hl, const SplitPar
     }
 }
 
+// The same two tests for the tree-growing kernels, on 32-bit sums (a leaf's gradient and hessian sums
+// fit 32 bits: checked when the rows are loaded) and with the per-leaf constants taken out.
+struct Admit32 {
+    int G;                             // totals of the leaf
+    uint32_t H, n_s, half;             // half = H / 2
+    unsigned long long x_min, x_end;   // row estimate within [min_data, n_s - min_data]  <=>  x_min <= X < x_end
+    uint32_t min_data;
+    int const_h;
+    float q_sure;                      // single-precision hessian sums from here on are certainly >= min_sum_h
+    double min_sum_h, dh;
+};
+
+__device__ inline Admit32 qg_admit32(const SplitParams &p, double dh) {
+    Admit32 a;
+    a.G = (int)p.G; a.H = (uint32_t)p.H; a.n_s = (uint32_t)p.n_s; a.half = a.H / 2;
+    a.min_data = (uint32_t)p.min_data;
+    a.const_h = p.const_h;
+    const long long k = p.n_s - p.min_data;
+    a.x_min = (unsigned long long)p.min_data * a.H;
+    a.x_end = k < 0 ? 0ull : (unsigned long long)(k + 1) * a.H;
+    // the single-precision product is off by less than 4 * 2^-24 relative; 2^-20 above the limit is safe
+    a.q_sure = __fmul_ru(__double2float_ru(p.min_sum_h), 1.00000095367431640625f);
+    a.min_sum_h = p.min_sum_h;
+    a.dh = dh;
+    return a;
+}
+
+// qg_candidate_admissible for left hessian sum hl, same decisions: the products with the interval
+// length are compared in single precision where that is certain, in double precision otherwise.
+__device__ inline bool qg_admissible32(uint32_t hl, const Admit32 &a, const GainScale &sc) {
+    const uint32_t hr = a.H - hl;
+    if (hl == 0 || hr == 0) return false;
+    if (a.const_h) {
+        if (!(hl >= a.min_data && a.n_s - hl >= a.min_data)) return false;
+    } else {
+        const unsigned long long X = (unsigned long long)hl * a.n_s + a.half;
+        if (X < a.x_min || X >= a.x_end) return false;
+    }
+    if (!(__fmul_rn((float)hl, sc.dh) >= a.q_sure) || !(__fmul_rn((float)hr, sc.dh) >= a.q_sure)) {
+        if (__dmul_rn((double)hl, a.dh) < a.min_sum_h || __dmul_rn((double)hr, a.dh) < a.min_sum_h) return false;
+    }
+    return true;
+}
+
+// qg_gain_bounds on 32-bit sums, with the fast division (2 units in the last place: every term of
+// Eq. 7 still comes out within 16 * 2^-24 relative, of which the bounds take four times).
+__device__ inline void qg_gain_bounds32(int gl, uint32_t hl, const Admit32 &a, const GainScale &sc, float tp,
+                                        float &lo, float &hi) {
+    const float gdl = __fmul_rn((float)gl, sc.dg), gdr = __fmul_rn((float)(a.G - gl), sc.dg);
+    const float hdl = __fadd_rn(__fmul_rn((float)hl, sc.dh), sc.lambda), hdr = __fadd_rn(__fmul_rn((float)(a.H - hl), sc.dh), sc.lambda);
+    const float tl = __fdividef(__fmul_rn(gdl, gdl), hdl), tr = __fdividef(__fmul_rn(gdr, gdr), hdr);
+    const float gain = __fmul_rn(0.5f, __fsub_rn(__fadd_rn(tl, tr), tp));
+    // 64 * 2^-24 of the terms, and room for results that left the normal range on the way
+    const float err = __fadd_rn(__fmul_rn(3.814697265625e-6f, __fadd_rn(__fadd_rn(tl, tr), tp)), 1.0e-37f);
+    lo = __fsub_rn(gain, err);
+    hi = __fadd_rn(gain, err);
+    // out of the range in which single precision (and its fast division) says anything: no information.
+    // (A non-zero gradient sum times dg >= 1e-15 squares to a normal number.)
+    if (!(fabsf(gain) <= 3.0e38f) || !(err <= 3.0e38f) || !(fmaxf(hdl, hdr) <= 1.0e30f) || !(fminf(hdl, hdr) >= 1.0e-30f) ||
+        !(sc.dg >= 1.0e-15f)) {
+        lo = -__int_as_float(0x7f800000);
+        hi = __int_as_float(0x7f800000);
+    }
+}
+
 // Running state of one feature's scan in one lane.
 struct ScanState {
     long long carry_g, carry_h;   // sums of the bins before the current group of 32

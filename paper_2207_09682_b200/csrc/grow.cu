@@ -56,7 +56,9 @@ struct GrowArgs {
     int32_t *m_feature, *m_bin, *m_left, *m_right;
     double *m_gain;
     cudaGraphConditionalHandle cond; // condition of the graph's while node
-    int use_cond;                    // 0: launched on a stream, the host reads gs->done
+    int use_cond;
+    int sep_reduce;                  // the best split over the features is taken by k_grow_reduce, not by the last
+                                     // block of the finishing kernel                    // 0: launched on a stream, the host reads gs->done
 };
 
 __global__ void k_grow_begin(GrowState *gs, NodeRec *recs, double *rec_gain, int32_t *rec_child, int32_t *rec_pos,
@@ -314,21 +316,105 @@ struct WarpBest {
 
 constexpr int FIN_THREADS = 128, FIN_WARPS = FIN_THREADS / 32, FIN_BLOCKS_PER_SM = 8;
 
+// Last step for one leaf being split (ROOT: for the root), by one block once every feature's best
+// thresholds are written: the best over all features (lowest feature on equal gain), then the growth
+// records of the two children (ROOT: the root's best split).
+struct TailIn {   // what the step needs of the job, read before the wait for the other blocks
+    int parent_slot, small_slot, child0, rec, buf;
+    uint32_t n, nl, off, n_all, nl_all;
+    long long gl, hl, PG, PH;
+};
+__device__ __forceinline__ TailIn tail_in(const GrowState *gs, int j) {
+    const GrowJob *job = gs->jobs + j;
+    TailIn t;
+    t.parent_slot = job->parent_slot; t.small_slot = job->small_slot; t.child0 = job->child0; t.rec = job->rec; t.buf = job->buf;
+    t.n = job->n; t.nl = job->nl; t.off = job->off; t.n_all = job->n_all; t.nl_all = (uint32_t)gs->nl_all[j];
+    t.gl = job->gl; t.hl = job->hl; t.PG = job->PG; t.PH = job->PH;
+    return t;
+}
+template <bool ROOT>
+__device__ __forceinline__ void finish_tail(const GrowArgs &a, const int j, const TailIn &t) {
+    __threadfence();
+    GrowState *gs = a.gs;
+    GrowJob *job = gs->jobs + j;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const SplitRec *cand = a.cand + (size_t)j * a.F * 2;
+    __shared__ SplitRec fin_rec[2][FIN_WARPS];
+    SplitRec bS = qg_invalid_rec(), bL = qg_invalid_rec();
+    for (int i2 = threadIdx.x; i2 < a.F; i2 += FIN_THREADS) {
+        const SplitRec x = load_rec_cg(cand + 2 * i2), y = load_rec_cg(cand + 2 * i2 + 1);
+        if (qg_rec_better(x, bS)) bS = x;
+        if (qg_rec_better(y, bL)) bL = y;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const SplitRec x = shfl_xor_rec(bS, o), y = shfl_xor_rec(bL, o);
+        if (qg_rec_better(x, bS)) bS = x;
+        if (qg_rec_better(y, bL)) bL = y;
+    }
+    if (lane == 0) { fin_rec[0][warp] = bS; fin_rec[1][warp] = bL; }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    bS = fin_rec[0][0];
+    bL = fin_rec[1][0];
+    for (int w = 1; w < FIN_WARPS; ++w) {
+        if (qg_rec_better(fin_rec[0][w], bS)) bS = fin_rec[0][w];
+        if (qg_rec_better(fin_rec[1][w], bL)) bL = fin_rec[1][w];
+    }
+    job->finish_count = 0;
+    job->lb[0] = job->lb[1] = 0;
+    const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
+    if (ROOT) {
+        a.recs[0].best = bS;
+        a.rec_gain[0] = bS.valid ? bS.gain : NEG;
+        return;
+    }
+    const int parent_slot = t.parent_slot, small_slot = t.small_slot;
+    const int child0 = t.child0, jrec = t.rec;
+    const uint32_t nl = t.nl, nr = t.n - nl, off = t.off;
+    const uint32_t nl_all = t.nl_all, nr_all = t.n_all - nl_all;
+    const long long gl = t.gl, hl = t.hl;
+    const bool small_is_left = nl_all <= nr_all;
+    const int dstbuf = t.buf == 0 ? 1 : 0;
+    NodeRec lf, rt;
+    lf.off = off; lf.n = nl; lf.n_all = nl_all; lf.buf = dstbuf;
+    lf.G = gl; lf.H = hl;
+    rt.off = off + nl; rt.n = nr; rt.n_all = nr_all; rt.buf = dstbuf;
+    rt.G = t.PG - gl; rt.H = t.PH - hl;
+    lf.slot = small_is_left ? small_slot : parent_slot;
+    rt.slot = small_is_left ? parent_slot : small_slot;
+    lf.best = small_is_left ? bS : bL;
+    rt.best = small_is_left ? bL : bS;
+    lf.state = rt.state = 0;
+    lf.child0 = rt.child0 = -1;
+    lf.nl = rt.nl = 0;
+    lf.parent_node = rt.parent_node = -1;
+    lf.parent_side = 0; rt.parent_side = 1;
+    a.recs[child0] = lf;
+    a.recs[child0 + 1] = rt;
+    a.recs[jrec].nl = nl;
+    a.rec_gain[child0] = lf.best.valid ? lf.best.gain : NEG;
+    a.rec_gain[child0 + 1] = rt.best.valid ? rt.best.gain : NEG;
+    a.rec_child[child0] = a.rec_child[child0 + 1] = -1;
+    a.rec_pos[child0] = a.rec_pos[child0 + 1] = -1;
+    a.rec_parent[child0] = a.rec_parent[child0 + 1] = jrec;
+}
+
 // One feature of one leaf being split (ROOT: of the root): the work of a block of k_grow_finish.
 // 128 threads, thread t owns bins 2 t and 2 t + 1 (n_bins <= 256).  A bin is one 64-bit word, the
 // gradient sum in the upper half and the hessian sum in the lower; the sums of a whole leaf fit the
 // halves (checked when the rows are loaded), so prefix sums are taken on the words themselves.
-template <bool ROOT>
+template <bool ROOT, bool SEP>
 __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const int j) {
     GrowState *gs = a.gs;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     GrowJob *job = gs->jobs + j;
     // everything the block needs from the state, at once (one round trip to memory)
-    const int parent_slot = ROOT ? 0 : job->parent_slot, small_slot = ROOT ? 0 : job->small_slot;
-    const int parts = job->parts, slot0 = job->slot0, child0 = job->child0, jrec = job->rec, jbuf = job->buf;
-    const uint32_t gs_n = job->n, gs_nl = job->nl, gs_off = job->off, gs_n_all = job->n_all;
-    const uint32_t gs_nl_all = (uint32_t)gs->nl_all[j];
-    const long long gs_gl = job->gl, gs_hl = job->hl, gs_PG = job->PG, gs_PH = job->PH;
+    const int parts = job->parts, slot0 = job->slot0;
+    const TailIn ti = tail_in(gs, j);
+    const int parent_slot = ROOT ? 0 : ti.parent_slot, small_slot = ROOT ? 0 : ti.small_slot;
+    constexpr bool sep_reduce = SEP;   // k_grow_reduce takes the last step
+    const uint32_t gs_n = ti.n, gs_nl = ti.nl, gs_n_all = ti.n_all, gs_nl_all = ti.nl_all;
+    const long long gs_gl = ti.gl, gs_hl = ti.hl, gs_PG = ti.PG, gs_PH = ti.PH;
     const long long tot_g = a.state->tot_g, tot_h = a.state->tot_h;
     const uint32_t gmax_bits = a.state->gmax_bits, hmax_bits = a.state->hmax_bits;
     const FeatRec fr = a.feat_rec[f];
@@ -492,78 +578,25 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
             if (r.bin >= 0) { x.valid = 1; x.gain = r.gain; x.bin = r.bin; x.gl = (long long)(int)(r.w >> 32); x.hl = (long long)(uint32_t)r.w; }
             cand[2 * f + c] = x;
         }
-        __threadfence();
-        is_last = atomicAdd(&job->finish_count, 1u) == (unsigned int)a.F - 1u;
+        if (!sep_reduce) {
+            __threadfence();
+            is_last = atomicAdd(&job->finish_count, 1u) == (unsigned int)a.F - 1u;
+        }
     }
+    if (sep_reduce) return;   // k_grow_reduce follows
     __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-
-    // ---- the last block of this leaf: best candidates over all features, then the growth records
-    //      of the two children (ROOT: the root's best split)
-    __shared__ SplitRec fin_rec[2][FIN_WARPS];
-    SplitRec bS = qg_invalid_rec(), bL = qg_invalid_rec();
-    for (int i2 = threadIdx.x; i2 < a.F; i2 += FIN_THREADS) {
-        const SplitRec x = load_rec_cg(cand + 2 * i2), y = load_rec_cg(cand + 2 * i2 + 1);
-        if (qg_rec_better(x, bS)) bS = x;
-        if (qg_rec_better(y, bL)) bL = y;
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        const SplitRec x = shfl_xor_rec(bS, o), y = shfl_xor_rec(bL, o);
-        if (qg_rec_better(x, bS)) bS = x;
-        if (qg_rec_better(y, bL)) bL = y;
-    }
-    if (lane == 0) { fin_rec[0][warp] = bS; fin_rec[1][warp] = bL; }
-    __syncthreads();
-    if (threadIdx.x != 0) return;
-    bS = fin_rec[0][0];
-    bL = fin_rec[1][0];
-    for (int w = 1; w < FIN_WARPS; ++w) {
-        if (qg_rec_better(fin_rec[0][w], bS)) bS = fin_rec[0][w];
-        if (qg_rec_better(fin_rec[1][w], bL)) bL = fin_rec[1][w];
-    }
-    job->finish_count = 0;
-    job->lb[0] = job->lb[1] = 0;
-    const double NEG = -__longlong_as_double(0x7FF0000000000000LL);
-    if (ROOT) {
-        a.recs[0].best = bS;
-        a.rec_gain[0] = bS.valid ? bS.gain : NEG;
-        return;
-    }
-    const int dstbuf = jbuf == 0 ? 1 : 0;
-    NodeRec lf, rt;
-    lf.off = gs_off; lf.n = nl; lf.n_all = nl_all; lf.buf = dstbuf;
-    lf.G = gs_gl; lf.H = gs_hl;
-    rt.off = gs_off + nl; rt.n = nr; rt.n_all = nr_all; rt.buf = dstbuf;
-    rt.G = gs_PG - gs_gl; rt.H = gs_PH - gs_hl;
-    lf.slot = small_is_left ? small_slot : parent_slot;
-    rt.slot = small_is_left ? parent_slot : small_slot;
-    lf.best = small_is_left ? bS : bL;
-    rt.best = small_is_left ? bL : bS;
-    lf.state = rt.state = 0;
-    lf.child0 = rt.child0 = -1;
-    lf.nl = rt.nl = 0;
-    lf.parent_node = rt.parent_node = -1;
-    lf.parent_side = 0; rt.parent_side = 1;
-    a.recs[child0] = lf;
-    a.recs[child0 + 1] = rt;
-    a.recs[jrec].nl = nl;
-    a.rec_gain[child0] = lf.best.valid ? lf.best.gain : NEG;
-    a.rec_gain[child0 + 1] = rt.best.valid ? rt.best.gain : NEG;
-    a.rec_child[child0] = a.rec_child[child0 + 1] = -1;
-    a.rec_pos[child0] = a.rec_pos[child0 + 1] = -1;
-    a.rec_parent[child0] = a.rec_parent[child0 + 1] = jrec;
+    if (is_last) finish_tail<ROOT>(a, j, ti);
 }
 
 // ROOT: scans the root histogram (pool slot 0), one block per feature.  Otherwise: completes the
 // splits of the current pass: the (leaf, feature) pairs of the batch, leaf-major, are dealt round-robin
 // to a grid sized to what the SMs hold at once, so that every block gets the same number of pairs to
 // within one, whatever the batch size.
-template <bool ROOT>
+template <bool ROOT, bool SEP>
 __global__ void __launch_bounds__(FIN_THREADS, FIN_BLOCKS_PER_SM) k_grow_finish(GrowArgs a) {
     if (a.gs->done) return;
     if (ROOT) {
-        finish_one<ROOT>(a, (int)blockIdx.x, 0);
+        finish_one<ROOT, SEP>(a, (int)blockIdx.x, 0);
         return;
     }
     const int items = a.gs->n_jobs * a.F;
@@ -571,8 +604,16 @@ __global__ void __launch_bounds__(FIN_THREADS, FIN_BLOCKS_PER_SM) k_grow_finish(
         const int j = it / a.F;
         // the shared arrays of finish_one need no barrier in between: each is last read before a
         // barrier that every thread passes before the next leaf's first write to it
-        finish_one<ROOT>(a, it - j * a.F, j);
+        finish_one<ROOT, SEP>(a, it - j * a.F, j);
     }
+}
+
+// With thousands of features the last step runs as a kernel of its own, one block per leaf of the
+// batch: left to whichever block of the finishing kernel comes last, a block that has fallen behind
+// takes that step for one leaf after the other and falls further behind each time.
+__global__ void __launch_bounds__(FIN_THREADS) k_grow_reduce(GrowArgs a) {
+    if (a.gs->done || (int)blockIdx.x >= a.gs->n_jobs) return;
+    finish_tail<false>(a, (int)blockIdx.x, tail_in(a.gs, (int)blockIdx.x));
 }
 
 // Sharded rows only: sums the partial histograms of every smaller child of the pass into its pool
@@ -1020,6 +1061,7 @@ void fill_args(qgbdt_ctx *c, GrowArgs &a) {
     a.m_gain = c->d_m_gain;
     a.cond = 0;
     a.use_cond = 0;
+    a.sep_reduce = c->F > 512;
 }
 
 int launch_commit(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st) {
@@ -1060,9 +1102,15 @@ int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st, int n_jobs = 
     if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
     {
         const int resident = c->sm_count * FIN_BLOCKS_PER_SM, all = c->F * a.K;
-        k_grow_finish<false><<<(unsigned)(all < resident ? all : resident), FIN_THREADS, 0, st>>>(a);
+        const unsigned grid = (unsigned)(all < resident ? all : resident);
+        if (a.sep_reduce) k_grow_finish<false, true><<<grid, FIN_THREADS, 0, st>>>(a);
+        else k_grow_finish<false, false><<<grid, FIN_THREADS, 0, st>>>(a);
     }
     QG_LAUNCH_CHECK(c);
+    if (a.sep_reduce) {
+        k_grow_reduce<<<(unsigned)a.K, FIN_THREADS, 0, st>>>(a);
+        QG_LAUNCH_CHECK(c);
+    }
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     return launch_commit(c, a, st);
 }
@@ -1180,7 +1228,7 @@ int qg_grow_tree(qgbdt_ctx *c, int tree_slot, cudaStream_t st) {
     if (rc != QGBDT_OK) return rc;
     if ((rc = qg_allreduce(c, c->d_hist_pool, (int64_t)c->F * c->nb, QGBDT_REDUCE_SUM_I64, st)) != QGBDT_OK) return rc;
     if ((rc = qg_phase_begin(c, QG_PHASE_FINISH, st)) != QGBDT_OK) return rc;
-    k_grow_finish<true><<<(unsigned)c->F, FIN_THREADS, 0, st>>>(a);
+    k_grow_finish<true, false><<<(unsigned)c->F, FIN_THREADS, 0, st>>>(a);
     QG_LAUNCH_CHECK(c);
     if ((rc = qg_phase_end(c, st)) != QGBDT_OK) return rc;
     if (c->prm.num_leaves < 2) return QGBDT_OK;

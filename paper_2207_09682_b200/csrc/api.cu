@@ -242,7 +242,7 @@ int load_common(qgbdt_ctx *c, const uint8_t *d_bins, int64_t n_rows, int32_t n_f
     if ((rc = dev_alloc(c, &c->d_idx_tmp, (size_t)n_rows)) != QGBDT_OK) return rc;
     // block counts of the step-wise partition (a block per 2048 rows), or the warp and block counts
     // of the partition launches of tree growth (nine words per block)
-    c->grow_pb_total = c->sm_count * 4 + GROW_MAX_JOBS;
+    c->grow_pb_total = c->sm_count * 8 + GROW_MAX_JOBS;
     {
         size_t need = (size_t)n_rows / 2048 + 8, grow = (size_t)c->grow_pb_total * 9 + 8;
         if ((rc = dev_alloc(c, &c->d_part_counts, need > grow ? need : grow)) != QGBDT_OK) return rc;

@@ -44,7 +44,7 @@ struct GrowArgs {
     uint32_t *counts;                // [pb_total * PART_WARPS] left rows per warp range, then [pb_total] per block
     int pb_total;                    // blocks of a partition launch
     unsigned long long *pool;        // [slots][F][nb]
-    const unsigned long long *partial;
+    unsigned long long *partial;       // per leaf of the batch and tile: sums of the smaller child's CTAs (zero between passes)
     SplitRec *cand;                  // [jobs][F][2] best candidates of every feature for the two children
     int F, nb, L;
     int K, slack;                    // leaves per pass; leaves that may be split ahead of their confirmation
@@ -136,10 +136,10 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
     if (lb * PART_WARPS >= active) return;                               // no warp of this block has work
     const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
     uint32_t lefts = 0;
-    for (uint32_t w = w0; w < w1; w += 4) {
-        uint32_t row[4], word[4];
+    for (uint32_t w = w0; w < w1; w += 8) {
+        uint32_t row[8], word[8];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < 8; ++k) {
             const uint32_t e = ((w + k) << 5) + lane;
             row[k] = (w + k < w1 && e < n) ? (src ? src[off + e].x : off + e) : 0xFFFFFFFFu;
         }
@@ -147,13 +147,13 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
         // DRAM granules), or, without that copy, a word of the tile (a granule per row)
         if (col8) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) word[k] = row[k] != 0xFFFFFFFFu ? (uint32_t)col8[row[k]] << shift : 0xFFFFFFFFu;
+            for (int k = 0; k < 8; ++k) word[k] = row[k] != 0xFFFFFFFFu ? (uint32_t)col8[row[k]] << shift : 0xFFFFFFFFu;
         } else {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) word[k] = row[k] != 0xFFFFFFFFu ? col[(size_t)row[k] << logW] : 0xFFFFFFFFu;
+            for (int k = 0; k < 8; ++k) word[k] = row[k] != 0xFFFFFFFFu ? col[(size_t)row[k] << logW] : 0xFFFFFFFFu;
         }
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < 8; ++k) {
             const bool left = row[k] != 0xFFFFFFFFu && ((word[k] >> shift) & 0xFFu) <= thr;
             const uint32_t b = __ballot_sync(0xffffffffu, left);
             if (w + k < w1) {
@@ -451,8 +451,8 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
     const int fl = fr.fl, W = 1 << fr.logW;
     const uint32_t P = (ROOT || a.merged) ? 1u : qg_grow_parts((uint32_t)parts, small_is_left ? nl : nr, a.rows_min);
     const size_t pstride = (size_t)4 * a.nb * 32;
-    const unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
-                                     (size_t)(fl & 3) * a.nb * W + (fl >> 2);
+    unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
+                               (size_t)(fl & 3) * a.nb * W + (fl >> 2);
     unsigned long long *S = a.pool + (size_t)small_slot * hw + (size_t)f * a.nb;
     unsigned long long *Pp = ROOT ? nullptr : a.pool + (size_t)parent_slot * hw + (size_t)f * a.nb;
     unsigned long long sv[2], lv[2];
@@ -464,7 +464,12 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
             sv[jb] = 0; lv[jb] = 0; pv[jb] = 0;
             if (b < a.nb) {
                 if (!ROOT) pv[jb] = Pp[b];
-                if (!ROOT && P > 1) {
+                if (!ROOT && P > 1 && fr.logW < QG_SHARED_PARTIAL_LOGW) {
+                    // the CTAs of the tile added their sums into its first partial slot: take them, leave zero
+                    unsigned long long *q = part + (size_t)b * W;
+                    sv[jb] = *q;
+                    *q = 0ull;
+                } else if (!ROOT && P > 1) {
                     const unsigned long long *q = part + (size_t)b * W;
                     for (uint32_t i0 = 0; i0 < P; i0 += 16) {   // 16 independent loads in flight
                         unsigned long long x[16];
@@ -634,18 +639,23 @@ __global__ void __launch_bounds__(256) k_grow_merge(GrowArgs a) {
         if (P <= 1) continue;   // a single CTA wrote the slot itself
         const int fl = fr.fl, W = 1 << fr.logW;
         const size_t pstride = (size_t)4 * a.nb * 32;
-        const unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
-                                         (size_t)(fl & 3) * a.nb * W + (fl >> 2);
+        unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
+                                   (size_t)(fl & 3) * a.nb * W + (fl >> 2);
         unsigned long long *S = a.pool + (size_t)small_slot * a.F * a.nb + (size_t)f * a.nb;
         for (int b = threadIdx.x; b < a.nb; b += 256) {
-            const unsigned long long *q = part + (size_t)b * W;
+            unsigned long long *q = part + (size_t)b * W;
             unsigned long long v = 0;
-            for (uint32_t i0 = 0; i0 < P; i0 += 8) {
-                unsigned long long x[8];
+            if (fr.logW < QG_SHARED_PARTIAL_LOGW) {   // one slot holds the sum: take it, leave zero
+                v = *q;
+                *q = 0ull;
+            } else {
+                for (uint32_t i0 = 0; i0 < P; i0 += 8) {
+                    unsigned long long x[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
+                    for (int k = 0; k < 8; ++k) x[k] = i0 + k < P ? q[(size_t)(i0 + k) * pstride] : 0ull;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) v += x[k];
+                    for (int k = 0; k < 8; ++k) v += x[k];
+                }
             }
             S[b] = v;
         }

@@ -114,6 +114,7 @@ struct Out {
     unsigned long long *ptr;   // partial slot of this CTA, or the final histogram
     bool direct;               // final layout hist[f][bin] instead of partial [k][bin][a]
     bool first;                // nothing stored yet: store instead of accumulate
+    bool shared_out;           // several CTAs add into the same (zeroed) output: reductions instead of stores
 };
 
 // Adds the CTA's local histogram into its output and clears it.  The R replicas of a column
@@ -165,8 +166,12 @@ __device__ inline void flush_local(int *hp, const TileDesc &td, const int logW, 
             if (fl < td.nf) {
                 unsigned long long *q = out.direct ? out.ptr + (size_t)(td.f0 + fl) * nb + bin
                                                    : out.ptr + (size_t)k * nb * W + e;
-                if (!out.first) v += *q;
-                *q = v;
+                if (out.shared_out) {
+                    if (v) atomicAdd(q, v);
+                } else {
+                    if (!out.first) v += *q;
+                    *q = v;
+                }
             }
         }
     }
@@ -281,8 +286,12 @@ __device__ __forceinline__ void hist_cta(const HistArgs &a, const TileDesc &td, 
 
     Out out;
     out.direct = P == 1;
-    out.first = true;   // the two passes of the 32+32 mode write different features
-    out.ptr = out.direct ? a.hist : a.partial + (size_t)(td.cta0 + part) * 4 * a.nb * 32;
+    // tree growth, rows of up to 64 bytes: the CTAs of a leaf's tile all add into the tile's first partial
+    // slot, which is zero before the launch (whoever reads it clears it); integer sums come out the same
+    // in any order.  (128-byte rows: 32 k reductions per CTA cost more than the partial slots' stores.)
+    out.shared_out = LIST == 2 && P > 1 && logW < QG_SHARED_PARTIAL_LOGW;
+    out.first = !out.shared_out;   // the two passes of the 32+32 mode write different features
+    out.ptr = out.direct ? a.hist : a.partial + (size_t)(td.cta0 + (out.shared_out ? 0u : part)) * 4 * a.nb * 32;
 
     // ---- range of this part in warp-units [0, q1) from its first unit, and the leftover rows /
     //      entries [s0, s1) that are done one by one

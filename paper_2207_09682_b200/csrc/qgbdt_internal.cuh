@@ -123,6 +123,10 @@ struct NodeRec {
 };
 
 // One leaf being split in the current pass.
+// Tiles narrower than 2^this words per row: the histogram CTAs of a leaf being split add into one
+// partial slot per tile; from this width on each CTA stores a partial slot of its own.
+constexpr int QG_SHARED_PARTIAL_LOGW = 5;
+
 struct GrowJob {
     int32_t rec;                     // its growth record
     int32_t feature, bin;            // the split

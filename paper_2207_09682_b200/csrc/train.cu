@@ -84,6 +84,13 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
         (rc = alloc_dev(c, &c->d_grow_partial, (size_t)c->grow_xcap * c->tiles.size() * 4 * c->nb * 32,
                         "partial histograms of tree growth")) != QGBDT_OK)
         return rc;
+    // the CTAs of a histogram build add into these sums and whoever reads them clears them: every call
+    // starts from zero, whatever state an earlier call that ended in an error left
+    bool shared_slots = false;
+    for (const auto &t : c->tiles) shared_slots = shared_slots || t.logW < QG_SHARED_PARTIAL_LOGW;
+    if (shared_slots)
+        QG_CUDA(c, cudaMemsetAsync(c->d_grow_partial, 0,
+                                   (size_t)c->grow_xcap * c->tiles.size() * 4 * c->nb * 32 * sizeof(unsigned long long), st));
     if (!c->d_ent0 && (rc = alloc_dev(c, &c->d_ent0, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_ent1 && (rc = alloc_dev(c, &c->d_ent1, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_leaf_id && (rc = alloc_dev(c, &c->d_leaf_id, (size_t)c->N, "leaf numbers")) != QGBDT_OK) return rc;

@@ -32,9 +32,10 @@ WORKLOAD_ROWS = {"large": 10_500_000, "tall": 1_000_000, "tiny": 50_000, "wide":
 # rows of the CPU arm: the same rows as the GPU arm (one oracle tree: about 9 s on 'large', 15 s on 'wide')
 CPU_SAMPLE_ROWS = dict(WORKLOAD_ROWS)
 FALLBACK_HBM_GBS = 6650.0
-# DRAM traffic of the histogram kernels on the 'large' workload from an ncu capture
-# (profiles/launch_list_large_10p5Mx28.md): 3.37 GB over the 255 builds of one tree.  Valid only for
-# the kernel sources the capture was taken with.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the histogram kernels on the 'large'
+# workload, per build, averaged over the builds of one tree, from an ncu capture of the same kernels on
+# 4 M rows scaled by the rows (traffic grows in proportion to them).  Valid only for the kernel sources
+# the capture was taken with.
 HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 13.21e6,
                 "sources_sha1": "331e037039ff3f9fab93e421716983d78c5b675e"}
 
@@ -294,7 +295,7 @@ def time_hist_builds(ctx, torch, synth, n, features, n_bins, cbytes, reps=10, ba
 
 def run_sweep(args):
     """Histogram-kernel sweep (rows x features x bins x gradient bits, root and 50 % subset builds);
-    prints one text line per point.  Not a benchmark line: a table for the design notes."""
+    prints one text line per point.  Not a benchmark line: a table of the kernel over tile widths, bit widths and row fractions."""
     import torch
     from paper_2207_09682_b200 import binding, synth
     torch.cuda.set_device(0)

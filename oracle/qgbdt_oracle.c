@@ -21,7 +21,7 @@
  *
  * Conventions the paper leaves open (random source, rounding arithmetic, validity
  * rules, tie-breaks, the deterministic sigmoid, fixed-point refit sums) are fixed
- * here exactly as the repository's design notes list them.
+ * here, each where it is used, with the reason beside it.
  *
  * Pins: every function here is pinned by the CPU tests (brute force, closed forms,
  * invariants, the paper's worked examples) except the exact output values of the

@@ -670,7 +670,7 @@ __host__ __device__ inline size_t commit_region_bytes(int L) {
     const size_t a = (size_t)L * (sizeof(double) + 3 * sizeof(int));
     size_t n = (size_t)(L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8);
     if (n < 1024) n = 1024;   // the sort works on a power of two of entries
-    const size_t b = n * (sizeof(double) + 2 * sizeof(int));
+    const size_t b = n * (sizeof(double) + 2 * sizeof(int)) + 1024 * (sizeof(double) + sizeof(int));   // + the sort's second buffer
     return ((a > b ? a : b) + 15) / 16 * 16;
 }
 __host__ __device__ inline size_t commit_smem_bytes(int L, int max_recs) {
@@ -893,34 +893,41 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
     if (n_cand > max_cand) n_cand = max_cand;   // cannot happen: the bound counts every record without a confirmed split
     // the open records in order: larger gain first, lower record on equal gain
     if (n_cand <= 1024) {
-        // bitonic sort of the (key, record) pairs, padded to a power of two with entries that sort last
+        // bitonic sort of the (key, record) pairs, one per thread in registers, padded to a power of two
+        // with entries that sort last.  Partners less than 32 apart exchange by shuffle; the others through
+        // shared memory, in two buffers used in turn (one barrier per such step).
         int m = 32;
         while (m < n_cand) m <<= 1;
-        for (int i = n_cand + tid; i < m; i += COMMIT_THREADS) {
-            cand_k[i] = 0ull;
-            cand_r[i] = 0x7FFFFFFF;
-        }
-        __syncthreads();
+        unsigned long long key = tid < n_cand ? cand_k[tid] : 0ull;
+        int rec = tid < n_cand ? cand_r[tid] : 0x7FFFFFFF;
+        unsigned long long *sort_k = reinterpret_cast<unsigned long long *>(by_rank + max_cand);   // [1024]
+        int *sort_r = reinterpret_cast<int *>(sort_k + 1024);                                       // [1024]
+        __syncthreads();   // every thread holds its pair: the arrays become the first exchange buffer
+        int pb = 0;
         for (int k = 2; k <= m; k <<= 1) {
+            const bool first_low = (tid & k) == 0;   // this run of k entries ends up with the first entry lowest
             for (int jj = k >> 1; jj > 0; jj >>= 1) {
-                const int i = tid, x = i ^ jj;
-                if (i < m && x > i) {
-                    const unsigned long long ka = cand_k[i], kb = cand_k[x];
-                    const int ra = cand_r[i], rb = cand_r[x];
-                    const bool a_first = ka > kb || (ka == kb && ra < rb);   // a belongs before b
-                    const bool want_a_first = (i & k) == 0;
-                    if (a_first != want_a_first) {
-                        cand_k[i] = kb; cand_k[x] = ka;
-                        cand_r[i] = rb; cand_r[x] = ra;
-                    }
+                unsigned long long ok;
+                int orr;
+                if (jj >= 32) {
+                    unsigned long long *bk = pb ? sort_k : cand_k;
+                    int *br = pb ? sort_r : cand_r;
+                    bk[tid] = key;
+                    br[tid] = rec;
+                    __syncthreads();
+                    ok = bk[tid ^ jj];
+                    orr = br[tid ^ jj];
+                    pb ^= 1;
+                } else {
+                    ok = __shfl_xor_sync(0xffffffffu, key, jj);
+                    orr = __shfl_xor_sync(0xffffffffu, rec, jj);
                 }
-                __syncthreads();
+                const bool mine_first = key > ok || (key == ok && rec < orr);   // mine belongs before the partner's
+                const bool lower = (tid & jj) == 0;
+                if (mine_first != (lower == first_low)) { key = ok; rec = orr; }
             }
         }
-        for (int i = tid; i < n_cand; i += COMMIT_THREADS) {
-            const int r = cand_r[i];
-            by_rank[i] = (i < budget && cs[r] == -1 && r != mand) ? r : -1;
-        }
+        if (tid < n_cand) by_rank[tid] = (tid < budget && cs[rec] == -1 && rec != mand) ? rec : -1;
     } else {
         for (int i = tid; i < n_cand; i += COMMIT_THREADS) {
             const unsigned long long g = cand_k[i];

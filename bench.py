@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 # workload, per build, averaged over the builds of one tree, from an ncu capture of the same kernels on
 # 4 M rows scaled by the rows (traffic grows in proportion to them).  Valid only for the kernel sources
 # the capture was taken with.
-HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 13.21e6,
-                "sources_sha1": "331e037039ff3f9fab93e421716983d78c5b675e"}
+HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 11.01e6,
+                "sources_sha1": "55e5c455e31cb166af9cb1aae244ded3febcbf60"}
 
 
 def hist_traffic(workload, rows):

@@ -99,6 +99,7 @@ void free_data(qgbdt_ctx *c) {
     dev_free(c->d_front);
     dev_free(c->d_grow_bits);
     dev_free(c->d_grow_partial);
+    dev_free(c->d_grow_prep);
     dev_free(c->d_ent0);
     dev_free(c->d_ent1);
     dev_free(c->d_leaf_id);

@@ -45,6 +45,7 @@ struct GrowArgs {
     int pb_total;                    // blocks of a partition launch
     unsigned long long *pool;        // [slots][F][nb]
     unsigned long long *partial;       // per leaf of the batch and tile: sums of the smaller child's CTAs (zero between passes)
+    JobPrep *prep;                   // [jobs] per-leaf constants (thousands of features: k_grow_prep writes them)
     SplitRec *cand;                  // [jobs][F][2] best candidates of every feature for the two children
     int F, nb, L;
     int K, slack;                    // leaves per pass; leaves that may be split ahead of their confirmation
@@ -413,43 +414,43 @@ __device__ __forceinline__ void finish_one(const GrowArgs &a, const int f, const
     const TailIn ti = tail_in(gs, j);
     const int parent_slot = ROOT ? 0 : ti.parent_slot, small_slot = ROOT ? 0 : ti.small_slot;
     constexpr bool sep_reduce = SEP;   // k_grow_reduce takes the last step
-    const uint32_t gs_n = ti.n, gs_nl = ti.nl, gs_n_all = ti.n_all, gs_nl_all = ti.nl_all;
-    const long long gs_gl = ti.gl, gs_hl = ti.hl, gs_PG = ti.PG, gs_PH = ti.PH;
-    const long long tot_g = a.state->tot_g, tot_h = a.state->tot_h;
-    const uint32_t gmax_bits = a.state->gmax_bits, hmax_bits = a.state->hmax_bits;
     const FeatRec fr = a.feat_rec[f];
     const size_t hw = (size_t)a.F * a.nb;
 
-    // the two children: "small" was built by Algorithm 1, "large" is parent - small
-    // rows of this context (nl, nr) and over all ranks (nl_all, nr_all); which child is "small" and
-    // every row count that enters the split search are the ones over all ranks
-    const uint32_t n = ROOT ? a.N : gs_n, nl = ROOT ? n : gs_nl, nr = n - nl;
-    const uint32_t n_all = ROOT ? a.N_all : gs_n_all, nl_all = ROOT ? n_all : gs_nl_all, nr_all = n_all - nl_all;
-    const bool small_is_left = nl_all <= nr_all;
+    // the two children: "small" was built by Algorithm 1, "large" is parent - small.  Which child is
+    // "small" and every row count that enters the split search are the ones over all ranks.  What is
+    // the same for every feature of the leaf comes from the histogram kernel of the pass (ROOT: is
+    // worked out here).
     SplitParams pS = a.sp, pL = a.sp;
+    double dg, dh, tpS, tpL = 0.0;
+    Admit32 aS, aL;
+    bool small_is_left = true;
+    uint32_t P = 1u;
     if (ROOT) {
-        pS.G = tot_g; pS.H = tot_h; pS.n_s = n_all;
+        pS.G = a.state->tot_g; pS.H = a.state->tot_h; pS.n_s = a.N_all;
+        qg_scales(a.state, pS, dg, dh);   // interval lengths of Eq. 5 from the maxima stored by the quantizer
+        tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
+        aS = qg_admit32(pS, dh);
+        aL = aS;
     } else {
-        const long long gl = gs_gl, hl = gs_hl, gr = gs_PG - gl, hr = gs_PH - hl;
-        pS.G = small_is_left ? gl : gr; pS.H = small_is_left ? hl : hr; pS.n_s = small_is_left ? nl_all : nr_all;
-        pL.G = small_is_left ? gr : gl; pL.H = small_is_left ? hr : hl; pL.n_s = small_is_left ? nr_all : nl_all;
+        // thousands of features: worked out once per leaf by k_grow_prep; else here, for every feature
+        const JobPrep pr = SEP ? a.prep[j] : qg_job_prep(gs, j, a.state, a.sp, a.rows_min);
+        dg = pr.dg; dh = pr.dh; tpS = pr.tpS; tpL = pr.tpL;
+        aS = pr.aS; aL = pr.aL;
+        small_is_left = pr.small_is_left != 0;
+        P = a.merged ? 1u : pr.P;
+        pS.G = aS.G; pS.H = aS.H; pS.n_s = aS.n_s;
+        pL.G = aL.G; pL.H = aL.H; pL.n_s = aL.n_s;
     }
     __shared__ WarpBest sm[2][FIN_WARPS];
     __shared__ bool is_last;
     __shared__ unsigned long long wtot[2][FIN_WARPS];
-    // interval lengths of Eq. 5 from the maxima stored by the quantizer
-    const double dg = __ddiv_rn((double)__uint_as_float(gmax_bits), (double)pS.kg);
-    const double dh = pS.const_h ? 1.0 : __ddiv_rn((double)__uint_as_float(hmax_bits), (double)pS.kh);
-    const double tpS = qg_gain_term(pS.G, pS.H, dg, dh, pS.lambda);
-    const double tpL = ROOT ? 0.0 : qg_gain_term(pL.G, pL.H, dg, dh, pL.lambda);
     GainScale sc;
     sc.dg = (float)dg; sc.dh = (float)dh; sc.lambda = (float)pS.lambda;
-    const Admit32 aS = qg_admit32(pS, dh), aL = qg_admit32(pL, dh);
 
     // ---- phase A: the smaller child's bins summed over the partial histograms, the larger child's
     //      by subtraction from the parent's
     const int fl = fr.fl, W = 1 << fr.logW;
-    const uint32_t P = (ROOT || a.merged) ? 1u : qg_grow_parts((uint32_t)parts, small_is_left ? nl : nr, a.rows_min);
     const size_t pstride = (size_t)4 * a.nb * 32;
     unsigned long long *part = a.partial + (size_t)(slot0 + fr.tile * parts) * pstride +
                                (size_t)(fl & 3) * a.nb * W + (fl >> 2);
@@ -611,6 +612,13 @@ __global__ void __launch_bounds__(FIN_THREADS, FIN_BLOCKS_PER_SM) k_grow_finish(
         // barrier that every thread passes before the next leaf's first write to it
         finish_one<ROOT, SEP>(a, it - j * a.F, j);
     }
+}
+
+// With thousands of features: lane j works out what is the same for all features of leaf j, once, before
+// the finishing kernel (one warp).
+__global__ void __launch_bounds__(32) k_grow_prep(GrowArgs a) {
+    if (a.gs->done || (int)threadIdx.x >= a.gs->n_jobs) return;
+    a.prep[threadIdx.x] = qg_job_prep(a.gs, (int)threadIdx.x, a.state, a.sp, a.rows_min);
 }
 
 // With thousands of features the last step runs as a kernel of its own, one block per leaf of the
@@ -1051,6 +1059,7 @@ void fill_args(qgbdt_ctx *c, GrowArgs &a) {
     a.pb_total = c->grow_pb_total;
     a.pool = c->d_hist_pool;
     a.partial = c->d_grow_partial;
+    a.prep = c->d_grow_prep;
     a.cand = c->d_cand;
     a.F = c->F;
     a.nb = c->nb;
@@ -1120,6 +1129,10 @@ int enqueue_pass(qgbdt_ctx *c, const GrowArgs &a, cudaStream_t st, int n_jobs = 
     {
         const int resident = c->sm_count * FIN_BLOCKS_PER_SM, all = c->F * a.K;
         const unsigned grid = (unsigned)(all < resident ? all : resident);
+        if (a.sep_reduce) {
+            k_grow_prep<<<1, 32, 0, st>>>(a);
+            QG_LAUNCH_CHECK(c);
+        }
         if (a.sep_reduce) k_grow_finish<false, true><<<grid, FIN_THREADS, 0, st>>>(a);
         else k_grow_finish<false, false><<<grid, FIN_THREADS, 0, st>>>(a);
     }

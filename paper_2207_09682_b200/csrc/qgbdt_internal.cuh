@@ -165,6 +165,26 @@ struct GrowState {
                                      // rank's count, a sharded run sums it over the ranks before the histograms)
 };
 
+// Per-leaf constants of the split search on 32-bit sums (the functions are in split_scan.cuh).
+struct Admit32 {
+    int G;                             // totals of the leaf
+    uint32_t H, n_s, half;             // half = H / 2
+    unsigned long long x_min, x_end;   // row estimate within [min_data, n_s - min_data]  <=>  x_min <= X < x_end
+    uint32_t min_data;
+    int const_h;
+    float q_sure;                      // single-precision hessian sums from here on are certainly >= min_sum_h
+    double min_sum_h, dh;
+};
+
+// Per leaf being split: what is the same for all its features in the finishing kernel.
+struct JobPrep {
+    double dg, dh;         // interval lengths of Eq. 5
+    double tpS, tpL;       // the leaf's own term of Eq. 7 for the smaller and the larger child
+    Admit32 aS, aL;
+    uint32_t P;            // histogram CTAs per tile that took part
+    int32_t small_is_left;
+};
+
 struct qgbdt_ctx {
     qgbdt_params prm;
     int device = 0;
@@ -220,6 +240,7 @@ struct qgbdt_ctx {
     int grow_rows_min = 1024;                   // rows per histogram CTA of tree growth, at least
     uint32_t *d_grow_bits = nullptr;            // [grow_jobs][bits_stride] predicate bits of the leaves being split
     size_t grow_bits_stride = 0;
+    JobPrep *d_grow_prep = nullptr;                 // [GROW_MAX_JOBS]
     unsigned long long *d_grow_partial = nullptr;   // [grow_xcap * tiles][4][nb][32] partial histograms of growth
     uint2 *d_ent0 = nullptr, *d_ent1 = nullptr; // [N] (row, gradient code) pairs of the leaves, two buffers
     uint16_t *d_leaf_id = nullptr;              // [N] leaf of every row in the tree just grown

@@ -93,16 +93,6 @@ __device__ inline void qg_gain_bounds(long long gl, long long hl, const SplitPar
 
 // The same two tests for the tree-growing kernels, on 32-bit sums (a leaf's gradient and hessian sums
 // fit 32 bits: checked when the rows are loaded) and with the per-leaf constants taken out.
-struct Admit32 {
-    int G;                             // totals of the leaf
-    uint32_t H, n_s, half;             // half = H / 2
-    unsigned long long x_min, x_end;   // row estimate within [min_data, n_s - min_data]  <=>  x_min <= X < x_end
-    uint32_t min_data;
-    int const_h;
-    float q_sure;                      // single-precision hessian sums from here on are certainly >= min_sum_h
-    double min_sum_h, dh;
-};
-
 __device__ inline Admit32 qg_admit32(const SplitParams &p, double dh) {
     Admit32 a;
     a.G = (int)p.G; a.H = (uint32_t)p.H; a.n_s = (uint32_t)p.n_s; a.half = a.H / 2;
@@ -154,6 +144,28 @@ __device__ inline void qg_gain_bounds32(int gl, uint32_t hl, const Admit32 &a, c
         lo = -__int_as_float(0x7f800000);
         hi = __int_as_float(0x7f800000);
     }
+}
+
+// What the finishing kernel needs of a leaf being split that is the same for all its features (known
+// once the rows of both sides are: after the partition of the pass).
+__device__ inline JobPrep qg_job_prep(const GrowState *gs, int j, const DevState *state, const SplitParams &sp,
+                                      uint32_t rows_min) {
+    const GrowJob *job = gs->jobs + j;
+    const uint32_t n = job->n, nl = job->nl, nr = n - nl;
+    const uint32_t n_all = job->n_all, nl_all = (uint32_t)gs->nl_all[j], nr_all = n_all - nl_all;
+    const long long gl = job->gl, hl = job->hl, gr = job->PG - gl, hr = job->PH - hl;
+    JobPrep r;
+    r.small_is_left = nl_all <= nr_all ? 1 : 0;
+    SplitParams pS = sp, pL = sp;
+    pS.G = r.small_is_left ? gl : gr; pS.H = r.small_is_left ? hl : hr; pS.n_s = r.small_is_left ? nl_all : nr_all;
+    pL.G = r.small_is_left ? gr : gl; pL.H = r.small_is_left ? hr : hl; pL.n_s = r.small_is_left ? nr_all : nl_all;
+    qg_scales(state, sp, r.dg, r.dh);
+    r.tpS = qg_gain_term(pS.G, pS.H, r.dg, r.dh, sp.lambda);
+    r.tpL = qg_gain_term(pL.G, pL.H, r.dg, r.dh, sp.lambda);
+    r.aS = qg_admit32(pS, r.dh);
+    r.aL = qg_admit32(pL, r.dh);
+    r.P = qg_grow_parts((uint32_t)job->parts, r.small_is_left ? nl : nr, rows_min);
+    return r;
 }
 
 // Running state of one feature's scan in one lane.

@@ -91,6 +91,7 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
     if (shared_slots)
         QG_CUDA(c, cudaMemsetAsync(c->d_grow_partial, 0,
                                    (size_t)c->grow_xcap * c->tiles.size() * 4 * c->nb * 32 * sizeof(unsigned long long), st));
+    if (!c->d_grow_prep && (rc = alloc_dev(c, &c->d_grow_prep, (size_t)GROW_MAX_JOBS, "per-leaf constants")) != QGBDT_OK) return rc;
     if (!c->d_ent0 && (rc = alloc_dev(c, &c->d_ent0, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_ent1 && (rc = alloc_dev(c, &c->d_ent1, (size_t)c->N, "row/code pairs")) != QGBDT_OK) return rc;
     if (!c->d_leaf_id && (rc = alloc_dev(c, &c->d_leaf_id, (size_t)c->N, "leaf numbers")) != QGBDT_OK) return rc;

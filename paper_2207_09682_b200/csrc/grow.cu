@@ -137,7 +137,26 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_flags(GrowArgs a) {
     if (lb * PART_WARPS >= active) return;                               // no warp of this block has work
     const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
     uint32_t lefts = 0;
-    for (uint32_t w = w0; w < w1; w += 8) {
+    uint32_t w = w0;
+    // whole groups of eight words of 32 rows, all rows inside the leaf: no tests in the loop
+    const uint32_t w_full = n >> 5;   // words below this one have 32 rows
+    if (src && col8) {
+        const uint2 *ps = src + off + lane;
+        for (; w + 8 <= w1 && w + 8 <= w_full; w += 8) {
+            uint32_t row[8], code[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) row[k] = ps[(size_t)(w + k) << 5].x;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) code[k] = col8[row[k]];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t b = __ballot_sync(0xffffffffu, code[k] <= thr);
+                if (lane == k) bits[w + k] = b;
+                lefts += __popc(b);
+            }
+        }
+    }
+    for (; w < w1; w += 8) {
         uint32_t row[8], word[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -228,7 +247,33 @@ __global__ void __launch_bounds__(PART_THREADS) k_grow_scatter(GrowArgs a) {
     }
     const uint2 *src = buf < 0 ? nullptr : (buf ? a.ent1 : a.ent0);
     uint2 *dst = buf == 0 ? a.ent1 : a.ent0;
-    for (uint32_t w = w0; w < w1; w += 4) {
+    uint32_t w = w0;
+    const uint32_t w_full = n >> 5;   // words below this one have 32 rows
+    if (src) {
+        // whole groups of four words, all rows inside the leaf: no tests in the loop
+        const uint2 *ps = src + off + lane;
+        uint2 *pd = dst + off;
+        const uint32_t below = (1u << lane) - 1u;
+        for (; w + 4 <= w1 && w + 4 <= w_full; w += 4) {
+            uint32_t bw[4];
+            uint2 ent[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                bw[k] = bits[w + k];
+                ent[k] = ps[(size_t)(w + k) << 5];
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t rank_l = __popc(bw[k] & below);
+                const bool left = (bw[k] >> lane) & 1u;
+                // left rows keep their order at the front; right rows theirs behind all `total` left rows
+                const uint32_t dest = left ? before + rank_l : total + (((w + k) << 5) - before) + (lane - rank_l);
+                pd[dest] = ent[k];
+                before += __popc(bw[k]);
+            }
+        }
+    }
+    for (; w < w1; w += 4) {
         uint32_t bw[4];
         uint2 ent[4];
 #pragma unroll

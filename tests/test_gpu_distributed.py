@@ -70,6 +70,7 @@ def same_trees(a, b, trees):
     ("tall", 30_001, dict(num_trees=2, num_leaves=63), (0.2, 0.55, 0.9)),       # four uneven ranks
     ("large", 40_000, dict(num_trees=2, num_leaves=31), (0.4,)),               # constant hessian
     ("tall", 20_000, dict(num_trees=2, num_leaves=31, bits=8), (0.3, 0.7)),     # 32+32 local bins
+    ("wide", 12_000, dict(num_trees=1, num_leaves=20), (0.45,)),                # 2000 features: 128-byte rows
 ])
 def test_sharded_ranks_train_the_single_context_trees(name, rows, over, cuts):
     wl = synth.CONFIGS[name](device="cpu", rows=rows)

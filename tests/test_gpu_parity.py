@@ -439,6 +439,8 @@ TRAIN_CASES = [
     ("tall", 30_000, dict(num_trees=3, num_leaves=63)),
     ("large", 40_000, dict(num_trees=3, num_leaves=63)),
     ("wide", 3_000, dict(num_trees=2, num_leaves=15)),
+    # more than 512 features: per-leaf constants and the best split over the features in kernels of their own
+    ("wide600", 9_000, dict(num_trees=2, num_leaves=40)),
     # 32+32 local bins inside tree growth (two passes over the smaller child's rows)
     ("tall", 30_000, dict(num_trees=3, num_leaves=63, bits=8)),
     ("tall", 30_000, dict(num_trees=3, num_leaves=63, bits=6)),
@@ -455,7 +457,10 @@ TRAIN_CASES = [
 
 
 def train_case(name, rows, over, column_copy=None, refit=True):
-    wl = synth.CONFIGS[name](device="cpu", rows=rows) if name != "wide" else synth.wide(device="cpu", rows=rows, features=300)
+    if name.startswith("wide"):
+        wl = synth.wide(device="cpu", rows=rows, features=600 if name == "wide600" else 300)
+    else:
+        wl = synth.CONFIGS[name](device="cpu", rows=rows)
     kw = dict(wl.params, seed=11)
     kw.update(over)
     data, y = wl.bins.numpy(), wl.labels.numpy()
@@ -478,7 +483,7 @@ def train_case(name, rows, over, column_copy=None, refit=True):
     return ctx
 
 
-@pytest.mark.parametrize("name,rows,over", [TRAIN_CASES[0], TRAIN_CASES[2], TRAIN_CASES[4]])
+@pytest.mark.parametrize("name,rows,over", [TRAIN_CASES[0], TRAIN_CASES[2], TRAIN_CASES[5]])
 def test_training_with_leaf_values_from_the_quantized_sums(name, rows, over):
     # Sec. 4.2 without refitting: w~ from the integer sums of every leaf; trees, values and scores as the oracle's
     train_case(name, rows, over, refit=False)

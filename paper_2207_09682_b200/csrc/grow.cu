@@ -785,18 +785,33 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
     __syncthreads();
 
     // ---- (1) warp 0 replays the best-first order.  Lane l keeps the best of the leaves l, l + 32, ...
-    //      and looks at them again only when one of them changes.
+    //      and looks at them again only when one of them changes.  Up to 256 leaves the keys of a
+    //      lane's leaves stay in its registers (the replay is one long chain of dependent steps: every
+    //      shared-memory round trip taken out of it counts); beyond, in the shared array.
     if (warp == 0) {
+        constexpr int RS = 8;
+        const bool reg_keys = L <= 32 * RS;
         int n_leaves = n_leaves0, mand = -1, done = 0, commits = 0;
-        const size_t no = (size_t)tree_slot * (L > 1 ? L - 1 : 1);
         unsigned long long lk = 0;   // key of the lane's best gain (0: the lane has no leaf)
         int li = 0x7FFFFFFF;
+        unsigned long long kreg[RS];
+#pragma unroll
+        for (int q = 0; q < RS; ++q) {
+            const int i = lane + 32 * q;
+            kreg[q] = (reg_keys && i < n_leaves) ? gain_key(fg[i]) : 0ull;
+        }
         auto rescan = [&]() {
             lk = 0;
             li = 0x7FFFFFFF;
-            for (int i = lane; i < n_leaves; i += 32) {
-                const unsigned long long k = gain_key(fg[i]);
-                if (k > lk) { lk = k; li = i; }
+            if (reg_keys) {
+#pragma unroll
+                for (int q = 0; q < RS; ++q)
+                    if (kreg[q] > lk) { lk = kreg[q]; li = lane + 32 * q; }
+            } else {
+                for (int i = lane; i < n_leaves; i += 32) {
+                    const unsigned long long k = gain_key(fg[i]);
+                    if (k > lk) { lk = k; li = i; }
+                }
             }
         };
         rescan();
@@ -812,14 +827,8 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
             const int r = sf[bi], c0 = cs[r];
             if (c0 < 0) { mand = r; break; }
             const int node = n_leaves - 1, right = n_leaves;
-            if (lane == 0) {
-                a.m_left[no + node] = ~bi;
-                a.m_right[no + node] = ~right;
-                const int p = spn[r];
-                if (p >= 0) {
-                    if ((p & 1) == 0) a.m_left[no + (p >> 1)] = node;
-                    else a.m_right[no + (p >> 1)] = node;
-                }
+            const double g0 = cg[c0], g1 = cg[c0 + 1];   // gains of the two new numbered leaves
+            if (lane == 0) {   // shared memory only: the node arrays are written after the replay, in parallel
                 spn[c0] = node << 1;
                 spn[c0 + 1] = node << 1 | 1;
                 sf[bi] = c0;
@@ -827,7 +836,16 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
                 cl_rec[commits] = r;
                 cl_leaf[commits] = bi;
             }
-            if (lane < 2) fg[lane == 0 ? bi : right] = cg[c0 + lane];   // gains of the two new numbered leaves
+            if (reg_keys) {
+                const unsigned long long k0 = gain_key(g0), k1 = gain_key(g1);
+#pragma unroll
+                for (int q = 0; q < RS; ++q) {
+                    if (lane + 32 * q == bi) kreg[q] = k0;
+                    if (lane + 32 * q == right) kreg[q] = k1;
+                }
+            } else if (lane < 2) {
+                fg[lane == 0 ? bi : right] = lane == 0 ? g0 : g1;
+            }
             __syncwarp();
             ++n_leaves;
             ++commits;
@@ -844,6 +862,18 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
         unsigned long long rows = 0;
         for (int t = tid; t < commits; t += COMMIT_THREADS) {
             const int r = cl_rec[t], node = n_leaves0 - 1 + t, c0 = cs[r];
+            // children of the node: a child that was confirmed in this launch too is a node (the place of
+            // its own children names it), else the leaf number the replay gave it (left: the parent's,
+            // right: the next free one at the time)
+            const int gl = cs[c0], gr = cs[c0 + 1];
+            a.m_left[no + node] = (gl >= 0 && spn[gl] >= 0) ? (spn[gl] >> 1) : ~cl_leaf[t];
+            a.m_right[no + node] = (gr >= 0 && spn[gr] >= 0) ? (spn[gr] >> 1) : ~(n_leaves0 + t);
+            // a parent from an earlier launch learns of its new child node here (one from this launch above)
+            const int p = spn[r];
+            if (p >= 0 && (p >> 1) < n_leaves0 - 1) {
+                if ((p & 1) == 0) a.m_left[no + (p >> 1)] = node;
+                else a.m_right[no + (p >> 1)] = node;
+            }
             const NodeRec *q = a.recs + r;
             a.m_feature[no + node] = q->best.feature;
             a.m_bin[no + node] = q->best.bin;

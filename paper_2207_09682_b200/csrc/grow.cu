@@ -719,10 +719,15 @@ __global__ void __launch_bounds__(256) k_grow_merge(GrowArgs a) {
 // growth record and the list of splits confirmed in this launch, and later the compacted list of
 // the records whose split is not confirmed (the gain that orders them, the record, and the records
 // by rank); then, per growth record, its gain, its children (or -1) and its place in the tree.
+// Records whose split may be open at once (at least the 1024 entries the sort pads to; a multiple of
+// four so that the arrays behind one another stay 16-byte aligned).
+__host__ __device__ inline int commit_max_cand(int L) {
+    const int n = L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8;
+    return n < 1024 ? 1024 : (n + 3) & ~3;
+}
 __host__ __device__ inline size_t commit_region_bytes(int L) {
     const size_t a = (size_t)L * (sizeof(double) + 3 * sizeof(int));
-    size_t n = (size_t)(L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8);
-    if (n < 1024) n = 1024;   // the sort works on a power of two of entries
+    const size_t n = (size_t)commit_max_cand(L);
     const size_t b = n * (sizeof(double) + 2 * sizeof(int)) + 1024 * (sizeof(double) + sizeof(int));   // + the sort's second buffer
     return ((a > b ? a : b) + 15) / 16 * 16;
 }
@@ -761,7 +766,7 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
     int *cl_rec = sf + L;                                       // [L] confirmed in this launch: the record split ...
     int *cl_leaf = cl_rec + L;                                  // [L] ... and the number of the leaf it was
     // the region, second use
-    const int max_cand = (L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8) < 1024 ? 1024 : (L + 2 * GROW_SLACK + 2 * GROW_MAX_JOBS + 8);
+    const int max_cand = commit_max_cand(L);
     unsigned long long *cand_k = reinterpret_cast<unsigned long long *>(smem_raw);   // [max_cand] ordering keys of the open records
     int *cand_r = reinterpret_cast<int *>(cand_k + max_cand);   // [max_cand] the records
     // per record
@@ -975,7 +980,35 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
     int n_cand = s_ncand;
     if (n_cand > max_cand) n_cand = max_cand;   // cannot happen: the bound counts every record without a confirmed split
     // the open records in order: larger gain first, lower record on equal gain
-    if (n_cand <= 1024) {
+    if (n_cand <= 448) {
+        // few enough to count: the rank of a pair is the number of pairs that belong before it.  Every
+        // thread reads all pairs from shared memory, four at a time (the list is padded to a multiple of
+        // four with pairs that belong after every other): fewer dependent steps than a sorting network.
+        const int n4 = (n_cand + 3) & ~3;
+        if (tid >= n_cand && tid < n4) {
+            cand_k[tid] = 0ull;
+            cand_r[tid] = 0x7FFFFFFF;
+        }
+        __syncthreads();
+        if (tid < n_cand) {
+            const unsigned long long key = cand_k[tid];
+            const int rec = cand_r[tid];
+            const ulonglong2 *k2 = reinterpret_cast<const ulonglong2 *>(cand_k);
+            const int4 *r4 = reinterpret_cast<const int4 *>(cand_r);
+            int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+#pragma unroll 2
+            for (int q = 0; q < (n4 >> 2); ++q) {
+                const ulonglong2 ka = k2[2 * q], kb = k2[2 * q + 1];
+                const int4 rr = r4[q];
+                c0 += (ka.x > key || (ka.x == key && rr.x < rec)) ? 1 : 0;
+                c1 += (ka.y > key || (ka.y == key && rr.y < rec)) ? 1 : 0;
+                c2 += (kb.x > key || (kb.x == key && rr.z < rec)) ? 1 : 0;
+                c3 += (kb.y > key || (kb.y == key && rr.w < rec)) ? 1 : 0;
+            }
+            const int rank = c0 + c1 + c2 + c3;
+            by_rank[rank] = (rank < budget && cs[rec] == -1 && rec != mand) ? rec : -1;
+        }
+    } else if (n_cand <= 1024) {
         // bitonic sort of the (key, record) pairs, one per thread in registers, padded to a power of two
         // with entries that sort last.  Partners less than 32 apart exchange by shuffle; the others through
         // shared memory, in two buffers used in turn (one barrier per such step).

@@ -901,7 +901,9 @@ __global__ void __launch_bounds__(COMMIT_THREADS) k_grow_commit(GrowArgs a) {
                 a.front[i] = r;
             }
         }
-        if (rows) atomicAdd(&s_rows, rows);
+        // one shared atomic per warp (64-bit shared atomics are compare-and-swap loops)
+        for (int o = 16; o > 0; o >>= 1) rows += __shfl_xor_sync(0xffffffffu, rows, o);
+        if (lane == 0 && rows) atomicAdd(&s_rows, rows);
     }
     __syncthreads();   // the region is free from here on
     if (tid == 0) {

@@ -61,7 +61,10 @@ int ensure_train_buffers(qgbdt_ctx *c, int num_trees, cudaStream_t st) {
     if (c->grow_jobs <= 1 || !c->d_recs) {
         int k = 65536 / (c->F > 0 ? c->F : 1);
         c->grow_jobs = k < 2 ? 2 : (k > GROW_MAX_JOBS ? GROW_MAX_JOBS : k);
-        c->grow_xcap = 2 * qg_grow_parts_cap(c) + c->grow_jobs;
+        // histogram CTAs per tile a pass may use: twice one leaf's share of the SMs, four times with several
+        // tiles (a leaf's share is then small, and CTAs of unequal leaves fill the SMs better in more pieces:
+        // 2 % per tree at 2000 features; six and eight times were slower again)
+        c->grow_xcap = (c->tiles.size() > 1 ? 4 : 2) * qg_grow_parts_cap(c) + c->grow_jobs;
         int max_logw = 0;
         for (const TileDesc &t : c->tiles) max_logw = t.logW > max_logw ? t.logW : max_logw;
         // rows per histogram CTA of a pass, at least.  Rows of up to 32 bytes: every CTA of a leaf adds its

@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # 4 M rows scaled by the rows (traffic grows in proportion to them).  Valid only for the kernel sources
 # the capture was taken with.
 HIST_TRAFFIC = {"workload": "large", "bytes_per_launch": 11.01e6,
-                "sources_sha1": "55e5c455e31cb166af9cb1aae244ded3febcbf60"}
+                "sources_sha1": "0ba02b51281a9401982eb480d803ad5ff840cfbe"}
 
 
 def hist_traffic(workload, rows):

@@ -123,8 +123,10 @@ __global__ void __launch_bounds__(HIST_THREADS, 1) k_hist_coop(HistArgs a) {
 // Tree growth: a launch builds the histograms of the smaller children (ties: the left one) of all
 // leaves being split in the current pass.  The rows are (row, code) pairs in the buffer the scatter
 // kernel wrote; a job owns the CTAs x in [cta0, cta0 + parts) of every tile and the partial slots
-// slot0 + tile * parts + part; the histogram goes to the job's pool slot.  The grid is
-// (CTAs per tile, tile - tile0).
+// slot0 + tile * parts + part.  One CTA for a child: the histogram goes straight to the job's pool
+// slot.  Several: on rows of up to 64 bytes they all add into the tile's first partial slot (zero
+// before the launch, cleared by its reader), on 128-byte rows each stores a slot of its own; the
+// finishing kernel moves the sums to the pool slot.  The grid is (CTAs per tile, tile - tile0).
 struct GrowHist {
     const GrowState *gs;
     const uint2 *ent0, *ent1;
@@ -435,8 +437,8 @@ int qg_hist_grow_configure(qgbdt_ctx *c) {
 }
 
 // Histograms of the smaller children of the leaves being split in the current pass (sizes known
-// only on the device): partial histograms or, for a small child, the finished histogram in its
-// pool slot.
+// only on the device): sums in partial slots or, for a child that one CTA builds, the finished
+// histogram in its pool slot.
 int qg_hist_grow(qgbdt_ctx *c, cudaStream_t st) {
     const int bits = c->prm.bits;
     const int kg = qg_levels_g(bits);

@@ -75,10 +75,11 @@ struct FeatRec {
 };
 
 // Histogram CTAs per tile that take part in building a child of n rows during tree growth: one per
-// `rows_min` rows, at most `parts`.  rows_min is 1024 for rows of up to 32 bytes and grows with the
-// width of the widest tile (4096 for 128-byte rows): a CTA of a wide tile writes a quarter of a
-// megabyte of partial histogram that the finishing kernel has to read back, and has four times the
-// work per row to make up for its fixed cost.
+// `rows_min` rows, at most `parts`.  rows_min is 3072 for rows of up to 32 bytes (every CTA adds its
+// whole local histogram into the leaf's sums) and 1024 per 32 bytes of the widest tile beyond (4096
+// for 128-byte rows: a CTA of a wide tile writes a quarter of a megabyte of partial histogram that
+// the finishing kernel has to read back, and has four times the work per row to make up for its
+// fixed cost).
 __device__ __host__ inline uint32_t qg_grow_parts(uint32_t parts, uint32_t n, uint32_t rows_min) {
     uint32_t want = (n + rows_min - 1) / rows_min;
     if (want < 1) want = 1;

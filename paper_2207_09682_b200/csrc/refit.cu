@@ -167,6 +167,13 @@ struct WalkNode {           // a node of the tree being walked, in shared memory
     int32_t feature;
 };
 
+// The same for a matrix of one tile of 32-byte rows, in 8 bytes (32 lanes at 32 different nodes: half the
+// shared-memory wavefronts of the 16-byte node): children in 16 bits each (a context takes at most 4096
+// leaves), then the threshold and the byte of the row.
+__device__ __forceinline__ uint2 pack_node8(int left, int right, int bin, int byte) {
+    return make_uint2(((uint32_t)left & 0xFFFFu) | ((uint32_t)right << 16), (uint32_t)(bin & 0xFF) | ((uint32_t)(byte & 0xFF) << 8));
+}
+
 constexpr int WALK_THREADS = 256;
 
 // *p (two adjacent 32-bit shared words, low then high) += v, with 32-bit atomics.
@@ -209,9 +216,14 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk(const GrowState *gs, cons
     WalkNode *nodes = reinterpret_cast<WalkNode *>(wsm);
     unsigned long long *acc = reinterpret_cast<unsigned long long *>(wsm + (size_t)(n_nodes > 0 ? n_nodes : 1) * sizeof(WalkNode));
     uint32_t *srow = reinterpret_cast<uint32_t *>(acc + (SUMS ? 2 * L : 0)) + threadIdx.x * 9;   // this thread's row
+    uint2 *nodes8 = reinterpret_cast<uint2 *>(wsm);   // ROW_LOGW == 3: 8-byte nodes in the same place
     for (int i = threadIdx.x; i < n_nodes; i += WALK_THREADS) {
         const int f = m_feature[i];
         const FeatRec fr = feat_rec[f];
+        if (ROW_LOGW == 3) {
+            nodes8[i] = pack_node8(m_left[i], m_right[i], m_bin[i], fr.fl);
+            continue;
+        }
         WalkNode w;
         w.left = m_left[i]; w.right = m_right[i];
         w.logW = (uint8_t)fr.logW; w.shift = (uint8_t)(8 * fr.byte); w.bin = (uint8_t)m_bin[i]; w.byte = (uint8_t)fr.fl;
@@ -236,15 +248,17 @@ __global__ void __launch_bounds__(WALK_THREADS) k_walk(const GrowState *gs, cons
             }
             int node = 0;
             for (;;) {
-                const WalkNode w = nodes[node];
-                uint32_t code;
+                int next;
                 if (ROW_LOGW == 3) {
-                    code = reinterpret_cast<const uint8_t *>(srow)[w.byte];
+                    const uint2 w = nodes8[node];
+                    const uint32_t code = reinterpret_cast<const uint8_t *>(srow)[(w.y >> 8) & 0xFFu];
+                    next = code <= (w.y & 0xFFu) ? (int)(short)(w.x & 0xFFFFu) : (int)w.x >> 16;
                 } else {
+                    const WalkNode w = nodes[node];
                     const FeatRec fr = feat_rec[w.feature];
-                    code = (fr.col[(size_t)r << w.logW] >> w.shift) & 0xFFu;
+                    const uint32_t code = (fr.col[(size_t)r << w.logW] >> w.shift) & 0xFFu;
+                    next = code <= w.bin ? w.left : w.right;
                 }
-                const int next = code <= w.bin ? w.left : w.right;
                 if (next < 0) { leaf = ~next; break; }
                 node = next;
             }
